@@ -1,0 +1,201 @@
+/*
+ * gls.h -- C ABI of libgls: Gumbel-max list sampling (GLS) sweeps for NVIDIA B200 (sm_100a).
+ *
+ * The library implements the data-parallel part of "List-Level Distribution Coupling with
+ * Applications to Speculative Decoding and Lossy Compression" (arXiv 2506.05632):
+ *
+ *   - Sec. 3, Algorithm 1: with K sets of i.i.d. Exp(1) variables S_i^(k),
+ *         X^(k) = argmin_i S_i^(k) / p_i          (draft side, one race per draft k)
+ *         Y     = argmin_i min_k S_i^(k) / q_i    (target side, list-combined race)
+ *         accept iff Y is one of X^(1..K).
+ *   - Sec. 4, Algorithm 2: the same races per position j with noise U_i^(j,k), an active set S of
+ *     drafts that is pruned position by position, and a bonus token after L accepted positions.
+ *   - Sec. 5.1 and Appendix C: the same races over (importance) weights, with random bin labels
+ *     l_i, message M = l_Y and K decoders that only consider candidates whose label equals M.
+ *
+ * Everything is evaluated in the log domain:  argmin_i S_i/p_i = argmax_i (logit_i/T - ln S_i),
+ * because the softmax normaliser of a row does not depend on i.  Where rows with different
+ * normalisers meet (the min over k inside Y), each row's log-sum-exp is subtracted first, so the
+ * quantity compared is -ln(S_i^(k) / q_i^(j,k)) with q a true probability, as Algorithm 2 writes it.
+ *
+ * SHARED RANDOMNESS.  The paper only asks for i.i.d. uniforms shared by both parties (Algorithm 1,
+ * first step).  Here they are never stored: S = -ln U is a pure function of
+ * (seed, sequence id, position id, draft index k, token index i), generated inside the kernels by
+ * a counter-based generator (Philox4x32, published by Salmon et al., SC'11):
+ *
+ *     key     = (seed & 0xffffffff, seed >> 32)
+ *     counter = (c0 = token block, c1 = k | (domain << 16), c2 = position id, c3 = sequence id)
+ *     domain  = 0 decoding noise, 1 compression noise, 2 / 3 the refinement streams of 0 / 1
+ *
+ *   noise_spec 1:  block = i >> 2, w = out[i & 3],                v = (w + 0.5) * 2^-32
+ *   noise_spec 2:  coarse  block = i >> 3 in `domain`:   h = 16-bit field (i & 7) of the 128 output
+ *                  bits, i.e. (out[(i & 7) >> 1] >> (16 * (i & 1))) & 0xffff;
+ *                  refine  block = i >> 2 in `domain + 2`: r = out[i & 3];
+ *                                                               v = (h * 2^32 + r + 0.5) * 2^-48
+ *   S = -log1p(-v)   (v is strictly inside (0,1), so S is finite and positive; this is the paper's
+ *                     S = -ln U with U = 1 - v)
+ *
+ * A draft call and a verify call that describe the same (seed, sequence, position, k, i) therefore
+ * see the same S -- that is the coupling.  Both specs are exact definitions; spec 2 merely lets a
+ * kernel decide most tokens from the 16 coarse bits and generate the 32 refinement bits only for
+ * the few tokens that can still win.
+ *
+ * CONVENTIONS
+ *   - Token / candidate indices are 0-based (the paper counts from 1).
+ *   - All pointers are DEVICE pointers owned by the caller unless the name ends in `_host`.
+ *     The library allocates no device memory, keeps no state between calls, enqueues its kernels
+ *     on the caller's stream and returns without synchronising.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).
+ *   - Rows: the token dimension is contiguous; strides are in ELEMENTS and may be 0 (broadcast).
+ *     Rows whose first element is 16-byte aligned take the vectorised path; others are still
+ *     handled (slower scalar loads).
+ *   - A logit of -inf is a legal "masked" token (top-K truncation, Sec. 4.4).  NaN and +inf
+ *     logits never win a race and are excluded from the log-sum-exp.
+ *   - Ties (measure zero in exact arithmetic): lowest token index, then lowest k.
+ *   - Errors the host can see (null pointers, sizes <= 0, K > GLS_MAX_K, V >= 2^31, bad dtype,
+ *     inv_temp not finite or <= 0, workspace too small, misaligned base pointer) return a status
+ *     and enqueue nothing.  A row with no finite logit yields token -1 and ORs GLS_DEV_EMPTY_SUPPORT
+ *     into *device_status; nothing traps.
+ *   - Scores are computed in fp64 for the handful of candidates per row that survive the filter,
+ *     and returned as fp32.
+ */
+#ifndef GLS_H_
+#define GLS_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define GLS_MAX_K 64
+
+typedef enum {
+  GLS_OK = 0,
+  GLS_ERR_INVALID_ARG = 1,
+  GLS_ERR_UNSUPPORTED = 2,
+  GLS_ERR_MISALIGNED = 3,
+  GLS_ERR_WORKSPACE = 4,
+  GLS_ERR_CUDA = 5
+} gls_status_t;
+
+/* bits OR-ed into *device_status by the kernels */
+#define GLS_DEV_EMPTY_SUPPORT 1u /* some row had no finite logit: its token is -1 */
+
+typedef enum { GLS_F32 = 0, GLS_BF16 = 1 } gls_dtype_t;
+
+/* A batch of rows indexed [b][k][j][i]; i (token) is contiguous. */
+typedef struct {
+  const void* data; /* device pointer to element [0][0][0][0]                       */
+  int32_t dtype;    /* gls_dtype_t                                                  */
+  int64_t stride_b; /* elements between consecutive b; 0 broadcasts                 */
+  int64_t stride_k; /* elements between consecutive k; 0 = one row shared by all k  */
+  int64_t stride_j; /* elements between consecutive positions j                     */
+} gls_rows_t;
+
+/* noise flags */
+#define GLS_NOISE_SHARED_ACROSS_K 1u /* every k uses the noise of k = 0: the comparison scheme of
+                                        Sec. 5.2 in which all decoders share one set of numbers */
+
+/* Shared randomness: MUST be identical in the draft call and the verify call of one step. */
+typedef struct {
+  uint64_t seed;           /* Philox key                                                       */
+  uint32_t seq_base;       /* sequence id of batch row b is seq_base + b ...                   */
+  const uint32_t* seq_ids; /* ... unless this optional DEVICE array [B] is given               */
+  uint32_t pos_base;       /* position id of index j is pos_base + j                           */
+  uint32_t noise_spec;     /* 1 or 2 (see above); 0 selects 2                                  */
+  uint32_t rounds;         /* Philox rounds, 0 selects 10; 7..16 accepted                      */
+  uint32_t flags;          /* GLS_NOISE_*                                                      */
+} gls_noise_t;
+
+/* verify flags */
+#define GLS_COMBINE_ACTIVE 0u /* Algorithm 2 as printed: the min over k runs over the active set */
+#define GLS_COMBINE_ALL 1u    /* Appendix B, strong drafter invariance: min over all k           */
+#define GLS_NO_BONUS 2u       /* target rows cover positions 0..L-1 only; no bonus token         */
+
+/* Library version, major * 10000 + minor * 100 + patch. */
+int gls_version(void);
+
+/* Human-readable name of a status code (static storage, never NULL). */
+const char* gls_status_string(int status);
+
+/* Bytes of device workspace that any of the three entry points below needs for a problem of
+ * B batch rows, K drafts (streams), J positions and V tokens (candidates).  The workspace holds
+ * the per-(row, vocabulary-slice) partial results of the split reduction; its contents on entry
+ * are ignored and it may be reused by the next call on the same stream. */
+size_t gls_workspace_bytes(int B, int K, int J, int64_t V);
+
+/*
+ * Draft side -- Sec. 3 step 2, Algorithm 1 (third step), Algorithm 2 draft loop:
+ *     X[b,k,j] = argmin_i S_i^(j,k) / p_i^(j,k) = argmax_i ( logits[b,k,j,i] * inv_temp_k - ln S )
+ * with S keyed by (seed, seq(b), pos_base + j, k, i), noise domain 0.
+ *
+ *   draft_logits          [B,K,J,V] rows (fp32 or bf16)
+ *   inv_temp              1 / temperature, used for every k unless ...
+ *   inv_temp_per_draft_host  ... this HOST array [K] is non-NULL (Sec. 4.3 varies draft temperatures)
+ *   out_tokens            [B,K,J] int32, -1 for a row without finite logits
+ *   out_scores            NULL or [B,K,J] fp32: the winning logit*inv_temp - ln S (unnormalised)
+ *   workspace, workspace_bytes  >= gls_workspace_bytes(B,K,J,V)
+ *   device_status         NULL or uint32[1]; bits are OR-ed in, the caller zeroes it
+ */
+int gls_draft_sample(const gls_rows_t* draft_logits, int B, int K, int J, int64_t V, float inv_temp,
+                     const float* inv_temp_per_draft_host, const gls_noise_t* noise,
+                     int32_t* out_tokens, float* out_scores, void* workspace,
+                     size_t workspace_bytes, uint32_t* device_status, void* stream);
+
+/*
+ * Target side and verification -- Sec. 3 step 1, Algorithm 2 from "Let the set of active drafts"
+ * to the end.  With S = {0..K-1} initially, for j = 0..L-1:
+ *     Y_j = i-component of argmin_{i, k in S} S_i^(j,k) / q_i^(j,k),
+ *           q^(j,k) = softmax(target_logits[b,k,j,:] * inv_temp)
+ *     accept[b,k,j] = (k in S and draft_tokens[b,k,j] == Y_j);  S <- {k in S : accept}
+ *     if S is empty: tau = j + 1, stop.
+ * If all L positions leave S non-empty, the bonus token Y_L is drawn the same way from the rows at
+ * position L and tau = L + 1 (with GLS_NO_BONUS: no such rows, tau = L).
+ * GLS_COMBINE_ALL takes the min over every k (Appendix B) while S still records the survivors.
+ * Algorithm 1 is the case L = 1 with GLS_NO_BONUS: accept iff some accept[b,k,0] is 1.
+ *
+ *   target_logits   [B,K,J,V] rows, J = L + 1 (J = L with GLS_NO_BONUS)
+ *   draft_tokens    [B,K,L] int32 (the X of the draft phase)
+ *   out_tokens      [B,J] int32, -1 at and beyond index tau
+ *   out_num_tokens  [B] int32 = tau
+ *   out_accept      [B,K,L] uint8
+ *   out_scores      NULL or [B,J] fp32: ln(q_Y / S) of each emitted token, 0 beyond tau
+ *   L = 0 is legal (bonus token only).
+ */
+int gls_target_sample_verify(const gls_rows_t* target_logits, int B, int K, int L, int64_t V,
+                             float inv_temp, const int32_t* draft_tokens, const gls_noise_t* noise,
+                             uint32_t flags, int32_t* out_tokens, int32_t* out_num_tokens,
+                             uint8_t* out_accept, float* out_scores, void* workspace,
+                             size_t workspace_bytes, uint32_t* device_status, void* stream);
+
+/*
+ * Compression -- Sec. 5.1 and Appendix C.  Per batch row b (one source sample):
+ *     encoder:   Y = argmin_i min_k S_i^(k) / lambda_q,i          lambda_q = softmax(enc_logw[b,:])
+ *                M = bins[Y]                                      (the log2(L_max)-bit message)
+ *     decoder k: X^(k) = argmin_{i : bins[i] == M} S_i^(k) / lambda_p,i^(k)
+ *                                                                 from dec_logw[b,k,:]
+ *     match = (Y is one of X^(1..K))
+ * Noise is keyed by (seed, seq(b), pos_base, k, i) in domain 1.  Normalising the weights cannot
+ * change a per-row argmin; it only enters the reported encoder score through the log-sum-exp.
+ *
+ *   enc_logw      rows [B,1,1,N]: stride_b (or 0) is used, stride_k / stride_j are ignored
+ *   dec_logw      rows [B,K,1,N]; NULL skips the decoders (out_dec_index / out_match then unused)
+ *   bins          NULL (every label equal, L_max = 1) or uint8 labels [N] (bins_stride_b = 0) or
+ *                 [B,N] (bins_stride_b = N)
+ *   out_enc_index [B] int32, out_message [B] uint8, out_dec_index [B,K] int32, out_match [B] uint8
+ *   out_scores    NULL or [B,1+K] fp32: encoder ln(lambda_q,Y / S), then each decoder's
+ *                 unnormalised winning logw - ln S
+ *   workspace     >= gls_workspace_bytes(B, K, 2, N)
+ */
+int gls_compress_select(const gls_rows_t* enc_logw, const gls_rows_t* dec_logw, const uint8_t* bins,
+                        int64_t bins_stride_b, int B, int K, int64_t N, const gls_noise_t* noise,
+                        int32_t* out_enc_index, uint8_t* out_message, int32_t* out_dec_index,
+                        uint8_t* out_match, float* out_scores, void* workspace,
+                        size_t workspace_bytes, uint32_t* device_status, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* GLS_H_ */
