@@ -153,7 +153,10 @@ int gls_draft_sample(const gls_rows_t* draft_logits, int B, int K, int J, int64_
  *     if S is empty: tau = j + 1, stop.
  * If all L positions leave S non-empty, the bonus token Y_L is drawn the same way from the rows at
  * position L and tau = L + 1 (with GLS_NO_BONUS: no such rows, tau = L).
- * GLS_COMBINE_ALL takes the min over every k (Appendix B) while S still records the survivors.
+ * GLS_COMBINE_ALL is Appendix B: Y_j = argmin_i min over ALL k of S_i^(j,k) / q_i with q the target
+ * distribution of the accepted prefix, while S still records the survivors.  It is implemented for
+ * target rows shared by all k (stride_k = 0, where each stream's race over the shared row is that
+ * quantity); per-draft target rows return GLS_ERR_UNSUPPORTED.
  * Algorithm 1 is the case L = 1 with GLS_NO_BONUS: accept iff some accept[b,k,0] is 1.
  *
  *   target_logits   [B,K,J,V] rows, J = L + 1 (J = L with GLS_NO_BONUS)
@@ -187,7 +190,7 @@ int gls_target_sample_verify(const gls_rows_t* target_logits, int B, int K, int 
  *   out_enc_index [B] int32, out_message [B] uint8, out_dec_index [B,K] int32, out_match [B] uint8
  *   out_scores    NULL or [B,1+K] fp32: encoder ln(lambda_q,Y / S), then each decoder's
  *                 unnormalised winning logw - ln S
- *   workspace     >= gls_workspace_bytes(B, K, 2, N)
+ *   workspace     >= gls_workspace_bytes(B, K, 1, N)  (the encoder and decoder phases reuse it)
  */
 int gls_compress_select(const gls_rows_t* enc_logw, const gls_rows_t* dec_logw, const uint8_t* bins,
                         int64_t bins_stride_b, int B, int K, int64_t N, const gls_noise_t* noise,

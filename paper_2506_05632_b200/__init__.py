@@ -1,1 +1,14 @@
-"""B200-native Gumbel-max list sampling: Python binding of libgls (see include/gls.h)."""
+"""B200-native Gumbel-max list sampling (arXiv 2506.05632): Python binding of libgls.
+
+The functions here only marshal arguments (torch tensors -> raw device pointers, strides in
+elements) into the C ABI declared in include/gls.h; every step of the method runs in the CUDA
+kernels of csrc/.  There is no CPU fallback: if libgls.so cannot be loaded the calls raise.
+
+    draft_sample(logits, ...)                 Algorithm 1 third step / Algorithm 2 draft loop
+    target_sample_verify(logits, tokens, ...) Algorithm 2 verification
+    compress_select(enc, dec, bins, ...)      Sec. 5.1 encoder / decoder index selection
+"""
+from .binding import (  # noqa: F401
+    COMBINE_ACTIVE, COMBINE_ALL, NO_BONUS, NOISE_SHARED_ACROSS_K, DEV_EMPTY_SUPPORT, GlsError,
+    build, compress_select, draft_sample, lib_path, load, status_string, target_sample_verify,
+    version, workspace_bytes)

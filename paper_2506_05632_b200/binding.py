@@ -1,0 +1,247 @@
+"""ctypes binding of libgls.so (C ABI in include/gls.h).  Argument marshalling only."""
+import ctypes as C
+import os
+import subprocess
+import threading
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_ROOT = os.path.dirname(_HERE)
+_SRC_DIR = os.path.join(_HERE, "csrc")
+_LIB = os.path.join(_HERE, "libgls.so")
+
+COMBINE_ACTIVE, COMBINE_ALL, NO_BONUS = 0, 1, 2
+NOISE_SHARED_ACROSS_K = 1
+DEV_EMPTY_SUPPORT = 1
+F32, BF16 = 0, 1
+
+_lock = threading.Lock()
+_lib = None
+
+
+class GlsError(RuntimeError):
+    pass
+
+
+def lib_path():
+    return _LIB
+
+
+def _sources():
+    return sorted(os.path.join(_SRC_DIR, f) for f in os.listdir(_SRC_DIR)
+                  if f.endswith((".cu", ".cuh"))) + [os.path.join(_ROOT, "include", "gls.h")]
+
+
+def build(force=False, verbose=False):
+    """Compile csrc/*.cu into libgls.so for sm_100a with nvcc (cross-compiles without a GPU)."""
+    srcs = _sources()
+    if (not force and os.path.exists(_LIB)
+            and os.path.getmtime(_LIB) >= max(os.path.getmtime(s) for s in srcs)):
+        return _LIB
+    cus = [s for s in srcs if s.endswith(".cu")]
+    tmp = _LIB + ".tmp%d" % os.getpid()
+    cmd = ["nvcc", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
+           "-shared", "-Xcompiler", "-fPIC", "-o", tmp] + cus
+    if verbose:
+        cmd.insert(1, "-Xptxas=-v")
+    subprocess.run(cmd, check=True)
+    os.replace(tmp, _LIB)
+    return _LIB
+
+
+class _Rows(C.Structure):
+    _fields_ = [("data", C.c_void_p), ("dtype", C.c_int32), ("stride_b", C.c_int64),
+                ("stride_k", C.c_int64), ("stride_j", C.c_int64)]
+
+
+class _Noise(C.Structure):
+    _fields_ = [("seed", C.c_uint64), ("seq_base", C.c_uint32), ("seq_ids", C.c_void_p),
+                ("pos_base", C.c_uint32), ("noise_spec", C.c_uint32), ("rounds", C.c_uint32),
+                ("flags", C.c_uint32)]
+
+
+def load():
+    """Load libgls.so (building it if the sources are newer and nvcc is present)."""
+    global _lib
+    with _lock:
+        if _lib is not None:
+            return _lib
+        if not os.path.exists(_LIB):
+            build()
+        L = C.CDLL(_LIB)
+        L.gls_version.restype = C.c_int
+        L.gls_status_string.restype = C.c_char_p
+        L.gls_status_string.argtypes = [C.c_int]
+        L.gls_workspace_bytes.restype = C.c_size_t
+        L.gls_workspace_bytes.argtypes = [C.c_int, C.c_int, C.c_int, C.c_int64]
+        L.gls_draft_sample.restype = C.c_int
+        L.gls_draft_sample.argtypes = [
+            C.POINTER(_Rows), C.c_int, C.c_int, C.c_int, C.c_int64, C.c_float, C.c_void_p,
+            C.POINTER(_Noise), C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p,
+            C.c_void_p]
+        L.gls_target_sample_verify.restype = C.c_int
+        L.gls_target_sample_verify.argtypes = [
+            C.POINTER(_Rows), C.c_int, C.c_int, C.c_int, C.c_int64, C.c_float, C.c_void_p,
+            C.POINTER(_Noise), C.c_uint32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
+            C.c_void_p, C.c_size_t, C.c_void_p, C.c_void_p]
+        L.gls_compress_select.restype = C.c_int
+        L.gls_compress_select.argtypes = [
+            C.POINTER(_Rows), C.POINTER(_Rows), C.c_void_p, C.c_int64, C.c_int, C.c_int,
+            C.c_int64, C.POINTER(_Noise), C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
+            C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p, C.c_void_p]
+        _lib = L
+        return _lib
+
+
+def version():
+    return int(load().gls_version())
+
+
+def status_string(rc):
+    return load().gls_status_string(int(rc)).decode()
+
+
+def workspace_bytes(B, K, J, V):
+    return int(load().gls_workspace_bytes(int(B), int(K), int(J), int(V)))
+
+
+def _check(rc):
+    if rc != 0:
+        raise GlsError(status_string(rc))
+
+
+def _rows(t, lead):
+    """gls_rows_t of a tensor whose last dim is contiguous; `lead` leading dims give strides."""
+    if not t.is_cuda:
+        raise GlsError("libgls takes device tensors; there is no CPU path")
+    if t.dtype == torch.float32:
+        dt = F32
+    elif t.dtype == torch.bfloat16:
+        dt = BF16
+    else:
+        raise GlsError("logits must be float32 or bfloat16")
+    if t.stride(-1) != 1 and t.shape[-1] > 1:
+        raise GlsError("the token dimension must be contiguous")
+    st = [t.stride(d) for d in range(lead)] + [0] * (3 - lead)
+    return _Rows(t.data_ptr(), dt, st[0], st[1], st[2])
+
+
+def _noise(seed, seq_base, seq_ids, pos_base, spec, rounds, flags):
+    ptr = None
+    if seq_ids is not None:
+        if seq_ids.dtype != torch.int32 or not seq_ids.is_cuda or not seq_ids.is_contiguous():
+            raise GlsError("seq_ids must be a contiguous int32 device tensor (bit pattern = uint32)")
+        ptr = seq_ids.data_ptr()
+    return _Noise(int(seed) & (2**64 - 1), int(seq_base), ptr, int(pos_base), int(spec),
+                  int(rounds), int(flags))
+
+
+def _ptr(t):
+    return None if t is None else t.data_ptr()
+
+
+def _stream():
+    return torch.cuda.current_stream().cuda_stream
+
+
+def _workspace(workspace, need, device):
+    if workspace is None:
+        workspace = torch.empty(need, dtype=torch.uint8, device=device)
+    return workspace
+
+
+def draft_sample(logits, inv_temp=1.0, inv_temp_per_draft=None, seed=0, seq_base=0, seq_ids=None,
+                 pos_base=0, spec=2, rounds=10, noise_flags=0, want_scores=True, workspace=None,
+                 status=None, out_tokens=None, out_scores=None):
+    """logits [B,K,J,V] (device, fp32/bf16) -> (tokens int32 [B,K,J], scores fp32 [B,K,J] | None)."""
+    L = load()
+    B, K, J, V = logits.shape
+    dev = logits.device
+    rows = _rows(logits, 3)
+    nz = _noise(seed, seq_base, seq_ids, pos_base, spec, rounds, noise_flags)
+    if out_tokens is None:
+        out_tokens = torch.empty((B, K, J), dtype=torch.int32, device=dev)
+    if out_scores is None and want_scores:
+        out_scores = torch.empty((B, K, J), dtype=torch.float32, device=dev)
+    need = workspace_bytes(B, K, J, V)
+    workspace = _workspace(workspace, need, dev)
+    itk = None
+    if inv_temp_per_draft is not None:
+        itk = (C.c_float * K)(*[float(x) for x in inv_temp_per_draft])
+    _check(L.gls_draft_sample(C.byref(rows), B, K, J, V, float(inv_temp),
+                              C.cast(itk, C.c_void_p) if itk is not None else None, C.byref(nz),
+                              _ptr(out_tokens), _ptr(out_scores), workspace.data_ptr(),
+                              workspace.numel(), _ptr(status), _stream()))
+    return out_tokens, out_scores
+
+
+def target_sample_verify(logits, draft_tokens, inv_temp=1.0, flags=0, seed=0, seq_base=0,
+                         seq_ids=None, pos_base=0, spec=2, rounds=10, noise_flags=0,
+                         want_scores=True, workspace=None, status=None, out=None):
+    """logits [B,K,J,V], draft_tokens int32 [B,K,L]; J = L+1 (L with NO_BONUS).
+
+    Returns dict(tokens [B,J], tau [B], accept [B,K,L], scores [B,J] | None)."""
+    L = load()
+    B, K, J, V = logits.shape
+    Ld = J if (flags & NO_BONUS) else J - 1
+    dev = logits.device
+    rows = _rows(logits, 3)
+    nz = _noise(seed, seq_base, seq_ids, pos_base, spec, rounds, noise_flags)
+    if Ld > 0:
+        if draft_tokens.dtype != torch.int32 or not draft_tokens.is_contiguous():
+            raise GlsError("draft_tokens must be contiguous int32")
+        assert tuple(draft_tokens.shape) == (B, K, Ld)
+    if out is None:
+        out = dict(tokens=torch.empty((B, J), dtype=torch.int32, device=dev),
+                   tau=torch.empty((B,), dtype=torch.int32, device=dev),
+                   accept=torch.empty((B, K, Ld), dtype=torch.uint8, device=dev),
+                   scores=torch.empty((B, J), dtype=torch.float32, device=dev)
+                   if want_scores else None)
+    need = workspace_bytes(B, K, J, V)
+    workspace = _workspace(workspace, need, dev)
+    _check(L.gls_target_sample_verify(
+        C.byref(rows), B, K, Ld, V, float(inv_temp), _ptr(draft_tokens) if Ld > 0 else None,
+        C.byref(nz), int(flags), _ptr(out["tokens"]), _ptr(out["tau"]),
+        _ptr(out["accept"]) if Ld > 0 else None, _ptr(out.get("scores")), workspace.data_ptr(),
+        workspace.numel(), _ptr(status), _stream()))
+    return out
+
+
+def compress_select(enc_logw, dec_logw=None, bins=None, K=None, seed=0, seq_base=0, seq_ids=None,
+                    pos_base=0, spec=2, rounds=10, noise_flags=0, want_scores=True, workspace=None,
+                    status=None, out=None):
+    """enc_logw [B,N], dec_logw [B,K,N] | None, bins uint8 [N] | [B,N] | None.
+
+    Returns dict(enc_index [B], message [B], dec_index [B,K], match [B], scores [B,1+K] | None)."""
+    L = load()
+    B, N = enc_logw.shape
+    dev = enc_logw.device
+    erows = _rows(enc_logw, 1)
+    drows = None
+    if dec_logw is not None:
+        assert dec_logw.shape[0] == B and dec_logw.shape[2] == N
+        K = dec_logw.shape[1]
+        drows = _rows(dec_logw, 2)
+    assert K is not None
+    bsb = 0
+    if bins is not None:
+        if bins.dtype != torch.uint8 or not bins.is_contiguous():
+            raise GlsError("bins must be contiguous uint8")
+        bsb = 0 if bins.dim() == 1 else N
+    nz = _noise(seed, seq_base, seq_ids, pos_base, spec, rounds, noise_flags)
+    if out is None:
+        out = dict(enc_index=torch.empty((B,), dtype=torch.int32, device=dev),
+                   message=torch.empty((B,), dtype=torch.uint8, device=dev),
+                   dec_index=torch.full((B, K), -1, dtype=torch.int32, device=dev),
+                   match=torch.zeros((B,), dtype=torch.uint8, device=dev),
+                   scores=torch.full((B, 1 + K), float("nan"), dtype=torch.float32, device=dev)
+                   if want_scores else None)
+    need = workspace_bytes(B, K, 1, N)
+    workspace = _workspace(workspace, need, dev)
+    _check(L.gls_compress_select(
+        C.byref(erows), C.byref(drows) if drows is not None else None, _ptr(bins), bsb, B, K, N,
+        C.byref(nz), _ptr(out["enc_index"]), _ptr(out["message"]), _ptr(out["dec_index"]),
+        _ptr(out["match"]), _ptr(out.get("scores")), workspace.data_ptr(), workspace.numel(),
+        _ptr(status), _stream()))
+    return out

@@ -1,0 +1,478 @@
+// gls_api.cu -- C ABI of libgls (see include/gls.h) and the small kernels around the sweep:
+// the split-vocabulary reduction with exact re-scoring of the winner, and the per-sequence
+// epilogues (Algorithm 2's active-set loop; the encoder / decoder bookkeeping of Sec. 5.1).
+//
+// All noise is evaluated by the device functions of gls_kernels.cuh, compiled once in this
+// translation unit, so the draft-side, target-side and compression entry points see bit-identical
+// shared randomness (the paper's analysis assumes identical floating-point behaviour on both
+// sides of the coupling, Sec. 5.3).
+#include <cmath>
+#include <cstring>
+
+#include "../../include/gls.h"
+#include "gls_kernels.cuh"
+
+namespace gls {
+
+constexpr int kNumSMs = 148;  // B200
+constexpr int kMinChunk = 2048;
+constexpr int kMaxChunk = 16384;
+
+struct Plan {
+  int chunk, splits;
+  long long rows, n_items;
+  size_t off_hints, off_partials, off_rows, total;
+};
+
+static size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+// Slice size: aim at ~8 work items per resident warp so that the static round-robin over warps
+// balances, but keep slices long enough to amortise the per-item reduction.
+static Plan make_plan(long long rows, long long V) {
+  Plan p;
+  const long long target_items = 8LL * kNumSMs * 32;
+  long long chunk = (rows * V + target_items - 1) / target_items;
+  chunk = (chunk + kWarpTokens - 1) / kWarpTokens * kWarpTokens;
+  if (chunk < kMinChunk) chunk = kMinChunk;
+  if (chunk > kMaxChunk) chunk = kMaxChunk;
+  const long long vceil = (V + kWarpTokens - 1) / kWarpTokens * kWarpTokens;
+  if (chunk > vceil) chunk = vceil;
+  p.chunk = (int)chunk;
+  p.splits = (int)((V + chunk - 1) / chunk);
+  p.rows = rows;
+  p.n_items = rows * p.splits;
+  p.off_hints = 0;
+  p.off_partials = align_up((size_t)rows * sizeof(uint32_t), 256);
+  p.off_rows = p.off_partials + align_up((size_t)p.n_items * sizeof(Partial), 256);
+  p.total = p.off_rows + align_up((size_t)rows * sizeof(RowResult), 256);
+  return p;
+}
+
+// ------------------------------------------------------------------------------------------
+// Split-V reduction: one warp per row merges the slices' partials, re-scores the leading
+// candidate(s) in fp64 and merges the softmax statistics.
+//   out_mode 0: write RowResult only; 1: also write tokens / scores (draft side).
+// ------------------------------------------------------------------------------------------
+template <int DT, int SPEC, int ROUNDS>
+__global__ void __launch_bounds__(128)
+finalize_rows_kernel(const __grid_constant__ SweepArgs A, int rows, int with_lse,
+                     RowResult* __restrict__ rowres, int32_t* __restrict__ out_tokens,
+                     float* __restrict__ out_scores, uint32_t* __restrict__ dev_status) {
+  const int lane = threadIdx.x & 31;
+  const int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  if (row >= rows) return;
+  constexpr int ES = DT == kBF16 ? 2 : 4;
+  const int j = row % A.J;
+  const int bk = row / A.J;
+  const int k = bk % A.K;
+  const int b = bk / A.K;
+  const float inv_t = A.inv_t[k];
+  const float c2 = inv_t * kLog2e;
+
+  Top2 best;
+  top2_init(best);
+  float lm = kLseFloor;
+  for (int s = lane; s < A.splits; s += 32) {
+    const Partial p = A.partials[(long long)row * A.splits + s];
+    top2_offer(best, p.s1, p.i1);
+    top2_offer(best, p.s2, p.i2);
+    lm = fmaxf(lm, p.lm);
+  }
+  top2_warp_merge(best);
+#pragma unroll
+  for (int d = 16; d > 0; d >>= 1) lm = fmaxf(lm, __shfl_xor_sync(0xffffffffu, lm, d));
+  double lsum = 0.0;
+  if (with_lse) {
+    for (int s = lane; s < A.splits; s += 32) {
+      const Partial p = A.partials[(long long)row * A.splits + s];
+      if (p.ls > 0.f) lsum += (double)p.ls * exp2((double)(p.lm - lm) * (double)c2);
+    }
+#pragma unroll
+    for (int d = 16; d > 0; d >>= 1) lsum += __shfl_xor_sync(0xffffffffu, lsum, d);
+  }
+  if (lane != 0) return;
+
+  RowResult r;
+  r.pad0 = r.pad1 = r.pad2 = 0;
+  r.lse = (with_lse && lsum > 0.0) ? (double)lm * (double)inv_t + log(lsum)
+                                   : -CUDART_INF;
+  if (best.i1 < 0) {
+    r.idx = -1;
+    r.score = -CUDART_INF;
+    if (dev_status) atomicOr(dev_status, GLS_DEV_EMPTY_SUPPORT);
+  } else {
+    const char* rowp = (const char*)A.data + (b * A.sb + k * A.sk + j * A.sj) * ES;
+    StreamKey sk;
+    sk.c1 = ((uint32_t)k & A.kmask) | (A.domain << 16);
+    sk.pos = A.pos_base + (uint32_t)j;
+    sk.seq = A.seq_ids ? A.seq_ids[b] : A.seq_base + (uint32_t)b;
+    double e1 = exact_score<DT, SPEC, ROUNDS>(A, rowp, sk, best.i1, inv_t);
+    int idx = best.i1;
+    // a runner-up closer than the fp32 error bound is re-scored too
+    const float window = 2.0f * 0x1p-17f * (36.0f + fabsf(best.s1));
+    if (best.i2 >= 0 && best.s1 - best.s2 <= window) {
+      const double e2 = exact_score<DT, SPEC, ROUNDS>(A, rowp, sk, best.i2, inv_t);
+      if (e2 > e1 || (e2 == e1 && best.i2 < idx)) {
+        e1 = e2;
+        idx = best.i2;
+      }
+    }
+    r.idx = idx;
+    r.score = e1;
+  }
+  if (rowres) rowres[row] = r;
+  if (out_tokens) out_tokens[row] = r.idx;
+  if (out_scores) out_scores[row] = r.idx >= 0 ? (float)r.score : CUDART_NAN_F;
+}
+
+// ------------------------------------------------------------------------------------------
+// Algorithm 2, from "Let the set of active drafts be S" to the end; one thread per sequence.
+// rows[(b*K + k)*J + j] holds the winner of row (b,k,j) under its own noise stream.
+// ------------------------------------------------------------------------------------------
+__global__ void verify_epilogue_kernel(const RowResult* __restrict__ rows, int B, int K, int L,
+                                       int J, uint32_t flags,
+                                       const int32_t* __restrict__ draft_tokens,
+                                       int32_t* __restrict__ out_tokens,
+                                       int32_t* __restrict__ out_num, uint8_t* __restrict__ accept,
+                                       float* __restrict__ out_scores,
+                                       uint32_t* __restrict__ dev_status) {
+  const int b = blockIdx.x * blockDim.x + threadIdx.x;
+  if (b >= B) return;
+  unsigned long long active = K >= 64 ? ~0ull : ((1ull << K) - 1ull);
+  for (int j = 0; j < J; ++j) {
+    out_tokens[(long long)b * J + j] = -1;
+    if (out_scores) out_scores[(long long)b * J + j] = 0.f;
+  }
+  for (long long t = 0; t < (long long)K * L; ++t) accept[(long long)b * K * L + t] = 0;
+  int n_out = 0;
+  for (int j = 0; j < J; ++j) {
+    // Y_j = argmin_i min_{k in S} S_i^(j,k) / q_i^(j,k)  ==  best of the rows' winners after
+    // subtracting each row's log-sum-exp; ties: lowest token, then lowest k
+    double bs = 0.0;
+    int bi = -1;
+    for (int k = 0; k < K; ++k) {
+      if (!((active >> k) & 1ull) && !(flags & GLS_COMBINE_ALL)) continue;
+      const RowResult r = rows[((long long)b * K + k) * J + j];
+      if (r.idx < 0) continue;
+      const double sc = r.score - r.lse;
+      if (bi < 0 || sc > bs || (sc == bs && r.idx < bi)) {
+        bs = sc;
+        bi = r.idx;
+      }
+    }
+    out_tokens[(long long)b * J + j] = bi;
+    if (out_scores) out_scores[(long long)b * J + j] = bi >= 0 ? (float)bs : CUDART_NAN_F;
+    if (bi < 0 && dev_status) atomicOr(dev_status, GLS_DEV_EMPTY_SUPPORT);
+    n_out = j + 1;
+    if (j == L) break;  // bonus token
+    unsigned long long next = 0ull;
+    for (int k = 0; k < K; ++k) {
+      const bool ok = ((active >> k) & 1ull) && bi >= 0 &&
+                      draft_tokens[((long long)b * K + k) * L + j] == bi;
+      accept[((long long)b * K + k) * L + j] = ok ? 1 : 0;
+      if (ok) next |= 1ull << k;
+    }
+    active = next;
+    if (active == 0ull) break;
+  }
+  out_num[b] = n_out;
+}
+
+// Sec. 5.1 encoder bookkeeping: Y = best over the K streams of the encoder row, M = l_Y.
+__global__ void encoder_epilogue_kernel(const RowResult* __restrict__ rows, int B, int K,
+                                        const uint8_t* __restrict__ bins, long long bins_sb,
+                                        int32_t* __restrict__ enc_index,
+                                        uint8_t* __restrict__ message,
+                                        float* __restrict__ out_scores,
+                                        uint32_t* __restrict__ dev_status) {
+  const int b = blockIdx.x * blockDim.x + threadIdx.x;
+  if (b >= B) return;
+  double bs = 0.0;
+  int bi = -1;
+  for (int k = 0; k < K; ++k) {
+    const RowResult r = rows[(long long)b * K + k];
+    if (r.idx < 0) continue;
+    const double sc = r.score - r.lse;
+    if (bi < 0 || sc > bs || (sc == bs && r.idx < bi)) {
+      bs = sc;
+      bi = r.idx;
+    }
+  }
+  enc_index[b] = bi;
+  message[b] = (bins && bi >= 0) ? bins[bins_sb * b + bi] : (uint8_t)0;
+  if (out_scores) out_scores[(long long)b * (1 + K)] = bi >= 0 ? (float)bs : CUDART_NAN_F;
+  if (bi < 0 && dev_status) atomicOr(dev_status, GLS_DEV_EMPTY_SUPPORT);
+}
+
+// Sec. 5.1 decoder bookkeeping: X^(k) per decoder and the match flag Y in {X^(k)}.
+__global__ void decoder_epilogue_kernel(const RowResult* __restrict__ rows, int B, int K,
+                                        const int32_t* __restrict__ enc_index,
+                                        int32_t* __restrict__ dec_index,
+                                        uint8_t* __restrict__ match,
+                                        float* __restrict__ out_scores) {
+  const int b = blockIdx.x * blockDim.x + threadIdx.x;
+  if (b >= B) return;
+  const int y = enc_index[b];
+  int hit = 0;
+  for (int k = 0; k < K; ++k) {
+    const RowResult r = rows[(long long)b * K + k];
+    dec_index[(long long)b * K + k] = r.idx;
+    if (out_scores)
+      out_scores[(long long)b * (1 + K) + 1 + k] = r.idx >= 0 ? (float)r.score : CUDART_NAN_F;
+    if (r.idx >= 0 && r.idx == y) hit = 1;
+  }
+  match[b] = (uint8_t)hit;
+}
+
+// ------------------------------------------------------------------------------------------
+// host side
+// ------------------------------------------------------------------------------------------
+static bool finite_pos(float x) { return std::isfinite(x) && x > 0.f; }
+
+static int fill_noise(SweepArgs& A, const gls_noise_t* nz, uint32_t domain, int* spec_out) {
+  const int rounds = nz->rounds ? (int)nz->rounds : 10;
+  if (rounds < 7 || rounds > 16) return GLS_ERR_INVALID_ARG;
+  const int spec = nz->noise_spec ? (int)nz->noise_spec : 2;
+  if (spec != 1 && spec != 2) return GLS_ERR_INVALID_ARG;
+  if (nz->flags & ~GLS_NOISE_SHARED_ACROSS_K) return GLS_ERR_INVALID_ARG;
+  uint32_t k0 = (uint32_t)(nz->seed & 0xffffffffu), k1 = (uint32_t)(nz->seed >> 32);
+  for (int r = 0; r < 16; ++r) {
+    A.rk[2 * r] = k0;
+    A.rk[2 * r + 1] = k1;
+    k0 += kPhiloxW0;
+    k1 += kPhiloxW1;
+  }
+  A.rounds = rounds;
+  A.seq_base = nz->seq_base;
+  A.seq_ids = nz->seq_ids;
+  A.pos_base = nz->pos_base;
+  A.domain = domain;
+  A.kmask = (nz->flags & GLS_NOISE_SHARED_ACROSS_K) ? 0u : 0xffffu;
+  *spec_out = spec;
+  return GLS_OK;
+}
+
+static int check_rows(const gls_rows_t* r) {
+  if (!r || !r->data) return GLS_ERR_INVALID_ARG;
+  if (r->dtype != GLS_F32 && r->dtype != GLS_BF16) return GLS_ERR_UNSUPPORTED;
+  const uintptr_t es = r->dtype == GLS_F32 ? 4 : 2;
+  if (((uintptr_t)r->data) % es) return GLS_ERR_MISALIGNED;
+  return GLS_OK;
+}
+
+template <int DT, int SPEC, int ROUNDS>
+static cudaError_t launch_sweep_t(const SweepArgs& A, bool lse, int grid, cudaStream_t st) {
+  if (lse)
+    sweep_kernel<DT, SPEC, true, ROUNDS><<<grid, kSweepThreads, 0, st>>>(A);
+  else
+    sweep_kernel<DT, SPEC, false, ROUNDS><<<grid, kSweepThreads, 0, st>>>(A);
+  return cudaGetLastError();
+}
+
+template <int DT, int SPEC, int ROUNDS>
+static cudaError_t launch_finalize_t(const SweepArgs& A, int rows, bool lse, RowResult* rowres,
+                                     int32_t* out_tokens, float* out_scores, uint32_t* status,
+                                     cudaStream_t st) {
+  const int wpb = 4;
+  finalize_rows_kernel<DT, SPEC, ROUNDS><<<(rows + wpb - 1) / wpb, wpb * 32, 0, st>>>(
+      A, rows, lse ? 1 : 0, rowres, out_tokens, out_scores, status);
+  return cudaGetLastError();
+}
+
+// sweep + split reduction of one batch of rows
+static int run_rows(SweepArgs& A, int dtype, int spec, const Plan& P, void* workspace, bool lse,
+                    int32_t* out_tokens, float* out_scores, uint32_t* status, cudaStream_t st) {
+  char* ws = (char*)workspace;
+  A.chunk = P.chunk;
+  A.splits = P.splits;
+  A.n_items = P.n_items;
+  A.hints = (uint32_t*)(ws + P.off_hints);
+  A.partials = (Partial*)(ws + P.off_partials);
+  RowResult* rowres = (RowResult*)(ws + P.off_rows);
+  if (cudaMemsetAsync(A.hints, 0, (size_t)P.rows * sizeof(uint32_t), st) != cudaSuccess)
+    return GLS_ERR_CUDA;
+  const long long want = (P.n_items + kSweepThreads / 32 - 1) / (kSweepThreads / 32);
+  const int grid = (int)(want < (long long)kNumSMs * 4 ? want : (long long)kNumSMs * 4);
+  cudaError_t err;
+#define SWEEP_CALL(...) launch_sweep_t<__VA_ARGS__>(A, lse, grid, st)
+  if (dtype == GLS_BF16) {
+    if (spec == 1) err = A.rounds == 10 ? SWEEP_CALL(kBF16, 1, 10) : SWEEP_CALL(kBF16, 1, 0);
+    else err = A.rounds == 10 ? SWEEP_CALL(kBF16, 2, 10) : SWEEP_CALL(kBF16, 2, 0);
+  } else {
+    if (spec == 1) err = A.rounds == 10 ? SWEEP_CALL(kF32, 1, 10) : SWEEP_CALL(kF32, 1, 0);
+    else err = A.rounds == 10 ? SWEEP_CALL(kF32, 2, 10) : SWEEP_CALL(kF32, 2, 0);
+  }
+#undef SWEEP_CALL
+  if (err != cudaSuccess) return GLS_ERR_CUDA;
+#define FIN_CALL(...) \
+  launch_finalize_t<__VA_ARGS__>(A, (int)P.rows, lse, rowres, out_tokens, out_scores, status, st)
+  if (dtype == GLS_BF16) {
+    if (spec == 1) err = A.rounds == 10 ? FIN_CALL(kBF16, 1, 10) : FIN_CALL(kBF16, 1, 0);
+    else err = A.rounds == 10 ? FIN_CALL(kBF16, 2, 10) : FIN_CALL(kBF16, 2, 0);
+  } else {
+    if (spec == 1) err = A.rounds == 10 ? FIN_CALL(kF32, 1, 10) : FIN_CALL(kF32, 1, 0);
+    else err = A.rounds == 10 ? FIN_CALL(kF32, 2, 10) : FIN_CALL(kF32, 2, 0);
+  }
+#undef FIN_CALL
+  return err == cudaSuccess ? GLS_OK : GLS_ERR_CUDA;
+}
+
+static bool sizes_ok(int B, int K, int J, int64_t V) {
+  if (B <= 0 || K <= 0 || K > GLS_MAX_K || J <= 0 || V <= 0) return false;
+  if (V >= (1LL << 31) - 2 * kWarpTokens) return false;
+  if ((long long)B * K * J >= (1LL << 31) / 64) return false;
+  return true;
+}
+
+}  // namespace gls
+
+using namespace gls;
+
+extern "C" {
+
+int gls_version(void) { return 100; }
+
+const char* gls_status_string(int status) {
+  switch (status) {
+    case GLS_OK: return "GLS_OK";
+    case GLS_ERR_INVALID_ARG: return "GLS_ERR_INVALID_ARG: null pointer, size or parameter out of range";
+    case GLS_ERR_UNSUPPORTED: return "GLS_ERR_UNSUPPORTED: dtype or flag combination not implemented";
+    case GLS_ERR_MISALIGNED: return "GLS_ERR_MISALIGNED: base pointer not aligned to its element size";
+    case GLS_ERR_WORKSPACE: return "GLS_ERR_WORKSPACE: workspace missing or smaller than gls_workspace_bytes()";
+    case GLS_ERR_CUDA: return "GLS_ERR_CUDA: a CUDA runtime call failed";
+    default: return "GLS: unknown status";
+  }
+}
+
+size_t gls_workspace_bytes(int B, int K, int J, int64_t V) {
+  if (!sizes_ok(B, K, J, V)) return 0;
+  return make_plan((long long)B * K * J, V).total;
+}
+
+int gls_draft_sample(const gls_rows_t* draft_logits, int B, int K, int J, int64_t V, float inv_temp,
+                     const float* inv_temp_per_draft_host, const gls_noise_t* noise,
+                     int32_t* out_tokens, float* out_scores, void* workspace,
+                     size_t workspace_bytes, uint32_t* device_status, void* stream) {
+  if (!noise || !out_tokens || !sizes_ok(B, K, J, V)) return GLS_ERR_INVALID_ARG;
+  int rc = check_rows(draft_logits);
+  if (rc != GLS_OK) return rc;
+  SweepArgs A;
+  std::memset(&A, 0, sizeof(A));
+  for (int k = 0; k < K; ++k) {
+    const float it = inv_temp_per_draft_host ? inv_temp_per_draft_host[k] : inv_temp;
+    if (!finite_pos(it)) return GLS_ERR_INVALID_ARG;
+    A.inv_t[k] = it;
+  }
+  int spec;
+  rc = fill_noise(A, noise, 0u, &spec);
+  if (rc != GLS_OK) return rc;
+  const Plan P = make_plan((long long)B * K * J, V);
+  if (!workspace || workspace_bytes < P.total) return GLS_ERR_WORKSPACE;
+  A.data = draft_logits->data;
+  A.sb = draft_logits->stride_b;
+  A.sk = draft_logits->stride_k;
+  A.sj = draft_logits->stride_j;
+  A.K = K;
+  A.J = J;
+  A.V = (int)V;
+  return run_rows(A, draft_logits->dtype, spec, P, workspace, false, out_tokens, out_scores,
+                  device_status, (cudaStream_t)stream);
+}
+
+int gls_target_sample_verify(const gls_rows_t* target_logits, int B, int K, int L, int64_t V,
+                             float inv_temp, const int32_t* draft_tokens, const gls_noise_t* noise,
+                             uint32_t flags, int32_t* out_tokens, int32_t* out_num_tokens,
+                             uint8_t* out_accept, float* out_scores, void* workspace,
+                             size_t workspace_bytes, uint32_t* device_status, void* stream) {
+  if (flags & ~(GLS_COMBINE_ALL | GLS_NO_BONUS)) return GLS_ERR_INVALID_ARG;
+  const int J = L + ((flags & GLS_NO_BONUS) ? 0 : 1);
+  if (!noise || !out_tokens || !out_num_tokens || L < 0 || !sizes_ok(B, K, J, V))
+    return GLS_ERR_INVALID_ARG;
+  if (L > 0 && (!draft_tokens || !out_accept)) return GLS_ERR_INVALID_ARG;
+  if (!finite_pos(inv_temp)) return GLS_ERR_INVALID_ARG;
+  int rc = check_rows(target_logits);
+  if (rc != GLS_OK) return rc;
+  // Appendix B couples every stream to the accepted prefix's distribution.  When all k share one
+  // target row per position (stride_k = 0) the rows' own winners already are that race.
+  if ((flags & GLS_COMBINE_ALL) && target_logits->stride_k != 0 && K > 1)
+    return GLS_ERR_UNSUPPORTED;
+  SweepArgs A;
+  std::memset(&A, 0, sizeof(A));
+  for (int k = 0; k < K; ++k) A.inv_t[k] = inv_temp;
+  int spec;
+  rc = fill_noise(A, noise, 0u, &spec);
+  if (rc != GLS_OK) return rc;
+  const Plan P = make_plan((long long)B * K * J, V);
+  if (!workspace || workspace_bytes < P.total) return GLS_ERR_WORKSPACE;
+  A.data = target_logits->data;
+  A.sb = target_logits->stride_b;
+  A.sk = target_logits->stride_k;
+  A.sj = target_logits->stride_j;
+  A.K = K;
+  A.J = J;
+  A.V = (int)V;
+  cudaStream_t st = (cudaStream_t)stream;
+  rc = run_rows(A, target_logits->dtype, spec, P, workspace, true, nullptr, nullptr, nullptr, st);
+  if (rc != GLS_OK) return rc;
+  const RowResult* rowres = (const RowResult*)((char*)workspace + P.off_rows);
+  verify_epilogue_kernel<<<(B + 127) / 128, 128, 0, st>>>(rowres, B, K, L, J, flags, draft_tokens,
+                                                         out_tokens, out_num_tokens, out_accept,
+                                                         out_scores, device_status);
+  return cudaGetLastError() == cudaSuccess ? GLS_OK : GLS_ERR_CUDA;
+}
+
+int gls_compress_select(const gls_rows_t* enc_logw, const gls_rows_t* dec_logw, const uint8_t* bins,
+                        int64_t bins_stride_b, int B, int K, int64_t N, const gls_noise_t* noise,
+                        int32_t* out_enc_index, uint8_t* out_message, int32_t* out_dec_index,
+                        uint8_t* out_match, float* out_scores, void* workspace,
+                        size_t workspace_bytes, uint32_t* device_status, void* stream) {
+  if (!noise || !out_enc_index || !out_message || !sizes_ok(B, K, 1, N))
+    return GLS_ERR_INVALID_ARG;
+  if (bins_stride_b != 0 && bins_stride_b < N) return GLS_ERR_INVALID_ARG;
+  int rc = check_rows(enc_logw);
+  if (rc != GLS_OK) return rc;
+  if (dec_logw) {
+    rc = check_rows(dec_logw);
+    if (rc != GLS_OK) return rc;
+    if (!out_dec_index || !out_match) return GLS_ERR_INVALID_ARG;
+  }
+  SweepArgs A;
+  std::memset(&A, 0, sizeof(A));
+  for (int k = 0; k < K; ++k) A.inv_t[k] = 1.0f;
+  int spec;
+  rc = fill_noise(A, noise, 1u, &spec);
+  if (rc != GLS_OK) return rc;
+  const Plan P = make_plan((long long)B * K, N);
+  if (!workspace || workspace_bytes < P.total) return GLS_ERR_WORKSPACE;
+  cudaStream_t st = (cudaStream_t)stream;
+  const RowResult* rowres = (const RowResult*)((char*)workspace + P.off_rows);
+  // encoder: the one row of sample b raced under each of the K streams (stride_k = 0)
+  A.data = enc_logw->data;
+  A.sb = enc_logw->stride_b;
+  A.sk = 0;
+  A.sj = 0;
+  A.K = K;
+  A.J = 1;
+  A.V = (int)N;
+  rc = run_rows(A, enc_logw->dtype, spec, P, workspace, true, nullptr, nullptr, nullptr, st);
+  if (rc != GLS_OK) return rc;
+  encoder_epilogue_kernel<<<(B + 127) / 128, 128, 0, st>>>(rowres, B, K, bins, bins_stride_b,
+                                                          out_enc_index, out_message, out_scores,
+                                                          device_status);
+  if (cudaGetLastError() != cudaSuccess) return GLS_ERR_CUDA;
+  if (!dec_logw) return GLS_OK;
+  // decoders: row (b,k) under stream k, restricted to candidates labelled M
+  A.data = dec_logw->data;
+  A.sb = dec_logw->stride_b;
+  A.sk = dec_logw->stride_k;
+  A.bins = bins;
+  A.bins_sb = bins_stride_b;
+  A.msg = out_message;
+  rc = run_rows(A, dec_logw->dtype, spec, P, workspace, false, nullptr, nullptr, device_status, st);
+  if (rc != GLS_OK) return rc;
+  decoder_epilogue_kernel<<<(B + 127) / 128, 128, 0, st>>>(rowres, B, K, out_enc_index,
+                                                          out_dec_index, out_match, out_scores);
+  return cudaGetLastError() == cudaSuccess ? GLS_OK : GLS_ERR_CUDA;
+}
+
+}  // extern "C"

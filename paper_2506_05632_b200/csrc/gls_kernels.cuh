@@ -1,0 +1,536 @@
+// gls_kernels.cuh -- device code of libgls: fused noise + score + argmax sweep for sm_100a.
+//
+// One pass over each row of logits computes, per (row, vocabulary slice):
+//   - the two best candidates of the Gumbel-max race  argmax_i (logit_i / T - ln S_i)
+//     (Sec. 3 step 2 / Algorithm 1 of arXiv 2506.05632, log domain), with S_i generated in
+//     registers from the counter-based generator described in include/gls.h;
+//   - optionally the running (max, sum) of the row's softmax normaliser, needed where rows
+//     with different normalisers meet in the min over k (Algorithm 2, the Y_j line).
+//
+// The sweep never evaluates a logarithm for a token that cannot win.  With m a lower bound on
+// the row's final best score, token i can only matter if  S_i <= exp(logit_i/T - m), and
+// S_i = -log1p(-v_i) >= v_i >= (coarse bits of v_i).  So per group of 8 consecutive tokens one
+// test "min coarse bits < 2^(max logit * c - m')" decides, and only groups that pass look at
+// their tokens one by one (fp32 score from the full-precision uniform).  The filter has no false
+// negatives (margins below), so the result equals a full evaluation.
+#pragma once
+#include <cuda_runtime.h>
+#include <math_constants.h>
+#include <stdint.h>
+
+namespace gls {
+
+constexpr int kMaxK = 64;
+constexpr int kWarpTokens = 256;  // tokens one warp consumes per iteration (8 per lane)
+constexpr float kLog2e = 1.4426950408889634f;
+
+enum : int { kF32 = 0, kBF16 = 1 };
+
+// Published Philox4x32 constants (Salmon et al., SC'11).
+constexpr uint32_t kPhiloxM0 = 0xD2511F53u;
+constexpr uint32_t kPhiloxM1 = 0xCD9E8D57u;
+constexpr uint32_t kPhiloxW0 = 0x9E3779B9u;
+constexpr uint32_t kPhiloxW1 = 0xBB67AE85u;
+
+// Per (row, slice) result of the sweep: the two best fp32 scores with their tokens, and the
+// slice's softmax statistics (lm = max logit seen, ls = sum 2^((logit - lm) * c)).
+struct __align__(16) Partial {
+  float s1;
+  int i1;
+  float s2;
+  int i2;
+  float lm;
+  float ls;
+  int pad0, pad1;
+};
+
+// Per row: exact (fp64) score of the winner, its token, and the row's log-sum-exp.
+struct __align__(16) RowResult {
+  double score;
+  double lse;
+  int idx;
+  int pad0, pad1, pad2;
+};
+
+struct SweepArgs {
+  const void* data;       // rows [B][K][J][V]
+  long long sb, sk, sj;   // element strides
+  int K, J, V;
+  int chunk;              // tokens per slice, a multiple of kWarpTokens
+  int splits;             // slices per row
+  long long n_items;      // rows * splits
+  float inv_t[kMaxK];     // 1/T per k
+  uint32_t rk[32];        // Philox round keys: rk[2r], rk[2r+1]
+  int rounds;
+  uint32_t seq_base;
+  const uint32_t* seq_ids;
+  uint32_t pos_base;
+  uint32_t domain;        // 0 decoding, 1 compression
+  uint32_t kmask;         // 0xffff, or 0 when every k shares the noise of k = 0
+  const uint8_t* bins;    // NULL, or candidate labels
+  long long bins_sb;
+  const uint8_t* msg;     // [B] label a candidate must carry (decoder side)
+  uint32_t* hints;        // [rows] ordered-int encoding of a lower bound on the row's best score
+  Partial* partials;      // [n_items]
+};
+
+// ------------------------------------------------------------------------------------------
+// small helpers
+// ------------------------------------------------------------------------------------------
+__device__ __forceinline__ float ex2_approx(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+__device__ __forceinline__ uint32_t min_u16x2(uint32_t a, uint32_t b) {
+  uint32_t d;
+  asm("min.u16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
+  return d;
+}
+__device__ __forceinline__ uint32_t max_bf16x2(uint32_t a, uint32_t b) {
+  uint32_t d;
+  asm("max.bf16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));  // a NaN operand is ignored
+  return d;
+}
+__device__ __forceinline__ float bf16_lo(uint32_t w) { return __uint_as_float(w << 16); }
+__device__ __forceinline__ float bf16_hi(uint32_t w) { return __uint_as_float(w & 0xffff0000u); }
+
+__device__ __forceinline__ uint4 ld_stream16(const void* p) {
+  uint4 v;
+  asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+               : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+               : "l"(p));
+  return v;
+}
+
+// order-preserving map float -> uint32 (for atomicMax); 0 decodes to -inf
+__device__ __forceinline__ uint32_t enc_ordered(float f) {
+  uint32_t b = __float_as_uint(f);
+  return (b & 0x80000000u) ? ~b : (b | 0x80000000u);
+}
+__device__ __forceinline__ float dec_ordered(uint32_t e) {
+  if (e <= 0x007fffffu) return -CUDART_INF_F;  // at or below the code of -inf (0 = never written)
+  uint32_t b = (e & 0x80000000u) ? (e & 0x7fffffffu) : ~e;
+  return __uint_as_float(b);
+}
+
+// ------------------------------------------------------------------------------------------
+// Philox4x32: (c0,c1,c2,c3) <- (hi(M1 c2)^c1^k0, lo(M1 c2), hi(M0 c0)^c3^k1, lo(M0 c0)) per round,
+// round keys precomputed on the host.
+// ------------------------------------------------------------------------------------------
+template <int ROUNDS>
+__device__ __forceinline__ void philox4x32(const uint32_t* __restrict__ rk, int rounds_rt,
+                                           uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3,
+                                           uint32_t (&out)[4]) {
+  const int n = ROUNDS > 0 ? ROUNDS : rounds_rt;
+#pragma unroll
+  for (int r = 0; r < n; ++r) {
+    const unsigned long long p0 = (unsigned long long)kPhiloxM0 * c0;
+    const unsigned long long p1 = (unsigned long long)kPhiloxM1 * c2;
+    const uint32_t n0 = (uint32_t)(p1 >> 32) ^ c1 ^ rk[2 * r];
+    const uint32_t n2 = (uint32_t)(p0 >> 32) ^ c3 ^ rk[2 * r + 1];
+    c1 = (uint32_t)p1;
+    c3 = (uint32_t)p0;
+    c0 = n0;
+    c2 = n2;
+  }
+  out[0] = c0;
+  out[1] = c1;
+  out[2] = c2;
+  out[3] = c3;
+}
+
+// Identity of one noise stream: everything of the counter except the token block.
+struct StreamKey {
+  uint32_t c1;  // k | domain << 16
+  uint32_t pos;
+  uint32_t seq;
+};
+
+// The uniform of token i under noise_spec SPEC, as the 48-bit (or 32-bit) integer numerator and
+// the scale 2^-bits: v = (num + 0.5) * 2^-bits.
+template <int SPEC, int ROUNDS>
+__device__ __forceinline__ double uniform_exact(const SweepArgs& A, const StreamKey& sk, int i) {
+  uint32_t o[4];
+  if (SPEC == 1) {
+    philox4x32<ROUNDS>(A.rk, A.rounds, (uint32_t)i >> 2, sk.c1, sk.pos, sk.seq, o);
+    return ((double)o[i & 3] + 0.5) * 0x1p-32;
+  } else {
+    philox4x32<ROUNDS>(A.rk, A.rounds, (uint32_t)i >> 3, sk.c1, sk.pos, sk.seq, o);
+    const uint32_t h = (o[(i & 7) >> 1] >> (16 * (i & 1))) & 0xffffu;
+    philox4x32<ROUNDS>(A.rk, A.rounds, (uint32_t)i >> 2, sk.c1 + (2u << 16), sk.pos, sk.seq, o);
+    return ((double)h * 4294967296.0 + (double)o[i & 3] + 0.5) * 0x1p-48;
+  }
+}
+
+template <int DT>
+__device__ __forceinline__ float load_logit(const void* row, long long i) {
+  if (DT == kF32) return __ldg((const float*)row + i);
+  return __uint_as_float((uint32_t)__ldg((const unsigned short*)row + i) << 16);
+}
+
+// Exact score of one token in fp64: logit/T - ln S, S = -log1p(-v)  (Sec. 3: S = -ln U, U = 1 - v).
+template <int DT, int SPEC, int ROUNDS>
+__device__ __noinline__ double exact_score(const SweepArgs& A, const void* row,
+                                           const StreamKey& sk, int i, float inv_t) {
+  const double a = (double)load_logit<DT>(row, i) * (double)inv_t;
+  const double v = uniform_exact<SPEC, ROUNDS>(A, sk, i);
+  return a - log(-log1p(-v));
+}
+
+// fp32 score from the full uniform; |error| is well below score_slack().
+__device__ __forceinline__ float score_f32(float a, float inv_t, float v, float* ln_s) {
+  const float s = -log1pf(-v);
+  const float l = logf(s);
+  *ln_s = l;
+  return fmaf(a, inv_t, -l);
+}
+// Bound on |fp32 score - exact score| used to (a) keep the filter's running bound below the
+// truth and (b) decide when two candidates must be re-evaluated in fp64.
+__device__ __forceinline__ float score_slack(float s, float ln_s) {
+  return 0x1p-17f * (1.0f + fabsf(s) + fabsf(ln_s));
+}
+
+// Exponent offset of the filter for a running lower bound m on the best score (natural-log
+// units): a token passes iff coarse(v) < 2^(logit * c + nm).  The margin covers the rounding of
+// c, of the fma and of ex2.approx (together < 1e-5 for |logit * c| < 2^10), so no token whose
+// exact score reaches m is ever rejected.
+__device__ __forceinline__ float filter_offset(float m) {
+  if (m == -CUDART_INF_F) return CUDART_INF_F;
+  const float ml = m * kLog2e;
+  return fmaf(fabsf(ml), 0x1p-20f, 0x1p-12f) - ml;
+}
+
+struct Top2 {
+  float s1;
+  int i1;
+  float s2;
+  int i2;
+};
+__device__ __forceinline__ void top2_init(Top2& t) {
+  t.s1 = -CUDART_INF_F;
+  t.i1 = -1;
+  t.s2 = -CUDART_INF_F;
+  t.i2 = -1;
+}
+// order: score descending, then token ascending
+__device__ __forceinline__ bool beats(float s, int i, float s0, int i0) {
+  return i0 < 0 || s > s0 || (s == s0 && i < i0);
+}
+__device__ __forceinline__ void top2_offer(Top2& t, float s, int i) {
+  if (i < 0) return;
+  if (beats(s, i, t.s1, t.i1)) {
+    t.s2 = t.s1;
+    t.i2 = t.i1;
+    t.s1 = s;
+    t.i1 = i;
+  } else if (beats(s, i, t.s2, t.i2)) {
+    t.s2 = s;
+    t.i2 = i;
+  }
+}
+__device__ __forceinline__ void top2_warp_merge(Top2& t) {
+#pragma unroll
+  for (int d = 16; d > 0; d >>= 1) {
+    const float os1 = __shfl_xor_sync(0xffffffffu, t.s1, d);
+    const int oi1 = __shfl_xor_sync(0xffffffffu, t.i1, d);
+    const float os2 = __shfl_xor_sync(0xffffffffu, t.s2, d);
+    const int oi2 = __shfl_xor_sync(0xffffffffu, t.i2, d);
+    top2_offer(t, os1, oi1);
+    top2_offer(t, os2, oi2);
+  }
+}
+
+// ------------------------------------------------------------------------------------------
+// Per-token examination of one lane's group of 8 tokens (rare path).
+//   a[8]   logits (excluded / out-of-range tokens hold -inf)
+//   w[]    coarse generator output of the group: SPEC 2: 4 words = 8 halfwords, SPEC 1: 8 words
+// ------------------------------------------------------------------------------------------
+template <int SPEC, int ROUNDS>
+__device__ __noinline__ void examine_group(const SweepArgs& A, const StreamKey sk, int tok0,
+                                           const float (&a)[8], const uint32_t* w, float inv_t,
+                                           float c2, float m, const uint8_t* bins, int msg,
+                                           Top2& best) {
+  float nm = filter_offset(m);
+  uint32_t fine[4];
+  int fine_block = -1;
+#pragma unroll 1
+  for (int t = 0; t < 8; ++t) {
+    const float at = a[t];
+    if (!(at < CUDART_INF_F)) continue;  // NaN and +inf never win
+    const float thr = ex2_approx(fmaf(at, c2, nm));
+    float v;
+    if (SPEC == 1) {
+      const uint32_t wt = w[t];
+      if (!(__uint2float_rd(wt) < thr * 4294967296.0f)) continue;
+      v = ((float)wt + 0.5f) * 0x1p-32f;
+    } else {
+      const uint32_t h = (w[t >> 1] >> (16 * (t & 1))) & 0xffffu;
+      if (!((float)h < thr * 65536.0f)) continue;
+      const int blk = (tok0 + t) >> 2;
+      if (blk != fine_block) {
+        philox4x32<ROUNDS>(A.rk, A.rounds, (uint32_t)blk, sk.c1 + (2u << 16), sk.pos, sk.seq, fine);
+        fine_block = blk;
+      }
+      const uint32_t r = fine[(tok0 + t) & 3];
+      v = fmaf((float)h, 0x1p-16f, fmaf((float)r, 0x1p-48f, 0x1p-49f));
+    }
+    const int i = tok0 + t;
+    if (bins != nullptr && (int)__ldg(bins + i) != msg) continue;
+    float ln_s;
+    const float s = score_f32(at, inv_t, v, &ln_s);
+    top2_offer(best, s, i);
+    const float lower = s - score_slack(s, ln_s);
+    if (lower > m) {
+      m = lower;
+      nm = filter_offset(m);
+    }
+  }
+}
+
+// running lower bound implied by a lane's best candidate
+__device__ __forceinline__ float lane_bound(const Top2& t) {
+  if (t.i1 < 0) return -CUDART_INF_F;
+  // ln S is not kept; |ln S| <= 34 for v >= 2^-49, use that worst case
+  return t.s1 - 0x1p-17f * (35.0f + fabsf(t.s1));
+}
+
+// ------------------------------------------------------------------------------------------
+// The sweep.  Each warp owns work items (row, slice); per iteration a lane takes 8 consecutive
+// tokens (one 16-byte load of bf16, two of fp32), so a warp reads 512 B / 1 KB contiguous.
+// ------------------------------------------------------------------------------------------
+constexpr int kSweepThreads = 256;
+
+template <int DT>
+struct Group {
+  uint4 q0, q1;  // q1 only used by fp32
+};
+
+template <int DT>
+__device__ __forceinline__ Group<DT> load_group_vec(const char* rowp, int tok) {
+  Group<DT> g;
+  if (DT == kBF16) {
+    g.q0 = ld_stream16(rowp + (size_t)tok * 2);
+    g.q1 = make_uint4(0, 0, 0, 0);
+  } else {
+    g.q0 = ld_stream16(rowp + (size_t)tok * 4);
+    g.q1 = ld_stream16(rowp + (size_t)tok * 4 + 16);
+  }
+  return g;
+}
+
+// scalar loader for ragged tails and rows that are not 16-byte aligned; out-of-range -> -inf
+template <int DT>
+__device__ __forceinline__ Group<DT> load_group_scalar(const char* rowp, int tok, int V) {
+  Group<DT> g;
+  uint32_t e[8];
+#pragma unroll
+  for (int t = 0; t < 8; ++t) {
+    const int i = tok + t;
+    if (DT == kBF16)
+      e[t] = i < V ? (uint32_t)__ldg((const unsigned short*)rowp + i) : 0xff80u;
+    else
+      e[t] = i < V ? __float_as_uint(__ldg((const float*)rowp + i)) : 0xff800000u;
+  }
+  if (DT == kBF16) {
+    g.q0 = make_uint4(e[0] | (e[1] << 16), e[2] | (e[3] << 16), e[4] | (e[5] << 16),
+                      e[6] | (e[7] << 16));
+    g.q1 = make_uint4(0, 0, 0, 0);
+  } else {
+    g.q0 = make_uint4(e[0], e[1], e[2], e[3]);
+    g.q1 = make_uint4(e[4], e[5], e[6], e[7]);
+  }
+  return g;
+}
+
+template <int DT>
+__device__ __forceinline__ void unpack_group(const Group<DT>& g, float (&a)[8]) {
+  if (DT == kBF16) {
+    a[0] = bf16_lo(g.q0.x); a[1] = bf16_hi(g.q0.x);
+    a[2] = bf16_lo(g.q0.y); a[3] = bf16_hi(g.q0.y);
+    a[4] = bf16_lo(g.q0.z); a[5] = bf16_hi(g.q0.z);
+    a[6] = bf16_lo(g.q0.w); a[7] = bf16_hi(g.q0.w);
+  } else {
+    a[0] = __uint_as_float(g.q0.x); a[1] = __uint_as_float(g.q0.y);
+    a[2] = __uint_as_float(g.q0.z); a[3] = __uint_as_float(g.q0.w);
+    a[4] = __uint_as_float(g.q1.x); a[5] = __uint_as_float(g.q1.y);
+    a[6] = __uint_as_float(g.q1.z); a[7] = __uint_as_float(g.q1.w);
+  }
+}
+
+// max over the group, ignoring NaN
+template <int DT>
+__device__ __forceinline__ float group_max(const Group<DT>& g) {
+  if (DT == kBF16) {
+    const uint32_t x = max_bf16x2(max_bf16x2(g.q0.x, g.q0.y), max_bf16x2(g.q0.z, g.q0.w));
+    return fmaxf(bf16_lo(x), bf16_hi(x));
+  } else {
+    const float x0 = fmaxf(fmaxf(__uint_as_float(g.q0.x), __uint_as_float(g.q0.y)),
+                           fmaxf(__uint_as_float(g.q0.z), __uint_as_float(g.q0.w)));
+    const float x1 = fmaxf(fmaxf(__uint_as_float(g.q1.x), __uint_as_float(g.q1.y)),
+                           fmaxf(__uint_as_float(g.q1.z), __uint_as_float(g.q1.w)));
+    return fmaxf(x0, x1);
+  }
+}
+
+// Softmax statistics of one group: lm = running max, ls = sum 2^((a - lm) * c2).
+// Fast path assumes finite-or-(-inf) logits; anything else is redone token by token.
+__device__ __forceinline__ void lse_group(const float (&a)[8], float amax, float c2, float& lm,
+                                          float& ls) {
+  bool careful = false;
+  if (amax > lm) {
+    if (amax == CUDART_INF_F) {
+      careful = true;
+    } else {
+      ls *= ex2_approx((lm - amax) * c2);
+      lm = amax;
+    }
+  }
+  float gs = 0.f;
+  if (!careful) {
+#pragma unroll
+    for (int t = 0; t < 8; ++t) gs += ex2_approx((a[t] - lm) * c2);
+    careful = !(gs <= 16.0f);  // a NaN logit poisons the sum
+  }
+  if (careful) {
+    float vmax = -CUDART_INF_F;
+#pragma unroll
+    for (int t = 0; t < 8; ++t)
+      if (a[t] < CUDART_INF_F) vmax = fmaxf(vmax, a[t]);  // false for NaN and +inf
+    if (vmax > lm) {
+      ls *= ex2_approx((lm - vmax) * c2);
+      lm = vmax;
+    }
+    gs = 0.f;
+#pragma unroll
+    for (int t = 0; t < 8; ++t)
+      if (a[t] < CUDART_INF_F) gs += ex2_approx((a[t] - lm) * c2);
+  }
+  ls += gs;
+}
+
+constexpr float kLseFloor = -3.0e38f;  // finite stand-in for "no finite logit seen yet"
+
+template <int DT, int SPEC, bool LSE, int ROUNDS>
+__global__ void __launch_bounds__(kSweepThreads, 4)
+sweep_kernel(const __grid_constant__ SweepArgs A) {
+  const int lane = threadIdx.x & 31;
+  const long long warp0 = (long long)blockIdx.x * (kSweepThreads / 32) + (threadIdx.x >> 5);
+  const long long nwarps = (long long)gridDim.x * (kSweepThreads / 32);
+  constexpr int ES = DT == kBF16 ? 2 : 4;
+
+  for (long long item = warp0; item < A.n_items; item += nwarps) {
+    const int row = (int)(item / A.splits);
+    const int split = (int)(item - (long long)row * A.splits);
+    const int j = row % A.J;
+    const int bk = row / A.J;
+    const int k = bk % A.K;
+    const int b = bk / A.K;
+    const char* rowp = (const char*)A.data + (b * A.sb + k * A.sk + j * A.sj) * ES;
+    StreamKey sk;
+    sk.c1 = ((uint32_t)k & A.kmask) | (A.domain << 16);
+    sk.pos = A.pos_base + (uint32_t)j;
+    sk.seq = A.seq_ids ? __ldg(A.seq_ids + b) : A.seq_base + (uint32_t)b;
+    const float inv_t = A.inv_t[k];
+    const float c2 = inv_t * kLog2e;
+    const uint8_t* bins = A.bins ? A.bins + A.bins_sb * b : nullptr;
+    const int msg = (A.bins && A.msg) ? (int)__ldg(A.msg + b) : 0;
+    const int tok_begin = split * A.chunk;
+    const int tok_end = min(A.V, tok_begin + A.chunk);
+    const bool aligned = (((uintptr_t)rowp) & 15) == 0;
+    // iterations whose 256 tokens are all in range can use vector loads
+    const int n_full = aligned ? (tok_end - tok_begin) / kWarpTokens : 0;
+    const int n_iter = (tok_end - tok_begin + kWarpTokens - 1) / kWarpTokens;
+
+    float m = dec_ordered(__ldcg(A.hints + row));  // best lower bound published so far
+    float nm = filter_offset(m);
+    Top2 best;
+    top2_init(best);
+    float lm = kLseFloor, ls = 0.f;
+
+    Group<DT> cur, nxt;
+    int tok = tok_begin + lane * 8;
+    if (n_full > 0) cur = load_group_vec<DT>(rowp, tok);
+    for (int it = 0; it < n_iter; ++it, tok += kWarpTokens) {
+      const bool full = it < n_full;
+      if (!full) cur = load_group_scalar<DT>(rowp, tok, tok_end);
+      if (it + 1 < n_full) nxt = load_group_vec<DT>(rowp, tok + kWarpTokens);
+
+      // coarse noise of the group and its smallest value
+      uint32_t w[SPEC == 1 ? 8 : 4];
+      float vlow;  // lower bound on min_t v_t, scaled by 2^16 (SPEC 2) or 2^32 (SPEC 1)
+      if (SPEC == 1) {
+        uint32_t o[4];
+        philox4x32<ROUNDS>(A.rk, A.rounds, (uint32_t)tok >> 2, sk.c1, sk.pos, sk.seq, o);
+        w[0] = o[0]; w[1] = o[1]; w[2] = o[2]; w[3] = o[3];
+        philox4x32<ROUNDS>(A.rk, A.rounds, ((uint32_t)tok >> 2) + 1u, sk.c1, sk.pos, sk.seq, o);
+        w[4] = o[0]; w[5] = o[1]; w[6] = o[2]; w[7] = o[3];
+        const uint32_t wm = min(min(min(w[0], w[1]), min(w[2], w[3])),
+                                min(min(w[4], w[5]), min(w[6], w[7])));
+        vlow = __uint2float_rd(wm);
+      } else {
+        uint32_t o[4];
+        philox4x32<ROUNDS>(A.rk, A.rounds, (uint32_t)tok >> 3, sk.c1, sk.pos, sk.seq, o);
+        w[0] = o[0]; w[1] = o[1]; w[2] = o[2]; w[3] = o[3];
+        const uint32_t mm = min_u16x2(min_u16x2(w[0], w[1]), min_u16x2(w[2], w[3]));
+        vlow = (float)min(mm & 0xffffu, mm >> 16);
+      }
+      const float amax = group_max<DT>(cur);
+      const float thr = ex2_approx(fmaf(amax, c2, nm)) * (SPEC == 1 ? 4294967296.0f : 65536.0f);
+      const bool pass = vlow < thr;
+
+      if (LSE) {
+        float a[8];
+        unpack_group<DT>(cur, a);
+        lse_group(a, amax, c2, lm, ls);
+      }
+
+      if (__any_sync(0xffffffffu, pass)) {
+        if (pass) {
+          float a[8];
+          unpack_group<DT>(cur, a);
+          examine_group<SPEC, ROUNDS>(A, sk, tok, a, w, inv_t, c2, m, bins, msg, best);
+        }
+        // share the improved bound with the warp and with the other slices of the row
+        float mb = lane_bound(best);
+#pragma unroll
+        for (int d = 16; d > 0; d >>= 1) mb = fmaxf(mb, __shfl_xor_sync(0xffffffffu, mb, d));
+        if (mb > m) {
+          m = mb;
+          if (lane == 0) atomicMax(A.hints + row, enc_ordered(m));
+        }
+        const float mg = dec_ordered(__ldcg(A.hints + row));
+        if (mg > m) m = mg;
+        nm = filter_offset(m);
+      } else if ((it & 15) == 15) {
+        const float mg = dec_ordered(__ldcg(A.hints + row));
+        if (mg > m) {
+          m = mg;
+          nm = filter_offset(m);
+        }
+      }
+      cur = nxt;
+    }
+
+    // combine the lanes
+    top2_warp_merge(best);
+    if (LSE) {
+      float wm = lm;
+#pragma unroll
+      for (int d = 16; d > 0; d >>= 1) wm = fmaxf(wm, __shfl_xor_sync(0xffffffffu, wm, d));
+      float s = ls * ex2_approx((lm - wm) * c2);
+#pragma unroll
+      for (int d = 16; d > 0; d >>= 1) s += __shfl_xor_sync(0xffffffffu, s, d);
+      lm = wm;
+      ls = s;
+    }
+    if (lane == 0) {
+      Partial p;
+      p.s1 = best.s1; p.i1 = best.i1; p.s2 = best.s2; p.i2 = best.i2;
+      p.lm = lm; p.ls = ls; p.pad0 = 0; p.pad1 = 0;
+      A.partials[item] = p;
+    }
+  }
+}
+
+}  // namespace gls

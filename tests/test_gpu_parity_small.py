@@ -1,0 +1,246 @@
+"""CUDA path vs CPU oracle, element by element, on small and adversarial shapes (through the C ABI)."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2506_05632_b200 import synth
+from tests import parity
+
+pytestmark = pytest.mark.gpu
+SEED = synth.NOISE_SEED + 77
+
+
+def _rand_logits(B, K, J, V, dtype, seed, scale=3.0):
+    g = torch.Generator(device="cuda").manual_seed(seed)
+    x = scale * torch.randn(B, K, J, V, generator=g, device="cuda", dtype=torch.float32)
+    return x.to(dtype)
+
+
+def _draft_both(gls, oracle, logits, **kw):
+    tok, sc = gls.draft_sample(logits, **kw)
+    torch.cuda.synchronize()
+    ref = oracle.draft_sample(synth.to_numpy_rows(logits), **kw)
+    return tok.cpu().numpy(), sc.cpu().numpy(), ref
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("spec", [1, 2])
+def test_draft_shapes(gls, oracle, dtype, spec):
+    """Ragged vocabularies around every tile boundary: one lane group (8), one warp iteration
+    (256), one slice (2048) and several slices."""
+    for n, (V, K, J, B) in enumerate([(1, 1, 1, 3), (3, 2, 1, 4), (7, 3, 2, 5), (8, 1, 1, 6),
+                                      (9, 2, 2, 3), (31, 1, 1, 7), (33, 3, 1, 4), (255, 2, 1, 5),
+                                      (256, 1, 2, 5), (257, 2, 1, 5), (2047, 1, 1, 9),
+                                      (2049, 2, 1, 6), (5000, 2, 2, 6), (40001, 1, 1, 5)]):
+        logits = _rand_logits(B, K, J, V, dtype, 100 + n)
+        tok, sc, ref = _draft_both(gls, oracle, logits, seed=SEED, spec=spec, inv_temp=0.8,
+                                   seq_base=5, pos_base=2)
+        parity.check_draft(tok, sc, ref, "V=%d" % V)
+
+
+def test_draft_rounds_and_flags(gls, oracle):
+    logits = _rand_logits(6, 3, 2, 3001, torch.float32, 7)
+    for rounds in (7, 10, 12):
+        tok, sc, ref = _draft_both(gls, oracle, logits, seed=SEED, rounds=rounds)
+        parity.check_draft(tok, sc, ref, "rounds=%d" % rounds)
+    tok, sc, ref = _draft_both(gls, oracle, logits, seed=SEED, noise_flags=1)
+    parity.check_draft(tok, sc, ref, "shared noise")
+    tok, sc, ref = _draft_both(gls, oracle, logits, seed=SEED, inv_temp_per_draft=[0.5, 1.0, 2.5])
+    parity.check_draft(tok, sc, ref, "per-draft temperature")
+    ids = torch.tensor([9, 3, 2**31 - 1, 0, 77, 1234567], dtype=torch.int32, device="cuda")
+    tok, sc = gls.draft_sample(logits, seed=SEED, seq_ids=ids)
+    ref = oracle.draft_sample(logits.cpu().numpy(), seed=SEED, seq_ids=ids.cpu().numpy())
+    parity.check_draft(tok.cpu().numpy(), sc.cpu().numpy(), ref, "seq_ids")
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+def test_draft_strides_and_misalignment(gls, oracle, dtype):
+    B, K, J, V = 4, 3, 2, 1000
+    base = _rand_logits(B, K, J, V + 9, dtype, 11)
+    # rows that start 1, 3 elements past a 16-byte boundary (scalar-load path)
+    for off in (1, 3, 8):
+        view = base[..., off:off + V]
+        tok, sc = gls.draft_sample(view, seed=SEED)
+        ref = oracle.draft_sample(synth.to_numpy_rows(view.contiguous()), seed=SEED)
+        parity.check_draft(tok.cpu().numpy(), sc.cpu().numpy(), ref, "offset %d" % off)
+    # broadcast over k and over b (stride 0), permuted memory order
+    one = _rand_logits(B, 1, J, V, dtype, 12)
+    view = one.expand(B, K, J, V)
+    tok, sc = gls.draft_sample(view, seed=SEED)
+    ref = oracle.draft_sample(synth.to_numpy_rows(view.contiguous()), seed=SEED)
+    parity.check_draft(tok.cpu().numpy(), sc.cpu().numpy(), ref, "stride_k=0")
+    perm = _rand_logits(J, B, K, V, dtype, 13).permute(1, 2, 0, 3)
+    tok, sc = gls.draft_sample(perm, seed=SEED)
+    ref = oracle.draft_sample(synth.to_numpy_rows(perm.contiguous()), seed=SEED)
+    parity.check_draft(tok.cpu().numpy(), sc.cpu().numpy(), ref, "permuted")
+
+
+def test_masked_nan_inf_and_empty_rows(gls, oracle):
+    B, K, J, V = 6, 2, 2, 777
+    logits = _rand_logits(B, K, J, V, torch.float32, 21)
+    g = torch.Generator(device="cuda").manual_seed(22)
+    mask = torch.rand(B, K, J, V, generator=g, device="cuda") < 0.9
+    logits[mask] = float("-inf")           # top-K style truncation (Sec. 4.4)
+    logits[0, 0, 0, 5] = float("nan")
+    logits[0, 0, 0, 6] = float("inf")
+    logits[1, 1, 1, :] = float("-inf")     # a row without support
+    logits[2, 0, 1, :] = float("-inf")
+    logits[2, 0, 1, 700] = -3.0            # a one-hot row
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    tok, sc = gls.draft_sample(logits, seed=SEED, status=status)
+    ref = oracle.draft_sample(logits.cpu().numpy(), seed=SEED)
+    t = tok.cpu().numpy()
+    parity.check_draft(t, sc.cpu().numpy(), ref, "masked")
+    assert t[1, 1, 1] == -1 and t[2, 0, 1] == 700
+    assert int(status.item()) & gls.DEV_EMPTY_SUPPORT
+    # target side with the same rows: -1 token, tau stops there, status bit set
+    status.zero_()
+    dt = torch.from_numpy(ref["tokens"][:, :, :1].copy()).cuda()
+    out = gls.target_sample_verify(logits, dt, seed=SEED, status=status)
+    refv = oracle.target_sample_verify(logits.cpu().numpy(), ref["tokens"][:, :, :1], seed=SEED)
+    parity.check_verify(parity.to_np(out), refv, "masked verify")
+    allneg = torch.full((2, 2, 2, 100), float("-inf"), device="cuda")
+    out = gls.target_sample_verify(allneg, torch.zeros(2, 2, 1, dtype=torch.int32, device="cuda"),
+                                   seed=SEED, status=status)
+    o = parity.to_np(out)
+    assert (o["tokens"][:, 0] == -1).all() and (o["tau"] == 1).all() and not o["accept"].any()
+    assert int(status.item()) & gls.DEV_EMPTY_SUPPORT
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("spec", [1, 2])
+def test_verify_small(gls, oracle, dtype, spec):
+    """Algorithm 2 end to end on reduced copies of the verify workloads, several shapes."""
+    for cfg, B, K, L, V in ((2, 16, 4, 4, 3000), (3, 8, 8, 5, 5001), (4, 6, 8, 8, 2500),
+                            (2, 5, 1, 3, 999), (3, 7, 2, 0, 1234)):
+        w = synth.verify_workload(cfg, "cuda", B=B, K=K, L=L, V=V)
+        d, t = w.draft_logits.to(dtype), w.target_logits.to(dtype)
+        kw = dict(seed=w.noise_seed, spec=spec, inv_temp=w.inv_temp)
+        if L > 0:
+            tok, sc = gls.draft_sample(d, **kw)
+            refd = oracle.draft_sample(synth.to_numpy_rows(d), **kw)
+            parity.check_draft(tok.cpu().numpy(), sc.cpu().numpy(), refd, "cfg%d draft" % cfg)
+            dtok = torch.from_numpy(refd["tokens"]).cuda()
+        else:
+            dtok = torch.zeros(B, K, 0, dtype=torch.int32, device="cuda")
+        out = gls.target_sample_verify(t, dtok, **kw)
+        refv = oracle.target_sample_verify(synth.to_numpy_rows(t), dtok.cpu().numpy(), **kw)
+        parity.check_verify(parity.to_np(out), refv, "cfg%d verify" % cfg)
+        if L > 0:
+            assert (refv["tau"] > 1).any()  # the workloads do accept something
+        # NO_BONUS drops the last row
+        if L > 0:
+            out = gls.target_sample_verify(t[:, :, :L], dtok, flags=gls.NO_BONUS, **kw)
+            refn = oracle.target_sample_verify(synth.to_numpy_rows(t[:, :, :L].contiguous()),
+                                               dtok.cpu().numpy(), flags=2, **kw)
+            parity.check_verify(parity.to_np(out), refn, "cfg%d no-bonus" % cfg)
+
+
+def test_verify_shared_target_row_and_combine_all(gls, oracle):
+    """Algorithm 1's single q (stride_k = 0) and the Appendix B variant on it."""
+    B, K, L, V = 40, 4, 3, 600
+    t1 = _rand_logits(B, 1, L + 1, V, torch.float32, 31, scale=1.5)
+    t = t1.expand(B, K, L + 1, V)
+    d = (t1[:, :, :L] + 0.5 * _rand_logits(B, 1, L, V, torch.float32, 32, 1.0)).expand(B, K, L, V)
+    tok, _ = gls.draft_sample(d, seed=SEED)
+    for flags in (0, gls.COMBINE_ALL):
+        out = gls.target_sample_verify(t, tok, flags=flags, seed=SEED)
+        ref = oracle.target_sample_verify(t.contiguous().cpu().numpy(), tok.cpu().numpy(),
+                                          flags=flags, seed=SEED)
+        parity.check_verify(parity.to_np(out), ref, "flags=%d" % flags)
+    with pytest.raises(gls.GlsError):  # per-draft rows with COMBINE_ALL are not implemented
+        gls.target_sample_verify(t.contiguous(), tok, flags=gls.COMBINE_ALL, seed=SEED)
+
+
+def test_identical_rows_accept_everything(gls):
+    """p = q: acceptance in every realisation (remark after Theorem 1); bit-identical draft and
+    target rows must therefore give tau = L + 1 for every sequence on the GPU too."""
+    w = synth.verify_workload(3, "cuda", B=32, K=4, L=4, V=20011)
+    d = w.draft_logits
+    t = torch.cat([d, d[:, :, :1]], dim=2)
+    tok, _ = gls.draft_sample(d, seed=SEED, inv_temp=w.inv_temp)
+    out = gls.target_sample_verify(t, tok, seed=SEED, inv_temp=w.inv_temp)
+    assert (out["tau"] == 5).all()
+    assert out["accept"].any(dim=1).all()
+    # one-hot drafts: X is the hot token whatever the noise
+    hot = torch.full((8, 3, 2, 5000), float("-inf"), device="cuda")
+    hot[..., 4321] = 1.0
+    tok, _ = gls.draft_sample(hot, seed=SEED)
+    assert (tok == 4321).all()
+
+
+def test_config1_statistics_on_gpu(gls, oracle):
+    """Configuration 1 through the CUDA path: 1e5 trials of Algorithm 1 with V = 16, K = 2; equal
+    to the oracle trial by trial, and the acceptance rate respects the list matching lemma."""
+    from tests import theory
+
+    ld, lt = synth.tiny_coupling("cuda")
+    n, K = 100_000, 2
+    d = ld.view(1, 1, 1, 16).expand(n, K, 1, 16)
+    t = lt.view(1, 1, 1, 16).expand(n, K, 1, 16)
+    seed = synth.NOISE_SEED + 1
+    tok, sc = gls.draft_sample(d, seed=seed)
+    out = gls.target_sample_verify(t, tok, flags=gls.NO_BONUS, seed=seed)
+    dn = np.broadcast_to(ld.cpu().numpy().reshape(1, 1, 1, 16), (n, K, 1, 16))
+    tn = np.broadcast_to(lt.cpu().numpy().reshape(1, 1, 1, 16), (n, K, 1, 16))
+    refd = oracle.draft_sample(dn, seed=seed)
+    refv = oracle.target_sample_verify(tn, refd["tokens"], flags=2, seed=seed)
+    parity.check_draft(tok.cpu().numpy(), sc.cpu().numpy(), refd, "cfg1 draft")
+    o = parity.to_np(out)
+    parity.check_verify(o, refv, "cfg1 verify")
+    acc = o["accept"][:, :, 0].any(axis=1).mean()
+    p, q = theory.softmax(ld.cpu().numpy()), theory.softmax(lt.cpu().numpy())
+    assert acc >= theory.lml_bound(p, q, K) - 4 * np.sqrt(acc * (1 - acc) / n)
+
+
+@pytest.mark.parametrize("spec", [1, 2])
+def test_compress_small(gls, oracle, spec):
+    for B, K, N, lmax in ((12, 1, 50, 1), (10, 4, 3000, 4), (6, 3, 70001, 16), (5, 2, 257, 2)):
+        w = synth.compress_workload("cuda", B=B, K=K, N=N, D=4, l_max=lmax, seed=40 + N)
+        bins = w.bins if lmax > 1 else None
+        out = gls.compress_select(w.enc_logw, w.dec_logw, bins, seed=w.noise_seed, spec=spec)
+        ref = oracle.compress_select(w.enc_logw.cpu().numpy(), w.dec_logw.cpu().numpy(),
+                                     None if bins is None else bins.cpu().numpy(),
+                                     seed=w.noise_seed, spec=spec)
+        parity.check_compress(parity.to_np(out), ref, "N=%d" % N)
+    # per-sample labels [B,N], encoder only, shared noise across decoders
+    w = synth.compress_workload("cuda", B=7, K=3, N=4099, D=4, l_max=8, seed=50)
+    g = torch.Generator(device="cuda").manual_seed(51)
+    bins2 = torch.randint(0, 8, (7, 4099), generator=g, device="cuda", dtype=torch.uint8)
+    out = gls.compress_select(w.enc_logw, w.dec_logw, bins2, seed=SEED, noise_flags=1)
+    ref = oracle.compress_select(w.enc_logw.cpu().numpy(), w.dec_logw.cpu().numpy(),
+                                 bins2.cpu().numpy(), seed=SEED, noise_flags=1)
+    parity.check_compress(parity.to_np(out), ref, "per-sample bins")
+    out = gls.compress_select(w.enc_logw, None, w.bins, K=3, seed=SEED)
+    ref = oracle.compress_select(w.enc_logw.cpu().numpy(), None, w.bins.cpu().numpy(), K=3,
+                                 seed=SEED)
+    o = parity.to_np(out)
+    assert np.array_equal(o["enc_index"], ref["enc_index"])
+    assert np.array_equal(o["message"], ref["message"])
+
+
+def test_host_detectable_errors(gls):
+    x = torch.zeros(2, 2, 2, 64, device="cuda")
+    tok = torch.zeros(2, 2, 1, dtype=torch.int32, device="cuda")
+    with pytest.raises(gls.GlsError):
+        gls.draft_sample(x, inv_temp=0.0)
+    with pytest.raises(gls.GlsError):
+        gls.draft_sample(x, inv_temp=float("nan"))
+    with pytest.raises(gls.GlsError):
+        gls.draft_sample(x, spec=3)
+    with pytest.raises(gls.GlsError):
+        gls.draft_sample(x, rounds=3)
+    with pytest.raises(gls.GlsError):
+        gls.draft_sample(x, workspace=torch.empty(16, dtype=torch.uint8, device="cuda"))
+    with pytest.raises(gls.GlsError):
+        gls.draft_sample(x.double())
+    with pytest.raises(gls.GlsError):
+        gls.draft_sample(x.cpu())
+    with pytest.raises(gls.GlsError):
+        gls.target_sample_verify(x, tok, flags=8)
+    with pytest.raises(gls.GlsError):
+        gls.draft_sample(torch.zeros(1, 65, 1, 8, device="cuda"))
+    # the context is still usable afterwards
+    t, _ = gls.draft_sample(x)
+    torch.cuda.synchronize()
+    assert t.shape == (2, 2, 2)
