@@ -1,0 +1,347 @@
+#!/usr/bin/env python
+"""Benchmark of the GLS hot path on B200: verified positions/s and achieved HBM GB/s.
+
+A step is one pass of the whole hot path over one batch of synthetic logits: draft-side sampling
+over the draft logits, then target-side sampling + verification over the target logits
+(noise generation, both races, split-V reduction, list combine and accept test).
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg2|cfg3|cfg4] [--impl reference]
+
+Under torchrun (N > 1) every rank runs the same workload on its own sequences (sharded by
+sequence id, no data-path collective): weak scaling.  Rank 0 prints ONE JSON line.
+`--impl reference` times the CPU oracle (the reference arm of this repository) on a bounded sample.
+"""
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "verified_positions_per_s"
+UNIT = "positions/s"
+WORKLOAD_DESC = {
+    "cfg2": "multi-draft verify B=8 K=4 L=4 V=32000 fp32 T=1.0",
+    "cfg3": "serving-scale verify B=64 K=8 L=5 V=128256 bf16 T=0.7",
+    "cfg4": "large-batch verify B=256 K=8 L=8 V=152064 bf16 T=1.0",
+}
+# dram__bytes_read+write per launch of the target-side sweep kernel divided by its algorithmic
+# bytes, from the ncu capture summarised in profiles/ (None until a capture exists).
+TRAFFIC_RATIO = None
+
+
+def _peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        return float(json.load(open(p))["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
+
+    Q = ("timestamp,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.rows = []
+        self.proc = None
+        self.index = index
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.Q,
+                 "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append((time.time(), line.strip()))
+
+    def wait_first(self, timeout=10.0):
+        t0 = time.time()
+        while self.proc is not None and not self.rows and time.time() - t0 < timeout:
+            time.sleep(0.05)
+
+    def stop(self, t_begin=None, t_end=None):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, smax, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        power = []
+        for ts, r in self.rows:
+            # a sample printed at ts describes the ~100 ms before it
+            if t_begin is not None and not (t_begin <= ts <= t_end + 0.15):
+                continue
+            f = [x.strip() for x in r.split(",")][1:]
+            if len(f) < 7:
+                continue
+            try:
+                sm.append(float(f[0]))
+                smax.append(float(f[1]))
+                power.append(float(f[2]))
+            except ValueError:
+                continue
+            for n, v in zip(names, f[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": statistics.median(sm) if sm else None,
+                "sm_max_mhz": max(smax) if smax else None, "reasons": sorted(reasons),
+                "samples": len(sm), "power_w_max": max(power) if power else None}
+
+
+def _cpu_baseline(cfg, seqs, threads=None):
+    """The oracle, as it stands, on `seqs` sequences of the workload (host cores)."""
+    import torch
+
+    from oracle import gls_oracle
+    from paper_2506_05632_b200 import synth
+
+    cfg_id = int(cfg[3:])
+    dev = "cuda" if torch.cuda.is_available() else "cpu"
+    w = synth.verify_workload(cfg_id, dev, B=seqs)
+    B, K, L, V = w.shape
+    d, t = synth.to_numpy_rows(w.draft_logits), synth.to_numpy_rows(w.target_logits)
+    del w
+    if threads:
+        gls_oracle.set_threads(threads)
+    cores = gls_oracle.max_threads()
+    kw = dict(seed=synth.NOISE_SEED + cfg_id, inv_temp=synth._INV_TEMP[cfg_id])
+    t0 = time.perf_counter()
+    rd = gls_oracle.draft_sample(d, **kw)
+    gls_oracle.target_sample_verify(t, rd["tokens"], **kw)
+    dt = time.perf_counter() - t0
+    return {"value": B * L / dt, "unit": UNIT, "cores": cores, "kind": "oracle",
+            "sample": "%d of the workload's sequences (all %d rows of each), one pass, %.1f s wall"
+                      % (B, K * (2 * L + 1), dt)}, dt, B * L
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    seqs = {"cfg2": 8, "cfg3": 4, "cfg4": 2}[args.workload]
+    vals, secs = [], []
+    for i in range(args.warmup + args.steps):
+        base, dt, npos = _cpu_baseline(args.workload, seqs)
+        if i >= args.warmup:
+            vals.append(npos)
+            secs.append(dt)
+    value = sum(vals) / sum(secs)
+    base["value"] = value
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT,
+            "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": 1e3 * sum(secs) / len(secs), "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": WORKLOAD_DESC[args.workload],
+                       "sample": "each step = %d sequences of the workload" % seqs},
+            "cpu_baseline": base,
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line))
+
+
+def _time_calls(fn, steps, warmup, flush=None):
+    """CUDA-event timing on the current stream: total ms and per-call event pairs."""
+    import torch
+
+    for _ in range(warmup):
+        fn(None)
+    torch.cuda.synchronize()
+    marks = [[] for _ in range(steps)]
+    start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    start.record()
+    for i in range(steps):
+        if flush is not None:
+            flush.add_(1)
+        fn(marks[i])
+    end.record()
+    torch.cuda.synchronize()
+    return start.elapsed_time(end), marks
+
+
+def _mark(lst):
+    import torch
+
+    if lst is not None:
+        e = torch.cuda.Event(enable_timing=True)
+        e.record()
+        lst.append(e)
+
+
+def run_ours(args):
+    import torch
+
+    import paper_2506_05632_b200 as pkg
+    from paper_2506_05632_b200 import pipeline, synth
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    assert torch.cuda.is_available(), "bench.py needs a CUDA device (no CPU fallback)"
+    torch.cuda.set_device(local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    pkg.load()
+    cfg_id = int(args.workload[3:])
+    w = synth.verify_workload(cfg_id, "cuda", B=args.batch)
+    B, K, L, V = w.shape
+    buf = pipeline.StepBuffers(B, K, L, V)
+    seq_base = rank * B  # ranks own disjoint sequence ids
+    kw = dict(inv_temp=w.inv_temp, seed=w.noise_seed, seq_base=seq_base, spec=args.spec)
+    dbytes = w.draft_logits.numel() * w.draft_logits.element_size()
+    tbytes = w.target_logits.numel() * w.target_logits.element_size()
+    small = dbytes + tbytes < 512e6  # fits the 126 MB L2 several times over? then flush
+    flush = torch.zeros(64 << 20, dtype=torch.float32, device="cuda") if small else None
+
+    def step(marks):
+        _mark(marks)
+        pkg.draft_sample(w.draft_logits, out_tokens=buf.draft_tokens, out_scores=buf.draft_scores,
+                         workspace=buf.workspace, status=buf.status, **kw)
+        _mark(marks)
+        pkg.target_sample_verify(w.target_logits, buf.draft_tokens, out=buf.out,
+                                 workspace=buf.workspace, status=buf.status, **kw)
+        _mark(marks)
+
+    for _ in range(max(args.warmup, 3)):
+        step(None)
+    torch.cuda.synchronize()
+    if dist is not None:
+        dist.barrier()
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+        sampler.wait_first()
+        for _ in range(3):
+            step(None)
+        torch.cuda.synchronize()
+    if dist is not None:
+        dist.barrier()
+    t_begin = time.time()
+    total_ms, marks = _time_calls(step, args.steps, 0, flush)
+    t_end = time.time()
+    if dist is not None:
+        dist.barrier()
+    clocks = sampler.stop(t_begin, t_end) if rank == 0 else None
+    draft_ms = statistics.mean(m[0].elapsed_time(m[1]) for m in marks)
+    verify_ms = statistics.mean(m[1].elapsed_time(m[2]) for m in marks)
+    if flush is not None:  # the flush writes are inside the wall bracket: use the per-call sums
+        total_ms = (draft_ms + verify_ms) * args.steps
+    t = torch.tensor([total_ms], dtype=torch.float64, device="cuda")
+    if dist is not None:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    total_ms = float(t.item())
+    ms_per_step = total_ms / args.steps
+    value = world * B * L / (ms_per_step * 1e-3)
+    tau_mean = float(buf.out["tau"].float().mean().item())
+    assert int(buf.status.item()) == 0
+
+    # end to end from pinned host buffers (H2D of the logits and D2H of the results inside the
+    # timed region)
+    e2e = None
+    if not args.no_e2e:
+        hs = pipeline.HostStepper(B, K, L, V, w.draft_logits.dtype,
+                                  chunk_seqs=max(1, min(16, B // 4)))
+        h_d = torch.empty(w.draft_logits.shape, dtype=w.draft_logits.dtype, pin_memory=True)
+        h_t = torch.empty(w.target_logits.shape, dtype=w.target_logits.dtype, pin_memory=True)
+        h_d.copy_(w.draft_logits)
+        h_t.copy_(w.target_logits)
+        hs.step(h_d, h_t, **kw)
+        n_e2e = max(1, min(args.steps, 5))
+        torch.cuda.synchronize()
+        if dist is not None:
+            dist.barrier()
+        t0 = time.perf_counter()
+        for _ in range(n_e2e):
+            res = hs.step(h_d, h_t, **kw)
+        torch.cuda.synchronize()
+        e_ms = (time.perf_counter() - t0) * 1e3 / n_e2e
+        te = torch.tensor([e_ms], dtype=torch.float64, device="cuda")
+        if dist is not None:
+            dist.all_reduce(te, op=dist.ReduceOp.MAX)
+        e_ms = float(te.item())
+        assert torch.equal(res["tau"], buf.out["tau"].cpu())
+        e2e = {"value": world * B * L / (e_ms * 1e-3), "unit": UNIT,
+               "h2d_bytes_per_step": hs.h2d_bytes, "d2h_bytes_per_step": hs.d2h_bytes,
+               "ms_per_step": e_ms, "steps": n_e2e}
+        del h_d, h_t, hs
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+
+    peak, which = _peaks()
+    achieved = tbytes / (verify_ms * 1e-3) / 1e9
+    roofline = {"bound": "hbm", "kernel": "sweep_kernel<%s,spec2,lse> (target side; the call also "
+                "runs three microsecond-scale helper kernels)" %
+                ("bf16" if w.target_logits.dtype == torch.bfloat16 else "f32"),
+                "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                "peak_source": "of " + which,
+                "traffic": (TRAFFIC_RATIO * tbytes) if TRAFFIC_RATIO else None,
+                "algorithmic_bytes": tbytes, "ms": verify_ms,
+                "draft_side": {"achieved": dbytes / (draft_ms * 1e-3) / 1e9, "ms": draft_ms,
+                               "frac": dbytes / (draft_ms * 1e-3) / 1e9 / peak},
+                "step": {"achieved": (dbytes + tbytes) / (ms_per_step * 1e-3) / 1e9,
+                         "frac_of_nominal_8TBs": (dbytes + tbytes) / (ms_per_step * 1e-3) / 8e12}}
+    del w, buf
+    torch.cuda.empty_cache()
+    cpu = None
+    if not args.no_cpu:
+        cpu, _, _ = _cpu_baseline(args.workload, {"cfg2": 8, "cfg3": 32, "cfg4": 16}[args.workload])
+    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": {"workload": WORKLOAD_DESC[args.workload] + (" (B overridden to %d)" % B if args.batch else ""),
+                       "noise_spec": args.spec,
+                       "philox_rounds": 10,
+                       "l2": "flushed between steps" if flush is not None
+                       else "inputs (%.2f GB) larger than L2" % ((dbytes + tbytes) / 1e9),
+                       "mean_tau": tau_mean},
+            "hbm_gbs": (dbytes + tbytes) / (ms_per_step * 1e-3) / 1e9,
+            "clocks": clocks, "e2e": e2e, "gpu_launches": 5 * args.steps,
+            "roofline": roofline, "cpu_baseline": cpu}
+    print(json.dumps(line))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="cfg4", choices=sorted(WORKLOAD_DESC))
+    ap.add_argument("--batch", type=int, default=None,
+                    help="override B (reduced copy of the workload, e.g. for an ncu capture)")
+    ap.add_argument("--spec", type=int, default=2, choices=[1, 2], help="noise_spec")
+    ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg")
+    ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle baseline leg")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

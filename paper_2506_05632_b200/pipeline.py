@@ -1,0 +1,92 @@
+"""One pass of the whole hot path over a batch, on device tensors or from host buffers.
+
+`spec_step` is what a serving loop calls per speculative-decoding step once both sets of logits
+are on the GPU: draft-side sampling (Algorithm 2, draft loop) followed by target-side sampling and
+verification (Algorithm 2, second half).  `HostStepper` is the same step for logits that live in
+(pinned) host memory: it streams sequence chunks to the device through two staging buffers so
+that the copy of chunk n+1 overlaps the sweep of chunk n, and returns the results to the host.
+Only copies, launches and bookkeeping happen here; all arithmetic is in the CUDA library.
+"""
+import torch
+
+from . import binding
+
+
+class StepBuffers:
+    """Preallocated outputs and workspace for `spec_step` on B sequences."""
+
+    def __init__(self, B, K, L, V, device="cuda"):
+        self.shape = (B, K, L, V)
+        self.draft_tokens = torch.empty((B, K, max(L, 0)), dtype=torch.int32, device=device)
+        self.draft_scores = torch.empty((B, K, max(L, 0)), dtype=torch.float32, device=device)
+        self.out = dict(tokens=torch.empty((B, L + 1), dtype=torch.int32, device=device),
+                        tau=torch.empty((B,), dtype=torch.int32, device=device),
+                        accept=torch.empty((B, K, L), dtype=torch.uint8, device=device),
+                        scores=torch.empty((B, L + 1), dtype=torch.float32, device=device))
+        need = max(binding.workspace_bytes(B, K, max(L, 1), V),
+                   binding.workspace_bytes(B, K, L + 1, V))
+        self.workspace = torch.empty(need, dtype=torch.uint8, device=device)
+        self.status = torch.zeros(1, dtype=torch.int32, device=device)
+
+
+def spec_step(draft_logits, target_logits, buf, inv_temp=1.0, seed=0, seq_base=0, pos_base=0,
+              spec=2, rounds=10):
+    """draft_logits [B,K,L,V], target_logits [B,K,L+1,V] on the device -> buf.out (device)."""
+    kw = dict(inv_temp=inv_temp, seed=seed, seq_base=seq_base, pos_base=pos_base, spec=spec,
+              rounds=rounds, workspace=buf.workspace, status=buf.status)
+    if draft_logits.shape[2] > 0:
+        binding.draft_sample(draft_logits, out_tokens=buf.draft_tokens,
+                             out_scores=buf.draft_scores, **kw)
+    binding.target_sample_verify(target_logits, buf.draft_tokens, out=buf.out, **kw)
+    return buf.out
+
+
+class HostStepper:
+    """Hot path from HOST logits: chunked, double-buffered H2D copies overlapped with the sweeps."""
+
+    def __init__(self, B, K, L, V, dtype, chunk_seqs=16, device="cuda"):
+        self.B, self.K, self.L, self.V = B, K, L, V
+        self.chunk = min(chunk_seqs, B)
+        self.copy_stream = torch.cuda.Stream(device=device)
+        self.stage = [dict(d=torch.empty((self.chunk, K, L, V), dtype=dtype, device=device),
+                           t=torch.empty((self.chunk, K, L + 1, V), dtype=dtype, device=device),
+                           ready=torch.cuda.Event(), free=torch.cuda.Event(),
+                           buf=StepBuffers(self.chunk, K, L, V, device))
+                      for _ in range(2)]
+        self.h_tokens = torch.empty((B, L + 1), dtype=torch.int32).pin_memory()
+        self.h_tau = torch.empty((B,), dtype=torch.int32).pin_memory()
+        self.h_accept = torch.empty((B, K, L), dtype=torch.uint8).pin_memory()
+        elt = torch.empty(0, dtype=dtype).element_size()
+        self.h2d_bytes = B * K * (2 * L + 1) * V * elt
+        self.d2h_bytes = self.h_tokens.numel() * 4 + self.h_tau.numel() * 4 + self.h_accept.numel()
+
+    def step(self, h_draft, h_target, inv_temp=1.0, seed=0, seq_base=0, spec=2, rounds=10):
+        """h_draft [B,K,L,V], h_target [B,K,L+1,V]: pinned host tensors.  Returns host results."""
+        main = torch.cuda.current_stream()
+        n = 0
+        for b0 in range(0, self.B, self.chunk):
+            b1 = min(self.B, b0 + self.chunk)
+            s = self.stage[n & 1]
+            nb = b1 - b0
+            with torch.cuda.stream(self.copy_stream):
+                if n >= 2:
+                    self.copy_stream.wait_event(s["free"])
+                s["d"][:nb].copy_(h_draft[b0:b1], non_blocking=True)
+                s["t"][:nb].copy_(h_target[b0:b1], non_blocking=True)
+                s["ready"].record(self.copy_stream)
+            main.wait_event(s["ready"])
+            buf = s["buf"]
+            if nb == self.chunk:
+                d, t, bb = s["d"], s["t"], buf
+            else:  # ragged last chunk
+                d, t = s["d"][:nb], s["t"][:nb]
+                bb = StepBuffers(nb, self.K, self.L, self.V, d.device)
+            out = spec_step(d, t, bb, inv_temp=inv_temp, seed=seed, seq_base=seq_base + b0,
+                            spec=spec, rounds=rounds)
+            self.h_tokens[b0:b1].copy_(out["tokens"], non_blocking=True)
+            self.h_tau[b0:b1].copy_(out["tau"], non_blocking=True)
+            self.h_accept[b0:b1].copy_(out["accept"], non_blocking=True)
+            s["free"].record(main)
+            n += 1
+        main.synchronize()
+        return dict(tokens=self.h_tokens, tau=self.h_tau, accept=self.h_accept)
