@@ -12,6 +12,15 @@ import torch
 from . import binding
 
 
+def shard_sequences(B, rank, world):
+    """Sequences [b0, b1) of a batch of B that rank `rank` of `world` owns (contiguous, sizes differ
+    by at most one).  Noise is keyed by the absolute sequence id, so a rank passes seq_base = b0
+    and the union of the ranks' results equals the unsharded result bit for bit."""
+    base, extra = divmod(int(B), int(world))
+    b0 = rank * base + min(rank, extra)
+    return b0, b0 + base + (1 if rank < extra else 0)
+
+
 class StepBuffers:
     """Preallocated outputs and workspace for `spec_step` on B sequences."""
 
