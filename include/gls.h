@@ -77,7 +77,8 @@ typedef enum {
   GLS_ERR_UNSUPPORTED = 2,
   GLS_ERR_MISALIGNED = 3,
   GLS_ERR_WORKSPACE = 4,
-  GLS_ERR_CUDA = 5
+  GLS_ERR_CUDA = 5,
+  GLS_ERR_STATIC_LIMIT = 6 /* problem needs more scratch than the built-in static buffer holds */
 } gls_status_t;
 
 /* bits OR-ed into *device_status by the kernels */
@@ -143,6 +144,41 @@ int gls_draft_sample(const gls_rows_t* draft_logits, int B, int K, int J, int64_
                      const float* inv_temp_per_draft_host, const gls_noise_t* noise,
                      int32_t* out_tokens, float* out_scores, void* workspace,
                      size_t workspace_bytes, uint32_t* device_status, void* stream);
+
+/*
+ * Draft-side sampling for callers that cannot allocate device memory.  The paper has no counterpart
+ * to this call; it exists for deployment only and computes exactly what gls_draft_sample computes.
+ *
+ * Who needs it: code that runs where cudaMalloc is off limits -- a step function inside a serving
+ * loop that must not take cudaMalloc's device-wide synchronisation, or a plug-in whose host has
+ * handed every byte of device memory to its own pool and offers no hook to borrow some.  Such a
+ * caller has nowhere to get the `workspace` that gls_draft_sample asks for.  Here the scratch
+ * (bound hints, per-slice partial results, per-row results) lives in a buffer of
+ * GLS_STATIC_SCRATCH_BYTES that is compiled into the library image: every GPU that loads the
+ * library carries it from load until the process exits.  The call itself performs no cudaMalloc,
+ * no cudaFree and no allocating library routine.
+ *
+ * Arguments are those of gls_draft_sample without workspace / workspace_bytes; inputs and outputs
+ * still belong to the caller.
+ *
+ * Limits and rules:
+ *   - A problem whose scratch need, gls_workspace_bytes(B, K, J, V), exceeds
+ *     GLS_STATIC_SCRATCH_BYTES is refused with GLS_ERR_STATIC_LIMIT and nothing is enqueued
+ *     (gls_static_scratch_bytes() returns the limit at run time).
+ *   - The first call on each device looks up the buffer's device address (one
+ *     cudaGetSymbolAddress with that device current) and remembers it.  Make that first call
+ *     outside any stream capture.
+ *   - Every call on a device shares the one buffer, which still holds the previous call's contents;
+ *     the call clears the part that must start at zero on `stream` before using it.  Two calls that
+ *     can overlap on the GPU (different streams without an ordering between them) race on the
+ *     buffer: order them, or use gls_draft_sample with separate workspaces.
+ */
+#define GLS_STATIC_SCRATCH_BYTES (4u << 20)
+size_t gls_static_scratch_bytes(void);
+int gls_draft_sample_static(const gls_rows_t* draft_logits, int B, int K, int J, int64_t V,
+                            float inv_temp, const float* inv_temp_per_draft_host,
+                            const gls_noise_t* noise, int32_t* out_tokens, float* out_scores,
+                            uint32_t* device_status, void* stream);
 
 /*
  * Target side and verification -- Sec. 3 step 1, Algorithm 2 from "Let the set of active drafts"

@@ -80,6 +80,11 @@ def load():
             C.POINTER(_Rows), C.c_int, C.c_int, C.c_int, C.c_int64, C.c_float, C.c_void_p,
             C.POINTER(_Noise), C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p,
             C.c_void_p]
+        L.gls_static_scratch_bytes.restype = C.c_size_t
+        L.gls_draft_sample_static.restype = C.c_int
+        L.gls_draft_sample_static.argtypes = [
+            C.POINTER(_Rows), C.c_int, C.c_int, C.c_int, C.c_int64, C.c_float, C.c_void_p,
+            C.POINTER(_Noise), C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
         L.gls_target_sample_verify.restype = C.c_int
         L.gls_target_sample_verify.argtypes = [
             C.POINTER(_Rows), C.c_int, C.c_int, C.c_int, C.c_int64, C.c_float, C.c_void_p,
@@ -173,6 +178,32 @@ def draft_sample(logits, inv_temp=1.0, inv_temp_per_draft=None, seed=0, seq_base
                               C.cast(itk, C.c_void_p) if itk is not None else None, C.byref(nz),
                               _ptr(out_tokens), _ptr(out_scores), workspace.data_ptr(),
                               workspace.numel(), _ptr(status), _stream()))
+    return out_tokens, out_scores
+
+
+def static_scratch_bytes():
+    return int(load().gls_static_scratch_bytes())
+
+
+def draft_sample_static(logits, out_tokens, out_scores=None, inv_temp=1.0, inv_temp_per_draft=None,
+                        seed=0, seq_base=0, seq_ids=None, pos_base=0, spec=2, rounds=10,
+                        noise_flags=0, status=None):
+    """gls_draft_sample_static: draft_sample for callers that may not allocate device memory.
+
+    The caller passes the outputs (int32 [B,K,J], optional fp32 [B,K,J]); this wrapper creates no
+    tensor and the library uses its built-in scratch buffer.  Raises GlsError when the problem
+    needs more scratch than static_scratch_bytes()."""
+    L = load()
+    B, K, J, V = logits.shape
+    rows = _rows(logits, 3)
+    nz = _noise(seed, seq_base, seq_ids, pos_base, spec, rounds, noise_flags)
+    itk = None
+    if inv_temp_per_draft is not None:
+        itk = (C.c_float * K)(*[float(x) for x in inv_temp_per_draft])
+    _check(L.gls_draft_sample_static(C.byref(rows), B, K, J, V, float(inv_temp),
+                                     C.cast(itk, C.c_void_p) if itk is not None else None,
+                                     C.byref(nz), _ptr(out_tokens), _ptr(out_scores), _ptr(status),
+                                     _stream()))
     return out_tokens, out_scores
 
 

@@ -8,6 +8,7 @@
 // sides of the coupling, Sec. 5.3).
 #include <cmath>
 #include <cstring>
+#include <mutex>
 
 #include "../../include/gls.h"
 #include "gls_kernels.cuh"
@@ -340,6 +341,9 @@ const char* gls_status_string(int status) {
     case GLS_ERR_MISALIGNED: return "GLS_ERR_MISALIGNED: base pointer not aligned to its element size";
     case GLS_ERR_WORKSPACE: return "GLS_ERR_WORKSPACE: workspace missing or smaller than gls_workspace_bytes()";
     case GLS_ERR_CUDA: return "GLS_ERR_CUDA: a CUDA runtime call failed";
+    case GLS_ERR_STATIC_LIMIT:
+      return "GLS_ERR_STATIC_LIMIT: the problem needs more scratch than GLS_STATIC_SCRATCH_BYTES; "
+             "use the entry point that takes a workspace";
     default: return "GLS: unknown status";
   }
 }
@@ -473,6 +477,63 @@ int gls_compress_select(const gls_rows_t* enc_logw, const gls_rows_t* dec_logw, 
   decoder_epilogue_kernel<<<(B + 127) / 128, 128, 0, st>>>(rowres, B, K, out_enc_index,
                                                           out_dec_index, out_match, out_scores);
   return cudaGetLastError() == cudaSuccess ? GLS_OK : GLS_ERR_CUDA;
+}
+
+}  // extern "C"
+
+// ------------------------------------------------------------------------------------------
+// Allocation-free draft sampling: scratch compiled into the library image.
+// ------------------------------------------------------------------------------------------
+namespace gls {
+
+// Scratch of gls_draft_sample_static.  In host code this name is only a handle for
+// cudaGetSymbolAddress; the kernels get the device address that call returns.
+static __device__ __align__(256) unsigned char g_static_scratch[GLS_STATIC_SCRATCH_BYTES];
+
+constexpr int kMaxDevices = 64;
+static std::mutex g_static_mutex;
+static void* g_static_ptr[kMaxDevices] = {};
+
+// Device address of the scratch on the current device, looked up once per device.
+static int static_scratch_address(void** out) {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess) return GLS_ERR_CUDA;
+  if (dev < 0 || dev >= kMaxDevices) return GLS_ERR_UNSUPPORTED;
+  std::lock_guard<std::mutex> lock(g_static_mutex);
+  if (g_static_ptr[dev] == nullptr) {
+    void* p = nullptr;
+    if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess || p == nullptr) {
+      (void)cudaGetLastError();
+      return GLS_ERR_CUDA;
+    }
+    g_static_ptr[dev] = p;
+  }
+  *out = g_static_ptr[dev];
+  return GLS_OK;
+}
+
+}  // namespace gls
+
+extern "C" {
+
+size_t gls_static_scratch_bytes(void) { return (size_t)GLS_STATIC_SCRATCH_BYTES; }
+
+int gls_draft_sample_static(const gls_rows_t* draft_logits, int B, int K, int J, int64_t V,
+                            float inv_temp, const float* inv_temp_per_draft_host,
+                            const gls_noise_t* noise, int32_t* out_tokens, float* out_scores,
+                            uint32_t* device_status, void* stream) {
+  if (!gls::sizes_ok(B, K, J, V)) return GLS_ERR_INVALID_ARG;
+  const size_t need = gls_workspace_bytes(B, K, J, V);
+  if (need == 0) return GLS_ERR_INVALID_ARG;
+  if (need > (size_t)GLS_STATIC_SCRATCH_BYTES) return GLS_ERR_STATIC_LIMIT;
+  void* scratch = nullptr;
+  const int rc = gls::static_scratch_address(&scratch);
+  if (rc != GLS_OK) return rc;
+  // Same path as the workspace-taking entry point; it clears the bound hints on `stream` before
+  // the sweep reads them, which is the only part of the scratch that must start at zero.
+  return gls_draft_sample(draft_logits, B, K, J, V, inv_temp, inv_temp_per_draft_host, noise,
+                          out_tokens, out_scores, scratch, (size_t)GLS_STATIC_SCRATCH_BYTES,
+                          device_status, stream);
 }
 
 }  // extern "C"
