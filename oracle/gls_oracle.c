@@ -85,7 +85,7 @@ void glso_philox4x32(const uint32_t ctr[4], const uint32_t key[2], int rounds, u
 typedef struct {
   uint64_t seed;
   int rounds;       /* Philox rounds (10 by default) */
-  int spec;         /* 1 or 2 */
+  int spec;         /* 1, 2 or 3 */
   uint32_t domain;  /* 0 decoding, 1 compression */
   uint32_t seq, pos, k;
 } glso_key_t;
@@ -99,6 +99,16 @@ double glso_uniform(const glso_key_t* nk, int64_t i) {
     glso_philox4x32(ctr, key, nk->rounds, out);
     uint32_t w = out[i & 3];
     return ((double)w + 0.5) * 0x1p-32;
+  } else if (nk->spec == 3) {
+    /* 8 coarse bits (16 tokens per generator call) + 40 refinement bits (2 tokens per call) */
+    uint32_t cc[4] = {(uint32_t)(i >> 4), nk->k | (nk->domain << 16), nk->pos, nk->seq};
+    glso_philox4x32(cc, key, nk->rounds, out);
+    uint32_t h = (out[(i & 15) >> 2] >> (8 * (i & 3))) & 0xffu;
+    uint32_t cr[4] = {(uint32_t)(i >> 1), nk->k | ((nk->domain + 2u) << 16), nk->pos, nk->seq};
+    glso_philox4x32(cr, key, nk->rounds, out);
+    uint64_t x = ((uint64_t)(out[2 * (i & 1) + 1] & 0xffu) << 32) | out[2 * (i & 1)];
+    /* h * 2^40 + x + 0.5 < 2^48 + 1: exact in fp64 */
+    return ((double)h * 1099511627776.0 + (double)x + 0.5) * 0x1p-48;
   } else {
     uint32_t cc[4] = {(uint32_t)(i >> 3), nk->k | (nk->domain << 16), nk->pos, nk->seq};
     glso_philox4x32(cc, key, nk->rounds, out);
@@ -248,7 +258,7 @@ typedef struct {
   uint32_t seq_base;
   const uint32_t* seq_ids; /* host array [B] or NULL */
   uint32_t pos_base;
-  uint32_t noise_spec; /* 1 or 2 */
+  uint32_t noise_spec; /* 1, 2 or 3 */
   uint32_t rounds;
   uint32_t flags;
 } glso_noise_t;

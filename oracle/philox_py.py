@@ -58,6 +58,13 @@ def uniform_numerator(seed, seq, pos, k, i, spec=2, domain=0, rounds=10):
     if spec == 1:
         out = philox4x32((i >> 2, k | (domain << 16), pos, seq), key, rounds)
         return out[i & 3], 32
+    if spec == 3:
+        coarse = philox4x32((i >> 4, k | (domain << 16), pos, seq), key, rounds)
+        bits128 = coarse[0] | (coarse[1] << 32) | (coarse[2] << 64) | (coarse[3] << 96)
+        h = (bits128 >> (8 * (i & 15))) & 0xFF
+        fine = philox4x32((i >> 1, k | ((domain + 2) << 16), pos, seq), key, rounds)
+        half = (fine[0] | (fine[1] << 32)) if (i & 1) == 0 else (fine[2] | (fine[3] << 32))
+        return (h << 40) | (half & ((1 << 40) - 1)), 48
     coarse = philox4x32((i >> 3, k | (domain << 16), pos, seq), key, rounds)
     bits128 = coarse[0] | (coarse[1] << 32) | (coarse[2] << 64) | (coarse[3] << 96)
     h = (bits128 >> (16 * (i & 7))) & 0xFFFF

@@ -67,7 +67,7 @@ def test_avalanche(oracle):
 
 def test_uniform_bit_fields_match_second_implementation(oracle):
     rng = np.random.default_rng(4)
-    for spec in (1, 2):
+    for spec in (1, 2, 3):
         for domain in (0, 1):
             for _ in range(400):
                 seq, pos = int(rng.integers(0, 2**32)), int(rng.integers(0, 2**32))
@@ -78,14 +78,14 @@ def test_uniform_bit_fields_match_second_implementation(oracle):
                 assert got == want
                 assert 0.0 < got < 1.0
     # consecutive tokens walk through all fields of a block
-    for spec in (1, 2):
+    for spec in (1, 2, 3):
         vals = [oracle.uniform(SEED, 5, 6, 7, i, spec=spec) for i in range(64)]
         assert len(set(vals)) == 64
 
 
 def test_noise_is_exp1_and_uniform(oracle):
     n = 1_000_000
-    for spec in (1, 2):
+    for spec in (1, 2, 3):
         S = oracle.exp_noise_row(SEED, seq=11, pos=3, k=1, V=n, spec=spec)
         assert np.all(S > 0) and np.all(np.isfinite(S))
         assert abs(S.mean() - 1.0) < 5e-3 and abs(S.var() - 1.0) < 1.5e-2
@@ -110,6 +110,7 @@ def test_streams_differ_across_key_components(oracle):
         oracle.exp_noise_row(SEED + 1, V=V, **base),
         oracle.exp_noise_row(SEED ^ (1 << 40), V=V, **base),
         oracle.exp_noise_row(SEED, V=V, spec=1, **base),
+        oracle.exp_noise_row(SEED, V=V, spec=3, **base),
     ]
     for o in others:
         assert not np.any(o == ref)
@@ -130,3 +131,20 @@ def test_spec2_coarse_bits_bound_the_uniform(oracle):
         v = oracle.uniform(SEED, 1, 2, 3, i, spec=2)
         assert h / 65536.0 <= v < (h + 1) / 65536.0
         assert -math.log1p(-v) >= v  # S >= v, so S >= h * 2^-16 as well
+
+
+def test_spec3_coarse_byte_bounds_the_uniform(oracle):
+    """With the 8 + 40 bit layout the coarse byte alone gives h / 256 <= v < (h + 1) / 256, and all
+    16 byte fields of one coarse generator call are used by 16 consecutive tokens."""
+    seen = set()
+    for i in range(0, 4096):
+        num, bits = philox_py.uniform_numerator(SEED, 1, 2, 3, i, 3, 0)
+        assert bits == 48
+        h = num >> 40
+        v = oracle.uniform(SEED, 1, 2, 3, i, spec=3)
+        assert h / 256.0 <= v < (h + 1) / 256.0
+        seen.add(h)
+    assert len(seen) == 256  # every byte value occurs among 4096 tokens (miss probability < 3e-5)
+    # tokens with a zero coarse byte are 1/256 of all: binomial(65536, 1/256), mean 256, sd 16
+    zeros = sum(philox_py.uniform_numerator(SEED, 9, 0, 0, i, 3, 0)[0] >> 40 == 0 for i in range(65536))
+    assert 256 - 5 * 16 < zeros < 256 + 5 * 16
