@@ -291,7 +291,7 @@ def run_ours(args):
 
     peak, which = _peaks()
     achieved = tbytes / (verify_ms * 1e-3) / 1e9
-    roofline = {"bound": "hbm", "kernel": "sweep_kernel<%s,spec2,lse> (target side; the call also "
+    roofline = {"bound": "hbm", "kernel": "sweep kernel <%s, lse> of the selected noise_spec (target side; the call also "
                 "runs three microsecond-scale helper kernels)" %
                 ("bf16" if w.target_logits.dtype == torch.bfloat16 else "f32"),
                 "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
@@ -333,7 +333,7 @@ def main():
     ap.add_argument("--workload", default="cfg4", choices=sorted(WORKLOAD_DESC))
     ap.add_argument("--batch", type=int, default=None,
                     help="override B (reduced copy of the workload, e.g. for an ncu capture)")
-    ap.add_argument("--spec", type=int, default=2, choices=[1, 2], help="noise_spec")
+    ap.add_argument("--spec", type=int, default=3, choices=[1, 2, 3], help="noise_spec")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle baseline leg")
     args = ap.parse_args()

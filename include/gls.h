@@ -32,13 +32,20 @@
  *                  bits, i.e. (out[(i & 7) >> 1] >> (16 * (i & 1))) & 0xffff;
  *                  refine  block = i >> 2 in `domain + 2`: r = out[i & 3];
  *                                                               v = (h * 2^32 + r + 0.5) * 2^-48
+ *   noise_spec 3:  coarse  block = i >> 4 in `domain`:   h = byte (i & 15) of the 128 output bits,
+ *                  i.e. (out[(i & 15) >> 2] >> (8 * (i & 3))) & 0xff;
+ *                  refine  block = i >> 1 in `domain + 2`: x = the low 40 bits of the 64-bit half
+ *                  (i & 1), i.e. ((out[2 (i & 1) + 1] & 0xff) << 32) | out[2 (i & 1)];
+ *                                                               v = (h * 2^40 + x + 0.5) * 2^-48
  *   S = -log1p(-v)   (v is strictly inside (0,1), so S is finite and positive; this is the paper's
  *                     S = -ln U with U = 1 - v)
  *
  * A draft call and a verify call that describe the same (seed, sequence, position, k, i) therefore
- * see the same S -- that is the coupling.  Both specs are exact definitions; spec 2 merely lets a
- * kernel decide most tokens from the 16 coarse bits and generate the 32 refinement bits only for
- * the few tokens that can still win.
+ * see the same S -- that is the coupling.  All three specs are exact definitions; specs 2 and 3 let
+ * a kernel decide most tokens from the coarse bits alone (16 bits for 8 tokens per generator call,
+ * or 8 bits for 16 tokens per call) and generate the refinement bits only for the few tokens that
+ * can still win.  Spec 3 is the default and the fastest: the generator's 32x32->64-bit multiplies
+ * are the scarcest resource of the sweep on sm_100a.
  *
  * CONVENTIONS
  *   - Token / candidate indices are 0-based (the paper counts from 1).
@@ -47,8 +54,8 @@
  *     on the caller's stream and returns without synchronising.
  *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).
  *   - Rows: the token dimension is contiguous; strides are in ELEMENTS and may be 0 (broadcast).
- *     Rows whose first element is 16-byte aligned take the vectorised path; others are still
- *     handled (slower scalar loads).
+ *     Rows whose first element is 32-byte aligned (16-byte for noise_spec 1 and 2) take the
+ *     vectorised path; others are still handled (slower scalar loads).
  *   - A logit of -inf is a legal "masked" token (top-K truncation, Sec. 4.4).  NaN and +inf
  *     logits never win a race and are excluded from the log-sum-exp.
  *   - Ties (measure zero in exact arithmetic): lowest token index, then lowest k.
@@ -105,7 +112,7 @@ typedef struct {
   uint32_t seq_base;       /* sequence id of batch row b is seq_base + b ...                   */
   const uint32_t* seq_ids; /* ... unless this optional DEVICE array [B] is given               */
   uint32_t pos_base;       /* position id of index j is pos_base + j                           */
-  uint32_t noise_spec;     /* 1 or 2 (see above); 0 selects 2                                  */
+  uint32_t noise_spec;     /* 1, 2 or 3 (see above); 0 selects 3                               */
   uint32_t rounds;         /* Philox rounds, 0 selects 10; 7..16 accepted                      */
   uint32_t flags;          /* GLS_NOISE_*                                                      */
 } gls_noise_t;

@@ -12,6 +12,7 @@
 
 #include "../../include/gls.h"
 #include "gls_kernels.cuh"
+#include "gls_sweep3.cuh"
 
 namespace gls {
 
@@ -20,16 +21,25 @@ constexpr int kMinChunk = 2048;
 constexpr int kMaxChunk = 16384;
 
 struct Plan {
-  int chunk, splits;
+  int chunk, splits, parts;
   long long rows, n_items;
   size_t off_hints, off_partials, off_rows, total;
 };
 
 static size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
-// Slice size: aim at ~8 work items per resident warp so that the static round-robin over warps
-// balances, but keep slices long enough to amortise the per-item reduction.
-static Plan make_plan(long long rows, long long V) {
+static void plan_layout(Plan& p) {
+  p.n_items = p.rows * p.splits;
+  p.off_hints = 0;
+  p.off_partials = align_up((size_t)p.rows * sizeof(uint32_t), 256);
+  p.off_rows = p.off_partials + align_up((size_t)p.rows * p.parts * sizeof(Partial), 256);
+  p.total = p.off_rows + align_up((size_t)p.rows * sizeof(RowResult), 256);
+}
+
+// noise_spec 1 and 2 (a warp per work item).  Slice size: aim at ~8 work items per resident warp
+// so that the static round-robin over warps balances, but keep slices long enough to amortise
+// the per-item reduction.
+static Plan make_plan12(long long rows, long long V) {
   Plan p;
   const long long target_items = 8LL * kNumSMs * 32;
   long long chunk = (rows * V + target_items - 1) / target_items;
@@ -40,13 +50,36 @@ static Plan make_plan(long long rows, long long V) {
   if (chunk > vceil) chunk = vceil;
   p.chunk = (int)chunk;
   p.splits = (int)((V + chunk - 1) / chunk);
+  p.parts = p.splits;
   p.rows = rows;
-  p.n_items = rows * p.splits;
-  p.off_hints = 0;
-  p.off_partials = align_up((size_t)rows * sizeof(uint32_t), 256);
-  p.off_rows = p.off_partials + align_up((size_t)p.n_items * sizeof(Partial), 256);
-  p.total = p.off_rows + align_up((size_t)rows * sizeof(RowResult), 256);
+  plan_layout(p);
   return p;
+}
+
+// noise_spec 3 (a CTA per work item, one partial per warp).  Whole rows when there are enough of
+// them to keep the static round-robin over the resident CTAs balanced (16 items per CTA),
+// otherwise the fewest slices that reach that count, never shorter than kS3MinChunk tokens.
+constexpr int kS3CtasPerSM = 4;
+constexpr int kS3MinChunk = 4 * kS3CtaTokens;
+static Plan make_plan3(long long rows, long long V) {
+  Plan p;
+  const long long target_items = 16LL * kNumSMs * kS3CtasPerSM;
+  long long splits = (target_items + rows - 1) / rows;
+  const long long max_splits = (V + kS3MinChunk - 1) / kS3MinChunk;
+  if (splits > max_splits) splits = max_splits;
+  if (splits < 1) splits = 1;
+  long long chunk = (V + splits - 1) / splits;
+  chunk = (chunk + kS3CtaTokens - 1) / kS3CtaTokens * kS3CtaTokens;
+  p.chunk = (int)chunk;
+  p.splits = (int)((V + chunk - 1) / chunk);
+  p.parts = p.splits * kSweepWarps3;
+  p.rows = rows;
+  plan_layout(p);
+  return p;
+}
+
+static Plan make_plan(long long rows, long long V, int spec) {
+  return spec == 3 ? make_plan3(rows, V) : make_plan12(rows, V);
 }
 
 // ------------------------------------------------------------------------------------------
@@ -73,8 +106,8 @@ finalize_rows_kernel(const __grid_constant__ SweepArgs A, int rows, int with_lse
   Top2 best;
   top2_init(best);
   float lm = kLseFloor;
-  for (int s = lane; s < A.splits; s += 32) {
-    const Partial p = A.partials[(long long)row * A.splits + s];
+  for (int s = lane; s < A.parts; s += 32) {
+    const Partial p = A.partials[(long long)row * A.parts + s];
     top2_offer(best, p.s1, p.i1);
     top2_offer(best, p.s2, p.i2);
     lm = fmaxf(lm, p.lm);
@@ -84,8 +117,8 @@ finalize_rows_kernel(const __grid_constant__ SweepArgs A, int rows, int with_lse
   for (int d = 16; d > 0; d >>= 1) lm = fmaxf(lm, __shfl_xor_sync(0xffffffffu, lm, d));
   double lsum = 0.0;
   if (with_lse) {
-    for (int s = lane; s < A.splits; s += 32) {
-      const Partial p = A.partials[(long long)row * A.splits + s];
+    for (int s = lane; s < A.parts; s += 32) {
+      const Partial p = A.partials[(long long)row * A.parts + s];
       if (p.ls > 0.f) lsum += (double)p.ls * exp2((double)(p.lm - lm) * (double)c2);
     }
 #pragma unroll
@@ -233,8 +266,8 @@ static bool finite_pos(float x) { return std::isfinite(x) && x > 0.f; }
 static int fill_noise(SweepArgs& A, const gls_noise_t* nz, uint32_t domain, int* spec_out) {
   const int rounds = nz->rounds ? (int)nz->rounds : 10;
   if (rounds < 7 || rounds > 16) return GLS_ERR_INVALID_ARG;
-  const int spec = nz->noise_spec ? (int)nz->noise_spec : 2;
-  if (spec != 1 && spec != 2) return GLS_ERR_INVALID_ARG;
+  const int spec = nz->noise_spec ? (int)nz->noise_spec : 3;
+  if (spec < 1 || spec > 3) return GLS_ERR_INVALID_ARG;
   if (nz->flags & ~GLS_NOISE_SHARED_ACROSS_K) return GLS_ERR_INVALID_ARG;
   uint32_t k0 = (uint32_t)(nz->seed & 0xffffffffu), k1 = (uint32_t)(nz->seed >> 32);
   for (int r = 0; r < 16; ++r) {
@@ -286,33 +319,51 @@ static int run_rows(SweepArgs& A, int dtype, int spec, const Plan& P, void* work
   char* ws = (char*)workspace;
   A.chunk = P.chunk;
   A.splits = P.splits;
+  A.parts = P.parts;
+  A.rows = (int)P.rows;
   A.n_items = P.n_items;
   A.hints = (uint32_t*)(ws + P.off_hints);
   A.partials = (Partial*)(ws + P.off_partials);
   RowResult* rowres = (RowResult*)(ws + P.off_rows);
   if (cudaMemsetAsync(A.hints, 0, (size_t)P.rows * sizeof(uint32_t), st) != cudaSuccess)
     return GLS_ERR_CUDA;
-  const long long want = (P.n_items + kSweepThreads / 32 - 1) / (kSweepThreads / 32);
-  const int grid = (int)(want < (long long)kNumSMs * 4 ? want : (long long)kNumSMs * 4);
   cudaError_t err;
-#define SWEEP_CALL(...) launch_sweep_t<__VA_ARGS__>(A, lse, grid, st)
-  if (dtype == GLS_BF16) {
-    if (spec == 1) err = A.rounds == 10 ? SWEEP_CALL(kBF16, 1, 10) : SWEEP_CALL(kBF16, 1, 0);
-    else err = A.rounds == 10 ? SWEEP_CALL(kBF16, 2, 10) : SWEEP_CALL(kBF16, 2, 0);
+  const bool r10 = A.rounds == 10;
+  const bool bf = dtype == GLS_BF16;
+  if (spec == 3) {
+    const long long cap = (long long)kNumSMs * kS3CtasPerSM;
+    const int grid = (int)(P.n_items < cap ? P.n_items : cap);
+#define SWEEP3(DT, R)                                                            \
+  (lse ? sweep3_kernel<DT, true, R><<<grid, kSweepWarps3 * 32, 0, st>>>(A)       \
+       : sweep3_kernel<DT, false, R><<<grid, kSweepWarps3 * 32, 0, st>>>(A))
+    if (bf) { if (r10) SWEEP3(kBF16, 10); else SWEEP3(kBF16, 0); }
+    else { if (r10) SWEEP3(kF32, 10); else SWEEP3(kF32, 0); }
+#undef SWEEP3
+    err = cudaGetLastError();
   } else {
-    if (spec == 1) err = A.rounds == 10 ? SWEEP_CALL(kF32, 1, 10) : SWEEP_CALL(kF32, 1, 0);
-    else err = A.rounds == 10 ? SWEEP_CALL(kF32, 2, 10) : SWEEP_CALL(kF32, 2, 0);
-  }
+    const long long want = (P.n_items + kSweepThreads / 32 - 1) / (kSweepThreads / 32);
+    const int grid = (int)(want < (long long)kNumSMs * 4 ? want : (long long)kNumSMs * 4);
+#define SWEEP_CALL(...) launch_sweep_t<__VA_ARGS__>(A, lse, grid, st)
+    if (bf) {
+      if (spec == 1) err = r10 ? SWEEP_CALL(kBF16, 1, 10) : SWEEP_CALL(kBF16, 1, 0);
+      else err = r10 ? SWEEP_CALL(kBF16, 2, 10) : SWEEP_CALL(kBF16, 2, 0);
+    } else {
+      if (spec == 1) err = r10 ? SWEEP_CALL(kF32, 1, 10) : SWEEP_CALL(kF32, 1, 0);
+      else err = r10 ? SWEEP_CALL(kF32, 2, 10) : SWEEP_CALL(kF32, 2, 0);
+    }
 #undef SWEEP_CALL
+  }
   if (err != cudaSuccess) return GLS_ERR_CUDA;
 #define FIN_CALL(...) \
   launch_finalize_t<__VA_ARGS__>(A, (int)P.rows, lse, rowres, out_tokens, out_scores, status, st)
-  if (dtype == GLS_BF16) {
-    if (spec == 1) err = A.rounds == 10 ? FIN_CALL(kBF16, 1, 10) : FIN_CALL(kBF16, 1, 0);
-    else err = A.rounds == 10 ? FIN_CALL(kBF16, 2, 10) : FIN_CALL(kBF16, 2, 0);
+  if (bf) {
+    if (spec == 1) err = r10 ? FIN_CALL(kBF16, 1, 10) : FIN_CALL(kBF16, 1, 0);
+    else if (spec == 2) err = r10 ? FIN_CALL(kBF16, 2, 10) : FIN_CALL(kBF16, 2, 0);
+    else err = r10 ? FIN_CALL(kBF16, 3, 10) : FIN_CALL(kBF16, 3, 0);
   } else {
-    if (spec == 1) err = A.rounds == 10 ? FIN_CALL(kF32, 1, 10) : FIN_CALL(kF32, 1, 0);
-    else err = A.rounds == 10 ? FIN_CALL(kF32, 2, 10) : FIN_CALL(kF32, 2, 0);
+    if (spec == 1) err = r10 ? FIN_CALL(kF32, 1, 10) : FIN_CALL(kF32, 1, 0);
+    else if (spec == 2) err = r10 ? FIN_CALL(kF32, 2, 10) : FIN_CALL(kF32, 2, 0);
+    else err = r10 ? FIN_CALL(kF32, 3, 10) : FIN_CALL(kF32, 3, 0);
   }
 #undef FIN_CALL
   return err == cudaSuccess ? GLS_OK : GLS_ERR_CUDA;
@@ -320,7 +371,7 @@ static int run_rows(SweepArgs& A, int dtype, int spec, const Plan& P, void* work
 
 static bool sizes_ok(int B, int K, int J, int64_t V) {
   if (B <= 0 || K <= 0 || K > GLS_MAX_K || J <= 0 || V <= 0) return false;
-  if (V >= (1LL << 31) - 2 * kWarpTokens) return false;
+  if (V >= (1LL << 31) - 2 * kS3CtaTokens) return false;
   if ((long long)B * K * J >= (1LL << 31) / 64) return false;
   return true;
 }
@@ -350,7 +401,9 @@ const char* gls_status_string(int status) {
 
 size_t gls_workspace_bytes(int B, int K, int J, int64_t V) {
   if (!sizes_ok(B, K, J, V)) return 0;
-  return make_plan((long long)B * K * J, V).total;
+  const size_t a = make_plan12((long long)B * K * J, V).total;
+  const size_t b = make_plan3((long long)B * K * J, V).total;
+  return a > b ? a : b;
 }
 
 int gls_draft_sample(const gls_rows_t* draft_logits, int B, int K, int J, int64_t V, float inv_temp,
@@ -370,7 +423,7 @@ int gls_draft_sample(const gls_rows_t* draft_logits, int B, int K, int J, int64_
   int spec;
   rc = fill_noise(A, noise, 0u, &spec);
   if (rc != GLS_OK) return rc;
-  const Plan P = make_plan((long long)B * K * J, V);
+  const Plan P = make_plan((long long)B * K * J, V, spec);
   if (!workspace || workspace_bytes < P.total) return GLS_ERR_WORKSPACE;
   A.data = draft_logits->data;
   A.sb = draft_logits->stride_b;
@@ -406,7 +459,7 @@ int gls_target_sample_verify(const gls_rows_t* target_logits, int B, int K, int 
   int spec;
   rc = fill_noise(A, noise, 0u, &spec);
   if (rc != GLS_OK) return rc;
-  const Plan P = make_plan((long long)B * K * J, V);
+  const Plan P = make_plan((long long)B * K * J, V, spec);
   if (!workspace || workspace_bytes < P.total) return GLS_ERR_WORKSPACE;
   A.data = target_logits->data;
   A.sb = target_logits->stride_b;
@@ -446,7 +499,7 @@ int gls_compress_select(const gls_rows_t* enc_logw, const gls_rows_t* dec_logw, 
   int spec;
   rc = fill_noise(A, noise, 1u, &spec);
   if (rc != GLS_OK) return rc;
-  const Plan P = make_plan((long long)B * K, N);
+  const Plan P = make_plan((long long)B * K, N, spec);
   if (!workspace || workspace_bytes < P.total) return GLS_ERR_WORKSPACE;
   cudaStream_t st = (cudaStream_t)stream;
   const RowResult* rowres = (const RowResult*)((char*)workspace + P.off_rows);

@@ -22,6 +22,7 @@ namespace gls {
 
 constexpr int kMaxK = 64;
 constexpr int kWarpTokens = 256;  // tokens one warp consumes per iteration (8 per lane)
+constexpr int kSweepWarps3 = 8;   // warps per CTA of the noise_spec 3 sweep
 constexpr float kLog2e = 1.4426950408889634f;
 
 enum : int { kF32 = 0, kBF16 = 1 };
@@ -56,8 +57,10 @@ struct SweepArgs {
   const void* data;       // rows [B][K][J][V]
   long long sb, sk, sj;   // element strides
   int K, J, V;
-  int chunk;              // tokens per slice, a multiple of kWarpTokens
+  int chunk;              // tokens per slice
   int splits;             // slices per row
+  int parts;              // partial results per row (slices x producers per slice)
+  int rows;               // B * K * J
   long long n_items;      // rows * splits
   float inv_t[kMaxK];     // 1/T per k
   uint32_t rk[32];        // Philox round keys: rk[2r], rk[2r+1]
@@ -155,6 +158,12 @@ __device__ __forceinline__ double uniform_exact(const SweepArgs& A, const Stream
   if (SPEC == 1) {
     philox4x32<ROUNDS>(A.rk, A.rounds, (uint32_t)i >> 2, sk.c1, sk.pos, sk.seq, o);
     return ((double)o[i & 3] + 0.5) * 0x1p-32;
+  } else if (SPEC == 3) {
+    philox4x32<ROUNDS>(A.rk, A.rounds, (uint32_t)i >> 4, sk.c1, sk.pos, sk.seq, o);
+    const uint32_t h = (o[(i & 15) >> 2] >> (8 * (i & 3))) & 0xffu;
+    philox4x32<ROUNDS>(A.rk, A.rounds, (uint32_t)i >> 1, sk.c1 + (2u << 16), sk.pos, sk.seq, o);
+    const uint32_t lo = (i & 1) ? o[2] : o[0], hi = ((i & 1) ? o[3] : o[1]) & 0xffu;
+    return ((double)h * 1099511627776.0 + (double)hi * 4294967296.0 + (double)lo + 0.5) * 0x1p-48;
   } else {
     philox4x32<ROUNDS>(A.rk, A.rounds, (uint32_t)i >> 3, sk.c1, sk.pos, sk.seq, o);
     const uint32_t h = (o[(i & 7) >> 1] >> (16 * (i & 1))) & 0xffffu;

@@ -1,0 +1,455 @@
+// gls_sweep3.cuh -- the vocabulary sweep for noise_spec 3 (8 coarse + 40 refinement bits).
+//
+// One Philox4x32 call yields the coarse bytes of 16 consecutive tokens, so the generator -- whose
+// 32x32->64-bit multiplies are the scarcest resource of this path on sm_100a -- runs once per 16
+// tokens.  With m a lower bound on the row's best score, token i can only matter if
+// S_i <= exp(logit_i/T - m), and S_i = -log1p(-v_i) >= v_i >= h_i / 256 with h_i its coarse byte.
+// Hence, per group of 16 tokens:
+//   - if 2^(max logit * c - m') <= 1/256 (the usual case), only tokens with h == 0 can matter:
+//     a zero-byte test on the four generator words settles the group;
+//   - otherwise the whole group is a candidate ("wide" group; a few per row).
+// Candidate groups are not examined on the spot: the lane pushes the group (its block index and
+// the four generator words) on a small per-warp queue in shared memory and the sweep goes on.
+// When 32 groups are queued the warp evaluates them together, one group per lane: refinement
+// bits from the second generator stream, the per-token filter on the 48-bit uniform, and for the
+// survivors the fp32 score logit/T - ln(-log1p(-v)).  Batching turns what would be a divergent
+// detour in most iterations (a zero byte turns up in 1 of 16 groups) into dense work done once
+// per ~16 iterations.  The filter has no false negatives, so the result equals a full evaluation
+// (Sec. 3 step 2 / Algorithm 2 draft loop and Y_j line of arXiv 2506.05632, log domain).
+//
+// Work decomposition: a work item is one (row, vocabulary slice), owned by a CTA of 8 warps; per
+// iteration a lane takes 16 consecutive tokens (one 32-byte load of bf16, two of fp32), a warp
+// 512 and the CTA 4096 contiguous tokens.  Warps never wait on one another: they share the bound
+// m through one tagged shared-memory word, each warp writes its own partial result, and the
+// split-V reduction merges them.
+#pragma once
+#include "gls_kernels.cuh"
+
+namespace gls {
+
+constexpr int kS3LaneTokens = 16;
+constexpr int kS3WarpTokens = 32 * kS3LaneTokens;               // 512
+constexpr int kS3CtaTokens = kSweepWarps3 * kS3WarpTokens;      // 4096
+constexpr int kS3QueueCap = 64;                                 // groups per warp queue
+constexpr int kS3EntryWords = 5;                                // block | wide flag, 4 words
+
+// 32 bytes per lane in one instruction (sm_100a): a warp reads 1 KB contiguous.
+struct Words8 {
+  uint32_t w[8];
+};
+__device__ __forceinline__ Words8 ld_stream32(const void* p) {
+  Words8 v;
+  asm volatile("ld.global.nc.L1::no_allocate.v8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+               : "=r"(v.w[0]), "=r"(v.w[1]), "=r"(v.w[2]), "=r"(v.w[3]), "=r"(v.w[4]),
+                 "=r"(v.w[5]), "=r"(v.w[6]), "=r"(v.w[7])
+               : "l"(p));
+  return v;
+}
+
+// two-wide fp32 arithmetic (sm_100a)
+__device__ __forceinline__ unsigned long long pack_f32x2(float a, float b) {
+  unsigned long long r;
+  asm("mov.b64 %0, {%1,%2};" : "=l"(r) : "f"(a), "f"(b));
+  return r;
+}
+__device__ __forceinline__ void unpack_f32x2(unsigned long long r, float& a, float& b) {
+  asm("mov.b64 {%0,%1}, %2;" : "=f"(a), "=f"(b) : "l"(r));
+}
+__device__ __forceinline__ unsigned long long fma_f32x2(unsigned long long a, unsigned long long b,
+                                                        unsigned long long c) {
+  unsigned long long d;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+  return d;
+}
+__device__ __forceinline__ unsigned long long add_f32x2(unsigned long long a, unsigned long long b) {
+  unsigned long long d;
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
+
+// 16 tokens of one lane: bf16 -> 8 words (two tokens each), fp32 -> 16 words
+template <int DT>
+struct Group16;
+template <>
+struct Group16<kBF16> {
+  Words8 a;
+};
+template <>
+struct Group16<kF32> {
+  Words8 a, b;
+};
+
+__device__ __forceinline__ void load16_vec(Group16<kBF16>& g, const char* p) { g.a = ld_stream32(p); }
+__device__ __forceinline__ void load16_vec(Group16<kF32>& g, const char* p) {
+  g.a = ld_stream32(p);
+  g.b = ld_stream32(p + 32);
+}
+// scalar loader for ragged tails and rows that are not 32-byte aligned; out of range -> -inf
+__device__ __forceinline__ void load16_scalar(Group16<kBF16>& g, const char* rowp, int tok, int end) {
+#pragma unroll
+  for (int t = 0; t < 8; ++t) {
+    const uint32_t lo = tok + 2 * t < end ? (uint32_t)__ldg((const unsigned short*)rowp + tok + 2 * t) : 0xff80u;
+    const uint32_t hi = tok + 2 * t + 1 < end ? (uint32_t)__ldg((const unsigned short*)rowp + tok + 2 * t + 1) : 0xff80u;
+    g.a.w[t] = lo | (hi << 16);
+  }
+}
+__device__ __forceinline__ void load16_scalar(Group16<kF32>& g, const char* rowp, int tok, int end) {
+#pragma unroll
+  for (int t = 0; t < 8; ++t) {
+    g.a.w[t] = tok + t < end ? __float_as_uint(__ldg((const float*)rowp + tok + t)) : 0xff800000u;
+    g.b.w[t] = tok + 8 + t < end ? __float_as_uint(__ldg((const float*)rowp + tok + 8 + t)) : 0xff800000u;
+  }
+}
+
+// max over the 16 logits, ignoring NaN
+__device__ __forceinline__ float group16_max(const Group16<kBF16>& g) {
+  const uint32_t x = max_bf16x2(max_bf16x2(max_bf16x2(g.a.w[0], g.a.w[1]), max_bf16x2(g.a.w[2], g.a.w[3])),
+                                max_bf16x2(max_bf16x2(g.a.w[4], g.a.w[5]), max_bf16x2(g.a.w[6], g.a.w[7])));
+  return fmaxf(bf16_lo(x), bf16_hi(x));
+}
+__device__ __forceinline__ float group16_max(const Group16<kF32>& g) {
+  float m = -CUDART_INF_F;
+#pragma unroll
+  for (int t = 0; t < 8; ++t)
+    m = fmaxf(m, fmaxf(__uint_as_float(g.a.w[t]), __uint_as_float(g.b.w[t])));
+  return m;
+}
+// logit t (0..15) of the group, t a compile-time constant after unrolling
+template <int DT>
+__device__ __forceinline__ float group16_get(const Group16<DT>& g, int t);
+template <>
+__device__ __forceinline__ float group16_get<kBF16>(const Group16<kBF16>& g, int t) {
+  return (t & 1) ? bf16_hi(g.a.w[t >> 1]) : bf16_lo(g.a.w[t >> 1]);
+}
+template <>
+__device__ __forceinline__ float group16_get<kF32>(const Group16<kF32>& g, int t) {
+  return __uint_as_float(t < 8 ? g.a.w[t] : g.b.w[t - 8]);
+}
+
+constexpr float kS3LseFloor = -1.0e30f;  // finite stand-in for "no finite logit seen yet"
+
+// Softmax statistics of 16 logits: lm = running max, ls2 = two partial sums of 2^((a - lm) c2).
+// The fast path assumes finite-or-(-inf) logits; anything else is redone token by token.
+template <int DT>
+__device__ __forceinline__ void lse16(const Group16<DT>& g, float amax, float c2, float& lm,
+                                      unsigned long long& ls2) {
+  bool careful = false;
+  if (amax > lm) {
+    if (amax == CUDART_INF_F) {
+      careful = true;
+    } else {
+      const float r = ex2_approx((lm - amax) * c2);
+      ls2 = fma_f32x2(ls2, pack_f32x2(r, r), 0ull);
+      lm = amax;
+    }
+  }
+  if (!careful) {
+    const float nl = -lm * c2;
+    const unsigned long long c22 = pack_f32x2(c2, c2), nl2 = pack_f32x2(nl, nl);
+    unsigned long long gs2 = 0ull;
+#pragma unroll
+    for (int t = 0; t < 16; t += 2) {
+      float e0, e1;
+      unpack_f32x2(fma_f32x2(pack_f32x2(group16_get<DT>(g, t), group16_get<DT>(g, t + 1)), c22, nl2), e0, e1);
+      gs2 = add_f32x2(gs2, pack_f32x2(ex2_approx(e0), ex2_approx(e1)));
+    }
+    float s0, s1;
+    unpack_f32x2(gs2, s0, s1);
+    if (s0 + s1 <= 32.0f) ls2 = add_f32x2(ls2, gs2);
+    else careful = true;  // a NaN logit poisons the sum
+  }
+  if (careful) {
+    float vmax = -CUDART_INF_F;
+#pragma unroll
+    for (int t = 0; t < 16; ++t) {
+      const float a = group16_get<DT>(g, t);
+      if (a < CUDART_INF_F) vmax = fmaxf(vmax, a);  // false for NaN and +inf
+    }
+    if (vmax > lm) {
+      const float r = ex2_approx((lm - vmax) * c2);
+      ls2 = fma_f32x2(ls2, pack_f32x2(r, r), 0ull);
+      lm = vmax;
+    }
+    float gs = 0.f;
+#pragma unroll
+    for (int t = 0; t < 16; ++t) {
+      const float a = group16_get<DT>(g, t);
+      if (a < CUDART_INF_F) gs += ex2_approx((a - lm) * c2);
+    }
+    ls2 = add_f32x2(ls2, pack_f32x2(gs, 0.f));
+  }
+}
+
+// Any zero byte among the 16 coarse bytes?  (exact as a yes / no for the four words together)
+__device__ __forceinline__ bool any_zero_byte(const uint32_t (&w)[4]) {
+  const uint32_t z = ((w[0] - 0x01010101u) & ~w[0]) | ((w[1] - 0x01010101u) & ~w[1]) |
+                     ((w[2] - 0x01010101u) & ~w[2]) | ((w[3] - 0x01010101u) & ~w[3]);
+  return (z & 0x80808080u) != 0u;
+}
+// bit t set iff byte t of the word is zero (exact per byte)
+__device__ __forceinline__ uint32_t zero_byte_mask4(uint32_t v) {
+  const uint32_t t = ~(((v & 0x7f7f7f7fu) + 0x7f7f7f7fu) | v | 0x7f7f7f7fu);  // 0x80 per zero byte
+  return (((t >> 7) * 0x00204081u) >> 21) & 0xfu;
+}
+
+// ------------------------------------------------------------------------------------------
+// Batched evaluation of queued groups: lane l < n takes entry l.  For every candidate token of
+// its group (tokens whose coarse byte is zero, or all 16 of a wide group) the lane draws the 40
+// refinement bits, applies the per-token filter to the 48-bit uniform and scores the survivors
+// in fp32.  Returns the best lower bound found (ordered code, 0 if none).
+// ------------------------------------------------------------------------------------------
+template <int DT, int ROUNDS>
+__device__ __noinline__ uint32_t s3_flush(const SweepArgs& A, const void* row, StreamKey sk,
+                                          float inv_t, float nm, const uint8_t* bins, int msg,
+                                          int tok_end, const uint32_t* entries, int n, Top2* best) {
+  const int lane = threadIdx.x & 31;
+  const uint32_t* e = entries + lane * kS3EntryWords;
+  uint32_t msk = 0u, blk = 0u;
+  if (lane < n) {
+    blk = e[0];
+    msk = zero_byte_mask4(e[1]) | (zero_byte_mask4(e[2]) << 4) | (zero_byte_mask4(e[3]) << 8) |
+          (zero_byte_mask4(e[4]) << 12);
+    if (blk & 0x80000000u) msk = 0xffffu;
+    blk &= 0x7fffffffu;
+  }
+  Top2 b = *best;
+  float lower = -CUDART_INF_F;
+  const float c2 = inv_t * kLog2e;
+  while (__any_sync(0xffffffffu, msk != 0u)) {
+    if (msk != 0u) {
+      const int t = __ffs(msk) - 1;
+      msk &= msk - 1u;
+      const int i = (int)(blk << 4) + t;
+      if (i < tok_end) {
+        const float a = load_logit<DT>(row, i);
+        if (a < CUDART_INF_F) {  // NaN and +inf never win
+          const uint32_t h = (e[1 + (t >> 2)] >> (8 * (t & 3))) & 0xffu;
+          uint32_t f[4];
+          philox4x32<ROUNDS>(A.rk, A.rounds, (uint32_t)i >> 1, sk.c1 + (2u << 16), sk.pos, sk.seq, f);
+          const uint32_t lo = (i & 1) ? f[2] : f[0], hi = ((i & 1) ? f[3] : f[1]) & 0xffu;
+          const float v = fmaf((float)h, 0x1p-8f,
+                               fmaf((float)hi, 0x1p-16f, fmaf((float)lo, 0x1p-48f, 0x1p-49f)));
+          if (v < ex2_approx(fmaf(a, c2, nm)) &&
+              (bins == nullptr || (int)__ldg(bins + i) == msg)) {
+            float ln_s;
+            const float s = score_f32(a, inv_t, v, &ln_s);
+            top2_offer(b, s, i);
+            lower = fmaxf(lower, s - score_slack(s, ln_s));
+          }
+        }
+      }
+    }
+  }
+  *best = b;
+  __syncwarp();
+  return __reduce_max_sync(0xffffffffu, enc_ordered(lower));
+}
+
+// ------------------------------------------------------------------------------------------
+// The kernel
+// ------------------------------------------------------------------------------------------
+struct S3Shared {
+  unsigned long long m_tag;  // (item tag << 32) | ordered code of the CTA-wide bound on the best score
+  Top2 best[kSweepWarps3 * 32];  // per-thread candidates, touched by the batched path only
+  uint32_t queue[kSweepWarps3][kS3QueueCap * kS3EntryWords];
+};
+
+template <int DT, bool LSE, int ROUNDS>
+__global__ void __launch_bounds__(kSweepWarps3 * 32, 4)
+sweep3_kernel(const __grid_constant__ SweepArgs A) {
+  __shared__ S3Shared sh;
+  const int lane = threadIdx.x & 31;
+  const int warp = threadIdx.x >> 5;
+  constexpr int ES = DT == kBF16 ? 2 : 4;
+  constexpr int DEPTH = DT == kBF16 ? 2 : 1;  // groups in flight per lane
+  constexpr int STEP = kS3CtaTokens * ES;      // bytes between a lane's consecutive groups
+  typedef Group16<DT> G;
+  uint32_t* const queue = sh.queue[warp];
+  Top2* const best = &sh.best[threadIdx.x];
+  volatile unsigned long long* const m_tag = &sh.m_tag;
+
+  if (threadIdx.x == 0) sh.m_tag = 0ull;
+  __syncthreads();
+
+  uint32_t tag = 0u;
+  for (long long item = blockIdx.x; item < A.n_items; item += gridDim.x) {
+    ++tag;
+    const int split = (int)(item / A.rows);
+    const int row = (int)(item - (long long)split * A.rows);
+    const int j = row % A.J;
+    const int bk = row / A.J;
+    const int k = bk % A.K;
+    const int b = bk / A.K;
+    const char* rowp = (const char*)A.data + (b * A.sb + k * A.sk + j * A.sj) * ES;
+    StreamKey sk;
+    sk.c1 = ((uint32_t)k & A.kmask) | (A.domain << 16);
+    sk.pos = A.pos_base + (uint32_t)j;
+    sk.seq = A.seq_ids ? __ldg(A.seq_ids + b) : A.seq_base + (uint32_t)b;
+    const float inv_t = A.inv_t[k];
+    const float c2 = inv_t * kLog2e;
+    const uint8_t* bins = A.bins ? A.bins + A.bins_sb * b : nullptr;
+    const int msg = (A.bins && A.msg) ? (int)__ldg(A.msg + b) : 0;
+    const int tok_begin = split * A.chunk;
+    const int tok_end = min(A.V, tok_begin + A.chunk);
+    const bool aligned = (((uintptr_t)rowp) & 31) == 0;
+    // this warp's iterations: tokens base_w + it * kS3CtaTokens + [0, 512)
+    const int base_w = tok_begin + warp * kS3WarpTokens;
+    const int span = tok_end - base_w;
+    const int n_iter = span > 0 ? (span + kS3CtaTokens - 1) / kS3CtaTokens : 0;
+    const int n_full = (aligned && span >= kS3WarpTokens) ? (span - kS3WarpTokens) / kS3CtaTokens + 1 : 0;
+    const int tok0 = base_w + lane * kS3LaneTokens;
+
+    uint32_t m_enc = __ldcg(A.hints + row);  // bound published by earlier slices of the row
+    top2_init(*best);
+    float lm = kS3LseFloor;
+    unsigned long long ls2 = 0ull;
+    int qn = 0;
+
+    // ---- warm start: a valid lower bound from the coarse bytes of the lane's first group -----
+    // v < (h + 1) / 256  =>  S = -log1p(-v) < x / (1 - x), x = (h + 1) / 256, so the token's score
+    // exceeds logit/T - ln(x / (1 - x)).  Each lane takes the best such bound over its 16 tokens.
+    if (n_iter > 0) {
+      G g;
+      if (n_full > 0) load16_vec(g, rowp + (size_t)tok0 * ES);
+      else load16_scalar(g, rowp, tok0, tok_end);
+      uint32_t cw[4];
+      philox4x32<ROUNDS>(A.rk, A.rounds, (uint32_t)tok0 >> 4, sk.c1, sk.pos, sk.seq, cw);
+      float lb2 = -CUDART_INF_F;  // log2 units
+      int tb = 0;
+#pragma unroll
+      for (int t = 0; t < 16; ++t) {
+        const float a = group16_get<DT>(g, t);
+        const uint32_t h = (cw[t >> 2] >> (8 * (t & 3))) & 0xffu;
+        float key;
+        asm("lg2.approx.ftz.f32 %0, %1;" : "=f"(key) : "f"((float)(255u - h) / (float)(h + 1u)));
+        key = fmaf(a, c2, key);  // log2 of exp(logit/T) (1 - x) / x
+        if (h < 255u && a < CUDART_INF_F && key > lb2) {
+          lb2 = key;
+          tb = t;
+        }
+      }
+      float lb = -CUDART_INF_F;
+      if (lb2 > -CUDART_INF_F && tok0 + tb < tok_end &&
+          (bins == nullptr || (int)__ldg(bins + tok0 + tb) == msg)) {
+        lb = lb2 * 0.6931471805599453f;
+        // lg2.approx, the division and the roundings are good to ~1e-6 relative of |lb2| + 8
+        lb -= 0x1p-16f * (16.0f + fabsf(lb));
+      }
+      const uint32_t e = __reduce_max_sync(0xffffffffu, enc_ordered(lb));
+      if (e > m_enc) m_enc = e;
+      if (lane == 0 && m_enc > 0u)
+        atomicMax((unsigned long long*)&sh.m_tag, ((unsigned long long)tag << 32) | m_enc);
+    }
+    float nm = filter_offset(dec_ordered(m_enc));
+    float nm8 = nm + 8.0f;
+
+    // one group of 16 tokens per lane
+    auto process = [&](const G& g, int tok) {
+      uint32_t cw[4];
+      philox4x32<ROUNDS>(A.rk, A.rounds, (uint32_t)tok >> 4, sk.c1, sk.pos, sk.seq, cw);
+      const float amax = group16_max(g);
+      const bool wide = fmaf(amax, c2, nm8) > 0.f;  // 2^(amax c + nm) > 1/256: any byte may matter
+      const bool pass = any_zero_byte(cw) | wide;
+      if (LSE) lse16<DT>(g, amax, c2, lm, ls2);
+      const unsigned long long mt = *m_tag;  // bound published by the other warps of the CTA
+      uint32_t m_new = ((uint32_t)(mt >> 32) == tag) ? (uint32_t)mt : 0u;
+      const unsigned bal = __ballot_sync(0xffffffffu, pass);
+      if (bal != 0u) {
+        if (pass) {
+          uint32_t* e = queue + (qn + __popc(bal & ((1u << lane) - 1u))) * kS3EntryWords;
+          e[0] = ((uint32_t)tok >> 4) | (wide ? 0x80000000u : 0u);
+          e[1] = cw[0]; e[2] = cw[1]; e[3] = cw[2]; e[4] = cw[3];
+        }
+        qn += __popc(bal);
+        if (qn >= 32) {
+          __syncwarp();
+          qn -= 32;
+          const uint32_t e = s3_flush<DT, ROUNDS>(A, rowp, sk, inv_t, nm, bins, msg, tok_end,
+                                                  queue + qn * kS3EntryWords, 32, best);
+          if (e > m_new) {
+            m_new = e;
+            if (lane == 0)
+              atomicMax((unsigned long long*)&sh.m_tag, ((unsigned long long)tag << 32) | e);
+          }
+        }
+      }
+      if (m_new > m_enc) {
+        m_enc = m_new;
+        nm = filter_offset(dec_ordered(m_enc));
+        nm8 = nm + 8.0f;
+      }
+    };
+
+    // ---- full iterations: DEPTH vector loads in flight per lane --------------------------------
+    {
+      const char* p = rowp + (size_t)tok0 * ES;
+      int tok = tok0;
+      const int nd = n_full / DEPTH * DEPTH;
+      if (nd >= DEPTH) {
+        G buf[DEPTH];
+#pragma unroll
+        for (int d = 0; d < DEPTH; ++d) load16_vec(buf[d], p + (size_t)d * STEP);
+        p += (size_t)DEPTH * STEP;
+        for (int it = DEPTH; it < nd; it += DEPTH) {
+#pragma unroll
+          for (int d = 0; d < DEPTH; ++d) {
+            const G g = buf[d];
+            load16_vec(buf[d], p + (size_t)d * STEP);
+            process(g, tok + d * kS3CtaTokens);
+          }
+          p += (size_t)DEPTH * STEP;
+          tok += DEPTH * kS3CtaTokens;
+        }
+#pragma unroll
+        for (int d = 0; d < DEPTH; ++d) process(buf[d], tok + d * kS3CtaTokens);
+        tok += DEPTH * kS3CtaTokens;
+      }
+      for (int it = nd; it < n_full; ++it) {
+        G g;
+        load16_vec(g, p);
+        process(g, tok);
+        p += STEP;
+        tok += kS3CtaTokens;
+      }
+      // ---- ragged tail and rows that are not 32-byte aligned ---------------------------------
+      for (int it = n_full; it < n_iter; ++it) {
+        G g;
+        load16_scalar(g, rowp, tok, tok_end);
+        process(g, tok);
+        tok += kS3CtaTokens;
+      }
+    }
+    // ---- drain the queue ---------------------------------------------------------------------
+    if (qn > 0) {
+      __syncwarp();
+      const uint32_t e = s3_flush<DT, ROUNDS>(A, rowp, sk, inv_t, nm, bins, msg, tok_end, queue, qn, best);
+      if (e > m_enc) m_enc = e;
+      qn = 0;
+    }
+
+    // ---- combine the lanes; every warp writes its own partial result ---------------------------
+    Top2 t2 = *best;
+    top2_warp_merge(t2);
+    float ls = 0.f;
+    if (LSE) {
+      float s0, s1;
+      unpack_f32x2(ls2, s0, s1);
+      float wm = lm;
+#pragma unroll
+      for (int d = 16; d > 0; d >>= 1) wm = fmaxf(wm, __shfl_xor_sync(0xffffffffu, wm, d));
+      ls = (s0 + s1) * ex2_approx((lm - wm) * c2);
+#pragma unroll
+      for (int d = 16; d > 0; d >>= 1) ls += __shfl_xor_sync(0xffffffffu, ls, d);
+      lm = wm;
+    }
+    if (lane == 0) {
+      Partial p;
+      p.s1 = t2.s1; p.i1 = t2.i1; p.s2 = t2.s2; p.i2 = t2.i2;
+      p.lm = lm; p.ls = ls; p.pad0 = 0; p.pad1 = 0;
+      A.partials[((long long)row * A.splits + split) * kSweepWarps3 + warp] = p;
+      if (A.splits > 1 && m_enc > 0u) atomicMax(A.hints + row, m_enc);
+    }
+  }
+}
+
+}  // namespace gls
