@@ -56,18 +56,25 @@ static Plan make_plan12(long long rows, long long V) {
   return p;
 }
 
-// noise_spec 3 (a CTA per work item, one partial per warp).  Whole rows when there are enough of
-// them to keep the static round-robin over the resident CTAs balanced (16 items per CTA),
-// otherwise the fewest slices that reach that count, never shorter than kS3MinChunk tokens.
-constexpr int kS3CtasPerSM = 4;
+// noise_spec 3 (a CTA per work item, one partial per warp).  Every item costs a fixed set-up and
+// merge, so rows are cut into as few slices as keep the static round-robin over the resident
+// CTAs balanced: the fewest slices for which the last round of items wastes at most 6 % of the
+// machine, or that give every CTA at least 12 items.  Slices are whole CTA iterations and at
+// least kS3MinChunk tokens long, except that small problems may go down to one CTA iteration.
+constexpr int kS3CtasPerSM = GLS_S3_MIN_CTAS;
 constexpr int kS3MinChunk = 4 * kS3CtaTokens;
 static Plan make_plan3(long long rows, long long V) {
   Plan p;
-  const long long target_items = 16LL * kNumSMs * kS3CtasPerSM;
-  long long splits = (target_items + rows - 1) / rows;
-  const long long max_splits = (V + kS3MinChunk - 1) / kS3MinChunk;
-  if (splits > max_splits) splits = max_splits;
-  if (splits < 1) splits = 1;
+  const long long grid = (long long)kNumSMs * kS3CtasPerSM;
+  long long max_splits = (V + kS3MinChunk - 1) / kS3MinChunk;
+  if (rows * max_splits < 2 * grid) max_splits = (V + kS3CtaTokens - 1) / kS3CtaTokens;
+  long long splits = 1;
+  for (; splits < max_splits; ++splits) {
+    const long long items = rows * splits;
+    if (items >= 12 * grid) break;
+    const long long rounds = (items + grid - 1) / grid;
+    if (items >= grid && (double)(rounds * grid - items) <= 0.06 * (double)(rounds * grid)) break;
+  }
   long long chunk = (V + splits - 1) / splits;
   chunk = (chunk + kS3CtaTokens - 1) / kS3CtaTokens * kS3CtaTokens;
   p.chunk = (int)chunk;
@@ -334,8 +341,8 @@ static int run_rows(SweepArgs& A, int dtype, int spec, const Plan& P, void* work
     const long long cap = (long long)kNumSMs * kS3CtasPerSM;
     const int grid = (int)(P.n_items < cap ? P.n_items : cap);
 #define SWEEP3(DT, R)                                                            \
-  (lse ? sweep3_kernel<DT, true, R><<<grid, kSweepWarps3 * 32, 0, st>>>(A)       \
-       : sweep3_kernel<DT, false, R><<<grid, kSweepWarps3 * 32, 0, st>>>(A))
+  (lse ? sweep3_kernel<DT, true, R><<<grid, kSweepWarps3 * 32, sizeof(S3Shared), st>>>(A)  \
+       : sweep3_kernel<DT, false, R><<<grid, kSweepWarps3 * 32, sizeof(S3Shared), st>>>(A))
     if (bf) { if (r10) SWEEP3(kBF16, 10); else SWEEP3(kBF16, 0); }
     else { if (r10) SWEEP3(kF32, 10); else SWEEP3(kF32, 0); }
 #undef SWEEP3

@@ -25,6 +25,10 @@
 #pragma once
 #include "gls_kernels.cuh"
 
+#ifndef GLS_S3_MIN_CTAS
+#define GLS_S3_MIN_CTAS 4
+#endif
+
 namespace gls {
 
 constexpr int kS3LaneTokens = 16;
@@ -44,6 +48,12 @@ __device__ __forceinline__ Words8 ld_stream32(const void* p) {
                  "=r"(v.w[5]), "=r"(v.w[6]), "=r"(v.w[7])
                : "l"(p));
   return v;
+}
+
+__device__ __forceinline__ float lg2_approx(float x) {
+  float y;
+  asm("lg2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
 }
 
 // two-wide fp32 arithmetic (sm_100a)
@@ -193,46 +203,81 @@ __device__ __forceinline__ uint32_t zero_byte_mask4(uint32_t v) {
 }
 
 // ------------------------------------------------------------------------------------------
-// Batched evaluation of queued groups: lane l < n takes entry l.  For every candidate token of
-// its group (tokens whose coarse byte is zero, or all 16 of a wide group) the lane draws the 40
-// refinement bits, applies the per-token filter to the 48-bit uniform and scores the survivors
+// Shared memory of the sweep CTA (dynamic, so that the batched path below can reach it too)
+// ------------------------------------------------------------------------------------------
+struct S3WarpCtx {  // what the batched path needs to know about the warp's current work item
+  const char* rowp;
+  const uint8_t* bins;
+  uint32_t c1, pos, seq;
+  float inv_t;
+  int msg, tok_end;
+};
+struct S3Shared {
+  unsigned long long m_tag;  // (item tag << 32) | ordered code of the CTA-wide bound on the best score
+  S3WarpCtx ctx[kSweepWarps3];
+  Top2 best[kSweepWarps3 * 32];  // per-thread candidates, touched by the batched path only
+  uint32_t queue[kSweepWarps3][kS3QueueCap * kS3EntryWords];
+};
+extern __shared__ __align__(16) unsigned char s3_smem_raw[];
+__device__ __forceinline__ S3Shared& s3_shared() { return *reinterpret_cast<S3Shared*>(s3_smem_raw); }
+
+// ------------------------------------------------------------------------------------------
+// Batched evaluation of queued groups: lane l < n takes entry first + l of its warp's queue.
+// Candidate tokens of a group: those whose coarse byte is zero; in a wide group, those whose
+// coarse byte passes the per-token test h < 256 * 2^(logit c + nm).  For every candidate the lane
+// draws the 40 refinement bits, applies the filter to the 48-bit uniform and scores the survivors
 // in fp32.  Returns the best lower bound found (ordered code, 0 if none).
 // ------------------------------------------------------------------------------------------
 template <int DT, int ROUNDS>
-__device__ __noinline__ uint32_t s3_flush(const SweepArgs& A, const void* row, StreamKey sk,
-                                          float inv_t, float nm, const uint8_t* bins, int msg,
-                                          int tok_end, const uint32_t* entries, int n, Top2* best) {
+__device__ __noinline__ uint32_t s3_flush(const SweepArgs& A, int first, int n, float nm) {
+  S3Shared& sh = s3_shared();
   const int lane = threadIdx.x & 31;
-  const uint32_t* e = entries + lane * kS3EntryWords;
+  const int warp = threadIdx.x >> 5;
+  const S3WarpCtx cx = sh.ctx[warp];
+  const uint32_t* e = sh.queue[warp] + (first + lane) * kS3EntryWords;
+  const float c2 = cx.inv_t * kLog2e;
   uint32_t msk = 0u, blk = 0u;
+  uint32_t w0 = 0u, w1 = 0u, w2 = 0u, w3 = 0u;
   if (lane < n) {
     blk = e[0];
-    msk = zero_byte_mask4(e[1]) | (zero_byte_mask4(e[2]) << 4) | (zero_byte_mask4(e[3]) << 8) |
-          (zero_byte_mask4(e[4]) << 12);
-    if (blk & 0x80000000u) msk = 0xffffu;
-    blk &= 0x7fffffffu;
+    w0 = e[1]; w1 = e[2]; w2 = e[3]; w3 = e[4];
+    if (blk & 0x80000000u) {
+      blk &= 0x7fffffffu;
+      Group16<DT> g;
+      load16_scalar(g, cx.rowp, (int)(blk << 4), cx.tok_end);
+      const float nm8 = nm + 8.0f;
+#pragma unroll
+      for (int t = 0; t < 16; ++t) {
+        const uint32_t wt = t < 4 ? w0 : t < 8 ? w1 : t < 12 ? w2 : w3;
+        const float h = (float)((wt >> (8 * (t & 3))) & 0xffu);
+        if (h < ex2_approx(fmaf(group16_get<DT>(g, t), c2, nm8))) msk |= 1u << t;  // false for NaN
+      }
+    } else {
+      msk = zero_byte_mask4(w0) | (zero_byte_mask4(w1) << 4) | (zero_byte_mask4(w2) << 8) |
+            (zero_byte_mask4(w3) << 12);
+    }
   }
-  Top2 b = *best;
+  Top2 b = sh.best[threadIdx.x];
   float lower = -CUDART_INF_F;
-  const float c2 = inv_t * kLog2e;
   while (__any_sync(0xffffffffu, msk != 0u)) {
     if (msk != 0u) {
       const int t = __ffs(msk) - 1;
       msk &= msk - 1u;
       const int i = (int)(blk << 4) + t;
-      if (i < tok_end) {
-        const float a = load_logit<DT>(row, i);
+      if (i < cx.tok_end) {
+        const float a = load_logit<DT>(cx.rowp, i);
         if (a < CUDART_INF_F) {  // NaN and +inf never win
-          const uint32_t h = (e[1 + (t >> 2)] >> (8 * (t & 3))) & 0xffu;
+          const uint32_t wt = t < 4 ? w0 : t < 8 ? w1 : t < 12 ? w2 : w3;
+          const uint32_t h = (wt >> (8 * (t & 3))) & 0xffu;
           uint32_t f[4];
-          philox4x32<ROUNDS>(A.rk, A.rounds, (uint32_t)i >> 1, sk.c1 + (2u << 16), sk.pos, sk.seq, f);
+          philox4x32<ROUNDS>(A.rk, A.rounds, (uint32_t)i >> 1, cx.c1 + (2u << 16), cx.pos, cx.seq, f);
           const uint32_t lo = (i & 1) ? f[2] : f[0], hi = ((i & 1) ? f[3] : f[1]) & 0xffu;
           const float v = fmaf((float)h, 0x1p-8f,
                                fmaf((float)hi, 0x1p-16f, fmaf((float)lo, 0x1p-48f, 0x1p-49f)));
           if (v < ex2_approx(fmaf(a, c2, nm)) &&
-              (bins == nullptr || (int)__ldg(bins + i) == msg)) {
+              (cx.bins == nullptr || (int)__ldg(cx.bins + i) == cx.msg)) {
             float ln_s;
-            const float s = score_f32(a, inv_t, v, &ln_s);
+            const float s = score_f32(a, cx.inv_t, v, &ln_s);
             top2_offer(b, s, i);
             lower = fmaxf(lower, s - score_slack(s, ln_s));
           }
@@ -240,7 +285,7 @@ __device__ __noinline__ uint32_t s3_flush(const SweepArgs& A, const void* row, S
       }
     }
   }
-  *best = b;
+  sh.best[threadIdx.x] = b;
   __syncwarp();
   return __reduce_max_sync(0xffffffffu, enc_ordered(lower));
 }
@@ -248,24 +293,17 @@ __device__ __noinline__ uint32_t s3_flush(const SweepArgs& A, const void* row, S
 // ------------------------------------------------------------------------------------------
 // The kernel
 // ------------------------------------------------------------------------------------------
-struct S3Shared {
-  unsigned long long m_tag;  // (item tag << 32) | ordered code of the CTA-wide bound on the best score
-  Top2 best[kSweepWarps3 * 32];  // per-thread candidates, touched by the batched path only
-  uint32_t queue[kSweepWarps3][kS3QueueCap * kS3EntryWords];
-};
-
 template <int DT, bool LSE, int ROUNDS>
-__global__ void __launch_bounds__(kSweepWarps3 * 32, 4)
+__global__ void __launch_bounds__(kSweepWarps3 * 32, GLS_S3_MIN_CTAS)
 sweep3_kernel(const __grid_constant__ SweepArgs A) {
-  __shared__ S3Shared sh;
+  S3Shared& sh = s3_shared();
   const int lane = threadIdx.x & 31;
   const int warp = threadIdx.x >> 5;
   constexpr int ES = DT == kBF16 ? 2 : 4;
-  constexpr int DEPTH = DT == kBF16 ? 2 : 1;  // groups in flight per lane
+  constexpr bool PREFETCH = DT == kBF16;       // fp32 groups are 16 registers: no second copy
   constexpr int STEP = kS3CtaTokens * ES;      // bytes between a lane's consecutive groups
   typedef Group16<DT> G;
   uint32_t* const queue = sh.queue[warp];
-  Top2* const best = &sh.best[threadIdx.x];
   volatile unsigned long long* const m_tag = &sh.m_tag;
 
   if (threadIdx.x == 0) sh.m_tag = 0ull;
@@ -276,21 +314,36 @@ sweep3_kernel(const __grid_constant__ SweepArgs A) {
     ++tag;
     const int split = (int)(item / A.rows);
     const int row = (int)(item - (long long)split * A.rows);
-    const int j = row % A.J;
-    const int bk = row / A.J;
-    const int k = bk % A.K;
-    const int b = bk / A.K;
-    const char* rowp = (const char*)A.data + (b * A.sb + k * A.sk + j * A.sj) * ES;
-    StreamKey sk;
-    sk.c1 = ((uint32_t)k & A.kmask) | (A.domain << 16);
-    sk.pos = A.pos_base + (uint32_t)j;
-    sk.seq = A.seq_ids ? __ldg(A.seq_ids + b) : A.seq_base + (uint32_t)b;
-    const float inv_t = A.inv_t[k];
-    const float c2 = inv_t * kLog2e;
-    const uint8_t* bins = A.bins ? A.bins + A.bins_sb * b : nullptr;
-    const int msg = (A.bins && A.msg) ? (int)__ldg(A.msg + b) : 0;
     const int tok_begin = split * A.chunk;
     const int tok_end = min(A.V, tok_begin + A.chunk);
+    uint32_t c1, pos, seq;
+    const char* rowp;
+    float c2;
+    {
+      const int j = row % A.J;
+      const int bk = row / A.J;
+      const int k = bk % A.K;
+      const int b = bk / A.K;
+      rowp = (const char*)A.data + (b * A.sb + k * A.sk + j * A.sj) * ES;
+      c1 = ((uint32_t)k & A.kmask) | (A.domain << 16);
+      pos = A.pos_base + (uint32_t)j;
+      seq = A.seq_ids ? __ldg(A.seq_ids + b) : A.seq_base + (uint32_t)b;
+      const float inv_t = A.inv_t[k];
+      c2 = inv_t * kLog2e;
+      __syncwarp();  // the previous item's batched path is done with the context
+      if (lane == 0) {
+        S3WarpCtx cx;
+        cx.rowp = rowp;
+        cx.bins = A.bins ? A.bins + A.bins_sb * b : nullptr;
+        cx.c1 = c1; cx.pos = pos; cx.seq = seq;
+        cx.inv_t = inv_t;
+        cx.msg = (A.bins && A.msg) ? (int)__ldg(A.msg + b) : 0;
+        cx.tok_end = tok_end;
+        sh.ctx[warp] = cx;
+      }
+      top2_init(sh.best[threadIdx.x]);
+      __syncwarp();
+    }
     const bool aligned = (((uintptr_t)rowp) & 31) == 0;
     // this warp's iterations: tokens base_w + it * kS3CtaTokens + [0, 512)
     const int base_w = tok_begin + warp * kS3WarpTokens;
@@ -300,7 +353,6 @@ sweep3_kernel(const __grid_constant__ SweepArgs A) {
     const int tok0 = base_w + lane * kS3LaneTokens;
 
     uint32_t m_enc = __ldcg(A.hints + row);  // bound published by earlier slices of the row
-    top2_init(*best);
     float lm = kS3LseFloor;
     unsigned long long ls2 = 0ull;
     int qn = 0;
@@ -313,26 +365,26 @@ sweep3_kernel(const __grid_constant__ SweepArgs A) {
       if (n_full > 0) load16_vec(g, rowp + (size_t)tok0 * ES);
       else load16_scalar(g, rowp, tok0, tok_end);
       uint32_t cw[4];
-      philox4x32<ROUNDS>(A.rk, A.rounds, (uint32_t)tok0 >> 4, sk.c1, sk.pos, sk.seq, cw);
+      philox4x32<ROUNDS>(A.rk, A.rounds, (uint32_t)tok0 >> 4, c1, pos, seq, cw);
       float lb2 = -CUDART_INF_F;  // log2 units
       int tb = 0;
 #pragma unroll
       for (int t = 0; t < 16; ++t) {
         const float a = group16_get<DT>(g, t);
         const uint32_t h = (cw[t >> 2] >> (8 * (t & 3))) & 0xffu;
-        float key;
-        asm("lg2.approx.ftz.f32 %0, %1;" : "=f"(key) : "f"((float)(255u - h) / (float)(h + 1u)));
-        key = fmaf(a, c2, key);  // log2 of exp(logit/T) (1 - x) / x
+        // log2 of exp(logit/T) (1 - x) / x
+        const float key = fmaf(a, c2, lg2_approx((float)(255u - h)) - lg2_approx((float)(h + 1u)));
         if (h < 255u && a < CUDART_INF_F && key > lb2) {
           lb2 = key;
           tb = t;
         }
       }
       float lb = -CUDART_INF_F;
+      const S3WarpCtx& cx = sh.ctx[warp];
       if (lb2 > -CUDART_INF_F && tok0 + tb < tok_end &&
-          (bins == nullptr || (int)__ldg(bins + tok0 + tb) == msg)) {
+          (cx.bins == nullptr || (int)__ldg(cx.bins + tok0 + tb) == cx.msg)) {
         lb = lb2 * 0.6931471805599453f;
-        // lg2.approx, the division and the roundings are good to ~1e-6 relative of |lb2| + 8
+        // lg2.approx and the roundings are good to ~1e-6 relative of |lb2| + 8
         lb -= 0x1p-16f * (16.0f + fabsf(lb));
       }
       const uint32_t e = __reduce_max_sync(0xffffffffu, enc_ordered(lb));
@@ -340,13 +392,12 @@ sweep3_kernel(const __grid_constant__ SweepArgs A) {
       if (lane == 0 && m_enc > 0u)
         atomicMax((unsigned long long*)&sh.m_tag, ((unsigned long long)tag << 32) | m_enc);
     }
-    float nm = filter_offset(dec_ordered(m_enc));
-    float nm8 = nm + 8.0f;
+    float nm8 = filter_offset(dec_ordered(m_enc)) + 8.0f;
 
     // one group of 16 tokens per lane
     auto process = [&](const G& g, int tok) {
       uint32_t cw[4];
-      philox4x32<ROUNDS>(A.rk, A.rounds, (uint32_t)tok >> 4, sk.c1, sk.pos, sk.seq, cw);
+      philox4x32<ROUNDS>(A.rk, A.rounds, (uint32_t)tok >> 4, c1, pos, seq, cw);
       const float amax = group16_max(g);
       const bool wide = fmaf(amax, c2, nm8) > 0.f;  // 2^(amax c + nm) > 1/256: any byte may matter
       const bool pass = any_zero_byte(cw) | wide;
@@ -364,8 +415,7 @@ sweep3_kernel(const __grid_constant__ SweepArgs A) {
         if (qn >= 32) {
           __syncwarp();
           qn -= 32;
-          const uint32_t e = s3_flush<DT, ROUNDS>(A, rowp, sk, inv_t, nm, bins, msg, tok_end,
-                                                  queue + qn * kS3EntryWords, 32, best);
+          const uint32_t e = s3_flush<DT, ROUNDS>(A, qn, 32, nm8 - 8.0f);
           if (e > m_new) {
             m_new = e;
             if (lane == 0)
@@ -375,60 +425,45 @@ sweep3_kernel(const __grid_constant__ SweepArgs A) {
       }
       if (m_new > m_enc) {
         m_enc = m_new;
-        nm = filter_offset(dec_ordered(m_enc));
-        nm8 = nm + 8.0f;
+        nm8 = filter_offset(dec_ordered(m_enc)) + 8.0f;
       }
     };
 
-    // ---- full iterations: DEPTH vector loads in flight per lane --------------------------------
+    // ---- the sweep: one call site for full (vector) and ragged (scalar) iterations; with
+    //      PREFETCH the next group's load is issued before the current one is used
     {
       const char* p = rowp + (size_t)tok0 * ES;
       int tok = tok0;
-      const int nd = n_full / DEPTH * DEPTH;
-      if (nd >= DEPTH) {
-        G buf[DEPTH];
-#pragma unroll
-        for (int d = 0; d < DEPTH; ++d) load16_vec(buf[d], p + (size_t)d * STEP);
-        p += (size_t)DEPTH * STEP;
-        for (int it = DEPTH; it < nd; it += DEPTH) {
-#pragma unroll
-          for (int d = 0; d < DEPTH; ++d) {
-            const G g = buf[d];
-            load16_vec(buf[d], p + (size_t)d * STEP);
-            process(g, tok + d * kS3CtaTokens);
-          }
-          p += (size_t)DEPTH * STEP;
-          tok += DEPTH * kS3CtaTokens;
-        }
-#pragma unroll
-        for (int d = 0; d < DEPTH; ++d) process(buf[d], tok + d * kS3CtaTokens);
-        tok += DEPTH * kS3CtaTokens;
-      }
-      for (int it = nd; it < n_full; ++it) {
+      G nxt;
+      if (PREFETCH && n_full > 0) load16_vec(nxt, p);
+#pragma unroll 1
+      for (int it = 0; it < n_iter; ++it) {
         G g;
-        load16_vec(g, p);
+        if (it < n_full) {
+          if (PREFETCH) {
+            g = nxt;
+            if (it + 1 < n_full) load16_vec(nxt, p + STEP);
+          } else {
+            load16_vec(g, p);
+          }
+        } else {
+          load16_scalar(g, rowp, tok, tok_end);
+        }
         process(g, tok);
         p += STEP;
-        tok += kS3CtaTokens;
-      }
-      // ---- ragged tail and rows that are not 32-byte aligned ---------------------------------
-      for (int it = n_full; it < n_iter; ++it) {
-        G g;
-        load16_scalar(g, rowp, tok, tok_end);
-        process(g, tok);
         tok += kS3CtaTokens;
       }
     }
     // ---- drain the queue ---------------------------------------------------------------------
     if (qn > 0) {
       __syncwarp();
-      const uint32_t e = s3_flush<DT, ROUNDS>(A, rowp, sk, inv_t, nm, bins, msg, tok_end, queue, qn, best);
+      const uint32_t e = s3_flush<DT, ROUNDS>(A, 0, qn, nm8 - 8.0f);
       if (e > m_enc) m_enc = e;
       qn = 0;
     }
 
     // ---- combine the lanes; every warp writes its own partial result ---------------------------
-    Top2 t2 = *best;
+    Top2 t2 = sh.best[threadIdx.x];
     top2_warp_merge(t2);
     float ls = 0.f;
     if (LSE) {
@@ -443,10 +478,10 @@ sweep3_kernel(const __grid_constant__ SweepArgs A) {
       lm = wm;
     }
     if (lane == 0) {
-      Partial p;
-      p.s1 = t2.s1; p.i1 = t2.i1; p.s2 = t2.s2; p.i2 = t2.i2;
-      p.lm = lm; p.ls = ls; p.pad0 = 0; p.pad1 = 0;
-      A.partials[((long long)row * A.splits + split) * kSweepWarps3 + warp] = p;
+      Partial pr;
+      pr.s1 = t2.s1; pr.i1 = t2.i1; pr.s2 = t2.s2; pr.i2 = t2.i2;
+      pr.lm = lm; pr.ls = ls; pr.pad0 = 0; pr.pad1 = 0;
+      A.partials[((long long)row * A.splits + split) * kSweepWarps3 + warp] = pr;
       if (A.splits > 1 && m_enc > 0u) atomicMax(A.hints + row, m_enc);
     }
   }
