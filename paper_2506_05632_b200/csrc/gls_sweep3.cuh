@@ -139,54 +139,62 @@ __device__ __forceinline__ float group16_get<kF32>(const Group16<kF32>& g, int t
 constexpr float kS3LseFloor = -1.0e30f;  // finite stand-in for "no finite logit seen yet"
 
 // Softmax statistics of 16 logits: lm = running max, ls2 = two partial sums of 2^((a - lm) c2).
-// The fast path assumes finite-or-(-inf) logits; anything else is redone token by token.
+// The fast path assumes finite-or-(-inf) logits; a group holding NaN or +inf is redone token by
+// token by lse16_careful (out of line: inlined, its 16 extra ex2 were issued for every group),
+// which returns the group's maximum over admissible logits and its sum relative to
+// max(lm, that maximum).
+struct LseFix {
+  float vmax, gs;
+};
+template <int DT>
+__device__ __noinline__ LseFix lse16_careful(Group16<DT> g, float c2, float lm) {
+  LseFix r;
+  r.vmax = -CUDART_INF_F;
+#pragma unroll
+  for (int t = 0; t < 16; ++t) {
+    const float a = group16_get<DT>(g, t);
+    if (a < CUDART_INF_F) r.vmax = fmaxf(r.vmax, a);  // false for NaN and +inf
+  }
+  const float ref = fmaxf(lm, r.vmax);
+  r.gs = 0.f;
+#pragma unroll
+  for (int t = 0; t < 16; ++t) {
+    const float a = group16_get<DT>(g, t);
+    if (a < CUDART_INF_F) r.gs += ex2_approx((a - ref) * c2);
+  }
+  return r;
+}
+
 template <int DT>
 __device__ __forceinline__ void lse16(const Group16<DT>& g, float amax, float c2, float& lm,
                                       unsigned long long& ls2) {
-  bool careful = false;
-  if (amax > lm) {
-    if (amax == CUDART_INF_F) {
-      careful = true;
-    } else {
-      const float r = ex2_approx((lm - amax) * c2);
-      ls2 = fma_f32x2(ls2, pack_f32x2(r, r), 0ull);
-      lm = amax;
-    }
+  // admissible maximum of the group: amax unless it is +inf (NaN never reaches amax)
+  if (amax > lm && amax < CUDART_INF_F) {
+    const float r = ex2_approx((lm - amax) * c2);
+    ls2 = fma_f32x2(ls2, pack_f32x2(r, r), 0ull);
+    lm = amax;
   }
-  if (!careful) {
-    const float nl = -lm * c2;
-    const unsigned long long c22 = pack_f32x2(c2, c2), nl2 = pack_f32x2(nl, nl);
-    unsigned long long gs2 = 0ull;
+  const float nl = -lm * c2;
+  const unsigned long long c22 = pack_f32x2(c2, c2), nl2 = pack_f32x2(nl, nl);
+  unsigned long long gs2 = 0ull;
 #pragma unroll
-    for (int t = 0; t < 16; t += 2) {
-      float e0, e1;
-      unpack_f32x2(fma_f32x2(pack_f32x2(group16_get<DT>(g, t), group16_get<DT>(g, t + 1)), c22, nl2), e0, e1);
-      gs2 = add_f32x2(gs2, pack_f32x2(ex2_approx(e0), ex2_approx(e1)));
-    }
-    float s0, s1;
-    unpack_f32x2(gs2, s0, s1);
-    if (s0 + s1 <= 32.0f) ls2 = add_f32x2(ls2, gs2);
-    else careful = true;  // a NaN logit poisons the sum
+  for (int t = 0; t < 16; t += 2) {
+    float e0, e1;
+    unpack_f32x2(fma_f32x2(pack_f32x2(group16_get<DT>(g, t), group16_get<DT>(g, t + 1)), c22, nl2), e0, e1);
+    gs2 = add_f32x2(gs2, pack_f32x2(ex2_approx(e0), ex2_approx(e1)));
   }
-  if (careful) {
-    float vmax = -CUDART_INF_F;
-#pragma unroll
-    for (int t = 0; t < 16; ++t) {
-      const float a = group16_get<DT>(g, t);
-      if (a < CUDART_INF_F) vmax = fmaxf(vmax, a);  // false for NaN and +inf
-    }
-    if (vmax > lm) {
-      const float r = ex2_approx((lm - vmax) * c2);
+  float s0, s1;
+  unpack_f32x2(gs2, s0, s1);
+  if (s0 + s1 <= 32.0f) {  // every term is at most 1 unless a NaN or +inf logit poisoned the sum
+    ls2 = add_f32x2(ls2, gs2);
+  } else {
+    const LseFix f = lse16_careful<DT>(g, c2, lm);
+    if (f.vmax > lm) {
+      const float r = ex2_approx((lm - f.vmax) * c2);
       ls2 = fma_f32x2(ls2, pack_f32x2(r, r), 0ull);
-      lm = vmax;
+      lm = f.vmax;
     }
-    float gs = 0.f;
-#pragma unroll
-    for (int t = 0; t < 16; ++t) {
-      const float a = group16_get<DT>(g, t);
-      if (a < CUDART_INF_F) gs += ex2_approx((a - lm) * c2);
-    }
-    ls2 = add_f32x2(ls2, pack_f32x2(gs, 0.f));
+    ls2 = add_f32x2(ls2, pack_f32x2(f.gs, 0.f));
   }
 }
 
@@ -412,16 +420,6 @@ sweep3_kernel(const __grid_constant__ SweepArgs A) {
           e[1] = cw[0]; e[2] = cw[1]; e[3] = cw[2]; e[4] = cw[3];
         }
         qn += __popc(bal);
-        if (qn >= 32) {
-          __syncwarp();
-          qn -= 32;
-          const uint32_t e = s3_flush<DT, ROUNDS>(A, qn, 32, nm8 - 8.0f);
-          if (e > m_new) {
-            m_new = e;
-            if (lane == 0)
-              atomicMax((unsigned long long*)&sh.m_tag, ((unsigned long long)tag << 32) | e);
-          }
-        }
       }
       if (m_new > m_enc) {
         m_enc = m_new;
@@ -429,29 +427,45 @@ sweep3_kernel(const __grid_constant__ SweepArgs A) {
       }
     };
 
-    // ---- the sweep: one call site for full (vector) and ragged (scalar) iterations; with
-    //      PREFETCH the next group's load is issued before the current one is used
+    // ---- the sweep.  The inner loop runs until 32 groups are queued; the batched evaluation is
+    //      called from the outer loop so that the inner loop carries no call (its state would
+    //      otherwise be spilled around the call on every iteration).  One call site serves full
+    //      (vector) and ragged (scalar) iterations; with PREFETCH the next group's load is issued
+    //      before the current one is used.
     {
       const char* p = rowp + (size_t)tok0 * ES;
       int tok = tok0;
+      int it = 0;
       G nxt;
       if (PREFETCH && n_full > 0) load16_vec(nxt, p);
+      for (;;) {
 #pragma unroll 1
-      for (int it = 0; it < n_iter; ++it) {
-        G g;
-        if (it < n_full) {
-          if (PREFETCH) {
-            g = nxt;
-            if (it + 1 < n_full) load16_vec(nxt, p + STEP);
+        for (; it < n_iter && qn < 32; ++it) {
+          G g;
+          if (it < n_full) {
+            if (PREFETCH) {
+              g = nxt;
+              if (it + 1 < n_full) load16_vec(nxt, p + STEP);
+            } else {
+              load16_vec(g, p);
+            }
           } else {
-            load16_vec(g, p);
+            load16_scalar(g, rowp, tok, tok_end);
           }
-        } else {
-          load16_scalar(g, rowp, tok, tok_end);
+          process(g, tok);
+          p += STEP;
+          tok += kS3CtaTokens;
         }
-        process(g, tok);
-        p += STEP;
-        tok += kS3CtaTokens;
+        if (qn < 32) break;
+        __syncwarp();
+        qn -= 32;
+        const uint32_t e = s3_flush<DT, ROUNDS>(A, qn, 32, nm8 - 8.0f);
+        if (e > m_enc) {
+          m_enc = e;
+          nm8 = filter_offset(dec_ordered(m_enc)) + 8.0f;
+          if (lane == 0)
+            atomicMax((unsigned long long*)&sh.m_tag, ((unsigned long long)tag << 32) | e);
+        }
       }
     }
     // ---- drain the queue ---------------------------------------------------------------------
