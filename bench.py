@@ -33,7 +33,7 @@ WORKLOAD_DESC = {
 }
 # dram__bytes_read+write per launch of the target-side sweep kernel divided by its algorithmic
 # bytes, from the ncu capture summarised in profiles/ (None until a capture exists).
-TRAFFIC_RATIO = None
+TRAFFIC_RATIO = 1.085  # profiles/sweep3_kernel_cfg4_b64.md (B=64 capture; traffic scales with the rows)
 
 
 def _peaks():
@@ -291,9 +291,11 @@ def run_ours(args):
 
     peak, which = _peaks()
     achieved = tbytes / (verify_ms * 1e-3) / 1e9
-    roofline = {"bound": "hbm", "kernel": "sweep kernel <%s, lse> of the selected noise_spec (target side; the call also "
-                "runs three microsecond-scale helper kernels)" %
-                ("bf16" if w.target_logits.dtype == torch.bfloat16 else "f32"),
+    kname = ("sweep3_kernel" if args.spec == 3 else "sweep_kernel") + "<%s, lse>" % (
+        "bf16" if w.target_logits.dtype == torch.bfloat16 else "f32")
+    roofline = {"bound": "hbm", "kernel": kname + " (target side: the dominant kernel; the call also "
+                "runs finalize_rows_kernel and verify_epilogue_kernel, microseconds each, inside "
+                "the same event bracket)",
                 "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                 "peak_source": "of " + which,
                 "traffic": (TRAFFIC_RATIO * tbytes) if TRAFFIC_RATIO else None,
