@@ -26,7 +26,7 @@
 #include "gls_kernels.cuh"
 
 #ifndef GLS_S3_MIN_CTAS
-#define GLS_S3_MIN_CTAS 4
+#define GLS_S3_MIN_CTAS 3
 #endif
 
 namespace gls {
@@ -35,7 +35,7 @@ constexpr int kS3LaneTokens = 16;
 constexpr int kS3WarpTokens = 32 * kS3LaneTokens;               // 512
 constexpr int kS3CtaTokens = kSweepWarps3 * kS3WarpTokens;      // 4096
 constexpr int kS3QueueCap = 64;                                 // groups per warp queue
-constexpr int kS3EntryWords = 5;                                // block | wide flag, 4 words
+constexpr int kS3EntryWords = 5;                                // block | kb << 28, 4 words
 
 // 32 bytes per lane in one instruction (sm_100a): a warp reads 1 KB contiguous.
 struct Words8 {
@@ -244,16 +244,20 @@ __device__ __noinline__ uint32_t s3_flush(const SweepArgs& A, int first, int n, 
   const S3WarpCtx cx = sh.ctx[warp];
   const uint32_t* e = sh.queue[warp] + (first + lane) * kS3EntryWords;
   const float c2 = cx.inv_t * kLog2e;
+  const float nm8 = nm + 8.0f;
   uint32_t msk = 0u, blk = 0u;
   uint32_t w0 = 0u, w1 = 0u, w2 = 0u, w3 = 0u;
   if (lane < n) {
     blk = e[0];
     w0 = e[1]; w1 = e[2]; w2 = e[3]; w3 = e[4];
-    if (blk & 0x80000000u) {
-      blk &= 0x7fffffffu;
+    // kb: the group's coarse bytes can matter only below 2^kb (0: zero bytes only)
+    const uint32_t kb = blk >> 28;
+    blk &= 0x0fffffffu;
+    if (kb > 3u) {
+      // very wide group: test every token's byte against the token's own threshold
       Group16<DT> g;
-      load16_scalar(g, cx.rowp, (int)(blk << 4), cx.tok_end);
-      const float nm8 = nm + 8.0f;
+      const int tokg = (int)(blk << 4);
+      load16_scalar(g, cx.rowp, tokg, cx.tok_end);
 #pragma unroll
       for (int t = 0; t < 16; ++t) {
         const uint32_t wt = t < 4 ? w0 : t < 8 ? w1 : t < 12 ? w2 : w3;
@@ -261,8 +265,10 @@ __device__ __noinline__ uint32_t s3_flush(const SweepArgs& A, int first, int n, 
         if (h < ex2_approx(fmaf(group16_get<DT>(g, t), c2, nm8))) msk |= 1u << t;  // false for NaN
       }
     } else {
-      msk = zero_byte_mask4(w0) | (zero_byte_mask4(w1) << 4) | (zero_byte_mask4(w2) << 8) |
-            (zero_byte_mask4(w3) << 12);
+      // bytes below 2^kb: clear their low kb bits and look for zero bytes
+      const uint32_t keep = 0x01010101u * ((0xffu << kb) & 0xffu);
+      msk = zero_byte_mask4(w0 & keep) | (zero_byte_mask4(w1 & keep) << 4) |
+            (zero_byte_mask4(w2 & keep) << 8) | (zero_byte_mask4(w3 & keep) << 12);
     }
   }
   Top2 b = sh.best[threadIdx.x];
@@ -274,9 +280,10 @@ __device__ __noinline__ uint32_t s3_flush(const SweepArgs& A, int first, int n, 
       const int i = (int)(blk << 4) + t;
       if (i < cx.tok_end) {
         const float a = load_logit<DT>(cx.rowp, i);
-        if (a < CUDART_INF_F) {  // NaN and +inf never win
-          const uint32_t wt = t < 4 ? w0 : t < 8 ? w1 : t < 12 ? w2 : w3;
-          const uint32_t h = (wt >> (8 * (t & 3))) & 0xffu;
+        const uint32_t wt = t < 4 ? w0 : t < 8 ? w1 : t < 12 ? w2 : w3;
+        const uint32_t h = (wt >> (8 * (t & 3))) & 0xffu;
+        // NaN and +inf never win; a non-zero byte must pass its own coarse test first
+        if (a < CUDART_INF_F && (h == 0u || (float)h < ex2_approx(fmaf(a, c2, nm8)))) {
           uint32_t f[4];
           philox4x32<ROUNDS>(A.rk, A.rounds, (uint32_t)i >> 1, cx.c1 + (2u << 16), cx.pos, cx.seq, f);
           const uint32_t lo = (i & 1) ? f[2] : f[0], hi = ((i & 1) ? f[3] : f[1]) & 0xffu;
@@ -407,7 +414,8 @@ sweep3_kernel(const __grid_constant__ SweepArgs A) {
       uint32_t cw[4];
       philox4x32<ROUNDS>(A.rk, A.rounds, (uint32_t)tok >> 4, c1, pos, seq, cw);
       const float amax = group16_max(g);
-      const bool wide = fmaf(amax, c2, nm8) > 0.f;  // 2^(amax c + nm) > 1/256: any byte may matter
+      const float x = fmaf(amax, c2, nm8);  // log2 of 256 * 2^(amax c + nm)
+      const bool wide = x > 0.f;             // non-zero coarse bytes may matter, those below 2^x
       const bool pass = any_zero_byte(cw) | wide;
       if (LSE) lse16<DT>(g, amax, c2, lm, ls2);
       const unsigned long long mt = *m_tag;  // bound published by the other warps of the CTA
@@ -416,7 +424,8 @@ sweep3_kernel(const __grid_constant__ SweepArgs A) {
       if (bal != 0u) {
         if (pass) {
           uint32_t* e = queue + (qn + __popc(bal & ((1u << lane) - 1u))) * kS3EntryWords;
-          e[0] = ((uint32_t)tok >> 4) | (wide ? 0x80000000u : 0u);
+          const uint32_t kb = wide ? (uint32_t)min(15, __float2int_ru(x)) : 0u;
+          e[0] = ((uint32_t)tok >> 4) | (kb << 28);
           e[1] = cw[0]; e[2] = cw[1]; e[3] = cw[2]; e[4] = cw[3];
         }
         qn += __popc(bal);
