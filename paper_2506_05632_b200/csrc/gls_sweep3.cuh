@@ -165,11 +165,16 @@ __device__ __noinline__ LseFix lse16_careful(Group16<DT> g, float c2, float lm) 
   return r;
 }
 
+// lm is a reference exponent, not a running maximum: it moves only when a group's maximum
+// exceeds it by more than 2^kLseHeadroom (then it jumps to that maximum), so the rescaling
+// branch is taken a handful of times per row instead of whenever any lane sees a new maximum.
+// Terms are at most 2^kLseHeadroom, far from fp32 overflow for any row length.
+constexpr float kLseHeadroom = 64.0f;
 template <int DT>
 __device__ __forceinline__ void lse16(const Group16<DT>& g, float amax, float c2, float& lm,
                                       unsigned long long& ls2) {
   // admissible maximum of the group: amax unless it is +inf (NaN never reaches amax)
-  if (amax > lm && amax < CUDART_INF_F) {
+  if (fmaf(amax - lm, c2, -kLseHeadroom) > 0.f && amax < CUDART_INF_F) {
     const float r = ex2_approx((lm - amax) * c2);
     ls2 = fma_f32x2(ls2, pack_f32x2(r, r), 0ull);
     lm = amax;
@@ -185,7 +190,8 @@ __device__ __forceinline__ void lse16(const Group16<DT>& g, float amax, float c2
   }
   float s0, s1;
   unpack_f32x2(gs2, s0, s1);
-  if (s0 + s1 <= 32.0f) {  // every term is at most 1 unless a NaN or +inf logit poisoned the sum
+  // every term is at most 2^kLseHeadroom unless a NaN or +inf logit poisoned the sum
+  if (s0 + s1 <= 0x1p69f) {
     ls2 = add_f32x2(ls2, gs2);
   } else {
     const LseFix f = lse16_careful<DT>(g, c2, lm);
