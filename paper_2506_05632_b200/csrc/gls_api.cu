@@ -340,9 +340,19 @@ static int run_rows(SweepArgs& A, int dtype, int spec, const Plan& P, void* work
   if (spec == 3) {
     const long long cap = (long long)kNumSMs * kS3CtasPerSM;
     const int grid = (int)(P.n_items < cap ? P.n_items : cap);
-#define SWEEP3(DT, R)                                                            \
-  (lse ? sweep3_kernel<DT, true, R><<<grid, kSweepWarps3 * 32, sizeof(S3Shared), st>>>(A)  \
-       : sweep3_kernel<DT, false, R><<<grid, kSweepWarps3 * 32, sizeof(S3Shared), st>>>(A))
+#define SWEEP3(DT, R)                                                                       \
+  do {                                                                                      \
+    const size_t smem = sizeof(S3Shared<DT>);                                               \
+    if (lse) {                                                                              \
+      cudaFuncSetAttribute(sweep3_kernel<DT, true, R>,                                      \
+                           cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);         \
+      sweep3_kernel<DT, true, R><<<grid, kSweepWarps3 * 32, smem, st>>>(A);                 \
+    } else {                                                                                \
+      cudaFuncSetAttribute(sweep3_kernel<DT, false, R>,                                     \
+                           cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);         \
+      sweep3_kernel<DT, false, R><<<grid, kSweepWarps3 * 32, smem, st>>>(A);                \
+    }                                                                                       \
+  } while (0)
     if (bf) { if (r10) SWEEP3(kBF16, 10); else SWEEP3(kBF16, 0); }
     else { if (r10) SWEEP3(kF32, 10); else SWEEP3(kF32, 0); }
 #undef SWEEP3

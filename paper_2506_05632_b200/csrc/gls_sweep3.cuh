@@ -35,7 +35,6 @@ constexpr int kS3LaneTokens = 16;
 constexpr int kS3WarpTokens = 32 * kS3LaneTokens;               // 512
 constexpr int kS3CtaTokens = kSweepWarps3 * kS3WarpTokens;      // 4096
 constexpr int kS3QueueCap = 64;                                 // groups per warp queue
-constexpr int kS3EntryWords = 5;                                // block | kb << 28, 4 words
 
 // 32 bytes per lane in one instruction (sm_100a): a warp reads 1 KB contiguous.
 struct Words8 {
@@ -136,6 +135,18 @@ __device__ __forceinline__ float group16_get<kF32>(const Group16<kF32>& g, int t
   return __uint_as_float(t < 8 ? g.a.w[t] : g.b.w[t - 8]);
 }
 
+// the group as loaded, to 16-byte aligned shared memory
+__device__ __forceinline__ void store_group16(uint32_t* dst, const Group16<kBF16>& g) {
+  reinterpret_cast<uint4*>(dst)[0] = make_uint4(g.a.w[0], g.a.w[1], g.a.w[2], g.a.w[3]);
+  reinterpret_cast<uint4*>(dst)[1] = make_uint4(g.a.w[4], g.a.w[5], g.a.w[6], g.a.w[7]);
+}
+__device__ __forceinline__ void store_group16(uint32_t* dst, const Group16<kF32>& g) {
+  reinterpret_cast<uint4*>(dst)[0] = make_uint4(g.a.w[0], g.a.w[1], g.a.w[2], g.a.w[3]);
+  reinterpret_cast<uint4*>(dst)[1] = make_uint4(g.a.w[4], g.a.w[5], g.a.w[6], g.a.w[7]);
+  reinterpret_cast<uint4*>(dst)[2] = make_uint4(g.b.w[0], g.b.w[1], g.b.w[2], g.b.w[3]);
+  reinterpret_cast<uint4*>(dst)[3] = make_uint4(g.b.w[4], g.b.w[5], g.b.w[6], g.b.w[7]);
+}
+
 constexpr float kS3LseFloor = -1.0e30f;  // finite stand-in for "no finite logit seen yet"
 
 // Softmax statistics of 16 logits: lm = running max, ls2 = two partial sums of 2^((a - lm) c2).
@@ -220,55 +231,103 @@ __device__ __forceinline__ uint32_t zero_byte_mask4(uint32_t v) {
 // Shared memory of the sweep CTA (dynamic, so that the batched path below can reach it too)
 // ------------------------------------------------------------------------------------------
 struct S3WarpCtx {  // what the batched path needs to know about the warp's current work item
-  const char* rowp;
   const uint8_t* bins;
   uint32_t c1, pos, seq;
+  uint32_t key0, key1;  // Philox key (round keys are key + r * Weyl constants)
   float inv_t;
   int msg, tok_end;
 };
+// A queue entry holds everything the batched path needs, so that it never goes back to global
+// memory for the logits: 4 generator words, block index | kb << 28, and the group's 16 logits as
+// loaded (8 words of bf16, 16 of fp32).  Entries are 16-byte aligned for 128-bit accesses.
+template <int DT>
+struct S3Entry {
+  static constexpr int kDataWords = DT == kBF16 ? 8 : 16;
+  static constexpr int kWords = 8 + (DT == kBF16 ? 8 : 24);  // 64 or 128 bytes
+};
+template <int DT>
 struct S3Shared {
   unsigned long long m_tag;  // (item tag << 32) | ordered code of the CTA-wide bound on the best score
   S3WarpCtx ctx[kSweepWarps3];
   Top2 best[kSweepWarps3 * 32];  // per-thread candidates, touched by the batched path only
-  uint32_t queue[kSweepWarps3][kS3QueueCap * kS3EntryWords];
+  __align__(16) uint32_t queue[kSweepWarps3][kS3QueueCap * S3Entry<DT>::kWords];
 };
 extern __shared__ __align__(16) unsigned char s3_smem_raw[];
-__device__ __forceinline__ S3Shared& s3_shared() { return *reinterpret_cast<S3Shared*>(s3_smem_raw); }
+template <int DT>
+__device__ __forceinline__ S3Shared<DT>& s3_shared() {
+  return *reinterpret_cast<S3Shared<DT>*>(s3_smem_raw);
+}
+
+// Philox4x32 with the round keys derived on the fly (the batched path runs out of line and has no
+// cheap access to the kernel parameter's precomputed round keys).
+template <int ROUNDS>
+__device__ __forceinline__ void philox4x32_keyed(uint32_t k0, uint32_t k1, int rounds_rt, uint32_t c0,
+                                                 uint32_t c1, uint32_t c2, uint32_t c3,
+                                                 uint32_t (&out)[4]) {
+  const int n = ROUNDS > 0 ? ROUNDS : rounds_rt;
+#pragma unroll
+  for (int r = 0; r < n; ++r) {
+    const unsigned long long p0 = (unsigned long long)kPhiloxM0 * c0;
+    const unsigned long long p1 = (unsigned long long)kPhiloxM1 * c2;
+    const uint32_t n0 = (uint32_t)(p1 >> 32) ^ c1 ^ k0;
+    const uint32_t n2 = (uint32_t)(p0 >> 32) ^ c3 ^ k1;
+    c1 = (uint32_t)p1;
+    c3 = (uint32_t)p0;
+    c0 = n0;
+    c2 = n2;
+    k0 += kPhiloxW0;
+    k1 += kPhiloxW1;
+  }
+  out[0] = c0;
+  out[1] = c1;
+  out[2] = c2;
+  out[3] = c3;
+}
+
+// logit t (0..15, a run-time index) of a queued group
+template <int DT>
+__device__ __forceinline__ float entry_logit(const uint32_t* data, int t) {
+  if (DT == kBF16) {
+    const uint32_t w = data[t >> 1];
+    return (t & 1) ? bf16_hi(w) : bf16_lo(w);
+  }
+  return __uint_as_float(data[t]);
+}
 
 // ------------------------------------------------------------------------------------------
 // Batched evaluation of queued groups: lane l < n takes entry first + l of its warp's queue.
-// Candidate tokens of a group: those whose coarse byte is zero; in a wide group, those whose
-// coarse byte passes the per-token test h < 256 * 2^(logit c + nm).  For every candidate the lane
-// draws the 40 refinement bits, applies the filter to the 48-bit uniform and scores the survivors
-// in fp32.  Returns the best lower bound found (ordered code, 0 if none).
+// Candidate tokens of a group: those whose coarse byte is below 2^kb (kb = 0, the usual case:
+// zero bytes only); in a very wide group (kb > 3) those whose byte passes the per-token test
+// h < 256 * 2^(logit c + nm).  A candidate with a non-zero byte takes that per-token test first;
+// then the lane draws its 40 refinement bits, applies the filter to the 48-bit uniform and scores
+// the survivors in fp32.  Returns the best lower bound found (ordered code, 0 if none).
 // ------------------------------------------------------------------------------------------
 template <int DT, int ROUNDS>
-__device__ __noinline__ uint32_t s3_flush(const SweepArgs& A, int first, int n, float nm) {
-  S3Shared& sh = s3_shared();
+__device__ __noinline__ uint32_t s3_flush(int rounds_rt, int first, int n, float nm) {
+  S3Shared<DT>& sh = s3_shared<DT>();
   const int lane = threadIdx.x & 31;
   const int warp = threadIdx.x >> 5;
   const S3WarpCtx cx = sh.ctx[warp];
-  const uint32_t* e = sh.queue[warp] + (first + lane) * kS3EntryWords;
+  const uint32_t* e = sh.queue[warp] + (first + lane) * S3Entry<DT>::kWords;
+  const uint32_t* data = e + 8;
   const float c2 = cx.inv_t * kLog2e;
   const float nm8 = nm + 8.0f;
   uint32_t msk = 0u, blk = 0u;
   uint32_t w0 = 0u, w1 = 0u, w2 = 0u, w3 = 0u;
   if (lane < n) {
-    blk = e[0];
-    w0 = e[1]; w1 = e[2]; w2 = e[3]; w3 = e[4];
+    const uint4 cw = *reinterpret_cast<const uint4*>(e);
+    w0 = cw.x; w1 = cw.y; w2 = cw.z; w3 = cw.w;
+    blk = e[4];
     // kb: the group's coarse bytes can matter only below 2^kb (0: zero bytes only)
     const uint32_t kb = blk >> 28;
     blk &= 0x0fffffffu;
     if (kb > 3u) {
       // very wide group: test every token's byte against the token's own threshold
-      Group16<DT> g;
-      const int tokg = (int)(blk << 4);
-      load16_scalar(g, cx.rowp, tokg, cx.tok_end);
 #pragma unroll
       for (int t = 0; t < 16; ++t) {
         const uint32_t wt = t < 4 ? w0 : t < 8 ? w1 : t < 12 ? w2 : w3;
         const float h = (float)((wt >> (8 * (t & 3))) & 0xffu);
-        if (h < ex2_approx(fmaf(group16_get<DT>(g, t), c2, nm8))) msk |= 1u << t;  // false for NaN
+        if (h < ex2_approx(fmaf(entry_logit<DT>(data, t), c2, nm8))) msk |= 1u << t;  // false for NaN
       }
     } else {
       // bytes below 2^kb: clear their low kb bits and look for zero bytes
@@ -285,13 +344,14 @@ __device__ __noinline__ uint32_t s3_flush(const SweepArgs& A, int first, int n, 
       msk &= msk - 1u;
       const int i = (int)(blk << 4) + t;
       if (i < cx.tok_end) {
-        const float a = load_logit<DT>(cx.rowp, i);
+        const float a = entry_logit<DT>(data, t);
         const uint32_t wt = t < 4 ? w0 : t < 8 ? w1 : t < 12 ? w2 : w3;
         const uint32_t h = (wt >> (8 * (t & 3))) & 0xffu;
         // NaN and +inf never win; a non-zero byte must pass its own coarse test first
         if (a < CUDART_INF_F && (h == 0u || (float)h < ex2_approx(fmaf(a, c2, nm8)))) {
           uint32_t f[4];
-          philox4x32<ROUNDS>(A.rk, A.rounds, (uint32_t)i >> 1, cx.c1 + (2u << 16), cx.pos, cx.seq, f);
+          philox4x32_keyed<ROUNDS>(cx.key0, cx.key1, rounds_rt, (uint32_t)i >> 1, cx.c1 + (2u << 16),
+                                   cx.pos, cx.seq, f);
           const uint32_t lo = (i & 1) ? f[2] : f[0], hi = ((i & 1) ? f[3] : f[1]) & 0xffu;
           const float v = fmaf((float)h, 0x1p-8f,
                                fmaf((float)hi, 0x1p-16f, fmaf((float)lo, 0x1p-48f, 0x1p-49f)));
@@ -317,7 +377,7 @@ __device__ __noinline__ uint32_t s3_flush(const SweepArgs& A, int first, int n, 
 template <int DT, bool LSE, int ROUNDS>
 __global__ void __launch_bounds__(kSweepWarps3 * 32, GLS_S3_MIN_CTAS)
 sweep3_kernel(const __grid_constant__ SweepArgs A) {
-  S3Shared& sh = s3_shared();
+  S3Shared<DT>& sh = s3_shared<DT>();
   const int lane = threadIdx.x & 31;
   const int warp = threadIdx.x >> 5;
   constexpr int ES = DT == kBF16 ? 2 : 4;
@@ -354,9 +414,9 @@ sweep3_kernel(const __grid_constant__ SweepArgs A) {
       __syncwarp();  // the previous item's batched path is done with the context
       if (lane == 0) {
         S3WarpCtx cx;
-        cx.rowp = rowp;
         cx.bins = A.bins ? A.bins + A.bins_sb * b : nullptr;
         cx.c1 = c1; cx.pos = pos; cx.seq = seq;
+        cx.key0 = A.rk[0]; cx.key1 = A.rk[1];
         cx.inv_t = inv_t;
         cx.msg = (A.bins && A.msg) ? (int)__ldg(A.msg + b) : 0;
         cx.tok_end = tok_end;
@@ -429,10 +489,11 @@ sweep3_kernel(const __grid_constant__ SweepArgs A) {
       const unsigned bal = __ballot_sync(0xffffffffu, pass);
       if (bal != 0u) {
         if (pass) {
-          uint32_t* e = queue + (qn + __popc(bal & ((1u << lane) - 1u))) * kS3EntryWords;
+          uint32_t* e = queue + (qn + __popc(bal & ((1u << lane) - 1u))) * S3Entry<DT>::kWords;
           const uint32_t kb = wide ? (uint32_t)min(15, __float2int_ru(x)) : 0u;
-          e[0] = ((uint32_t)tok >> 4) | (kb << 28);
-          e[1] = cw[0]; e[2] = cw[1]; e[3] = cw[2]; e[4] = cw[3];
+          *reinterpret_cast<uint4*>(e) = make_uint4(cw[0], cw[1], cw[2], cw[3]);
+          e[4] = ((uint32_t)tok >> 4) | (kb << 28);
+          store_group16(e + 8, g);
         }
         qn += __popc(bal);
       }
@@ -474,7 +535,7 @@ sweep3_kernel(const __grid_constant__ SweepArgs A) {
         if (qn < 32) break;
         __syncwarp();
         qn -= 32;
-        const uint32_t e = s3_flush<DT, ROUNDS>(A, qn, 32, nm8 - 8.0f);
+        const uint32_t e = s3_flush<DT, ROUNDS>(A.rounds, qn, 32, nm8 - 8.0f);
         if (e > m_enc) {
           m_enc = e;
           nm8 = filter_offset(dec_ordered(m_enc)) + 8.0f;
@@ -486,7 +547,7 @@ sweep3_kernel(const __grid_constant__ SweepArgs A) {
     // ---- drain the queue ---------------------------------------------------------------------
     if (qn > 0) {
       __syncwarp();
-      const uint32_t e = s3_flush<DT, ROUNDS>(A, 0, qn, nm8 - 8.0f);
+      const uint32_t e = s3_flush<DT, ROUNDS>(A.rounds, 0, qn, nm8 - 8.0f);
       if (e > m_enc) m_enc = e;
       qn = 0;
     }
