@@ -319,7 +319,7 @@ def run_ours(args):
                        else "inputs (%.2f GB) larger than L2" % ((dbytes + tbytes) / 1e9),
                        "mean_tau": tau_mean},
             "hbm_gbs": (dbytes + tbytes) / (ms_per_step * 1e-3) / 1e9,
-            "clocks": clocks, "e2e": e2e, "gpu_launches": 5 * args.steps,
+            "clocks": clocks, "e2e": e2e, "gpu_launches": 4 * args.steps,
             "roofline": roofline, "cpu_baseline": cpu}
     print(json.dumps(line))
     if dist is not None:

@@ -94,14 +94,11 @@ static Plan make_plan(long long rows, long long V, int spec) {
 // candidate(s) in fp64 and merges the softmax statistics.
 //   out_mode 0: write RowResult only; 1: also write tokens / scores (draft side).
 // ------------------------------------------------------------------------------------------
+// Warp-collective; the result is valid in lane 0.
 template <int DT, int SPEC, int ROUNDS>
-__global__ void __launch_bounds__(128)
-finalize_rows_kernel(const __grid_constant__ SweepArgs A, int rows, int with_lse,
-                     RowResult* __restrict__ rowres, int32_t* __restrict__ out_tokens,
-                     float* __restrict__ out_scores, uint32_t* __restrict__ dev_status) {
+__device__ __forceinline__ RowResult finalize_row(const SweepArgs& A, int row, int with_lse,
+                                                  uint32_t* __restrict__ dev_status) {
   const int lane = threadIdx.x & 31;
-  const int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
-  if (row >= rows) return;
   constexpr int ES = DT == kBF16 ? 2 : 4;
   const int j = row % A.J;
   const int bk = row / A.J;
@@ -131,15 +128,15 @@ finalize_rows_kernel(const __grid_constant__ SweepArgs A, int rows, int with_lse
 #pragma unroll
     for (int d = 16; d > 0; d >>= 1) lsum += __shfl_xor_sync(0xffffffffu, lsum, d);
   }
-  if (lane != 0) return;
-
   RowResult r;
   r.pad0 = r.pad1 = r.pad2 = 0;
+  r.idx = -1;
+  r.score = -CUDART_INF;
+  r.lse = -CUDART_INF;
+  if (lane != 0) return r;
   r.lse = (with_lse && lsum > 0.0) ? (double)lm * (double)inv_t + log(lsum)
                                    : -CUDART_INF;
   if (best.i1 < 0) {
-    r.idx = -1;
-    r.score = -CUDART_INF;
     if (dev_status) atomicOr(dev_status, GLS_DEV_EMPTY_SUPPORT);
   } else {
     const char* rowp = (const char*)A.data + (b * A.sb + k * A.sk + j * A.sj) * ES;
@@ -161,6 +158,18 @@ finalize_rows_kernel(const __grid_constant__ SweepArgs A, int rows, int with_lse
     r.idx = idx;
     r.score = e1;
   }
+  return r;
+}
+
+template <int DT, int SPEC, int ROUNDS>
+__global__ void __launch_bounds__(128)
+finalize_rows_kernel(const __grid_constant__ SweepArgs A, int rows, int with_lse,
+                     RowResult* __restrict__ rowres, int32_t* __restrict__ out_tokens,
+                     float* __restrict__ out_scores, uint32_t* __restrict__ dev_status) {
+  const int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  if (row >= rows) return;
+  const RowResult r = finalize_row<DT, SPEC, ROUNDS>(A, row, with_lse, dev_status);
+  if ((threadIdx.x & 31) != 0) return;
   if (rowres) rowres[row] = r;
   if (out_tokens) out_tokens[row] = r.idx;
   if (out_scores) out_scores[row] = r.idx >= 0 ? (float)r.score : CUDART_NAN_F;
@@ -170,15 +179,12 @@ finalize_rows_kernel(const __grid_constant__ SweepArgs A, int rows, int with_lse
 // Algorithm 2, from "Let the set of active drafts be S" to the end; one thread per sequence.
 // rows[(b*K + k)*J + j] holds the winner of row (b,k,j) under its own noise stream.
 // ------------------------------------------------------------------------------------------
-__global__ void verify_epilogue_kernel(const RowResult* __restrict__ rows, int B, int K, int L,
-                                       int J, uint32_t flags,
-                                       const int32_t* __restrict__ draft_tokens,
-                                       int32_t* __restrict__ out_tokens,
-                                       int32_t* __restrict__ out_num, uint8_t* __restrict__ accept,
-                                       float* __restrict__ out_scores,
-                                       uint32_t* __restrict__ dev_status) {
-  const int b = blockIdx.x * blockDim.x + threadIdx.x;
-  if (b >= B) return;
+// `rows` points at the K x J results of sequence b: rows[k * J + j].
+__device__ void verify_sequence(const RowResult* rows, int b, int K, int L, int J, uint32_t flags,
+                                const int32_t* __restrict__ draft_tokens,
+                                int32_t* __restrict__ out_tokens, int32_t* __restrict__ out_num,
+                                uint8_t* __restrict__ accept, float* __restrict__ out_scores,
+                                uint32_t* __restrict__ dev_status) {
   unsigned long long active = K >= 64 ? ~0ull : ((1ull << K) - 1ull);
   for (int j = 0; j < J; ++j) {
     out_tokens[(long long)b * J + j] = -1;
@@ -193,7 +199,7 @@ __global__ void verify_epilogue_kernel(const RowResult* __restrict__ rows, int B
     int bi = -1;
     for (int k = 0; k < K; ++k) {
       if (!((active >> k) & 1ull) && !(flags & GLS_COMBINE_ALL)) continue;
-      const RowResult r = rows[((long long)b * K + k) * J + j];
+      const RowResult r = rows[(long long)k * J + j];
       if (r.idx < 0) continue;
       const double sc = r.score - r.lse;
       if (bi < 0 || sc > bs || (sc == bs && r.idx < bi)) {
@@ -217,6 +223,49 @@ __global__ void verify_epilogue_kernel(const RowResult* __restrict__ rows, int B
     if (active == 0ull) break;
   }
   out_num[b] = n_out;
+}
+
+__global__ void verify_epilogue_kernel(const RowResult* __restrict__ rows, int B, int K, int L,
+                                       int J, uint32_t flags,
+                                       const int32_t* __restrict__ draft_tokens,
+                                       int32_t* __restrict__ out_tokens,
+                                       int32_t* __restrict__ out_num, uint8_t* __restrict__ accept,
+                                       float* __restrict__ out_scores,
+                                       uint32_t* __restrict__ dev_status) {
+  const int b = blockIdx.x * blockDim.x + threadIdx.x;
+  if (b >= B) return;
+  verify_sequence(rows + (long long)b * K * J, b, K, L, J, flags, draft_tokens, out_tokens, out_num,
+                  accept, out_scores, dev_status);
+}
+
+// Split-V reduction and Algorithm 2's loop in one launch: a CTA per sequence finalises the
+// sequence's K x J rows into shared memory (a warp per row), then one thread walks the positions.
+struct VerifyArgs {
+  int B, K, L, J;
+  uint32_t flags;
+  const int32_t* draft_tokens;
+  int32_t* out_tokens;
+  int32_t* out_num;
+  uint8_t* accept;
+  float* out_scores;
+  uint32_t* dev_status;
+};
+constexpr int kFusedVerifyMaxWarps = 32;  // one warp per row result, up to a full CTA
+constexpr size_t kFusedVerifyMaxSmem = 48 * 1024;
+template <int DT, int SPEC, int ROUNDS>
+__global__ void __launch_bounds__(kFusedVerifyMaxWarps * 32)
+finalize_verify_kernel(const __grid_constant__ SweepArgs A, const VerifyArgs va) {
+  RowResult* srows = reinterpret_cast<RowResult*>(s3_smem_raw);
+  const int b = blockIdx.x;
+  const int nrows = va.K * va.J;
+  for (int r = threadIdx.x >> 5; r < nrows; r += (int)(blockDim.x >> 5)) {
+    const RowResult rr = finalize_row<DT, SPEC, ROUNDS>(A, b * nrows + r, 1, nullptr);
+    if ((threadIdx.x & 31) == 0) srows[r] = rr;
+  }
+  __syncthreads();
+  if (threadIdx.x == 0)
+    verify_sequence(srows, b, va.K, va.L, va.J, va.flags, va.draft_tokens, va.out_tokens, va.out_num,
+                    va.accept, va.out_scores, va.dev_status);
 }
 
 // Sec. 5.1 encoder bookkeeping: Y = best over the K streams of the encoder row, M = l_Y.
@@ -321,8 +370,21 @@ static cudaError_t launch_finalize_t(const SweepArgs& A, int rows, bool lse, Row
 }
 
 // sweep + split reduction of one batch of rows
+template <int DT, int SPEC, int ROUNDS>
+static cudaError_t launch_fused_verify_t(const SweepArgs& A, const VerifyArgs& va, cudaStream_t st) {
+  const size_t smem = (size_t)va.K * va.J * sizeof(RowResult);
+  const int nrows = va.K * va.J;
+  const int warps = nrows < kFusedVerifyMaxWarps ? nrows : kFusedVerifyMaxWarps;
+  finalize_verify_kernel<DT, SPEC, ROUNDS><<<va.B, warps * 32, smem, st>>>(A, va);
+  return cudaGetLastError();
+}
+
+// sweep + split reduction of one batch of rows.  With `va` (verification) and a sequence's
+// K x J row results fitting in shared memory, the reduction and Algorithm 2's loop run as one
+// launch and *fused is set; otherwise the rows' results are left in the workspace.
 static int run_rows(SweepArgs& A, int dtype, int spec, const Plan& P, void* workspace, bool lse,
-                    int32_t* out_tokens, float* out_scores, uint32_t* status, cudaStream_t st) {
+                    int32_t* out_tokens, float* out_scores, uint32_t* status, cudaStream_t st,
+                    const VerifyArgs* va = nullptr, bool* fused = nullptr) {
   char* ws = (char*)workspace;
   A.chunk = P.chunk;
   A.splits = P.splits;
@@ -371,8 +433,13 @@ static int run_rows(SweepArgs& A, int dtype, int spec, const Plan& P, void* work
 #undef SWEEP_CALL
   }
   if (err != cudaSuccess) return GLS_ERR_CUDA;
-#define FIN_CALL(...) \
-  launch_finalize_t<__VA_ARGS__>(A, (int)P.rows, lse, rowres, out_tokens, out_scores, status, st)
+  const bool fuse = va != nullptr &&
+                    (size_t)va->K * va->J * sizeof(RowResult) <= kFusedVerifyMaxSmem;
+  if (fused) *fused = fuse;
+#define FIN_CALL(...)                                                                          \
+  (fuse ? launch_fused_verify_t<__VA_ARGS__>(A, *va, st)                                       \
+        : launch_finalize_t<__VA_ARGS__>(A, (int)P.rows, lse, rowres, out_tokens, out_scores, \
+                                         status, st))
   if (bf) {
     if (spec == 1) err = r10 ? FIN_CALL(kBF16, 1, 10) : FIN_CALL(kBF16, 1, 0);
     else if (spec == 2) err = r10 ? FIN_CALL(kBF16, 2, 10) : FIN_CALL(kBF16, 2, 0);
@@ -486,8 +553,20 @@ int gls_target_sample_verify(const gls_rows_t* target_logits, int B, int K, int 
   A.J = J;
   A.V = (int)V;
   cudaStream_t st = (cudaStream_t)stream;
-  rc = run_rows(A, target_logits->dtype, spec, P, workspace, true, nullptr, nullptr, nullptr, st);
+  VerifyArgs va;
+  va.B = B; va.K = K; va.L = L; va.J = J;
+  va.flags = flags;
+  va.draft_tokens = draft_tokens;
+  va.out_tokens = out_tokens;
+  va.out_num = out_num_tokens;
+  va.accept = out_accept;
+  va.out_scores = out_scores;
+  va.dev_status = device_status;
+  bool fused = false;
+  rc = run_rows(A, target_logits->dtype, spec, P, workspace, true, nullptr, nullptr, nullptr, st,
+                &va, &fused);
   if (rc != GLS_OK) return rc;
+  if (fused) return GLS_OK;
   const RowResult* rowres = (const RowResult*)((char*)workspace + P.off_rows);
   verify_epilogue_kernel<<<(B + 127) / 128, 128, 0, st>>>(rowres, B, K, L, J, flags, draft_tokens,
                                                          out_tokens, out_num_tokens, out_accept,

@@ -220,6 +220,19 @@ def test_compress_small(gls, oracle, spec):
     assert np.array_equal(o["message"], ref["message"])
 
 
+def test_verify_long_drafts_take_the_two_launch_epilogue(gls, oracle):
+    """K x (L+1) row results beyond what one CTA's shared memory holds (more than 1536 rows per
+    sequence): the reduction and Algorithm 2's loop then run as separate launches."""
+    B, K, L, V = 2, 64, 24, 300
+    w = synth.verify_workload(2, "cuda", B=B, K=K, L=L, V=V)
+    kw = dict(seed=w.noise_seed, inv_temp=w.inv_temp)
+    refd = oracle.draft_sample(synth.to_numpy_rows(w.draft_logits), **kw)
+    dtok = torch.from_numpy(refd["tokens"]).cuda()
+    out = gls.target_sample_verify(w.target_logits, dtok, **kw)
+    refv = oracle.target_sample_verify(synth.to_numpy_rows(w.target_logits), refd["tokens"], **kw)
+    parity.check_verify(parity.to_np(out), refv, "long drafts")
+
+
 def test_host_detectable_errors(gls):
     x = torch.zeros(2, 2, 2, 64, device="cuda")
     tok = torch.zeros(2, 2, 1, dtype=torch.int32, device="cuda")
