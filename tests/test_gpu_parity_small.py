@@ -233,6 +233,30 @@ def test_verify_long_drafts_take_the_two_launch_epilogue(gls, oracle):
     parity.check_verify(parity.to_np(out), refv, "long drafts")
 
 
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+def test_flat_and_peaked_rows(gls, oracle, dtype):
+    """Distributions that stress the coarse-byte filter of the default noise layout: flat rows
+    (every group is "wide": all tokens within a few nats of the best score), rows with one
+    dominant token, a few hundred equally strong tokens, very low and very high temperature."""
+    B, K, J, V = 3, 2, 2, 20000
+    g = torch.Generator(device="cuda").manual_seed(5)
+    flat = 0.01 * torch.randn(B, K, J, V, generator=g, device="cuda")
+    peaked = torch.randn(B, K, J, V, generator=g, device="cuda")
+    peaked[..., 1234] += 30.0
+    plateau = torch.randn(B, K, J, V, generator=g, device="cuda") - 20.0
+    plateau[..., 5000:5300] += 25.0
+    for name, x, it in (("flat", flat, 1.0), ("peaked", peaked, 1.0), ("plateau", plateau, 1.0),
+                        ("cold", peaked, 8.0), ("hot", plateau, 0.05)):
+        x = x.to(dtype)
+        kw = dict(seed=SEED + 5, inv_temp=it)
+        tok, sc, ref = _draft_both(gls, oracle, x, **kw)
+        parity.check_draft(tok, sc, ref, name)
+        dtok = torch.from_numpy(ref["tokens"][:, :, :1].copy()).cuda()
+        out = gls.target_sample_verify(x, dtok, **kw)
+        refv = oracle.target_sample_verify(synth.to_numpy_rows(x), ref["tokens"][:, :, :1], **kw)
+        parity.check_verify(parity.to_np(out), refv, name + " verify")
+
+
 def test_host_detectable_errors(gls):
     x = torch.zeros(2, 2, 2, 64, device="cuda")
     tok = torch.zeros(2, 2, 1, dtype=torch.int32, device="cuda")
