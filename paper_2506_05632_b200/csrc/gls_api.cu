@@ -144,15 +144,28 @@ __device__ __forceinline__ RowResult finalize_row(const SweepArgs& A, int row, i
     sk.c1 = ((uint32_t)k & A.kmask) | (A.domain << 16);
     sk.pos = A.pos_base + (uint32_t)j;
     sk.seq = A.seq_ids ? A.seq_ids[b] : A.seq_base + (uint32_t)b;
-    double e1 = exact_score<DT, SPEC, ROUNDS>(A, rowp, sk, best.i1, inv_t);
-    int idx = best.i1;
+    // In the fused multi-stream race a candidate is (token << 3) | stream; ordering by that
+    // code is "lowest token, then lowest stream", the tie rule.
+    const bool multi = A.multi_k > 0;
+    StreamKey sk1 = sk, sk2 = sk;
+    int t1 = best.i1, t2 = best.i2;
+    if (multi) {
+      sk1.c1 = sk.c1 + ((uint32_t)best.i1 & 7u);
+      t1 = (int)((uint32_t)best.i1 >> 3);
+      if (best.i2 >= 0) {
+        sk2.c1 = sk.c1 + ((uint32_t)best.i2 & 7u);
+        t2 = (int)((uint32_t)best.i2 >> 3);
+      }
+    }
+    double e1 = exact_score<DT, SPEC, ROUNDS>(A, rowp, sk1, t1, inv_t);
+    int code = best.i1, idx = t1;
     // a runner-up closer than the fp32 error bound is re-scored too
     const float window = 2.0f * 0x1p-17f * (36.0f + fabsf(best.s1));
     if (best.i2 >= 0 && best.s1 - best.s2 <= window) {
-      const double e2 = exact_score<DT, SPEC, ROUNDS>(A, rowp, sk, best.i2, inv_t);
-      if (e2 > e1 || (e2 == e1 && best.i2 < idx)) {
+      const double e2 = exact_score<DT, SPEC, ROUNDS>(A, rowp, sk2, t2, inv_t);
+      if (e2 > e1 || (e2 == e1 && best.i2 < code)) {
         e1 = e2;
-        idx = best.i2;
+        idx = t2;
       }
     }
     r.idx = idx;
@@ -274,7 +287,7 @@ __global__ void encoder_epilogue_kernel(const RowResult* __restrict__ rows, int 
                                         int32_t* __restrict__ enc_index,
                                         uint8_t* __restrict__ message,
                                         float* __restrict__ out_scores,
-                                        uint32_t* __restrict__ dev_status) {
+                                        uint32_t* __restrict__ dev_status, int score_stride) {
   const int b = blockIdx.x * blockDim.x + threadIdx.x;
   if (b >= B) return;
   double bs = 0.0;
@@ -290,7 +303,7 @@ __global__ void encoder_epilogue_kernel(const RowResult* __restrict__ rows, int 
   }
   enc_index[b] = bi;
   message[b] = (bins && bi >= 0) ? bins[bins_sb * b + bi] : (uint8_t)0;
-  if (out_scores) out_scores[(long long)b * (1 + K)] = bi >= 0 ? (float)bs : CUDART_NAN_F;
+  if (out_scores) out_scores[(long long)b * score_stride] = bi >= 0 ? (float)bs : CUDART_NAN_F;
   if (bi < 0 && dev_status) atomicOr(dev_status, GLS_DEV_EMPTY_SUPPORT);
 }
 
@@ -405,7 +418,11 @@ static int run_rows(SweepArgs& A, int dtype, int spec, const Plan& P, void* work
 #define SWEEP3(DT, R)                                                                       \
   do {                                                                                      \
     const size_t smem = sizeof(S3Shared<DT>);                                               \
-    if (lse) {                                                                              \
+    if (A.multi_k > 0) {                                                                    \
+      cudaFuncSetAttribute(sweep3_kernel<DT, true, R, true>,                                \
+                           cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);         \
+      sweep3_kernel<DT, true, R, true><<<grid, kSweepWarps3 * 32, smem, st>>>(A);           \
+    } else if (lse) {                                                                       \
       cudaFuncSetAttribute(sweep3_kernel<DT, true, R>,                                      \
                            cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);         \
       sweep3_kernel<DT, true, R><<<grid, kSweepWarps3 * 32, smem, st>>>(A);                 \
@@ -485,9 +502,12 @@ const char* gls_status_string(int status) {
 
 size_t gls_workspace_bytes(int B, int K, int J, int64_t V) {
   if (!sizes_ok(B, K, J, V)) return 0;
-  const size_t a = make_plan12((long long)B * K * J, V).total;
+  size_t need = make_plan12((long long)B * K * J, V).total;
   const size_t b = make_plan3((long long)B * K * J, V).total;
-  return a > b ? a : b;
+  const size_t c = make_plan3((long long)B * J, V).total;  // fused multi-stream encoder
+  if (b > need) need = b;
+  if (c > need) need = c;
+  return need;
 }
 
 int gls_draft_sample(const gls_rows_t* draft_logits, int B, int K, int J, int64_t V, float inv_temp,
@@ -599,21 +619,41 @@ int gls_compress_select(const gls_rows_t* enc_logw, const gls_rows_t* dec_logw, 
   if (!workspace || workspace_bytes < P.total) return GLS_ERR_WORKSPACE;
   cudaStream_t st = (cudaStream_t)stream;
   const RowResult* rowres = (const RowResult*)((char*)workspace + P.off_rows);
-  // encoder: the one row of sample b raced under each of the K streams (stride_k = 0)
   A.data = enc_logw->data;
   A.sb = enc_logw->stride_b;
   A.sk = 0;
   A.sj = 0;
-  A.K = K;
   A.J = 1;
   A.V = (int)N;
-  rc = run_rows(A, enc_logw->dtype, spec, P, workspace, true, nullptr, nullptr, nullptr, st);
-  if (rc != GLS_OK) return rc;
-  encoder_epilogue_kernel<<<(B + 127) / 128, 128, 0, st>>>(rowres, B, K, bins, bins_stride_b,
-                                                          out_enc_index, out_message, out_scores,
-                                                          device_status);
+  // The encoder index is one race over tokens and streams, Y = argmin_{i,k} S_i^(k) / lambda_q,i.
+  // With the default noise layout, up to 8 streams and N < 2^28 it runs fused: each row is read
+  // and summed once and the K streams share one bound; otherwise every stream sweeps the row on
+  // its own and the epilogue takes the best of the K winners.
+  const bool fused_enc = spec == 3 && K <= 8 && N < (1LL << 28);
+  if (fused_enc) {
+    const Plan PE = make_plan((long long)B, N, spec);
+    if (workspace_bytes < PE.total) return GLS_ERR_WORKSPACE;
+    A.K = 1;
+    A.multi_k = K;
+    rc = run_rows(A, enc_logw->dtype, spec, PE, workspace, true, nullptr, nullptr, nullptr, st);
+    A.multi_k = 0;
+    if (rc != GLS_OK) return rc;
+    const RowResult* rr = (const RowResult*)((char*)workspace + PE.off_rows);
+    encoder_epilogue_kernel<<<(B + 127) / 128, 128, 0, st>>>(rr, B, 1, bins, bins_stride_b,
+                                                            out_enc_index, out_message, out_scores,
+                                                            device_status, 1 + K);
+  } else {
+    // the one row of sample b raced under each of the K streams (stride_k = 0)
+    A.K = K;
+    rc = run_rows(A, enc_logw->dtype, spec, P, workspace, true, nullptr, nullptr, nullptr, st);
+    if (rc != GLS_OK) return rc;
+    encoder_epilogue_kernel<<<(B + 127) / 128, 128, 0, st>>>(rowres, B, K, bins, bins_stride_b,
+                                                            out_enc_index, out_message, out_scores,
+                                                            device_status, 1 + K);
+  }
   if (cudaGetLastError() != cudaSuccess) return GLS_ERR_CUDA;
   if (!dec_logw) return GLS_OK;
+  A.K = K;
   // decoders: row (b,k) under stream k, restricted to candidates labelled M
   A.data = dec_logw->data;
   A.sb = dec_logw->stride_b;

@@ -61,6 +61,7 @@ struct SweepArgs {
   int splits;             // slices per row
   int parts;              // partial results per row (slices x producers per slice)
   int rows;               // B * K * J
+  int multi_k;            // > 0: one race per row over this many noise streams (fused encoder)
   long long n_items;      // rows * splits
   float inv_t[kMaxK];     // 1/T per k
   uint32_t rk[32];        // Philox round keys: rk[2r], rk[2r+1]
@@ -227,7 +228,7 @@ __device__ __forceinline__ bool beats(float s, int i, float s0, int i0) {
   return i0 < 0 || s > s0 || (s == s0 && i < i0);
 }
 __device__ __forceinline__ void top2_offer(Top2& t, float s, int i) {
-  if (i < 0) return;
+  if (i < 0 || i == t.i1 || i == t.i2) return;  // the two leaders are distinct candidates
   if (beats(s, i, t.s1, t.i1)) {
     t.s2 = t.s1;
     t.i2 = t.i1;

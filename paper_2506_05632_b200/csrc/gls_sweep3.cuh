@@ -302,7 +302,7 @@ __device__ __forceinline__ float entry_logit(const uint32_t* data, int t) {
 // then the lane draws its 40 refinement bits, applies the filter to the 48-bit uniform and scores
 // the survivors in fp32.  Returns the best lower bound found (ordered code, 0 if none).
 // ------------------------------------------------------------------------------------------
-template <int DT, int ROUNDS>
+template <int DT, int ROUNDS, bool MULTI>
 __device__ __noinline__ uint32_t s3_flush(int rounds_rt, int first, int n, float nm) {
   S3Shared<DT>& sh = s3_shared<DT>();
   const int lane = threadIdx.x & 31;
@@ -314,10 +314,12 @@ __device__ __noinline__ uint32_t s3_flush(int rounds_rt, int first, int n, float
   const float nm8 = nm + 8.0f;
   uint32_t msk = 0u, blk = 0u;
   uint32_t w0 = 0u, w1 = 0u, w2 = 0u, w3 = 0u;
+  uint32_t ks = 0u;  // noise stream of the entry (fused multi-stream race only)
   if (lane < n) {
     const uint4 cw = *reinterpret_cast<const uint4*>(e);
     w0 = cw.x; w1 = cw.y; w2 = cw.z; w3 = cw.w;
     blk = e[4];
+    if (MULTI) ks = e[5];
     // kb: the group's coarse bytes can matter only below 2^kb (0: zero bytes only)
     const uint32_t kb = blk >> 28;
     blk &= 0x0fffffffu;
@@ -350,8 +352,8 @@ __device__ __noinline__ uint32_t s3_flush(int rounds_rt, int first, int n, float
         // NaN and +inf never win; a non-zero byte must pass its own coarse test first
         if (a < CUDART_INF_F && (h == 0u || (float)h < ex2_approx(fmaf(a, c2, nm8)))) {
           uint32_t f[4];
-          philox4x32_keyed<ROUNDS>(cx.key0, cx.key1, rounds_rt, (uint32_t)i >> 1, cx.c1 + (2u << 16),
-                                   cx.pos, cx.seq, f);
+          philox4x32_keyed<ROUNDS>(cx.key0, cx.key1, rounds_rt, (uint32_t)i >> 1,
+                                   cx.c1 + ks + (2u << 16), cx.pos, cx.seq, f);
           const uint32_t lo = (i & 1) ? f[2] : f[0], hi = ((i & 1) ? f[3] : f[1]) & 0xffu;
           const float v = fmaf((float)h, 0x1p-8f,
                                fmaf((float)hi, 0x1p-16f, fmaf((float)lo, 0x1p-48f, 0x1p-49f)));
@@ -359,7 +361,8 @@ __device__ __noinline__ uint32_t s3_flush(int rounds_rt, int first, int n, float
               (cx.bins == nullptr || (int)__ldg(cx.bins + i) == cx.msg)) {
             float ln_s;
             const float s = score_f32(a, cx.inv_t, v, &ln_s);
-            top2_offer(b, s, i);
+            // fused race: the candidate is (token, stream), ordered by token first
+            top2_offer(b, s, MULTI ? (int)(((uint32_t)i << 3) | ks) : i);
             lower = fmaxf(lower, s - score_slack(s, ln_s));
           }
         }
@@ -374,7 +377,7 @@ __device__ __noinline__ uint32_t s3_flush(int rounds_rt, int first, int n, float
 // ------------------------------------------------------------------------------------------
 // The kernel
 // ------------------------------------------------------------------------------------------
-template <int DT, bool LSE, int ROUNDS>
+template <int DT, bool LSE, int ROUNDS, bool MULTI = false>
 __global__ void __launch_bounds__(kSweepWarps3 * 32, GLS_S3_MIN_CTAS)
 sweep3_kernel(const __grid_constant__ SweepArgs A) {
   S3Shared<DT>& sh = s3_shared<DT>();
@@ -503,6 +506,66 @@ sweep3_kernel(const __grid_constant__ SweepArgs A) {
       }
     };
 
+    // ---- fused multi-stream race (Sec. 5.1 encoder: Y = argmin over tokens AND streams of
+    //      S_i^(k) / weight_i): the group is loaded, maximised and summed once, then each of the
+    //      multi_k noise streams takes its turn as one step of the inner loop.
+    if constexpr (MULTI) {
+      const int ns = A.multi_k;
+      const uint32_t smask = A.kmask;
+      const char* p = rowp + (size_t)tok0 * ES;
+      int tok = tok0;
+      int it = 0, st = 0;
+      G g;
+      float amax = 0.f;
+      for (;;) {
+#pragma unroll 1
+        while (it < n_iter && qn < 32) {
+          if (st == 0) {
+            if (it < n_full) load16_vec(g, p);
+            else load16_scalar(g, rowp, tok, tok_end);
+            amax = group16_max(g);
+            if (LSE) lse16<DT>(g, amax, c2, lm, ls2);
+          }
+          uint32_t cw[4];
+          philox4x32<ROUNDS>(A.rk, A.rounds, (uint32_t)tok >> 4, c1 + ((uint32_t)st & smask), pos, seq, cw);
+          const float x = fmaf(amax, c2, nm8);
+          const bool wide = x > 0.f;
+          const bool pass = any_zero_byte(cw) | wide;
+          const unsigned long long mt = *m_tag;
+          const uint32_t m_new = ((uint32_t)(mt >> 32) == tag) ? (uint32_t)mt : 0u;
+          const unsigned bal = __ballot_sync(0xffffffffu, pass);
+          if (pass) {
+            uint32_t* e = queue + (qn + __popc(bal & ((1u << lane) - 1u))) * S3Entry<DT>::kWords;
+            const uint32_t kb = wide ? (uint32_t)min(15, __float2int_ru(x)) : 0u;
+            *reinterpret_cast<uint4*>(e) = make_uint4(cw[0], cw[1], cw[2], cw[3]);
+            e[4] = ((uint32_t)tok >> 4) | (kb << 28);
+            e[5] = (uint32_t)st & smask;
+            store_group16(e + 8, g);
+          }
+          qn += __popc(bal);
+          if (m_new > m_enc) {
+            m_enc = m_new;
+            nm8 = filter_offset(dec_ordered(m_enc)) + 8.0f;
+          }
+          if (++st == ns) {
+            st = 0;
+            ++it;
+            p += STEP;
+            tok += kS3CtaTokens;
+          }
+        }
+        if (qn < 32) break;
+        __syncwarp();
+        qn -= 32;
+        const uint32_t e = s3_flush<DT, ROUNDS, MULTI>(A.rounds, qn, 32, nm8 - 8.0f);
+        if (e > m_enc) {
+          m_enc = e;
+          nm8 = filter_offset(dec_ordered(m_enc)) + 8.0f;
+          if (lane == 0)
+            atomicMax((unsigned long long*)&sh.m_tag, ((unsigned long long)tag << 32) | e);
+        }
+      }
+    } else
     // ---- the sweep.  The inner loop runs until 32 groups are queued; the batched evaluation is
     //      called from the outer loop so that the inner loop carries no call (its state would
     //      otherwise be spilled around the call on every iteration).  One call site serves full
@@ -535,7 +598,7 @@ sweep3_kernel(const __grid_constant__ SweepArgs A) {
         if (qn < 32) break;
         __syncwarp();
         qn -= 32;
-        const uint32_t e = s3_flush<DT, ROUNDS>(A.rounds, qn, 32, nm8 - 8.0f);
+        const uint32_t e = s3_flush<DT, ROUNDS, MULTI>(A.rounds, qn, 32, nm8 - 8.0f);
         if (e > m_enc) {
           m_enc = e;
           nm8 = filter_offset(dec_ordered(m_enc)) + 8.0f;
@@ -547,7 +610,7 @@ sweep3_kernel(const __grid_constant__ SweepArgs A) {
     // ---- drain the queue ---------------------------------------------------------------------
     if (qn > 0) {
       __syncwarp();
-      const uint32_t e = s3_flush<DT, ROUNDS>(A.rounds, 0, qn, nm8 - 8.0f);
+      const uint32_t e = s3_flush<DT, ROUNDS, MULTI>(A.rounds, 0, qn, nm8 - 8.0f);
       if (e > m_enc) m_enc = e;
       qn = 0;
     }
