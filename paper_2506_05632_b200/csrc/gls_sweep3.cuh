@@ -4,24 +4,28 @@
 // 32x32->64-bit multiplies are the scarcest resource of this path on sm_100a -- runs once per 16
 // tokens.  With m a lower bound on the row's best score, token i can only matter if
 // S_i <= exp(logit_i/T - m), and S_i = -log1p(-v_i) >= v_i >= h_i / 256 with h_i its coarse byte.
-// Hence, per group of 16 tokens:
-//   - if 2^(max logit * c - m') <= 1/256 (the usual case), only tokens with h == 0 can matter:
-//     a zero-byte test on the four generator words settles the group;
-//   - otherwise the whole group is a candidate ("wide" group; a few per row).
-// Candidate groups are not examined on the spot: the lane pushes the group (its block index and
-// the four generator words) on a small per-warp queue in shared memory and the sweep goes on.
-// When 32 groups are queued the warp evaluates them together, one group per lane: refinement
-// bits from the second generator stream, the per-token filter on the 48-bit uniform, and for the
-// survivors the fp32 score logit/T - ln(-log1p(-v)).  Batching turns what would be a divergent
-// detour in most iterations (a zero byte turns up in 1 of 16 groups) into dense work done once
-// per ~16 iterations.  The filter has no false negatives, so the result equals a full evaluation
-// (Sec. 3 step 2 / Algorithm 2 draft loop and Y_j line of arXiv 2506.05632, log domain).
+// Hence, per group of 16 tokens, with 2^x = 256 * 2^(max logit * c - m'):
+//   - if x <= 0 (the usual case), only tokens with h == 0 can matter: a zero-byte test on the
+//     four generator words settles the group;
+//   - otherwise the group is "wide" (a few dozen per row): bytes below 2^x can matter.
+// Candidate groups are not examined on the spot: the lane pushes the group (the four generator
+// words, its block index tagged with ceil(x), and its 16 logits as loaded) on a small per-warp
+// queue in shared memory and the sweep goes on.  When 32 groups are queued the warp evaluates
+// them together, one group per lane: per-token test on the coarse byte, refinement bits from the
+// second generator stream, the filter on the 48-bit uniform, and for the survivors the fp32 score
+// logit/T - ln(-log1p(-v)).  Batching turns what would be a divergent detour in most iterations
+// (a zero byte turns up in 1 of 16 groups) into dense work done once per ~10 iterations, and
+// because the entry carries the logits the batched path never goes back to global memory.  The
+// filter has no false negatives, so the result equals a full evaluation (Sec. 3 step 2 /
+// Algorithm 2 draft loop and Y_j line of arXiv 2506.05632, log domain).
 //
 // Work decomposition: a work item is one (row, vocabulary slice), owned by a CTA of 8 warps; per
 // iteration a lane takes 16 consecutive tokens (one 32-byte load of bf16, two of fp32), a warp
 // 512 and the CTA 4096 contiguous tokens.  Warps never wait on one another: they share the bound
 // m through one tagged shared-memory word, each warp writes its own partial result, and the
-// split-V reduction merges them.
+// split-V reduction merges them.  The batched evaluation is called from an outer loop so that
+// the hot loop contains no call.  A fused variant (MULTI) races one row under several noise
+// streams at once for the compression encoder of Sec. 5.1.
 #pragma once
 #include "gls_kernels.cuh"
 
