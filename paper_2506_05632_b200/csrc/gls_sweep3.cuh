@@ -153,70 +153,55 @@ __device__ __forceinline__ void store_group16(uint32_t* dst, const Group16<kF32>
 
 constexpr float kS3LseFloor = -1.0e30f;  // finite stand-in for "no finite logit seen yet"
 
-// Softmax statistics of 16 logits: lm = running max, ls2 = two partial sums of 2^((a - lm) c2).
-// The fast path assumes finite-or-(-inf) logits; a group holding NaN or +inf is redone token by
-// token by lse16_careful (out of line: inlined, its 16 extra ex2 were issued for every group),
-// which returns the group's maximum over admissible logits and its sum relative to
-// max(lm, that maximum).
-struct LseFix {
-  float vmax, gs;
-};
-template <int DT>
-__device__ __noinline__ LseFix lse16_careful(Group16<DT> g, float c2, float lm) {
-  LseFix r;
-  r.vmax = -CUDART_INF_F;
-#pragma unroll
-  for (int t = 0; t < 16; ++t) {
-    const float a = group16_get<DT>(g, t);
-    if (a < CUDART_INF_F) r.vmax = fmaxf(r.vmax, a);  // false for NaN and +inf
-  }
-  const float ref = fmaxf(lm, r.vmax);
-  r.gs = 0.f;
-#pragma unroll
-  for (int t = 0; t < 16; ++t) {
-    const float a = group16_get<DT>(g, t);
-    if (a < CUDART_INF_F) r.gs += ex2_approx((a - ref) * c2);
-  }
-  return r;
-}
-
-// lm is a reference exponent, not a running maximum: it moves only when a group's maximum
-// exceeds it by more than 2^kLseHeadroom (then it jumps to that maximum), so the rescaling
-// branch is taken a handful of times per row instead of whenever any lane sees a new maximum.
-// Terms are at most 2^kLseHeadroom, far from fp32 overflow for any row length.
+// Softmax statistics of 16 logits: lm = reference exponent, ls2 = two partial sums of
+// 2^((a - lm) c2).  lm is not a running maximum: it moves only when a group's maximum exceeds it
+// by more than 2^kLseHeadroom (then it jumps to that maximum), so the rescaling branch is taken a
+// handful of times per row instead of whenever any lane sees a new maximum; terms are at most
+// 2^kLseHeadroom, far from fp32 overflow for any row length.  The loop assumes finite-or-(-inf)
+// logits and checks nothing: a NaN or +inf logit turns the lane's sum into NaN or +inf, which
+// the caller detects once at the end of the work item and repairs with lse_redo_careful().
 constexpr float kLseHeadroom = 64.0f;
 template <int DT>
 __device__ __forceinline__ void lse16(const Group16<DT>& g, float amax, float c2, float& lm,
                                       unsigned long long& ls2) {
-  // admissible maximum of the group: amax unless it is +inf (NaN never reaches amax)
-  if (fmaf(amax - lm, c2, -kLseHeadroom) > 0.f && amax < CUDART_INF_F) {
-    const float r = ex2_approx((lm - amax) * c2);
-    ls2 = fma_f32x2(ls2, pack_f32x2(r, r), 0ull);
-    lm = amax;
+  if (fmaf(amax - lm, c2, -kLseHeadroom) > 0.f) {
+    if (amax < CUDART_INF_F) {
+      const float r = ex2_approx((lm - amax) * c2);
+      ls2 = fma_f32x2(ls2, pack_f32x2(r, r), 0ull);
+      lm = amax;
+    }
   }
   const float nl = -lm * c2;
   const unsigned long long c22 = pack_f32x2(c2, c2), nl2 = pack_f32x2(nl, nl);
-  unsigned long long gs2 = 0ull;
 #pragma unroll
   for (int t = 0; t < 16; t += 2) {
     float e0, e1;
     unpack_f32x2(fma_f32x2(pack_f32x2(group16_get<DT>(g, t), group16_get<DT>(g, t + 1)), c22, nl2), e0, e1);
-    gs2 = add_f32x2(gs2, pack_f32x2(ex2_approx(e0), ex2_approx(e1)));
+    ls2 = add_f32x2(ls2, pack_f32x2(ex2_approx(e0), ex2_approx(e1)));
   }
-  float s0, s1;
-  unpack_f32x2(gs2, s0, s1);
-  // every term is at most 2^kLseHeadroom unless a NaN or +inf logit poisoned the sum
-  if (s0 + s1 <= 0x1p69f) {
-    ls2 = add_f32x2(ls2, gs2);
-  } else {
-    const LseFix f = lse16_careful<DT>(g, c2, lm);
-    if (f.vmax > lm) {
-      const float r = ex2_approx((lm - f.vmax) * c2);
-      ls2 = fma_f32x2(ls2, pack_f32x2(r, r), 0ull);
-      lm = f.vmax;
+}
+
+// The lane's share of a work item again, token by token, leaving out NaN and +inf logits (they
+// cannot define a probability).  Rare: only rows that hold such values come here.
+template <int DT>
+__device__ __noinline__ void lse_redo_careful(const char* rowp, int tok0, int n_iter, int tok_end,
+                                              float c2, float* lm_out, float* ls_out) {
+  float lm = kS3LseFloor, ls = 0.f;
+  for (int it = 0; it < n_iter; ++it) {
+    const int tok = tok0 + it * kS3CtaTokens;
+    for (int t = 0; t < kS3LaneTokens; ++t) {
+      if (tok + t >= tok_end) break;
+      const float a = load_logit<DT>(rowp, tok + t);
+      if (!(a < CUDART_INF_F) || a == -CUDART_INF_F) continue;
+      if (a > lm) {
+        ls *= ex2_approx((lm - a) * c2);
+        lm = a;
+      }
+      ls += ex2_approx((a - lm) * c2);
     }
-    ls2 = add_f32x2(ls2, pack_f32x2(f.gs, 0.f));
   }
+  *lm_out = lm;
+  *ls_out = ls;
 }
 
 // Any zero byte among the 16 coarse bytes?  (exact as a yes / no for the four words together)
@@ -626,6 +611,13 @@ sweep3_kernel(const __grid_constant__ SweepArgs A) {
     if (LSE) {
       float s0, s1;
       unpack_f32x2(ls2, s0, s1);
+      if (__any_sync(0xffffffffu, !(s0 + s1 < CUDART_INF_F))) {  // NaN or +inf logits in the slice
+        float rl, rs;
+        lse_redo_careful<DT>(rowp, tok0, n_iter, tok_end, c2, &rl, &rs);
+        lm = rl;
+        s0 = rs;
+        s1 = 0.f;
+      }
       float wm = lm;
 #pragma unroll
       for (int d = 16; d > 0; d >>= 1) wm = fmaxf(wm, __shfl_xor_sync(0xffffffffu, wm, d));
