@@ -38,7 +38,6 @@ namespace gls {
 constexpr int kS3LaneTokens = 16;
 constexpr int kS3WarpTokens = 32 * kS3LaneTokens;               // 512
 constexpr int kS3CtaTokens = kSweepWarps3 * kS3WarpTokens;      // 4096
-constexpr int kS3QueueCap = 64;                                 // groups per warp queue
 
 // 32 bytes per lane in one instruction (sm_100a): a warp reads 1 KB contiguous.
 struct Words8 {
@@ -233,13 +232,16 @@ template <int DT>
 struct S3Entry {
   static constexpr int kDataWords = DT == kBF16 ? 8 : 16;
   static constexpr int kWords = 8 + (DT == kBF16 ? 8 : 24);  // 64 or 128 bytes
+  // Groups per warp queue: a batch is taken at 32 queued groups, and one step of the sweep can
+  // add 32 more (64 for bf16, whose sweep handles two groups per lane and step).
+  static constexpr int kCap = DT == kBF16 ? 96 : 64;
 };
 template <int DT>
 struct S3Shared {
   unsigned long long m_tag;  // (item tag << 32) | ordered code of the CTA-wide bound on the best score
   S3WarpCtx ctx[kSweepWarps3];
   Top2 best[kSweepWarps3 * 32];  // per-thread candidates, touched by the batched path only
-  __align__(16) uint32_t queue[kSweepWarps3][kS3QueueCap * S3Entry<DT>::kWords];
+  __align__(16) uint32_t queue[kSweepWarps3][S3Entry<DT>::kCap * S3Entry<DT>::kWords];
 };
 extern __shared__ __align__(16) unsigned char s3_smem_raw[];
 template <int DT>
@@ -495,6 +497,46 @@ sweep3_kernel(const __grid_constant__ SweepArgs A) {
       }
     };
 
+    // two groups per lane in one step (bf16): two independent generator chains in flight hide
+    // each other's latency, and the loop and polling overhead is paid once for 32 tokens
+    auto process2 = [&](const G& g0, const G& g1, int tok) {
+      uint32_t cw0[4], cw1[4];
+      philox4x32<ROUNDS>(A.rk, A.rounds, (uint32_t)tok >> 4, c1, pos, seq, cw0);
+      philox4x32<ROUNDS>(A.rk, A.rounds, (uint32_t)(tok + kS3CtaTokens) >> 4, c1, pos, seq, cw1);
+      const float amax0 = group16_max(g0), amax1 = group16_max(g1);
+      const float x0 = fmaf(amax0, c2, nm8), x1 = fmaf(amax1, c2, nm8);
+      const bool wide0 = x0 > 0.f, wide1 = x1 > 0.f;
+      const bool pass0 = any_zero_byte(cw0) | wide0, pass1 = any_zero_byte(cw1) | wide1;
+      if (LSE) {
+        lse16<DT>(g0, amax0, c2, lm, ls2);
+        lse16<DT>(g1, amax1, c2, lm, ls2);
+      }
+      const unsigned long long mt = *m_tag;
+      const uint32_t m_new = ((uint32_t)(mt >> 32) == tag) ? (uint32_t)mt : 0u;
+      const unsigned bal0 = __ballot_sync(0xffffffffu, pass0);
+      const unsigned bal1 = __ballot_sync(0xffffffffu, pass1);
+      if (pass0) {
+        uint32_t* e = queue + (qn + __popc(bal0 & ((1u << lane) - 1u))) * S3Entry<DT>::kWords;
+        const uint32_t kb = wide0 ? (uint32_t)min(15, __float2int_ru(x0)) : 0u;
+        *reinterpret_cast<uint4*>(e) = make_uint4(cw0[0], cw0[1], cw0[2], cw0[3]);
+        e[4] = ((uint32_t)tok >> 4) | (kb << 28);
+        store_group16(e + 8, g0);
+      }
+      qn += __popc(bal0);
+      if (pass1) {
+        uint32_t* e = queue + (qn + __popc(bal1 & ((1u << lane) - 1u))) * S3Entry<DT>::kWords;
+        const uint32_t kb = wide1 ? (uint32_t)min(15, __float2int_ru(x1)) : 0u;
+        *reinterpret_cast<uint4*>(e) = make_uint4(cw1[0], cw1[1], cw1[2], cw1[3]);
+        e[4] = ((uint32_t)(tok + kS3CtaTokens) >> 4) | (kb << 28);
+        store_group16(e + 8, g1);
+      }
+      qn += __popc(bal1);
+      if (m_new > m_enc) {
+        m_enc = m_new;
+        nm8 = filter_offset(dec_ordered(m_enc)) + 8.0f;
+      }
+    };
+
     // ---- fused multi-stream race (Sec. 5.1 encoder: Y = argmin over tokens AND streams of
     //      S_i^(k) / weight_i): the group is loaded, maximised and summed once, then each of the
     //      multi_k noise streams takes its turn as one step of the inner loop.
@@ -564,30 +606,64 @@ sweep3_kernel(const __grid_constant__ SweepArgs A) {
       const char* p = rowp + (size_t)tok0 * ES;
       int tok = tok0;
       int it = 0;
-      G nxt;
-      if (PREFETCH && n_full > 0) load16_vec(nxt, p);
+      constexpr bool PAIR = DT == kBF16;
+      G nxt, nxt1;
+      if (PAIR) {
+        if (n_full >= 2) {
+          load16_vec(nxt, p);
+          load16_vec(nxt1, p + STEP);
+        }
+      } else if (PREFETCH && n_full > 0) {
+        load16_vec(nxt, p);
+      }
       for (;;) {
+        if (PAIR) {
+          // pairs of full iterations, the next pair's loads in flight
 #pragma unroll 1
-        for (; it < n_iter && qn < 32; ++it) {
-          G g;
-          if (it < n_full) {
-            if (PREFETCH) {
-              g = nxt;
-              if (it + 1 < n_full) load16_vec(nxt, p + STEP);
-            } else {
-              load16_vec(g, p);
+          for (; it + 2 <= n_full && qn < 32; it += 2) {
+            const G g0 = nxt, g1 = nxt1;
+            if (it + 4 <= n_full) {
+              load16_vec(nxt, p + 2 * STEP);
+              load16_vec(nxt1, p + 3 * STEP);
             }
-          } else {
-            load16_scalar(g, rowp, tok, tok_end);
+            process2(g0, g1, tok);
+            p += 2 * STEP;
+            tok += 2 * kS3CtaTokens;
           }
-          process(g, tok);
-          p += STEP;
-          tok += kS3CtaTokens;
+          // what is left: at most one full iteration, then the ragged ones
+#pragma unroll 1
+          for (; it + 2 > n_full && it < n_iter && qn < 32; ++it) {
+            G g;
+            if (it < n_full) load16_vec(g, p);
+            else load16_scalar(g, rowp, tok, tok_end);
+            process(g, tok);
+            p += STEP;
+            tok += kS3CtaTokens;
+          }
+        } else {
+#pragma unroll 1
+          for (; it < n_iter && qn < 32; ++it) {
+            G g;
+            if (it < n_full) {
+              if (PREFETCH) {
+                g = nxt;
+                if (it + 1 < n_full) load16_vec(nxt, p + STEP);
+              } else {
+                load16_vec(g, p);
+              }
+            } else {
+              load16_scalar(g, rowp, tok, tok_end);
+            }
+            process(g, tok);
+            p += STEP;
+            tok += kS3CtaTokens;
+          }
         }
         if (qn < 32) break;
         __syncwarp();
-        qn -= 32;
-        const uint32_t e = s3_flush<DT, ROUNDS, MULTI>(A.rounds, qn, 32, nm8 - 8.0f);
+        const int nb = min(qn, 32);
+        qn -= nb;
+        const uint32_t e = s3_flush<DT, ROUNDS, MULTI>(A.rounds, qn, nb, nm8 - 8.0f);
         if (e > m_enc) {
           m_enc = e;
           nm8 = filter_offset(dec_ordered(m_enc)) + 8.0f;
