@@ -35,7 +35,7 @@ WORKLOAD_DESC = {
 }
 # dram__bytes_read+write per launch of the target-side sweep kernel divided by its algorithmic
 # bytes, from the ncu capture summarised in profiles/ (None until a capture exists).
-TRAFFIC_RATIO = 1.021  # profiles/sweep3_kernel_cfg4_b64.md (B=64 capture; traffic scales with the rows)
+TRAFFIC_RATIO = 1.015  # profiles/sweep3_kernel_cfg4_b64.md (B=64 capture; traffic scales with the rows)
 
 
 def _peaks():
