@@ -217,6 +217,41 @@ int gls_target_sample_verify(const gls_rows_t* target_logits, int B, int K, int 
                              size_t workspace_bytes, uint32_t* device_status, void* stream);
 
 /*
+ * Sparse rows -- Sec. 4.4 ("enabling top-K sampling ... allows us to throw away all but M << N
+ * high-probability tokens") and Appendix D.1 (the experiments keep the top 50 tokens).  A row is a
+ * list of M kept tokens: their ids in the full vocabulary and their logits; every other token has
+ * probability zero.  The races are those of the dense entry points on the row with -inf outside
+ * the list, with the noise of each kept token keyed by its ORIGINAL id, so a sparse call and a
+ * dense call on the correspondingly masked row return the same tokens and scores.  All kept tokens
+ * are scored directly (fp64); no workspace is needed.
+ *
+ *   token_ids  int32 [B,K,J,M] (strides below, M contiguous); -1 marks an empty slot; the ids of
+ *              one row must be distinct
+ *   logits     fp32, same indexing
+ *   strides    in elements, shared by both arrays; stride_k = 0 shares one list among all k
+ */
+typedef struct {
+  const int32_t* token_ids;
+  const float* logits;
+  int64_t stride_b, stride_k, stride_j;
+  int32_t M;
+} gls_sparse_rows_t;
+
+/* gls_draft_sample on sparse rows: out_tokens holds vocabulary ids (-1 for an empty row). */
+int gls_draft_sample_sparse(const gls_sparse_rows_t* draft_rows, int B, int K, int J, float inv_temp,
+                            const float* inv_temp_per_draft_host, const gls_noise_t* noise,
+                            int32_t* out_tokens, float* out_scores, uint32_t* device_status,
+                            void* stream);
+
+/* gls_target_sample_verify on sparse rows (same flags, same outputs).  Each list is normalised
+ * over its kept tokens, as top-K sampling does.  K * J must not exceed 1536. */
+int gls_target_sample_verify_sparse(const gls_sparse_rows_t* target_rows, int B, int K, int L,
+                                    float inv_temp, const int32_t* draft_tokens,
+                                    const gls_noise_t* noise, uint32_t flags, int32_t* out_tokens,
+                                    int32_t* out_num_tokens, uint8_t* out_accept, float* out_scores,
+                                    uint32_t* device_status, void* stream);
+
+/*
  * Compression -- Sec. 5.1 and Appendix C.  Per batch row b (one source sample):
  *     encoder:   Y = argmin_i min_k S_i^(k) / lambda_q,i          lambda_q = softmax(enc_logw[b,:])
  *                M = bins[Y]                                      (the log2(L_max)-bit message)

@@ -55,6 +55,11 @@ class _Rows(C.Structure):
                 ("stride_k", C.c_int64), ("stride_j", C.c_int64)]
 
 
+class _SparseRows(C.Structure):
+    _fields_ = [("token_ids", C.c_void_p), ("logits", C.c_void_p), ("stride_b", C.c_int64),
+                ("stride_k", C.c_int64), ("stride_j", C.c_int64), ("M", C.c_int32)]
+
+
 class _Noise(C.Structure):
     _fields_ = [("seed", C.c_uint64), ("seq_base", C.c_uint32), ("seq_ids", C.c_void_p),
                 ("pos_base", C.c_uint32), ("noise_spec", C.c_uint32), ("rounds", C.c_uint32),
@@ -85,6 +90,15 @@ def load():
         L.gls_draft_sample_static.argtypes = [
             C.POINTER(_Rows), C.c_int, C.c_int, C.c_int, C.c_int64, C.c_float, C.c_void_p,
             C.POINTER(_Noise), C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
+        L.gls_draft_sample_sparse.restype = C.c_int
+        L.gls_draft_sample_sparse.argtypes = [
+            C.POINTER(_SparseRows), C.c_int, C.c_int, C.c_int, C.c_float, C.c_void_p,
+            C.POINTER(_Noise), C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
+        L.gls_target_sample_verify_sparse.restype = C.c_int
+        L.gls_target_sample_verify_sparse.argtypes = [
+            C.POINTER(_SparseRows), C.c_int, C.c_int, C.c_int, C.c_float, C.c_void_p,
+            C.POINTER(_Noise), C.c_uint32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
+            C.c_void_p, C.c_void_p]
         L.gls_target_sample_verify.restype = C.c_int
         L.gls_target_sample_verify.argtypes = [
             C.POINTER(_Rows), C.c_int, C.c_int, C.c_int, C.c_int64, C.c_float, C.c_void_p,
@@ -205,6 +219,68 @@ def draft_sample_static(logits, out_tokens, out_scores=None, inv_temp=1.0, inv_t
                                      C.byref(nz), _ptr(out_tokens), _ptr(out_scores), _ptr(status),
                                      _stream()))
     return out_tokens, out_scores
+
+
+def _sparse(ids, logits):
+    """gls_sparse_rows_t of ids int32 [B,K,J,M] and logits fp32 with the same shape and strides."""
+    if not (ids.is_cuda and logits.is_cuda):
+        raise GlsError("libgls takes device tensors; there is no CPU path")
+    if ids.dtype != torch.int32 or logits.dtype != torch.float32:
+        raise GlsError("sparse rows are int32 token ids and float32 logits")
+    if ids.shape != logits.shape or ids.stride() != logits.stride():
+        raise GlsError("token_ids and logits must share shape and strides")
+    if ids.stride(-1) != 1 and ids.shape[-1] > 1:
+        raise GlsError("the kept-token dimension must be contiguous")
+    return _SparseRows(ids.data_ptr(), logits.data_ptr(), ids.stride(0), ids.stride(1),
+                       ids.stride(2), ids.shape[3])
+
+
+def draft_sample_sparse(token_ids, logits, inv_temp=1.0, inv_temp_per_draft=None, seed=0,
+                        seq_base=0, seq_ids=None, pos_base=0, spec=3, rounds=10, noise_flags=0,
+                        want_scores=True, status=None):
+    """Sparse rows (kept token ids and their logits, [B,K,J,M]) -> (vocabulary ids int32 [B,K,J],
+    scores fp32 [B,K,J] | None).  Same races as draft_sample on the row masked to the kept tokens."""
+    L = load()
+    B, K, J, M = token_ids.shape
+    rows = _sparse(token_ids, logits)
+    nz = _noise(seed, seq_base, seq_ids, pos_base, spec, rounds, noise_flags)
+    dev = token_ids.device
+    out_tokens = torch.empty((B, K, J), dtype=torch.int32, device=dev)
+    out_scores = torch.empty((B, K, J), dtype=torch.float32, device=dev) if want_scores else None
+    itk = None
+    if inv_temp_per_draft is not None:
+        itk = (C.c_float * K)(*[float(x) for x in inv_temp_per_draft])
+    _check(L.gls_draft_sample_sparse(C.byref(rows), B, K, J, float(inv_temp),
+                                     C.cast(itk, C.c_void_p) if itk is not None else None,
+                                     C.byref(nz), _ptr(out_tokens), _ptr(out_scores), _ptr(status),
+                                     _stream()))
+    return out_tokens, out_scores
+
+
+def target_sample_verify_sparse(token_ids, logits, draft_tokens, inv_temp=1.0, flags=0, seed=0,
+                                seq_base=0, seq_ids=None, pos_base=0, spec=3, rounds=10,
+                                noise_flags=0, want_scores=True, status=None):
+    """Sparse target rows [B,K,J,M] (J = L+1, or L with NO_BONUS) and draft_tokens int32 [B,K,L]
+    -> dict(tokens [B,J], tau [B], accept [B,K,L], scores [B,J] | None)."""
+    L = load()
+    B, K, J, M = token_ids.shape
+    Ld = J if (flags & NO_BONUS) else J - 1
+    rows = _sparse(token_ids, logits)
+    nz = _noise(seed, seq_base, seq_ids, pos_base, spec, rounds, noise_flags)
+    dev = token_ids.device
+    if Ld > 0:
+        if draft_tokens.dtype != torch.int32 or not draft_tokens.is_contiguous():
+            raise GlsError("draft_tokens must be contiguous int32")
+        assert tuple(draft_tokens.shape) == (B, K, Ld)
+    out = dict(tokens=torch.empty((B, J), dtype=torch.int32, device=dev),
+               tau=torch.empty((B,), dtype=torch.int32, device=dev),
+               accept=torch.empty((B, K, Ld), dtype=torch.uint8, device=dev),
+               scores=torch.empty((B, J), dtype=torch.float32, device=dev) if want_scores else None)
+    _check(L.gls_target_sample_verify_sparse(
+        C.byref(rows), B, K, Ld, float(inv_temp), _ptr(draft_tokens) if Ld > 0 else None,
+        C.byref(nz), int(flags), _ptr(out["tokens"]), _ptr(out["tau"]),
+        _ptr(out["accept"]) if Ld > 0 else None, _ptr(out.get("scores")), _ptr(status), _stream()))
+    return out
 
 
 def target_sample_verify(logits, draft_tokens, inv_temp=1.0, flags=0, seed=0, seq_base=0,

@@ -328,6 +328,110 @@ __global__ void decoder_epilogue_kernel(const RowResult* __restrict__ rows, int 
 }
 
 // ------------------------------------------------------------------------------------------
+// Sparse rows (Sec. 4.4: top-K truncation keeps M << N tokens).  A warp scores all kept tokens of
+// a row directly in fp64 -- logit/T - ln(-log1p(-v)), v keyed by the token's vocabulary id -- so
+// no filter, queue or workspace is involved.  Warp-collective; the result is valid in lane 0.
+// ------------------------------------------------------------------------------------------
+struct SparseArgs {
+  const int32_t* ids;
+  const float* logits;
+  long long sb, sk, sj;
+  int M;
+};
+
+__device__ __forceinline__ bool sparse_keep(int id, float a) {
+  return id >= 0 && a < CUDART_INF_F && a > -CUDART_INF_F;  // false for NaN, +inf and masked tokens
+}
+
+template <int SPEC, int ROUNDS>
+__device__ __forceinline__ RowResult sparse_row(const SweepArgs& A, const SparseArgs& S, int row,
+                                                uint32_t* __restrict__ dev_status) {
+  const int lane = threadIdx.x & 31;
+  const int j = row % A.J;
+  const int bk = row / A.J;
+  const int k = bk % A.K;
+  const int b = bk / A.K;
+  const long long base = b * S.sb + k * S.sk + j * S.sj;
+  const double inv_t = (double)A.inv_t[k];
+  StreamKey sk;
+  sk.c1 = ((uint32_t)k & A.kmask) | (A.domain << 16);
+  sk.pos = A.pos_base + (uint32_t)j;
+  sk.seq = A.seq_ids ? A.seq_ids[b] : A.seq_base + (uint32_t)b;
+  double best = -CUDART_INF, amax = -CUDART_INF;
+  int bid = -1;
+  for (int m = lane; m < S.M; m += 32) {
+    const int id = __ldg(S.ids + base + m);
+    const float a = __ldg(S.logits + base + m);
+    if (!sparse_keep(id, a)) continue;
+    const double al = (double)a * inv_t;
+    amax = fmax(amax, al);
+    const double v = uniform_exact<SPEC, ROUNDS>(A, sk, id);
+    const double sc = al - log(-log1p(-v));
+    if (bid < 0 || sc > best || (sc == best && id < bid)) {
+      best = sc;
+      bid = id;
+    }
+  }
+#pragma unroll
+  for (int d = 16; d > 0; d >>= 1) {
+    const double ob = __shfl_xor_sync(0xffffffffu, best, d);
+    const int oi = __shfl_xor_sync(0xffffffffu, bid, d);
+    amax = fmax(amax, __shfl_xor_sync(0xffffffffu, amax, d));
+    if (oi >= 0 && (bid < 0 || ob > best || (ob == best && oi < bid))) {
+      best = ob;
+      bid = oi;
+    }
+  }
+  double sum = 0.0;
+  if (bid >= 0) {
+    for (int m = lane; m < S.M; m += 32) {
+      const int id = __ldg(S.ids + base + m);
+      const float a = __ldg(S.logits + base + m);
+      if (sparse_keep(id, a)) sum += exp((double)a * inv_t - amax);
+    }
+  }
+#pragma unroll
+  for (int d = 16; d > 0; d >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, d);
+  RowResult r;
+  r.pad0 = r.pad1 = r.pad2 = 0;
+  r.idx = bid;
+  r.score = bid >= 0 ? best : -CUDART_INF;
+  r.lse = bid >= 0 ? amax + log(sum) : -CUDART_INF;
+  if (bid < 0 && dev_status && lane == 0) atomicOr(dev_status, GLS_DEV_EMPTY_SUPPORT);
+  return r;
+}
+
+template <int SPEC, int ROUNDS>
+__global__ void __launch_bounds__(128)
+sparse_draft_kernel(const __grid_constant__ SweepArgs A, const SparseArgs S, int rows,
+                    int32_t* __restrict__ out_tokens, float* __restrict__ out_scores,
+                    uint32_t* __restrict__ dev_status) {
+  const int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  if (row >= rows) return;
+  const RowResult r = sparse_row<SPEC, ROUNDS>(A, S, row, dev_status);
+  if ((threadIdx.x & 31) != 0) return;
+  out_tokens[row] = r.idx;
+  if (out_scores) out_scores[row] = r.idx >= 0 ? (float)r.score : CUDART_NAN_F;
+}
+
+// a CTA per sequence: a warp per row result into shared memory, then Algorithm 2's loop
+template <int SPEC, int ROUNDS>
+__global__ void __launch_bounds__(kFusedVerifyMaxWarps * 32)
+sparse_verify_kernel(const __grid_constant__ SweepArgs A, const SparseArgs S, const VerifyArgs va) {
+  RowResult* srows = reinterpret_cast<RowResult*>(s3_smem_raw);
+  const int b = blockIdx.x;
+  const int nrows = va.K * va.J;
+  for (int r = threadIdx.x >> 5; r < nrows; r += (int)(blockDim.x >> 5)) {
+    const RowResult rr = sparse_row<SPEC, ROUNDS>(A, S, b * nrows + r, nullptr);
+    if ((threadIdx.x & 31) == 0) srows[r] = rr;
+  }
+  __syncthreads();
+  if (threadIdx.x == 0)
+    verify_sequence(srows, b, va.K, va.L, va.J, va.flags, va.draft_tokens, va.out_tokens, va.out_num,
+                    va.accept, va.out_scores, va.dev_status);
+}
+
+// ------------------------------------------------------------------------------------------
 // host side
 // ------------------------------------------------------------------------------------------
 static bool finite_pos(float x) { return std::isfinite(x) && x > 0.f; }
@@ -591,6 +695,104 @@ int gls_target_sample_verify(const gls_rows_t* target_logits, int B, int K, int 
   verify_epilogue_kernel<<<(B + 127) / 128, 128, 0, st>>>(rowres, B, K, L, J, flags, draft_tokens,
                                                          out_tokens, out_num_tokens, out_accept,
                                                          out_scores, device_status);
+  return cudaGetLastError() == cudaSuccess ? GLS_OK : GLS_ERR_CUDA;
+}
+
+static int check_sparse(const gls_sparse_rows_t* r) {
+  if (!r || !r->token_ids || !r->logits || r->M <= 0) return GLS_ERR_INVALID_ARG;
+  if (((uintptr_t)r->token_ids) % 4 || ((uintptr_t)r->logits) % 4) return GLS_ERR_MISALIGNED;
+  return GLS_OK;
+}
+
+int gls_draft_sample_sparse(const gls_sparse_rows_t* draft_rows, int B, int K, int J, float inv_temp,
+                            const float* inv_temp_per_draft_host, const gls_noise_t* noise,
+                            int32_t* out_tokens, float* out_scores, uint32_t* device_status,
+                            void* stream) {
+  if (!noise || !out_tokens || !sizes_ok(B, K, J, 1)) return GLS_ERR_INVALID_ARG;
+  int rc = check_sparse(draft_rows);
+  if (rc != GLS_OK) return rc;
+  SweepArgs A;
+  std::memset(&A, 0, sizeof(A));
+  for (int k = 0; k < K; ++k) {
+    const float it = inv_temp_per_draft_host ? inv_temp_per_draft_host[k] : inv_temp;
+    if (!finite_pos(it)) return GLS_ERR_INVALID_ARG;
+    A.inv_t[k] = it;
+  }
+  int spec;
+  rc = fill_noise(A, noise, 0u, &spec);
+  if (rc != GLS_OK) return rc;
+  A.K = K;
+  A.J = J;
+  SparseArgs S;
+  S.ids = draft_rows->token_ids;
+  S.logits = draft_rows->logits;
+  S.sb = draft_rows->stride_b;
+  S.sk = draft_rows->stride_k;
+  S.sj = draft_rows->stride_j;
+  S.M = draft_rows->M;
+  const int rows = B * K * J;
+  cudaStream_t st = (cudaStream_t)stream;
+  const int wpb = 4;
+  const int grid = (rows + wpb - 1) / wpb;
+#define SPARSE_DRAFT(SPEC, R) \
+  sparse_draft_kernel<SPEC, R><<<grid, wpb * 32, 0, st>>>(A, S, rows, out_tokens, out_scores, device_status)
+  const bool r10 = A.rounds == 10;
+  if (spec == 1) { if (r10) SPARSE_DRAFT(1, 10); else SPARSE_DRAFT(1, 0); }
+  else if (spec == 2) { if (r10) SPARSE_DRAFT(2, 10); else SPARSE_DRAFT(2, 0); }
+  else { if (r10) SPARSE_DRAFT(3, 10); else SPARSE_DRAFT(3, 0); }
+#undef SPARSE_DRAFT
+  return cudaGetLastError() == cudaSuccess ? GLS_OK : GLS_ERR_CUDA;
+}
+
+int gls_target_sample_verify_sparse(const gls_sparse_rows_t* target_rows, int B, int K, int L,
+                                    float inv_temp, const int32_t* draft_tokens,
+                                    const gls_noise_t* noise, uint32_t flags, int32_t* out_tokens,
+                                    int32_t* out_num_tokens, uint8_t* out_accept, float* out_scores,
+                                    uint32_t* device_status, void* stream) {
+  if (flags & ~(GLS_COMBINE_ALL | GLS_NO_BONUS)) return GLS_ERR_INVALID_ARG;
+  const int J = L + ((flags & GLS_NO_BONUS) ? 0 : 1);
+  if (!noise || !out_tokens || !out_num_tokens || L < 0 || !sizes_ok(B, K, J, 1))
+    return GLS_ERR_INVALID_ARG;
+  if (L > 0 && (!draft_tokens || !out_accept)) return GLS_ERR_INVALID_ARG;
+  if (!finite_pos(inv_temp)) return GLS_ERR_INVALID_ARG;
+  int rc = check_sparse(target_rows);
+  if (rc != GLS_OK) return rc;
+  if ((flags & GLS_COMBINE_ALL) && target_rows->stride_k != 0 && K > 1) return GLS_ERR_UNSUPPORTED;
+  const size_t smem = (size_t)K * J * sizeof(RowResult);
+  if (smem > kFusedVerifyMaxSmem) return GLS_ERR_UNSUPPORTED;
+  SweepArgs A;
+  std::memset(&A, 0, sizeof(A));
+  for (int k = 0; k < K; ++k) A.inv_t[k] = inv_temp;
+  int spec;
+  rc = fill_noise(A, noise, 0u, &spec);
+  if (rc != GLS_OK) return rc;
+  A.K = K;
+  A.J = J;
+  SparseArgs S;
+  S.ids = target_rows->token_ids;
+  S.logits = target_rows->logits;
+  S.sb = target_rows->stride_b;
+  S.sk = target_rows->stride_k;
+  S.sj = target_rows->stride_j;
+  S.M = target_rows->M;
+  VerifyArgs va;
+  va.B = B; va.K = K; va.L = L; va.J = J;
+  va.flags = flags;
+  va.draft_tokens = draft_tokens;
+  va.out_tokens = out_tokens;
+  va.out_num = out_num_tokens;
+  va.accept = out_accept;
+  va.out_scores = out_scores;
+  va.dev_status = device_status;
+  cudaStream_t st = (cudaStream_t)stream;
+  const int nrows = K * J;
+  const int warps = nrows < kFusedVerifyMaxWarps ? nrows : kFusedVerifyMaxWarps;
+#define SPARSE_VERIFY(SPEC, R) sparse_verify_kernel<SPEC, R><<<B, warps * 32, smem, st>>>(A, S, va)
+  const bool r10 = A.rounds == 10;
+  if (spec == 1) { if (r10) SPARSE_VERIFY(1, 10); else SPARSE_VERIFY(1, 0); }
+  else if (spec == 2) { if (r10) SPARSE_VERIFY(2, 10); else SPARSE_VERIFY(2, 0); }
+  else { if (r10) SPARSE_VERIFY(3, 10); else SPARSE_VERIFY(3, 0); }
+#undef SPARSE_VERIFY
   return cudaGetLastError() == cudaSuccess ? GLS_OK : GLS_ERR_CUDA;
 }
 
