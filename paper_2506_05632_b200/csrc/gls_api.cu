@@ -58,35 +58,39 @@ static Plan make_plan12(long long rows, long long V) {
 
 // noise_spec 3 (a CTA per work item, one partial per warp).  Every item costs a fixed set-up and
 // merge, so rows are cut into as few slices as keep the static round-robin over the resident
-// CTAs balanced: the fewest slices for which the last round of items wastes at most 6 % of the
+// CTAs balanced: the fewest slices for which the last round of items wastes at most 15 % of the
 // machine, or that give every CTA at least 12 items.  Slices are whole CTA iterations and at
-// least kS3MinChunk tokens long, except that small problems may go down to one CTA iteration.
-constexpr int kS3CtasPerSM = GLS_S3_MIN_CTAS;
-constexpr int kS3MinChunk = 4 * kS3CtaTokens;
-static Plan make_plan3(long long rows, long long V) {
+// least four of them long, except that small problems may go down to one CTA iteration.
+template <int DT>
+static Plan make_plan3_t(long long rows, long long V) {
   Plan p;
-  const long long grid = (long long)kNumSMs * kS3CtasPerSM;
-  long long max_splits = (V + kS3MinChunk - 1) / kS3MinChunk;
-  if (rows * max_splits < 2 * grid) max_splits = (V + kS3CtaTokens - 1) / kS3CtaTokens;
+  constexpr int kCtaTok = S3Cfg<DT>::kCtaTokens;
+  constexpr int kMinChunk = 4 * kCtaTok;
+  const long long grid = (long long)kNumSMs * S3Cfg<DT>::kCtasPerSM;
+  long long max_splits = (V + kMinChunk - 1) / kMinChunk;
+  if (rows * max_splits < 2 * grid) max_splits = (V + kCtaTok - 1) / kCtaTok;
   long long splits = 1;
   for (; splits < max_splits; ++splits) {
     const long long items = rows * splits;
     if (items >= 12 * grid) break;
     const long long rounds = (items + grid - 1) / grid;
-    if (items >= grid && (double)(rounds * grid - items) <= 0.06 * (double)(rounds * grid)) break;
+    if (items >= grid && (double)(rounds * grid - items) <= 0.15 * (double)(rounds * grid)) break;
   }
   long long chunk = (V + splits - 1) / splits;
-  chunk = (chunk + kS3CtaTokens - 1) / kS3CtaTokens * kS3CtaTokens;
+  chunk = (chunk + kCtaTok - 1) / kCtaTok * kCtaTok;
   p.chunk = (int)chunk;
   p.splits = (int)((V + chunk - 1) / chunk);
-  p.parts = p.splits * kSweepWarps3;
+  p.parts = p.splits * S3Cfg<DT>::kWarps;
   p.rows = rows;
   plan_layout(p);
   return p;
 }
+static Plan make_plan3(long long rows, long long V, int dtype) {
+  return dtype == GLS_BF16 ? make_plan3_t<kBF16>(rows, V) : make_plan3_t<kF32>(rows, V);
+}
 
-static Plan make_plan(long long rows, long long V, int spec) {
-  return spec == 3 ? make_plan3(rows, V) : make_plan12(rows, V);
+static Plan make_plan(long long rows, long long V, int spec, int dtype) {
+  return spec == 3 ? make_plan3(rows, V, dtype) : make_plan12(rows, V);
 }
 
 // ------------------------------------------------------------------------------------------
@@ -517,7 +521,7 @@ static int run_rows(SweepArgs& A, int dtype, int spec, const Plan& P, void* work
   const bool r10 = A.rounds == 10;
   const bool bf = dtype == GLS_BF16;
   if (spec == 3) {
-    const long long cap = (long long)kNumSMs * kS3CtasPerSM;
+    const long long cap = (long long)kNumSMs * (bf ? S3Cfg<kBF16>::kCtasPerSM : S3Cfg<kF32>::kCtasPerSM);
     const int grid = (int)(P.n_items < cap ? P.n_items : cap);
 #define SWEEP3(DT, R)                                                                       \
   do {                                                                                      \
@@ -525,15 +529,15 @@ static int run_rows(SweepArgs& A, int dtype, int spec, const Plan& P, void* work
     if (A.multi_k > 0) {                                                                    \
       cudaFuncSetAttribute(sweep3_kernel<DT, true, R, true>,                                \
                            cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);         \
-      sweep3_kernel<DT, true, R, true><<<grid, kSweepWarps3 * 32, smem, st>>>(A);           \
+      sweep3_kernel<DT, true, R, true><<<grid, S3Cfg<DT>::kWarps * 32, smem, st>>>(A);           \
     } else if (lse) {                                                                       \
       cudaFuncSetAttribute(sweep3_kernel<DT, true, R>,                                      \
                            cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);         \
-      sweep3_kernel<DT, true, R><<<grid, kSweepWarps3 * 32, smem, st>>>(A);                 \
+      sweep3_kernel<DT, true, R><<<grid, S3Cfg<DT>::kWarps * 32, smem, st>>>(A);                 \
     } else {                                                                                \
       cudaFuncSetAttribute(sweep3_kernel<DT, false, R>,                                     \
                            cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);         \
-      sweep3_kernel<DT, false, R><<<grid, kSweepWarps3 * 32, smem, st>>>(A);                \
+      sweep3_kernel<DT, false, R><<<grid, S3Cfg<DT>::kWarps * 32, smem, st>>>(A);                \
     }                                                                                       \
   } while (0)
     if (bf) { if (r10) SWEEP3(kBF16, 10); else SWEEP3(kBF16, 0); }
@@ -576,7 +580,7 @@ static int run_rows(SweepArgs& A, int dtype, int spec, const Plan& P, void* work
 
 static bool sizes_ok(int B, int K, int J, int64_t V) {
   if (B <= 0 || K <= 0 || K > GLS_MAX_K || J <= 0 || V <= 0) return false;
-  if (V >= (1LL << 31) - 2 * kS3CtaTokens) return false;
+  if (V >= (1LL << 31) - 4 * kS3MaxCtaTokens) return false;
   if ((long long)B * K * J >= (1LL << 31) / 64) return false;
   return true;
 }
@@ -606,11 +610,14 @@ const char* gls_status_string(int status) {
 
 size_t gls_workspace_bytes(int B, int K, int J, int64_t V) {
   if (!sizes_ok(B, K, J, V)) return 0;
+  // the largest need over the noise layouts and element types (the call may use any of them)
   size_t need = make_plan12((long long)B * K * J, V).total;
-  const size_t b = make_plan3((long long)B * K * J, V).total;
-  const size_t c = make_plan3((long long)B * J, V).total;  // fused multi-stream encoder
-  if (b > need) need = b;
-  if (c > need) need = c;
+  for (int dt = 0; dt < 2; ++dt) {
+    const size_t b = make_plan3((long long)B * K * J, V, dt).total;
+    const size_t c = make_plan3((long long)B * J, V, dt).total;  // fused multi-stream encoder
+    if (b > need) need = b;
+    if (c > need) need = c;
+  }
   return need;
 }
 
@@ -631,7 +638,7 @@ int gls_draft_sample(const gls_rows_t* draft_logits, int B, int K, int J, int64_
   int spec;
   rc = fill_noise(A, noise, 0u, &spec);
   if (rc != GLS_OK) return rc;
-  const Plan P = make_plan((long long)B * K * J, V, spec);
+  const Plan P = make_plan((long long)B * K * J, V, spec, draft_logits->dtype);
   if (!workspace || workspace_bytes < P.total) return GLS_ERR_WORKSPACE;
   A.data = draft_logits->data;
   A.sb = draft_logits->stride_b;
@@ -667,7 +674,7 @@ int gls_target_sample_verify(const gls_rows_t* target_logits, int B, int K, int 
   int spec;
   rc = fill_noise(A, noise, 0u, &spec);
   if (rc != GLS_OK) return rc;
-  const Plan P = make_plan((long long)B * K * J, V, spec);
+  const Plan P = make_plan((long long)B * K * J, V, spec, target_logits->dtype);
   if (!workspace || workspace_bytes < P.total) return GLS_ERR_WORKSPACE;
   A.data = target_logits->data;
   A.sb = target_logits->stride_b;
@@ -817,7 +824,7 @@ int gls_compress_select(const gls_rows_t* enc_logw, const gls_rows_t* dec_logw, 
   int spec;
   rc = fill_noise(A, noise, 1u, &spec);
   if (rc != GLS_OK) return rc;
-  const Plan P = make_plan((long long)B * K, N, spec);
+  const Plan P = make_plan((long long)B * K, N, spec, enc_logw->dtype);
   if (!workspace || workspace_bytes < P.total) return GLS_ERR_WORKSPACE;
   cudaStream_t st = (cudaStream_t)stream;
   const RowResult* rowres = (const RowResult*)((char*)workspace + P.off_rows);
@@ -833,7 +840,7 @@ int gls_compress_select(const gls_rows_t* enc_logw, const gls_rows_t* dec_logw, 
   // its own and the epilogue takes the best of the K winners.
   const bool fused_enc = spec == 3 && K <= 8 && N < (1LL << 28);
   if (fused_enc) {
-    const Plan PE = make_plan((long long)B, N, spec);
+    const Plan PE = make_plan((long long)B, N, spec, enc_logw->dtype);
     if (workspace_bytes < PE.total) return GLS_ERR_WORKSPACE;
     A.K = 1;
     A.multi_k = K;
@@ -863,9 +870,12 @@ int gls_compress_select(const gls_rows_t* enc_logw, const gls_rows_t* dec_logw, 
   A.bins = bins;
   A.bins_sb = bins_stride_b;
   A.msg = out_message;
-  rc = run_rows(A, dec_logw->dtype, spec, P, workspace, false, nullptr, nullptr, device_status, st);
+  const Plan PD = make_plan((long long)B * K, N, spec, dec_logw->dtype);
+  if (workspace_bytes < PD.total) return GLS_ERR_WORKSPACE;
+  rc = run_rows(A, dec_logw->dtype, spec, PD, workspace, false, nullptr, nullptr, device_status, st);
   if (rc != GLS_OK) return rc;
-  decoder_epilogue_kernel<<<(B + 127) / 128, 128, 0, st>>>(rowres, B, K, out_enc_index,
+  const RowResult* rowres_d = (const RowResult*)((char*)workspace + PD.off_rows);
+  decoder_epilogue_kernel<<<(B + 127) / 128, 128, 0, st>>>(rowres_d, B, K, out_enc_index,
                                                           out_dec_index, out_match, out_scores);
   return cudaGetLastError() == cudaSuccess ? GLS_OK : GLS_ERR_CUDA;
 }

@@ -22,7 +22,6 @@ namespace gls {
 
 constexpr int kMaxK = 64;
 constexpr int kWarpTokens = 256;  // tokens one warp consumes per iteration (8 per lane)
-constexpr int kSweepWarps3 = 8;   // warps per CTA of the noise_spec 3 sweep
 constexpr float kLog2e = 1.4426950408889634f;
 
 enum : int { kF32 = 0, kBF16 = 1 };

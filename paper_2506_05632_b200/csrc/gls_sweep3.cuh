@@ -29,15 +29,24 @@
 #pragma once
 #include "gls_kernels.cuh"
 
-#ifndef GLS_S3_MIN_CTAS
-#define GLS_S3_MIN_CTAS 3
-#endif
-
 namespace gls {
 
 constexpr int kS3LaneTokens = 16;
 constexpr int kS3WarpTokens = 32 * kS3LaneTokens;               // 512
-constexpr int kS3CtaTokens = kSweepWarps3 * kS3WarpTokens;      // 4096
+
+// Launch shape per element type, chosen by measurement.  bf16 rows are bound by the noise
+// arithmetic: few warps per row and ~100 registers per thread (2 warps x 10 CTAs per SM) beat
+// wider CTAs by 15 %, because longer per-warp items amortise the per-item set-up and more
+// registers let the two generator chains of a step overlap.  fp32 rows are bound by HBM and want
+// the memory parallelism of 8 warps x 3 CTAs.
+template <int DT>
+struct S3Cfg {
+  static constexpr int kWarps = DT == kBF16 ? 2 : 8;
+  static constexpr int kCtasPerSM = DT == kBF16 ? 10 : 3;
+  static constexpr int kCtaTokens = kWarps * kS3WarpTokens;  // tokens one CTA consumes per iteration
+};
+constexpr int kS3MaxWarps = 8;
+constexpr int kS3MaxCtaTokens = kS3MaxWarps * kS3WarpTokens;
 
 // 32 bytes per lane in one instruction (sm_100a): a warp reads 1 KB contiguous.
 struct Words8 {
@@ -187,7 +196,7 @@ __device__ __noinline__ void lse_redo_careful(const char* rowp, int tok0, int n_
                                               float c2, float* lm_out, float* ls_out) {
   float lm = kS3LseFloor, ls = 0.f;
   for (int it = 0; it < n_iter; ++it) {
-    const int tok = tok0 + it * kS3CtaTokens;
+    const int tok = tok0 + it * S3Cfg<DT>::kCtaTokens;
     for (int t = 0; t < kS3LaneTokens; ++t) {
       if (tok + t >= tok_end) break;
       const float a = load_logit<DT>(rowp, tok + t);
@@ -239,9 +248,9 @@ struct S3Entry {
 template <int DT>
 struct S3Shared {
   unsigned long long m_tag;  // (item tag << 32) | ordered code of the CTA-wide bound on the best score
-  S3WarpCtx ctx[kSweepWarps3];
-  Top2 best[kSweepWarps3 * 32];  // per-thread candidates, touched by the batched path only
-  __align__(16) uint32_t queue[kSweepWarps3][S3Entry<DT>::kCap * S3Entry<DT>::kWords];
+  S3WarpCtx ctx[S3Cfg<DT>::kWarps];
+  Top2 best[S3Cfg<DT>::kWarps * 32];  // per-thread candidates, touched by the batched path only
+  __align__(16) uint32_t queue[S3Cfg<DT>::kWarps][S3Entry<DT>::kCap * S3Entry<DT>::kWords];
 };
 extern __shared__ __align__(16) unsigned char s3_smem_raw[];
 template <int DT>
@@ -369,13 +378,15 @@ __device__ __noinline__ uint32_t s3_flush(int rounds_rt, int first, int n, float
 // The kernel
 // ------------------------------------------------------------------------------------------
 template <int DT, bool LSE, int ROUNDS, bool MULTI = false>
-__global__ void __launch_bounds__(kSweepWarps3 * 32, GLS_S3_MIN_CTAS)
+__global__ void __launch_bounds__(S3Cfg<DT>::kWarps * 32, S3Cfg<DT>::kCtasPerSM)
 sweep3_kernel(const __grid_constant__ SweepArgs A) {
   S3Shared<DT>& sh = s3_shared<DT>();
   const int lane = threadIdx.x & 31;
   const int warp = threadIdx.x >> 5;
   constexpr int ES = DT == kBF16 ? 2 : 4;
   constexpr bool PREFETCH = DT == kBF16;       // fp32 groups are 16 registers: no second copy
+  constexpr int kS3CtaTokens = S3Cfg<DT>::kCtaTokens;
+  constexpr int kSweepWarps3 = S3Cfg<DT>::kWarps;
   constexpr int STEP = kS3CtaTokens * ES;      // bytes between a lane's consecutive groups
   typedef Group16<DT> G;
   uint32_t* const queue = sh.queue[warp];
