@@ -24,6 +24,8 @@
  *     (token block, k | domain << 16, position id, sequence id); see gls_uniform() below.
  *   - U is taken in the open interval: v = (integer + 0.5) * 2^-32 or 2^-48, U = 1 - v,
  *     S = -ln U = -log1p(-v).
+ *   - noise_spec 4 builds each group of 16 exponentials from its minimum (an exact sampler of
+ *     16 i.i.d. Exp(1) values; see exp_noise_group_min() below).
  *   - NaN and +inf logits are excluded (they cannot define a probability); -inf is a masked token.
  *
  * Pins (tests/test_oracle_*.py): a second pure-Python Philox, inversion of the Philox round,
@@ -85,13 +87,15 @@ void glso_philox4x32(const uint32_t ctr[4], const uint32_t key[2], int rounds, u
 typedef struct {
   uint64_t seed;
   int rounds;       /* Philox rounds (10 by default) */
-  int spec;         /* 1, 2 or 3 */
+  int spec;         /* 1, 2, 3 or 4 */
   uint32_t domain;  /* 0 decoding, 1 compression */
   uint32_t seq, pos, k;
 } glso_key_t;
 
 /* The uniform v in (0,1) of token i under the given key: Algorithm 1's U_i^(k) is 1 - v. */
+double glso_exp_noise(const glso_key_t* nk, int64_t i);
 double glso_uniform(const glso_key_t* nk, int64_t i) {
+  if (nk->spec == 4) return -expm1(-glso_exp_noise(nk, i)); /* derived: v = 1 - exp(-S) */
   uint32_t key[2] = {(uint32_t)(nk->seed & 0xffffffffu), (uint32_t)(nk->seed >> 32)};
   uint32_t out[4];
   if (nk->spec == 1) {
@@ -121,14 +125,59 @@ double glso_uniform(const glso_key_t* nk, int64_t i) {
   }
 }
 
+/*
+ * noise_spec 4: the 16 exponentials of tokens 16g .. 16g+15 ("group" g) are built from their
+ * minimum.  If E_0..E_15 are i.i.d. Exp(1), then M = min_t E_t ~ Exp(16), its position is uniform
+ * on 0..15 and independent of M, and the other fifteen, less M, are again i.i.d. Exp(1) and
+ * independent of both (memorylessness; Renyi's representation of exponential order statistics).
+ * Read backwards this is a sampler of 16 i.i.d. Exp(1) variables, i.e. of Sec. 3's S_i = -ln U_i:
+ *     M   = -log1p(-v0) / 16,   v0 = (w * 2^16 + r + 0.5) * 2^-48
+ *     S_i = M                   if (i mod 16) == loc
+ *     S_i = M + (-log1p(-v_i))  otherwise,  v_i = (u_i + 0.5) * 2^-32
+ * with, for the stream (seed, seq, pos, k, domain):
+ *     w   = word (g >> 5) & 3 of Philox(counter ((g >> 7) << 5 | (g & 31), k | domain << 16, pos, seq))
+ *           (128 consecutive groups share 32 generator calls, group g and g + 32 the same call)
+ *     r   = low 16 bits, loc = bits 16..19 of word 0 of Philox((g, k | (domain + 2) << 16, pos, seq))
+ *     u_i = word i & 3 of Philox((i >> 2, k | (domain + 4) << 16, pos, seq)).
+ * A sweep that knows w alone already knows S_i >= M >= w * 2^-36 for all 16 tokens of the group.
+ */
+static double exp_noise_group_min(const glso_key_t* nk, int64_t i) {
+  uint32_t key[2] = {(uint32_t)(nk->seed & 0xffffffffu), (uint32_t)(nk->seed >> 32)};
+  uint32_t out[4];
+  const int64_t g = i >> 4;
+  uint32_t cc[4] = {(uint32_t)(((g >> 7) << 5) | (g & 31)), nk->k | (nk->domain << 16), nk->pos, nk->seq};
+  glso_philox4x32(cc, key, nk->rounds, out);
+  const uint32_t w = out[(g >> 5) & 3];
+  uint32_t cr[4] = {(uint32_t)g, nk->k | ((nk->domain + 2u) << 16), nk->pos, nk->seq};
+  glso_philox4x32(cr, key, nk->rounds, out);
+  const uint32_t r = out[0] & 0xffffu;
+  const int loc = (int)((out[0] >> 16) & 15u);
+  /* w * 2^16 + r + 0.5 < 2^48 + 1: exact in fp64 */
+  const double v0 = ((double)w * 65536.0 + (double)r + 0.5) * 0x1p-48;
+  const double M = -log1p(-v0) / 16.0;
+  if ((int)(i & 15) == loc) return M;
+  uint32_t ct[4] = {(uint32_t)(i >> 2), nk->k | ((nk->domain + 4u) << 16), nk->pos, nk->seq};
+  glso_philox4x32(ct, key, nk->rounds, out);
+  const double vi = ((double)out[i & 3] + 0.5) * 0x1p-32;
+  return M + (-log1p(-vi));
+}
+
 /* S = -ln U = -log1p(-v) ~ Exp(1)  (Sec. 3, "S_i^(k) = -ln U_i^(k)") */
-double glso_exp_noise(const glso_key_t* nk, int64_t i) { return -log1p(-glso_uniform(nk, i)); }
+double glso_exp_noise(const glso_key_t* nk, int64_t i) {
+  if (nk->spec == 4) return exp_noise_group_min(nk, i);
+  return -log1p(-glso_uniform(nk, i));
+}
 
 /* Flat wrappers for the Python side (ctypes cannot pass the struct by value portably). */
 double glso_uniform_flat(uint64_t seed, int rounds, int spec, uint32_t domain, uint32_t seq,
                          uint32_t pos, uint32_t k, int64_t i) {
   glso_key_t nk = {seed, rounds, spec, domain, seq, pos, k};
   return glso_uniform(&nk, i);
+}
+double glso_exp_noise_flat(uint64_t seed, int rounds, int spec, uint32_t domain, uint32_t seq,
+                           uint32_t pos, uint32_t k, int64_t i) {
+  glso_key_t nk = {seed, rounds, spec, domain, seq, pos, k};
+  return glso_exp_noise(&nk, i);
 }
 void glso_exp_noise_row(uint64_t seed, int rounds, int spec, uint32_t domain, uint32_t seq,
                         uint32_t pos, uint32_t k, int64_t V, double* out) {
@@ -258,7 +307,7 @@ typedef struct {
   uint32_t seq_base;
   const uint32_t* seq_ids; /* host array [B] or NULL */
   uint32_t pos_base;
-  uint32_t noise_spec; /* 1, 2 or 3 */
+  uint32_t noise_spec; /* 1, 2, 3 or 4 */
   uint32_t rounds;
   uint32_t flags;
 } glso_noise_t;

@@ -93,6 +93,13 @@ def uniform(seed, seq, pos, k, i, spec=3, domain=0, rounds=10):
                                          int(pos), int(k), int(i)))
 
 
+def exp_noise(seed, seq, pos, k, i, spec=3, domain=0, rounds=10):
+    f = lib().glso_exp_noise_flat
+    f.restype = C.c_double
+    return float(f(C.c_uint64(int(seed)), C.c_int(int(rounds)), C.c_int(int(spec)), C.c_uint32(int(domain)),
+                   C.c_uint32(int(seq)), C.c_uint32(int(pos)), C.c_uint32(int(k)), C.c_int64(int(i))))
+
+
 def exp_noise_row(seed, seq, pos, k, V, spec=3, domain=0, rounds=10):
     """S_i = -ln U_i for i < V under one (sequence, position, draft) key, fp64."""
     out = np.empty(int(V), dtype=np.float64)

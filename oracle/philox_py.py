@@ -70,3 +70,28 @@ def uniform_numerator(seed, seq, pos, k, i, spec=2, domain=0, rounds=10):
     h = (bits128 >> (16 * (i & 7))) & 0xFFFF
     fine = philox4x32((i >> 2, k | ((domain + 2) << 16), pos, seq), key, rounds)
     return (h << 32) | fine[i & 3], 48
+
+
+def group_min_fields(seed, seq, pos, k, i, domain=0, rounds=10):
+    """noise_spec 4, the integer fields behind token i's exponential: (w, r, loc, u).
+
+    w: 32 coarse bits of the group's minimum, r: its 16 refinement bits, loc: position of the
+    minimum in the group of 16, u: the token's own 32-bit word (unused when i % 16 == loc)."""
+    key = (seed & MASK, (seed >> 32) & MASK)
+    g = i // 16
+    call, word = (g // 128) * 32 + g % 32, (g // 32) % 4
+    w = philox4x32((call, k | (domain << 16), pos, seq), key, rounds)[word]
+    first = philox4x32((g, k | ((domain + 2) << 16), pos, seq), key, rounds)[0]
+    r, loc = first % 65536, (first // 65536) % 16
+    u = philox4x32((i // 4, k | ((domain + 4) << 16), pos, seq), key, rounds)[i % 4]
+    return w, r, loc, u
+
+
+def exp_noise_group_min(seed, seq, pos, k, i, domain=0, rounds=10):
+    """noise_spec 4: S_i = M at the group's minimum position, M + Exp(1) elsewhere, M ~ Exp(16)."""
+    import math
+    w, r, loc, u = group_min_fields(seed, seq, pos, k, i, domain, rounds)
+    m = -math.log1p(-((w * 65536 + r) + 0.5) / 2.0**48) / 16.0
+    if i % 16 == loc:
+        return m
+    return m + -math.log1p(-(u + 0.5) / 2.0**32)

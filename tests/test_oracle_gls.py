@@ -35,7 +35,7 @@ def _chi2_p(samples, probs):
     return stats.chisquare(counts, probs * counts.sum()).pvalue
 
 
-@pytest.mark.parametrize("spec", [1, 2, 3])
+@pytest.mark.parametrize("spec", [1, 2, 3, 4])
 def test_config1_marginals_and_lml(oracle, spec):
     """Proposition 1 (X^(k) ~ p, Y ~ q) and Theorem 1 (acceptance >= LML) on configuration 1:
     V = 16, K = 2, 1e5 trials."""
@@ -161,7 +161,7 @@ def test_exact_joint_from_the_proof(oracle):
         assert abs(got - want) < 4 * np.sqrt(want * (1 - want) / n)
 
 
-@pytest.mark.parametrize("spec", [1, 2, 3])
+@pytest.mark.parametrize("spec", [1, 2, 3, 4])
 def test_brute_force_linear_domain(oracle, spec):
     """A second, deliberately naive evaluator: explicit probabilities, S/p ratios in the linear
     domain, min over k then argmin over i exactly as Algorithm 1 is printed."""

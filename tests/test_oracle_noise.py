@@ -85,7 +85,7 @@ def test_uniform_bit_fields_match_second_implementation(oracle):
 
 def test_noise_is_exp1_and_uniform(oracle):
     n = 1_000_000
-    for spec in (1, 2, 3):
+    for spec in (1, 2, 3, 4):
         S = oracle.exp_noise_row(SEED, seq=11, pos=3, k=1, V=n, spec=spec)
         assert np.all(S > 0) and np.all(np.isfinite(S))
         assert abs(S.mean() - 1.0) < 5e-3 and abs(S.var() - 1.0) < 1.5e-2
@@ -111,6 +111,7 @@ def test_streams_differ_across_key_components(oracle):
         oracle.exp_noise_row(SEED ^ (1 << 40), V=V, **base),
         oracle.exp_noise_row(SEED, V=V, spec=1, **base),
         oracle.exp_noise_row(SEED, V=V, spec=2, **base),
+        oracle.exp_noise_row(SEED, V=V, spec=4, **base),
     ]
     for o in others:
         assert not np.any(o == ref)
@@ -148,3 +149,61 @@ def test_spec3_coarse_byte_bounds_the_uniform(oracle):
     # tokens with a zero coarse byte are 1/256 of all: binomial(65536, 1/256), mean 256, sd 16
     zeros = sum(philox_py.uniform_numerator(SEED, 9, 0, 0, i, 3, 0)[0] >> 40 == 0 for i in range(65536))
     assert 256 - 5 * 16 < zeros < 256 + 5 * 16
+
+
+def test_spec4_matches_second_implementation(oracle):
+    rng = np.random.default_rng(5)
+    for domain in (0, 1):
+        for _ in range(600):
+            seq, pos = int(rng.integers(0, 2**32)), int(rng.integers(0, 2**32))
+            k, i = int(rng.integers(0, 64)), int(rng.integers(0, 2**31 - 1))
+            want = philox_py.exp_noise_group_min(SEED, seq, pos, k, i, domain)
+            assert oracle.exp_noise(SEED, seq, pos, k, i, spec=4, domain=domain) == want
+    # whole rows, bit for bit (same libm on both sides), across several groups and call blocks
+    row = oracle.exp_noise_row(SEED, seq=3, pos=4, k=5, V=5000, spec=4)
+    for i in list(range(0, 5000, 37)) + [15, 16, 511, 512, 2047, 2048, 4095, 4096, 4999]:
+        assert row[i] == philox_py.exp_noise_group_min(SEED, 3, 4, 5, i)
+
+
+def test_spec4_group_structure(oracle):
+    """The construction behind noise_spec 4: the group minimum is Exp(16), sits at a uniform
+    position, the other fifteen exceed it by Exp(1), and the coarse word bounds all sixteen."""
+    G = 40000
+    S = oracle.exp_noise_row(SEED, seq=21, pos=1, k=0, V=16 * G, spec=4).reshape(G, 16)
+    M = S.min(axis=1)
+    assert stats.kstest(16.0 * M, "expon").pvalue > 1e-3
+    loc = S.argmin(axis=1)
+    assert stats.chisquare(np.bincount(loc, minlength=16)).pvalue > 1e-4
+    rest = (S - M[:, None])[np.arange(16)[None, :] != loc[:, None]]
+    assert rest.size == 15 * G and np.all(rest > 0)
+    assert stats.kstest(rest, "expon").pvalue > 1e-3
+    # the position and the fields are the ones the second implementation reads
+    for g in range(0, G, 997):
+        w, r, lo, _ = philox_py.group_min_fields(SEED, 21, 1, 0, 16 * g)
+        assert lo == loc[g]
+        assert M[g] >= w * 2.0**-36  # what a sweep may conclude from the coarse word alone
+        assert M[g] == -math.log1p(-((w * 65536 + r) + 0.5) / 2.0**48) / 16.0
+
+
+def test_spec4_tokens_of_a_group_are_independent(oracle):
+    """Joint law: within a group the sixteen values are i.i.d. Exp(1), so their sum is Gamma(16),
+    pairs are uncorrelated (also in the log domain, where the race is decided), and the minimum
+    is independent of where it sits."""
+    G = 60000
+    S = oracle.exp_noise_row(SEED, seq=22, pos=2, k=3, V=16 * G, spec=4).reshape(G, 16)
+    assert stats.kstest(S.sum(axis=1), "gamma", args=(16,)).pvalue > 1e-3
+    assert stats.kstest(S[:, :2].sum(axis=1), "gamma", args=(2,)).pvalue > 1e-3
+    c = np.corrcoef(S.T)
+    assert np.max(np.abs(c - np.eye(16))) < 5.0 / math.sqrt(G)
+    cl = np.corrcoef(np.log(S).T)
+    assert np.max(np.abs(cl - np.eye(16))) < 5.0 / math.sqrt(G)
+    # second smallest minus smallest is Exp(15) (gap between order statistics)
+    srt = np.sort(S, axis=1)
+    assert stats.kstest(15.0 * (srt[:, 1] - srt[:, 0]), "expon").pvalue > 1e-3
+    # neighbouring groups, and groups 32 apart (same generator call), are unrelated
+    M = S.min(axis=1)
+    assert abs(np.corrcoef(M[:-1], M[1:])[0, 1]) < 5.0 / math.sqrt(G)
+    assert abs(np.corrcoef(M[:-32], M[32:])[0, 1]) < 5.0 / math.sqrt(G)
+    # every token's marginal is Exp(1) on its own
+    for t in (0, 7, 15):
+        assert stats.kstest(S[:, t], "expon").pvalue > 1e-3
