@@ -13,6 +13,7 @@
 #include "../../include/gls.h"
 #include "gls_kernels.cuh"
 #include "gls_sweep3.cuh"
+#include "gls_sweep4.cuh"
 
 namespace gls {
 
@@ -89,8 +90,38 @@ static Plan make_plan3(long long rows, long long V, int dtype) {
   return dtype == GLS_BF16 ? make_plan3_t<kBF16>(rows, V) : make_plan3_t<kF32>(rows, V);
 }
 
+// noise_spec 4: the same rule with that sweep's CTA shape (a warp step is 2048 tokens).
+template <int DT>
+static Plan make_plan4_t(long long rows, long long V) {
+  Plan p;
+  constexpr int kCtaTok = S4Cfg<DT>::kCtaTokens;
+  constexpr int kMinChunk = 4 * kCtaTok;
+  const long long grid = (long long)kNumSMs * S4Cfg<DT>::kCtasPerSM;
+  long long max_splits = (V + kMinChunk - 1) / kMinChunk;
+  if (rows * max_splits < 2 * grid) max_splits = (V + kCtaTok - 1) / kCtaTok;
+  long long splits = 1;
+  for (; splits < max_splits; ++splits) {
+    const long long items = rows * splits;
+    if (items >= 12 * grid) break;
+    const long long rounds = (items + grid - 1) / grid;
+    if (items >= grid && (double)(rounds * grid - items) <= 0.15 * (double)(rounds * grid)) break;
+  }
+  long long chunk = (V + splits - 1) / splits;
+  chunk = (chunk + kCtaTok - 1) / kCtaTok * kCtaTok;
+  p.chunk = (int)chunk;
+  p.splits = (int)((V + chunk - 1) / chunk);
+  p.parts = p.splits * S4Cfg<DT>::kWarps;
+  p.rows = rows;
+  plan_layout(p);
+  return p;
+}
+static Plan make_plan4(long long rows, long long V, int dtype) {
+  return dtype == GLS_BF16 ? make_plan4_t<kBF16>(rows, V) : make_plan4_t<kF32>(rows, V);
+}
+
 static Plan make_plan(long long rows, long long V, int spec, int dtype) {
-  return spec == 3 ? make_plan3(rows, V, dtype) : make_plan12(rows, V);
+  return spec == 4 ? make_plan4(rows, V, dtype)
+                   : spec == 3 ? make_plan3(rows, V, dtype) : make_plan12(rows, V);
 }
 
 // ------------------------------------------------------------------------------------------
@@ -369,8 +400,7 @@ __device__ __forceinline__ RowResult sparse_row(const SweepArgs& A, const Sparse
     if (!sparse_keep(id, a)) continue;
     const double al = (double)a * inv_t;
     amax = fmax(amax, al);
-    const double v = uniform_exact<SPEC, ROUNDS>(A, sk, id);
-    const double sc = al - log(-log1p(-v));
+    const double sc = al - log(noise_exact<SPEC, ROUNDS>(A, sk, id));
     if (bid < 0 || sc > best || (sc == best && id < bid)) {
       best = sc;
       bid = id;
@@ -444,7 +474,7 @@ static int fill_noise(SweepArgs& A, const gls_noise_t* nz, uint32_t domain, int*
   const int rounds = nz->rounds ? (int)nz->rounds : 10;
   if (rounds < 7 || rounds > 16) return GLS_ERR_INVALID_ARG;
   const int spec = nz->noise_spec ? (int)nz->noise_spec : 3;
-  if (spec < 1 || spec > 3) return GLS_ERR_INVALID_ARG;
+  if (spec < 1 || spec > 4) return GLS_ERR_INVALID_ARG;
   if (nz->flags & ~GLS_NOISE_SHARED_ACROSS_K) return GLS_ERR_INVALID_ARG;
   uint32_t k0 = (uint32_t)(nz->seed & 0xffffffffu), k1 = (uint32_t)(nz->seed >> 32);
   for (int r = 0; r < 16; ++r) {
@@ -520,7 +550,24 @@ static int run_rows(SweepArgs& A, int dtype, int spec, const Plan& P, void* work
   cudaError_t err;
   const bool r10 = A.rounds == 10;
   const bool bf = dtype == GLS_BF16;
-  if (spec == 3) {
+  if (spec == 4) {
+    const long long cap = (long long)kNumSMs * (bf ? S4Cfg<kBF16>::kCtasPerSM : S4Cfg<kF32>::kCtasPerSM);
+    const int grid = (int)(P.n_items < cap ? P.n_items : cap);
+#define SWEEP4(DT, R)                                                                       \
+  do {                                                                                      \
+    const size_t smem = sizeof(S4Shared<DT>);                                               \
+    if (A.multi_k > 0)                                                                      \
+      sweep4_kernel<DT, true, R, true><<<grid, S4Cfg<DT>::kWarps * 32, smem, st>>>(A);      \
+    else if (lse)                                                                           \
+      sweep4_kernel<DT, true, R><<<grid, S4Cfg<DT>::kWarps * 32, smem, st>>>(A);            \
+    else                                                                                    \
+      sweep4_kernel<DT, false, R><<<grid, S4Cfg<DT>::kWarps * 32, smem, st>>>(A);           \
+  } while (0)
+    if (bf) { if (r10) SWEEP4(kBF16, 10); else SWEEP4(kBF16, 0); }
+    else { if (r10) SWEEP4(kF32, 10); else SWEEP4(kF32, 0); }
+#undef SWEEP4
+    err = cudaGetLastError();
+  } else if (spec == 3) {
     const long long cap = (long long)kNumSMs * (bf ? S3Cfg<kBF16>::kCtasPerSM : S3Cfg<kF32>::kCtasPerSM);
     const int grid = (int)(P.n_items < cap ? P.n_items : cap);
 #define SWEEP3(DT, R)                                                                       \
@@ -568,11 +615,13 @@ static int run_rows(SweepArgs& A, int dtype, int spec, const Plan& P, void* work
   if (bf) {
     if (spec == 1) err = r10 ? FIN_CALL(kBF16, 1, 10) : FIN_CALL(kBF16, 1, 0);
     else if (spec == 2) err = r10 ? FIN_CALL(kBF16, 2, 10) : FIN_CALL(kBF16, 2, 0);
-    else err = r10 ? FIN_CALL(kBF16, 3, 10) : FIN_CALL(kBF16, 3, 0);
+    else if (spec == 3) err = r10 ? FIN_CALL(kBF16, 3, 10) : FIN_CALL(kBF16, 3, 0);
+    else err = r10 ? FIN_CALL(kBF16, 4, 10) : FIN_CALL(kBF16, 4, 0);
   } else {
     if (spec == 1) err = r10 ? FIN_CALL(kF32, 1, 10) : FIN_CALL(kF32, 1, 0);
     else if (spec == 2) err = r10 ? FIN_CALL(kF32, 2, 10) : FIN_CALL(kF32, 2, 0);
-    else err = r10 ? FIN_CALL(kF32, 3, 10) : FIN_CALL(kF32, 3, 0);
+    else if (spec == 3) err = r10 ? FIN_CALL(kF32, 3, 10) : FIN_CALL(kF32, 3, 0);
+    else err = r10 ? FIN_CALL(kF32, 4, 10) : FIN_CALL(kF32, 4, 0);
   }
 #undef FIN_CALL
   return err == cudaSuccess ? GLS_OK : GLS_ERR_CUDA;
@@ -580,7 +629,7 @@ static int run_rows(SweepArgs& A, int dtype, int spec, const Plan& P, void* work
 
 static bool sizes_ok(int B, int K, int J, int64_t V) {
   if (B <= 0 || K <= 0 || K > GLS_MAX_K || J <= 0 || V <= 0) return false;
-  if (V >= (1LL << 31) - 4 * kS3MaxCtaTokens) return false;
+  if (V >= (1LL << 31) - 4 * kS4MaxCtaTokens) return false;
   if ((long long)B * K * J >= (1LL << 31) / 64) return false;
   return true;
 }
@@ -617,6 +666,10 @@ size_t gls_workspace_bytes(int B, int K, int J, int64_t V) {
     const size_t c = make_plan3((long long)B * J, V, dt).total;  // fused multi-stream encoder
     if (b > need) need = b;
     if (c > need) need = c;
+    const size_t d = make_plan4((long long)B * K * J, V, dt).total;
+    const size_t e = make_plan4((long long)B * J, V, dt).total;
+    if (d > need) need = d;
+    if (e > need) need = e;
   }
   return need;
 }
@@ -746,7 +799,8 @@ int gls_draft_sample_sparse(const gls_sparse_rows_t* draft_rows, int B, int K, i
   const bool r10 = A.rounds == 10;
   if (spec == 1) { if (r10) SPARSE_DRAFT(1, 10); else SPARSE_DRAFT(1, 0); }
   else if (spec == 2) { if (r10) SPARSE_DRAFT(2, 10); else SPARSE_DRAFT(2, 0); }
-  else { if (r10) SPARSE_DRAFT(3, 10); else SPARSE_DRAFT(3, 0); }
+  else if (spec == 3) { if (r10) SPARSE_DRAFT(3, 10); else SPARSE_DRAFT(3, 0); }
+  else { if (r10) SPARSE_DRAFT(4, 10); else SPARSE_DRAFT(4, 0); }
 #undef SPARSE_DRAFT
   return cudaGetLastError() == cudaSuccess ? GLS_OK : GLS_ERR_CUDA;
 }
@@ -798,7 +852,8 @@ int gls_target_sample_verify_sparse(const gls_sparse_rows_t* target_rows, int B,
   const bool r10 = A.rounds == 10;
   if (spec == 1) { if (r10) SPARSE_VERIFY(1, 10); else SPARSE_VERIFY(1, 0); }
   else if (spec == 2) { if (r10) SPARSE_VERIFY(2, 10); else SPARSE_VERIFY(2, 0); }
-  else { if (r10) SPARSE_VERIFY(3, 10); else SPARSE_VERIFY(3, 0); }
+  else if (spec == 3) { if (r10) SPARSE_VERIFY(3, 10); else SPARSE_VERIFY(3, 0); }
+  else { if (r10) SPARSE_VERIFY(4, 10); else SPARSE_VERIFY(4, 0); }
 #undef SPARSE_VERIFY
   return cudaGetLastError() == cudaSuccess ? GLS_OK : GLS_ERR_CUDA;
 }
@@ -838,7 +893,7 @@ int gls_compress_select(const gls_rows_t* enc_logw, const gls_rows_t* dec_logw, 
   // With the default noise layout, up to 8 streams and N < 2^28 it runs fused: each row is read
   // and summed once and the K streams share one bound; otherwise every stream sweeps the row on
   // its own and the epilogue takes the best of the K winners.
-  const bool fused_enc = spec == 3 && K <= 8 && N < (1LL << 28);
+  const bool fused_enc = spec >= 3 && K <= 8 && N < (1LL << 28);
   if (fused_enc) {
     const Plan PE = make_plan((long long)B, N, spec, enc_logw->dtype);
     if (workspace_bytes < PE.total) return GLS_ERR_WORKSPACE;

@@ -172,6 +172,28 @@ __device__ __forceinline__ double uniform_exact(const SweepArgs& A, const Stream
   }
 }
 
+// The exponential S_i of token i in fp64.  noise_spec 1-3: S = -log1p(-v) (Sec. 3: S = -ln U,
+// U = 1 - v).  noise_spec 4: the group of 16 is built from its minimum M = -log1p(-v0) / 16,
+// v0 = (w * 2^16 + r + 0.5) * 2^-48: S = M at position loc of the group, M - log1p(-v_i) at the
+// others, v_i = (u_i + 0.5) * 2^-32 (an exact sampler of 16 i.i.d. Exp(1) values).
+template <int SPEC, int ROUNDS>
+__device__ __forceinline__ double noise_exact(const SweepArgs& A, const StreamKey& sk, int i) {
+  if (SPEC != 4) return -log1p(-uniform_exact<SPEC, ROUNDS>(A, sk, i));
+  uint32_t o[4];
+  const uint32_t g = (uint32_t)i >> 4;
+  philox4x32<ROUNDS>(A.rk, A.rounds, ((g >> 7) << 5) | (g & 31u), sk.c1, sk.pos, sk.seq, o);
+  const uint32_t j = (g >> 5) & 3u;
+  const uint32_t w = j == 0 ? o[0] : j == 1 ? o[1] : j == 2 ? o[2] : o[3];
+  philox4x32<ROUNDS>(A.rk, A.rounds, g, sk.c1 + (2u << 16), sk.pos, sk.seq, o);
+  const uint32_t r = o[0] & 0xffffu, loc = (o[0] >> 16) & 15u;
+  const double m = -log1p(-((double)w * 65536.0 + (double)r + 0.5) * 0x1p-48) / 16.0;
+  if (((uint32_t)i & 15u) == loc) return m;
+  philox4x32<ROUNDS>(A.rk, A.rounds, (uint32_t)i >> 2, sk.c1 + (4u << 16), sk.pos, sk.seq, o);
+  const uint32_t t = (uint32_t)i & 3u;
+  const uint32_t u = t == 0 ? o[0] : t == 1 ? o[1] : t == 2 ? o[2] : o[3];
+  return m + (-log1p(-((double)u + 0.5) * 0x1p-32));
+}
+
 template <int DT>
 __device__ __forceinline__ float load_logit(const void* row, long long i) {
   if (DT == kF32) return __ldg((const float*)row + i);
@@ -183,8 +205,7 @@ template <int DT, int SPEC, int ROUNDS>
 __device__ __noinline__ double exact_score(const SweepArgs& A, const void* row,
                                            const StreamKey& sk, int i, float inv_t) {
   const double a = (double)load_logit<DT>(row, i) * (double)inv_t;
-  const double v = uniform_exact<SPEC, ROUNDS>(A, sk, i);
-  return a - log(-log1p(-v));
+  return a - log(noise_exact<SPEC, ROUNDS>(A, sk, i));
 }
 
 // fp32 score from the full uniform; |error| is well below score_slack().

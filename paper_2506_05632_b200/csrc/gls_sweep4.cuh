@@ -1,0 +1,448 @@
+// gls_sweep4.cuh -- the vocabulary sweep for noise_spec 4 (groups of 16 exponentials built from
+// their minimum).
+//
+// Under noise_spec 4 the 16 tokens 16g .. 16g+15 of group g share one number M_g ~ Exp(16), the
+// smallest of their 16 exponentials: S_i = M_g at one uniformly placed token and M_g + Exp(1) at
+// the other fifteen -- an exact sampler of 16 i.i.d. Exp(1) values (memorylessness), i.e. of
+// Sec. 3's S_i = -ln U_i of arXiv 2506.05632.  One Philox4x32 call yields the 32 coarse bits w of
+// M for FOUR groups, so the generator -- whose 32x32->64-bit multiplies are the scarcest
+// resource of this path on sm_100a -- runs once per 64 tokens, and
+//     S_i >= M_g = -log1p(-v0) / 16 >= v0 / 16 >= w * 2^-36        for every token of the group.
+// With m a lower bound on the row's best score, a token can only matter if S_i <= exp(a_i - m)
+// (a_i = logit_i / T), hence a group only if  w * 2^-32 <= 16 * exp(max a - m): one fused
+// multiply-add, one ex2 and one compare per 16 tokens.  A few dozen groups per row pass.  They
+// are not examined on the spot: the lane pushes (w, g) on a small per-warp queue in shared
+// memory and the sweep goes on; when 32 groups are queued the warp evaluates them together, one
+// group per lane (the 16 refinement bits and the position of the minimum from a second
+// generator stream, a per-token test against M, and for the survivors their own Exp(1) from a
+// third stream and the fp32 score a_i - ln S_i).  The filter has no false negatives, so the
+// result equals a full evaluation (Sec. 3 step 2 / Algorithm 2 draft loop and Y_j line, log
+// domain).
+//
+// Work decomposition: a work item is one (row, vocabulary slice), owned by one CTA.  Per step a
+// warp takes 2048 contiguous tokens: lane l holds groups l, l + 32, l + 64, l + 96 of the step
+// (four 32-byte loads of bf16, eight of fp32, each warp-wide load 1 KB contiguous), which are
+// exactly the four groups served by its generator call.  Warps never wait on one another: they
+// share the bound m through one tagged shared-memory word, each warp writes its own partial
+// result, and the split-V reduction merges them.  The batched evaluation is called from an outer
+// loop so that the hot loop contains no call.  A fused variant (MULTI) races one row under
+// several noise streams at once for the compression encoder of Sec. 5.1.
+#pragma once
+#include "gls_sweep3.cuh"
+
+namespace gls {
+
+#ifndef GLS_S4_BF16_WARPS
+#define GLS_S4_BF16_WARPS 2
+#define GLS_S4_BF16_CTAS 10
+#endif
+#ifndef GLS_S4_F32_WARPS
+#define GLS_S4_F32_WARPS 4
+#define GLS_S4_F32_CTAS 4
+#endif
+constexpr int kS4LaneGroups = 4;                                // groups per lane and step
+constexpr int kS4WarpGroups = 32 * kS4LaneGroups;               // 128
+constexpr int kS4WarpTokens = 16 * kS4WarpGroups;               // 2048
+// Groups per warp queue: a batch is taken at 32 queued groups, and one step can add 128 more.
+constexpr int kS4QueueCap = 32 + kS4WarpGroups;
+
+// Launch shape per element type.  A lane holds its four groups in registers (32 for bf16, 64 for
+// fp32), so fp32 rows run with a 128-register budget.
+template <int DT>
+struct S4Cfg {
+  static constexpr int kWarps = DT == kBF16 ? GLS_S4_BF16_WARPS : GLS_S4_F32_WARPS;
+  static constexpr int kCtasPerSM = DT == kBF16 ? GLS_S4_BF16_CTAS : GLS_S4_F32_CTAS;
+  static constexpr int kCtaTokens = kWarps * kS4WarpTokens;
+};
+constexpr int kS4MaxCtaTokens = 8 * kS4WarpTokens;
+
+struct S4WarpCtx {  // what the batched path needs to know about the warp's current work item
+  const char* rowp;
+  const uint8_t* bins;
+  uint32_t c1, pos, seq;
+  uint32_t key0, key1;
+  float inv_t;
+  int msg, tok_end;
+};
+template <int DT>
+struct S4Shared {
+  unsigned long long m_tag;  // (item tag << 32) | ordered code of the CTA-wide bound on the best score
+  S4WarpCtx ctx[S4Cfg<DT>::kWarps];
+  Top2 best[S4Cfg<DT>::kWarps * 32];
+  uint2 queue[S4Cfg<DT>::kWarps][kS4QueueCap];  // (coarse word, group | stream << 28)
+};
+template <int DT>
+__device__ __forceinline__ S4Shared<DT>& s4_shared() {
+  return *reinterpret_cast<S4Shared<DT>*>(s3_smem_raw);
+}
+
+// Exp(1) from the uniform v = (word + frac) * 2^-32, frac in (0, 1) standing for further bits
+// and the half-step offset: -log1p(-v), through the complement 1 - v = (~word + 1 - frac) * 2^-32
+// when v > 1/2, so that the conversion of the word to fp32 can never round v up to 1.
+__device__ __forceinline__ float exp1_from_word(uint32_t word, float frac) {
+  if (word & 0x80000000u) return -logf(fmaf((float)(~word), 0x1p-32f, (1.0f - frac) * 0x1p-32f));
+  return -log1pf(-fmaf((float)word, 0x1p-32f, frac * 0x1p-32f));
+}
+
+// lower bound on word * 2^-32 from its top 23 bits, without an integer-to-float conversion
+__device__ __forceinline__ float coarse_lower(uint32_t w) {
+  return __uint_as_float(0x3f800000u | (w >> 9)) - 1.0f;
+}
+
+// generator call that serves group g (and g + 32, g + 64, g + 96 when g mod 128 < 32)
+__device__ __forceinline__ uint32_t s4_call_index(uint32_t g) { return ((g >> 7) << 5) | (g & 31u); }
+
+// ------------------------------------------------------------------------------------------
+// Batched evaluation of queued groups: lane l < n takes entry first + l of its warp's queue.
+// The lane draws the group's refinement bits and the position of its minimum, computes M, keeps
+// the tokens with a_t - ln M above the bound (S_t >= M), and scores the survivors in fp32, one
+// per round, drawing the token's own exponential unless it is the group's minimum.  Returns the
+// best lower bound found (ordered code, 0 if none).
+// ------------------------------------------------------------------------------------------
+template <int DT, int ROUNDS, bool MULTI>
+__device__ __noinline__ uint32_t s4_flush(int rounds_rt, int first, int n, float nm) {
+  S4Shared<DT>& sh = s4_shared<DT>();
+  const int lane = threadIdx.x & 31;
+  const int warp = threadIdx.x >> 5;
+  const S4WarpCtx cx = sh.ctx[warp];
+  const float c2 = cx.inv_t * kLog2e;
+  uint32_t msk = 0u, g = 0u, ks = 0u;
+  int loc = -1;
+  float M = 1.f;
+  float lb = -CUDART_INF_F;
+  if (lane < n) {
+    const uint2 e = sh.queue[warp][first + lane];
+    g = e.y;
+    if (MULTI) {
+      ks = g >> 28;
+      g &= 0x0fffffffu;
+    }
+    uint32_t f[4];
+    philox4x32_keyed<ROUNDS>(cx.key0, cx.key1, rounds_rt, g, cx.c1 + ks + (2u << 16), cx.pos, cx.seq, f);
+    loc = (int)((f[0] >> 16) & 15u);
+    M = exp1_from_word(e.x, ((float)(f[0] & 0xffffu) + 0.5f) * 0x1p-16f) * 0.0625f;
+    // the token at the minimum has S = M exactly: its score is a lower bound for the row at once
+    const int il = (int)(g << 4) + loc;
+    if (il < cx.tok_end && (cx.bins == nullptr || (int)__ldg(cx.bins + il) == cx.msg)) {
+      const float a = load_logit<DT>(cx.rowp, il);
+      if (a < CUDART_INF_F) {  // false for NaN
+        const float ln_s = logf(M);
+        const float s = fmaf(a, cx.inv_t, -ln_s);
+        lb = s - score_slack(s, ln_s);
+      }
+    }
+  }
+  nm = fminf(nm, filter_offset(dec_ordered(__reduce_max_sync(0xffffffffu, enc_ordered(lb)))));
+  if (lane < n) {
+    // token t can matter only if a_t c2 + nm - log2(M) >= 0 (S_t >= M); lg2.approx and the
+    // rounding of M are good to 2^-20, the extra 2^-10 covers them
+    const float nmM = nm - lg2_approx(M) + 0x1p-10f;
+    const int i0 = (int)(g << 4);
+#pragma unroll
+    for (int t = 0; t < 16; ++t) {
+      if (i0 + t < cx.tok_end) {
+        const float a = load_logit<DT>(cx.rowp, i0 + t);
+        if (a < CUDART_INF_F && fmaf(a, c2, nmM) >= 0.f) msk |= 1u << t;  // false for NaN
+      }
+    }
+  }
+  Top2 b = sh.best[threadIdx.x];
+  float lower = -CUDART_INF_F;
+  while (__any_sync(0xffffffffu, msk != 0u)) {
+    if (msk != 0u) {
+      const int t = __ffs(msk) - 1;
+      msk &= msk - 1u;
+      const int i = (int)(g << 4) + t;
+      if (cx.bins == nullptr || (int)__ldg(cx.bins + i) == cx.msg) {
+        const float a = load_logit<DT>(cx.rowp, i);
+        float s_noise = M;
+        if (t != loc) {
+          uint32_t f[4];
+          philox4x32_keyed<ROUNDS>(cx.key0, cx.key1, rounds_rt, (uint32_t)i >> 2,
+                                   cx.c1 + ks + (4u << 16), cx.pos, cx.seq, f);
+          const uint32_t u = (i & 2) ? ((i & 1) ? f[3] : f[2]) : ((i & 1) ? f[1] : f[0]);
+          s_noise = M + exp1_from_word(u, 0.5f);
+        }
+        const float ln_s = logf(s_noise);
+        const float s = fmaf(a, cx.inv_t, -ln_s);
+        // fused race: the candidate is (token, stream), ordered by token first
+        top2_offer(b, s, MULTI ? (int)(((uint32_t)i << 3) | ks) : i);
+        lower = fmaxf(lower, s - score_slack(s, ln_s));
+      }
+    }
+  }
+  sh.best[threadIdx.x] = b;
+  __syncwarp();
+  return __reduce_max_sync(0xffffffffu, enc_ordered(lower));
+}
+
+// The lane's share of a work item again for the softmax sum, token by token, leaving out NaN and
+// +inf logits (they cannot define a probability).  Rare: only rows that hold such values.
+template <int DT>
+__device__ __noinline__ void lse4_redo_careful(const char* rowp, int tok0, int n_steps, int tok_end,
+                                               float c2, float* lm_out, float* ls_out) {
+  float lm = kS3LseFloor, ls = 0.f;
+  for (int s = 0; s < n_steps; ++s) {
+    for (int j = 0; j < kS4LaneGroups; ++j) {
+      const int tok = tok0 + s * S4Cfg<DT>::kCtaTokens + j * 512;
+      for (int t = 0; t < 16; ++t) {
+        if (tok + t >= tok_end) break;
+        const float a = load_logit<DT>(rowp, tok + t);
+        if (!(a < CUDART_INF_F) || a == -CUDART_INF_F) continue;
+        if (a > lm) {
+          ls *= ex2_approx((lm - a) * c2);
+          lm = a;
+        }
+        ls += ex2_approx((a - lm) * c2);
+      }
+    }
+  }
+  *lm_out = lm;
+  *ls_out = ls;
+}
+
+// ------------------------------------------------------------------------------------------
+// The kernel
+// ------------------------------------------------------------------------------------------
+template <int DT, bool LSE, int ROUNDS, bool MULTI = false>
+__global__ void __launch_bounds__(S4Cfg<DT>::kWarps * 32, S4Cfg<DT>::kCtasPerSM)
+sweep4_kernel(const __grid_constant__ SweepArgs A) {
+  S4Shared<DT>& sh = s4_shared<DT>();
+  const int lane = threadIdx.x & 31;
+  const int warp = threadIdx.x >> 5;
+  constexpr int ES = DT == kBF16 ? 2 : 4;
+  constexpr int kWarps = S4Cfg<DT>::kWarps;
+  constexpr int kCtaTokens = S4Cfg<DT>::kCtaTokens;
+  typedef Group16<DT> G;
+  uint2* const queue = sh.queue[warp];
+  volatile unsigned long long* const m_tag = &sh.m_tag;
+
+  if (threadIdx.x == 0) sh.m_tag = 0ull;
+  __syncthreads();
+
+  uint32_t tag = 0u;
+  for (long long item = blockIdx.x; item < A.n_items; item += gridDim.x) {
+    ++tag;
+    const int split = (int)(item / A.rows);
+    const int row = (int)(item - (long long)split * A.rows);
+    const int tok_begin = split * A.chunk;  // a multiple of 2048
+    const int tok_end = min(A.V, tok_begin + A.chunk);
+    uint32_t c1, pos, seq;
+    const char* rowp;
+    float c2;
+    {
+      const int j = row % A.J;
+      const int bk = row / A.J;
+      const int k = bk % A.K;
+      const int b = bk / A.K;
+      rowp = (const char*)A.data + (b * A.sb + k * A.sk + j * A.sj) * ES;
+      c1 = ((uint32_t)k & A.kmask) | (A.domain << 16);
+      pos = A.pos_base + (uint32_t)j;
+      seq = A.seq_ids ? __ldg(A.seq_ids + b) : A.seq_base + (uint32_t)b;
+      const float inv_t = A.inv_t[k];
+      c2 = inv_t * kLog2e;
+      __syncwarp();  // the previous item's batched path is done with the context
+      if (lane == 0) {
+        S4WarpCtx cx;
+        cx.rowp = rowp;
+        cx.bins = A.bins ? A.bins + A.bins_sb * b : nullptr;
+        cx.c1 = c1; cx.pos = pos; cx.seq = seq;
+        cx.key0 = A.rk[0]; cx.key1 = A.rk[1];
+        cx.inv_t = inv_t;
+        cx.msg = (A.bins && A.msg) ? (int)__ldg(A.msg + b) : 0;
+        cx.tok_end = tok_end;
+        sh.ctx[warp] = cx;
+      }
+      top2_init(sh.best[threadIdx.x]);
+      __syncwarp();
+    }
+    const bool aligned = (((uintptr_t)rowp) & 31) == 0;
+    // this warp's steps: tokens base_w + s * kCtaTokens + [0, 2048)
+    const int base_w = tok_begin + warp * kS4WarpTokens;
+    const int span = tok_end - base_w;
+    const int n_steps = span > 0 ? (span + kCtaTokens - 1) / kCtaTokens : 0;
+    const int n_full = (aligned && span >= kS4WarpTokens) ? (span - kS4WarpTokens) / kCtaTokens + 1 : 0;
+    const int tok0 = base_w + lane * 16;  // the lane's first group; its others follow at +512 tokens
+
+    uint32_t m_enc = __ldcg(A.hints + row);  // bound published by earlier slices of the row
+    float lm = kS3LseFloor;
+    unsigned long long ls2 = 0ull;
+    int qn = 0;
+
+    // the lane's four groups of step s
+    auto load_step = [&](G (&g)[kS4LaneGroups], int s) {
+      const int tok = tok0 + s * kCtaTokens;
+      if (s < n_full) {
+        const char* p = rowp + (size_t)tok * ES;
+#pragma unroll
+        for (int j = 0; j < kS4LaneGroups; ++j) load16_vec(g[j], p + j * 512 * ES);
+      } else {
+#pragma unroll
+        for (int j = 0; j < kS4LaneGroups; ++j) load16_scalar(g[j], rowp, tok + j * 512, tok_end);
+      }
+    };
+    // coarse words of the lane's four groups of step s under noise stream c1s
+    auto coarse_step = [&](uint32_t (&cw)[4], int s, uint32_t c1s) {
+      const uint32_t g0 = (uint32_t)(tok0 + s * kCtaTokens) >> 4;  // g0 mod 128 == lane
+      philox4x32<ROUNDS>(A.rk, A.rounds, s4_call_index(g0), c1s, pos, seq, cw);
+    };
+
+    // ---- warm start: evaluate, per lane, the most promising group of the first step ------------
+    if (n_steps > 0) {
+      G g[kS4LaneGroups];
+      uint32_t cw[4];
+      load_step(g, 0);
+      coarse_step(cw, 0, c1);
+      float bkey = -CUDART_INF_F;
+      int bj = -1;
+#pragma unroll
+      for (int j = 0; j < kS4LaneGroups; ++j) {
+        // log2 of an upper bound on exp(score) of the group's tokens, up to a constant
+        const float key = fmaf(group16_max(g[j]), c2, -lg2_approx(coarse_lower(cw[j]) + 0x1p-24f));
+        if (key > bkey && tok0 + j * 512 < tok_end) {  // false for NaN
+          bkey = key;
+          bj = j;
+        }
+      }
+      const bool pass = bj >= 0;
+      const unsigned bal = __ballot_sync(0xffffffffu, pass);
+      if (pass) {
+        const uint32_t w = bj == 0 ? cw[0] : bj == 1 ? cw[1] : bj == 2 ? cw[2] : cw[3];
+        queue[__popc(bal & ((1u << lane) - 1u))] = make_uint2(w, ((uint32_t)tok0 >> 4) + 32u * bj);
+      }
+      const int nb = __popc(bal);
+      __syncwarp();
+      if (nb > 0) {
+        const uint32_t e = s4_flush<DT, ROUNDS, MULTI>(A.rounds, 0, nb, filter_offset(dec_ordered(m_enc)));
+        if (e > m_enc) m_enc = e;
+      }
+      if (lane == 0 && m_enc > 0u)
+        atomicMax((unsigned long long*)&sh.m_tag, ((unsigned long long)tag << 32) | m_enc);
+    }
+    float nm4 = filter_offset(dec_ordered(m_enc)) + 4.0f;
+
+    // one group: candidate iff coarse_lower(w) <= 2^(amax c2 + nm + 4)   (false for NaN)
+    auto test_group = [&](float amax, uint32_t w, uint32_t gidx) {
+      const bool pass = coarse_lower(w) <= ex2_approx(fmaf(amax, c2, nm4));
+      const unsigned bal = __ballot_sync(0xffffffffu, pass);
+      if (bal != 0u) {
+        if (pass) queue[qn + __popc(bal & ((1u << lane) - 1u))] = make_uint2(w, gidx);
+        qn += __popc(bal);
+      }
+    };
+    auto poll_bound = [&]() {
+      const unsigned long long mt = *m_tag;  // bound published by the other warps of the CTA
+      const uint32_t m_new = ((uint32_t)(mt >> 32) == tag) ? (uint32_t)mt : 0u;
+      if (m_new > m_enc) {
+        m_enc = m_new;
+        nm4 = filter_offset(dec_ordered(m_enc)) + 4.0f;
+      }
+    };
+    auto flush_batch = [&]() {
+      __syncwarp();
+      const int nb = min(qn, 32);
+      qn -= nb;
+      const uint32_t e = s4_flush<DT, ROUNDS, MULTI>(A.rounds, qn, nb, nm4 - 4.0f);
+      if (e > m_enc) {
+        m_enc = e;
+        nm4 = filter_offset(dec_ordered(m_enc)) + 4.0f;
+        if (lane == 0)
+          atomicMax((unsigned long long*)&sh.m_tag, ((unsigned long long)tag << 32) | e);
+      }
+    };
+
+    if constexpr (MULTI) {
+      // ---- fused multi-stream race (Sec. 5.1 encoder: Y = argmin over tokens AND streams of
+      //      S_i^(k) / weight_i): a step is loaded, maximised and summed once, then each of the
+      //      multi_k noise streams takes its turn as one pass of the inner loop.
+      const int ns = A.multi_k;
+      const uint32_t smask = A.kmask;
+      G g[kS4LaneGroups];
+      float amax[kS4LaneGroups];
+      int s = 0, st = 0;
+      for (;;) {
+#pragma unroll 1
+        while (s < n_steps && qn < 32) {
+          if (st == 0) {
+            load_step(g, s);
+#pragma unroll
+            for (int j = 0; j < kS4LaneGroups; ++j) {
+              amax[j] = group16_max(g[j]);
+              if (LSE) lse16<DT>(g[j], amax[j], c2, lm, ls2);
+            }
+          }
+          const uint32_t ks = (uint32_t)st & smask;
+          uint32_t cw[4];
+          coarse_step(cw, s, c1 + ks);
+          const uint32_t g0 = (uint32_t)(tok0 + s * kCtaTokens) >> 4;
+#pragma unroll
+          for (int j = 0; j < kS4LaneGroups; ++j) test_group(amax[j], cw[j], (g0 + 32u * j) | (ks << 28));
+          poll_bound();
+          if (++st == ns) {
+            st = 0;
+            ++s;
+          }
+        }
+        if (qn < 32) break;
+        flush_batch();
+      }
+    } else {
+      // ---- the sweep.  The inner loop runs until 32 groups are queued; the batched evaluation
+      //      is called from the outer loop so that the inner loop carries no call.
+      int s = 0;
+      for (;;) {
+#pragma unroll 1
+        for (; s < n_steps && qn < 32; ++s) {
+          G g[kS4LaneGroups];
+          uint32_t cw[4];
+          load_step(g, s);
+          coarse_step(cw, s, c1);
+          const uint32_t g0 = (uint32_t)(tok0 + s * kCtaTokens) >> 4;
+#pragma unroll
+          for (int j = 0; j < kS4LaneGroups; ++j) {
+            const float amax = group16_max(g[j]);
+            if (LSE) lse16<DT>(g[j], amax, c2, lm, ls2);
+            test_group(amax, cw[j], g0 + 32u * j);
+          }
+          poll_bound();
+        }
+        if (qn < 32) break;
+        flush_batch();
+      }
+    }
+    // ---- drain the queue ---------------------------------------------------------------------
+    while (qn > 0) flush_batch();
+
+    // ---- combine the lanes; every warp writes its own partial result ---------------------------
+    Top2 t2 = sh.best[threadIdx.x];
+    top2_warp_merge(t2);
+    float ls = 0.f;
+    if (LSE) {
+      float s0, s1;
+      unpack_f32x2(ls2, s0, s1);
+      if (__any_sync(0xffffffffu, !(s0 + s1 < CUDART_INF_F))) {  // NaN or +inf logits in the slice
+        float rl, rs;
+        lse4_redo_careful<DT>(rowp, tok0, n_steps, tok_end, c2, &rl, &rs);
+        lm = rl;
+        s0 = rs;
+        s1 = 0.f;
+      }
+      float wm = lm;
+#pragma unroll
+      for (int d = 16; d > 0; d >>= 1) wm = fmaxf(wm, __shfl_xor_sync(0xffffffffu, wm, d));
+      ls = (s0 + s1) * ex2_approx((lm - wm) * c2);
+#pragma unroll
+      for (int d = 16; d > 0; d >>= 1) ls += __shfl_xor_sync(0xffffffffu, ls, d);
+      lm = wm;
+    }
+    if (lane == 0) {
+      Partial pr;
+      pr.s1 = t2.s1; pr.i1 = t2.i1; pr.s2 = t2.s2; pr.i2 = t2.i2;
+      pr.lm = lm; pr.ls = ls; pr.pad0 = 0; pr.pad1 = 0;
+      A.partials[((long long)row * A.splits + split) * kWarps + warp] = pr;
+      if (A.splits > 1 && m_enc > 0u) atomicMax(A.hints + row, m_enc);
+    }
+  }
+}
+
+}  // namespace gls

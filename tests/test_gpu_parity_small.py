@@ -24,7 +24,7 @@ def _draft_both(gls, oracle, logits, **kw):
 
 
 @pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
-@pytest.mark.parametrize("spec", [1, 2, 3])
+@pytest.mark.parametrize("spec", [1, 2, 3, 4])
 def test_draft_shapes(gls, oracle, dtype, spec):
     """Ragged vocabularies around every tile boundary: one lane group (8 or 16 tokens), one warp
     iteration (256 or 512), one CTA iteration (2048 or 4096), one slice and several slices."""
@@ -109,7 +109,7 @@ def test_masked_nan_inf_and_empty_rows(gls, oracle):
 
 
 @pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
-@pytest.mark.parametrize("spec", [1, 2, 3])
+@pytest.mark.parametrize("spec", [1, 2, 3, 4])
 def test_verify_small(gls, oracle, dtype, spec):
     """Algorithm 2 end to end on reduced copies of the verify workloads, several shapes."""
     for cfg, B, K, L, V in ((2, 16, 4, 4, 3000), (3, 8, 8, 5, 5001), (4, 6, 8, 8, 2500),
@@ -194,7 +194,7 @@ def test_config1_statistics_on_gpu(gls, oracle):
     assert acc >= theory.lml_bound(p, q, K) - 4 * np.sqrt(acc * (1 - acc) / n)
 
 
-@pytest.mark.parametrize("spec", [1, 2, 3])
+@pytest.mark.parametrize("spec", [1, 2, 3, 4])
 def test_compress_small(gls, oracle, spec):
     for B, K, N, lmax in ((12, 1, 50, 1), (10, 4, 3000, 4), (6, 3, 70001, 16), (5, 2, 257, 2)):
         w = synth.compress_workload("cuda", B=B, K=K, N=N, D=4, l_max=lmax, seed=40 + N)
@@ -265,7 +265,7 @@ def test_host_detectable_errors(gls):
     with pytest.raises(gls.GlsError):
         gls.draft_sample(x, inv_temp=float("nan"))
     with pytest.raises(gls.GlsError):
-        gls.draft_sample(x, spec=4)
+        gls.draft_sample(x, spec=5)
     with pytest.raises(gls.GlsError):
         gls.draft_sample(x, rounds=3)
     with pytest.raises(gls.GlsError):
