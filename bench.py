@@ -293,7 +293,7 @@ def run_ours(args):
 
     peak, which = _peaks()
     achieved = tbytes / (verify_ms * 1e-3) / 1e9
-    kname = ("sweep3_kernel" if args.spec == 3 else "sweep_kernel") + "<%s, lse>" % (
+    kname = {4: "sweep4_kernel", 3: "sweep3_kernel"}.get(args.spec, "sweep_kernel") + "<%s, lse>" % (
         "bf16" if w.target_logits.dtype == torch.bfloat16 else "f32")
     roofline = {"bound": "hbm", "kernel": kname + " (target side: the dominant kernel; the call also "
                 "runs finalize_rows_kernel and verify_epilogue_kernel, microseconds each, inside "
@@ -403,7 +403,7 @@ def main():
     ap.add_argument("--workload", default="cfg4", choices=sorted(WORKLOAD_DESC))
     ap.add_argument("--batch", type=int, default=None,
                     help="override B (reduced copy of the workload, e.g. for an ncu capture)")
-    ap.add_argument("--spec", type=int, default=3, choices=[1, 2, 3], help="noise_spec")
+    ap.add_argument("--spec", type=int, default=4, choices=[1, 2, 3, 4], help="noise_spec")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle baseline leg")
     args = ap.parse_args()

@@ -25,7 +25,8 @@
  *
  *     key     = (seed & 0xffffffff, seed >> 32)
  *     counter = (c0 = token block, c1 = k | (domain << 16), c2 = position id, c3 = sequence id)
- *     domain  = 0 decoding noise, 1 compression noise, 2 / 3 the refinement streams of 0 / 1
+ *     domain  = 0 decoding noise, 1 compression noise, 2 / 3 the refinement streams of 0 / 1,
+ *               4 / 5 the per-token streams of 0 / 1 (noise_spec 4)
  *
  *   noise_spec 1:  block = i >> 2, w = out[i & 3],                v = (w + 0.5) * 2^-32
  *   noise_spec 2:  coarse  block = i >> 3 in `domain`:   h = 16-bit field (i & 7) of the 128 output
@@ -40,12 +41,26 @@
  *   S = -log1p(-v)   (v is strictly inside (0,1), so S is finite and positive; this is the paper's
  *                     S = -ln U with U = 1 - v)
  *
+ *   noise_spec 4 builds the 16 exponentials of the tokens 16g .. 16g+15 ("group" g) from their
+ *   minimum.  If E_0..E_15 are i.i.d. Exp(1), then M = min E_t is Exp(16), its position is uniform
+ *   and independent of M, and the other fifteen exceed M by i.i.d. Exp(1) amounts independent of
+ *   both (memorylessness).  Read backwards this is an exact sampler of 16 i.i.d. Exp(1) values:
+ *                  coarse  block = ((g >> 7) << 5) | (g & 31) in `domain`: w = out[(g >> 5) & 3]
+ *                          (128 consecutive groups share 32 calls; groups g, g+32, g+64, g+96 one call)
+ *                  refine  block = g in `domain + 2`: r = out[0] & 0xffff, loc = (out[0] >> 16) & 15
+ *                  token   block = i >> 2 in `domain + 4`: u = out[i & 3]
+ *                  M   = -log1p(-v0) / 16,  v0 = (w * 2^16 + r + 0.5) * 2^-48
+ *                  S_i = M                           if (i & 15) == loc
+ *                  S_i = M - log1p(-(u + 0.5) 2^-32) otherwise
+ *
  * A draft call and a verify call that describe the same (seed, sequence, position, k, i) therefore
- * see the same S -- that is the coupling.  All three specs are exact definitions; specs 2 and 3 let
- * a kernel decide most tokens from the coarse bits alone (16 bits for 8 tokens per generator call,
- * or 8 bits for 16 tokens per call) and generate the refinement bits only for the few tokens that
- * can still win.  Spec 3 is the default and the fastest: the generator's 32x32->64-bit multiplies
- * are the scarcest resource of the sweep on sm_100a.
+ * see the same S -- that is the coupling.  All four specs are exact definitions of i.i.d. Exp(1)
+ * noise.  Specs 2 and 3 let a kernel decide most tokens from the coarse bits alone (16 bits for 8
+ * tokens per generator call, or 8 bits for 16 tokens per call) and generate the refinement bits
+ * only for the few tokens that can still win.  Spec 4 goes further: one generator call covers 64
+ * tokens, and a whole group is settled by the bound S_i >= M >= w * 2^-36 (a few dozen groups
+ * per row need a closer look).  Spec 4 is the default and the fastest: the generator's
+ * 32x32->64-bit multiplies are the scarcest resource of the sweep on sm_100a.
  *
  * CONVENTIONS
  *   - Token / candidate indices are 0-based (the paper counts from 1).
@@ -112,7 +127,7 @@ typedef struct {
   uint32_t seq_base;       /* sequence id of batch row b is seq_base + b ...                   */
   const uint32_t* seq_ids; /* ... unless this optional DEVICE array [B] is given               */
   uint32_t pos_base;       /* position id of index j is pos_base + j                           */
-  uint32_t noise_spec;     /* 1, 2 or 3 (see above); 0 selects 3                               */
+  uint32_t noise_spec;     /* 1, 2, 3 or 4 (see above); 0 selects 4                            */
   uint32_t rounds;         /* Philox rounds, 0 selects 10; 7..16 accepted                      */
   uint32_t flags;          /* GLS_NOISE_*                                                      */
 } gls_noise_t;

@@ -316,7 +316,7 @@ static glso_key_t make_key(const glso_noise_t* nz, uint32_t domain, int b, int j
   glso_key_t nk;
   nk.seed = nz->seed;
   nk.rounds = nz->rounds ? (int)nz->rounds : 10;
-  nk.spec = nz->noise_spec ? (int)nz->noise_spec : 3;
+  nk.spec = nz->noise_spec ? (int)nz->noise_spec : 4;
   nk.domain = domain;
   nk.seq = nz->seq_ids ? nz->seq_ids[b] : nz->seq_base + (uint32_t)b;
   nk.pos = nz->pos_base + (uint32_t)j;

@@ -88,19 +88,19 @@ def philox4x32(ctr, key, rounds=10):
     return out
 
 
-def uniform(seed, seq, pos, k, i, spec=3, domain=0, rounds=10):
+def uniform(seed, seq, pos, k, i, spec=4, domain=0, rounds=10):
     return float(lib().glso_uniform_flat(int(seed), int(rounds), int(spec), int(domain), int(seq),
                                          int(pos), int(k), int(i)))
 
 
-def exp_noise(seed, seq, pos, k, i, spec=3, domain=0, rounds=10):
+def exp_noise(seed, seq, pos, k, i, spec=4, domain=0, rounds=10):
     f = lib().glso_exp_noise_flat
     f.restype = C.c_double
     return float(f(C.c_uint64(int(seed)), C.c_int(int(rounds)), C.c_int(int(spec)), C.c_uint32(int(domain)),
                    C.c_uint32(int(seq)), C.c_uint32(int(pos)), C.c_uint32(int(k)), C.c_int64(int(i))))
 
 
-def exp_noise_row(seed, seq, pos, k, V, spec=3, domain=0, rounds=10):
+def exp_noise_row(seed, seq, pos, k, V, spec=4, domain=0, rounds=10):
     """S_i = -ln U_i for i < V under one (sequence, position, draft) key, fp64."""
     out = np.empty(int(V), dtype=np.float64)
     lib().glso_exp_noise_row(int(seed), int(rounds), int(spec), int(domain), int(seq), int(pos),
@@ -108,7 +108,7 @@ def exp_noise_row(seed, seq, pos, k, V, spec=3, domain=0, rounds=10):
     return out
 
 
-def exp_noise_batch(seed, B, K, V, pos=0, seq_base=0, spec=3, domain=0, rounds=10):
+def exp_noise_batch(seed, B, K, V, pos=0, seq_base=0, spec=4, domain=0, rounds=10):
     """S[b,k,i] for sequences seq_base..seq_base+B-1, drafts 0..K-1, one position, fp64."""
     out = np.empty((int(B), int(K), int(V)), dtype=np.float64)
     f = lib().glso_exp_noise_batch
@@ -149,7 +149,7 @@ def _noise(seed, seq_base, seq_ids, pos_base, spec, rounds, flags):
 
 
 def draft_sample(logits, inv_temp=1.0, inv_temp_per_draft=None, seed=0, seq_base=0, seq_ids=None,
-                 pos_base=0, spec=3, rounds=10, noise_flags=0):
+                 pos_base=0, spec=4, rounds=10, noise_flags=0):
     """logits [B,K,J,V] (strided views allowed) -> dict(tokens, scores, gaps), each [B,K,J]."""
     logits, dt = _as_rows(logits)
     B, K, J, V = logits.shape
@@ -174,7 +174,7 @@ def draft_sample(logits, inv_temp=1.0, inv_temp_per_draft=None, seed=0, seq_base
 
 
 def target_sample_verify(logits, draft_tokens, inv_temp=1.0, flags=0, seed=0, seq_base=0,
-                         seq_ids=None, pos_base=0, spec=3, rounds=10, noise_flags=0):
+                         seq_ids=None, pos_base=0, spec=4, rounds=10, noise_flags=0):
     """logits [B,K,J,V], draft_tokens [B,K,L] with J = L+1 (L with NO_BONUS).
 
     Returns dict(tokens [B,J], tau [B], accept [B,K,L], scores [B,J], gaps [B,J], row_lse [B,K,J]).
@@ -204,7 +204,7 @@ def target_sample_verify(logits, draft_tokens, inv_temp=1.0, flags=0, seed=0, se
 
 
 def compress_select(enc_logw, dec_logw=None, bins=None, seed=0, seq_base=0, seq_ids=None,
-                    pos_base=0, spec=3, rounds=10, noise_flags=0, K=None):
+                    pos_base=0, spec=4, rounds=10, noise_flags=0, K=None):
     """enc_logw [B,N]; dec_logw [B,K,N] or None (then K must be given); bins None, [N] or [B,N].
 
     Returns dict(enc_index [B], message [B], dec_index [B,K], match [B], scores, gaps [B,1+K]).

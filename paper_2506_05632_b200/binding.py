@@ -171,7 +171,7 @@ def _workspace(workspace, need, device):
 
 
 def draft_sample(logits, inv_temp=1.0, inv_temp_per_draft=None, seed=0, seq_base=0, seq_ids=None,
-                 pos_base=0, spec=3, rounds=10, noise_flags=0, want_scores=True, workspace=None,
+                 pos_base=0, spec=4, rounds=10, noise_flags=0, want_scores=True, workspace=None,
                  status=None, out_tokens=None, out_scores=None):
     """logits [B,K,J,V] (device, fp32/bf16) -> (tokens int32 [B,K,J], scores fp32 [B,K,J] | None)."""
     L = load()
@@ -200,7 +200,7 @@ def static_scratch_bytes():
 
 
 def draft_sample_static(logits, out_tokens, out_scores=None, inv_temp=1.0, inv_temp_per_draft=None,
-                        seed=0, seq_base=0, seq_ids=None, pos_base=0, spec=3, rounds=10,
+                        seed=0, seq_base=0, seq_ids=None, pos_base=0, spec=4, rounds=10,
                         noise_flags=0, status=None):
     """gls_draft_sample_static: draft_sample for callers that may not allocate device memory.
 
@@ -236,7 +236,7 @@ def _sparse(ids, logits):
 
 
 def draft_sample_sparse(token_ids, logits, inv_temp=1.0, inv_temp_per_draft=None, seed=0,
-                        seq_base=0, seq_ids=None, pos_base=0, spec=3, rounds=10, noise_flags=0,
+                        seq_base=0, seq_ids=None, pos_base=0, spec=4, rounds=10, noise_flags=0,
                         want_scores=True, status=None):
     """Sparse rows (kept token ids and their logits, [B,K,J,M]) -> (vocabulary ids int32 [B,K,J],
     scores fp32 [B,K,J] | None).  Same races as draft_sample on the row masked to the kept tokens."""
@@ -258,7 +258,7 @@ def draft_sample_sparse(token_ids, logits, inv_temp=1.0, inv_temp_per_draft=None
 
 
 def target_sample_verify_sparse(token_ids, logits, draft_tokens, inv_temp=1.0, flags=0, seed=0,
-                                seq_base=0, seq_ids=None, pos_base=0, spec=3, rounds=10,
+                                seq_base=0, seq_ids=None, pos_base=0, spec=4, rounds=10,
                                 noise_flags=0, want_scores=True, status=None):
     """Sparse target rows [B,K,J,M] (J = L+1, or L with NO_BONUS) and draft_tokens int32 [B,K,L]
     -> dict(tokens [B,J], tau [B], accept [B,K,L], scores [B,J] | None)."""
@@ -284,7 +284,7 @@ def target_sample_verify_sparse(token_ids, logits, draft_tokens, inv_temp=1.0, f
 
 
 def target_sample_verify(logits, draft_tokens, inv_temp=1.0, flags=0, seed=0, seq_base=0,
-                         seq_ids=None, pos_base=0, spec=3, rounds=10, noise_flags=0,
+                         seq_ids=None, pos_base=0, spec=4, rounds=10, noise_flags=0,
                          want_scores=True, workspace=None, status=None, out=None):
     """logits [B,K,J,V], draft_tokens int32 [B,K,L]; J = L+1 (L with NO_BONUS).
 
@@ -316,7 +316,7 @@ def target_sample_verify(logits, draft_tokens, inv_temp=1.0, flags=0, seed=0, se
 
 
 def compress_select(enc_logw, dec_logw=None, bins=None, K=None, seed=0, seq_base=0, seq_ids=None,
-                    pos_base=0, spec=3, rounds=10, noise_flags=0, want_scores=True, workspace=None,
+                    pos_base=0, spec=4, rounds=10, noise_flags=0, want_scores=True, workspace=None,
                     status=None, out=None):
     """enc_logw [B,N], dec_logw [B,K,N] | None, bins uint8 [N] | [B,N] | None.
 

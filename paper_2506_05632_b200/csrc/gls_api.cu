@@ -473,7 +473,7 @@ static bool finite_pos(float x) { return std::isfinite(x) && x > 0.f; }
 static int fill_noise(SweepArgs& A, const gls_noise_t* nz, uint32_t domain, int* spec_out) {
   const int rounds = nz->rounds ? (int)nz->rounds : 10;
   if (rounds < 7 || rounds > 16) return GLS_ERR_INVALID_ARG;
-  const int spec = nz->noise_spec ? (int)nz->noise_spec : 3;
+  const int spec = nz->noise_spec ? (int)nz->noise_spec : 4;
   if (spec < 1 || spec > 4) return GLS_ERR_INVALID_ARG;
   if (nz->flags & ~GLS_NOISE_SHARED_ACROSS_K) return GLS_ERR_INVALID_ARG;
   uint32_t k0 = (uint32_t)(nz->seed & 0xffffffffu), k1 = (uint32_t)(nz->seed >> 32);

@@ -39,7 +39,7 @@ class StepBuffers:
 
 
 def spec_step(draft_logits, target_logits, buf, inv_temp=1.0, seed=0, seq_base=0, pos_base=0,
-              spec=3, rounds=10):
+              spec=4, rounds=10):
     """draft_logits [B,K,L,V], target_logits [B,K,L+1,V] on the device -> buf.out (device)."""
     kw = dict(inv_temp=inv_temp, seed=seed, seq_base=seq_base, pos_base=pos_base, spec=spec,
               rounds=rounds, workspace=buf.workspace, status=buf.status)
@@ -69,7 +69,7 @@ class HostStepper:
         self.h2d_bytes = B * K * (2 * L + 1) * V * elt
         self.d2h_bytes = self.h_tokens.numel() * 4 + self.h_tau.numel() * 4 + self.h_accept.numel()
 
-    def step(self, h_draft, h_target, inv_temp=1.0, seed=0, seq_base=0, spec=3, rounds=10):
+    def step(self, h_draft, h_target, inv_temp=1.0, seed=0, seq_base=0, spec=4, rounds=10):
         """h_draft [B,K,L,V], h_target [B,K,L+1,V]: pinned host tensors.  Returns host results."""
         main = torch.cuda.current_stream()
         n = 0

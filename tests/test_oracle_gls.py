@@ -16,7 +16,7 @@ NO_BONUS = 2
 COMBINE_ALL = 1
 
 
-def _alg1(oracle, ld, lt, K, trials, seed=SEED, spec=3, inv_temp=1.0, noise_flags=0):
+def _alg1(oracle, ld, lt, K, trials, seed=SEED, spec=4, inv_temp=1.0, noise_flags=0):
     """Algorithm 1 run `trials` times: one sequence id per trial, shared rows (stride 0)."""
     V = ld.shape[-1]
     d = np.broadcast_to(np.asarray(ld, np.float32).reshape(1, 1, 1, V), (trials, K, 1, V))
