@@ -35,7 +35,7 @@ WORKLOAD_DESC = {
 }
 # dram__bytes_read+write per launch of the target-side sweep kernel divided by its algorithmic
 # bytes, from the ncu capture summarised in profiles/ (None until a capture exists).
-TRAFFIC_RATIO = 1.015  # profiles/sweep3_kernel_cfg4_b64.md (B=64 capture; traffic scales with the rows)
+TRAFFIC_RATIO = 1.013  # profiles/sweep4_kernel_cfg4_b64.md (noise_spec 4, B=64 capture; traffic scales with the rows)
 
 
 def _peaks():
@@ -300,7 +300,7 @@ def run_ours(args):
                 "the same event bracket)",
                 "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                 "peak_source": "of " + which,
-                "traffic": (TRAFFIC_RATIO * tbytes) if TRAFFIC_RATIO else None,
+                "traffic": (TRAFFIC_RATIO * tbytes) if (TRAFFIC_RATIO and args.spec == 4) else None,
                 "algorithmic_bytes": tbytes, "ms": verify_ms,
                 "draft_side": {"achieved": dbytes / (draft_ms * 1e-3) / 1e9, "ms": draft_ms,
                                "frac": dbytes / (draft_ms * 1e-3) / 1e9 / peak},
@@ -380,7 +380,7 @@ def run_compress(args):
                        "l2": "inputs (%.2f GB) larger than L2" % ((eb + db) / 1e9),
                        "match_rate": float(out["match"].float().mean().item())},
             "clocks": clocks, "e2e": None, "gpu_launches": 6 * args.steps,
-            "roofline": {"bound": "hbm", "kernel": "sweep3_kernel<f32> (the K decoder sweeps: the "
+            "roofline": {"bound": "hbm", "kernel": "sweep4_kernel<f32> (the K decoder sweeps: the "
                          "dominant kernel; time = whole call minus an encoder-only call)",
                          "achieved": db / (dec_ms * 1e-3) / 1e9, "peak": peak, "unit": "GB/s",
                          "frac": db / (dec_ms * 1e-3) / 1e9 / peak, "peak_source": "of " + which,
