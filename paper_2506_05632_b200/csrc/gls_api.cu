@@ -91,11 +91,15 @@ static Plan make_plan3(long long rows, long long V, int dtype) {
 }
 
 // noise_spec 4: the same rule with that sweep's CTA shape (a warp step is 2048 tokens).
+#ifndef GLS_S4_WASTE
+#define GLS_S4_WASTE 0.15
+#define GLS_S4_MIN_STEPS 4
+#endif
 template <int DT>
 static Plan make_plan4_t(long long rows, long long V) {
   Plan p;
   constexpr int kCtaTok = S4Cfg<DT>::kCtaTokens;
-  constexpr int kMinChunk = 4 * kCtaTok;
+  constexpr int kMinChunk = GLS_S4_MIN_STEPS * kCtaTok;
   const long long grid = (long long)kNumSMs * S4Cfg<DT>::kCtasPerSM;
   long long max_splits = (V + kMinChunk - 1) / kMinChunk;
   if (rows * max_splits < 2 * grid) max_splits = (V + kCtaTok - 1) / kCtaTok;
@@ -104,7 +108,7 @@ static Plan make_plan4_t(long long rows, long long V) {
     const long long items = rows * splits;
     if (items >= 12 * grid) break;
     const long long rounds = (items + grid - 1) / grid;
-    if (items >= grid && (double)(rounds * grid - items) <= 0.15 * (double)(rounds * grid)) break;
+    if (items >= grid && (double)(rounds * grid - items) <= GLS_S4_WASTE * (double)(rounds * grid)) break;
   }
   long long chunk = (V + splits - 1) / splits;
   chunk = (chunk + kCtaTok - 1) / kCtaTok * kCtaTok;

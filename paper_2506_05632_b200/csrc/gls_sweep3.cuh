@@ -19,9 +19,9 @@
 // filter has no false negatives, so the result equals a full evaluation (Sec. 3 step 2 /
 // Algorithm 2 draft loop and Y_j line of arXiv 2506.05632, log domain).
 //
-// Work decomposition: a work item is one (row, vocabulary slice), owned by a CTA of 8 warps; per
-// iteration a lane takes 16 consecutive tokens (one 32-byte load of bf16, two of fp32), a warp
-// 512 and the CTA 4096 contiguous tokens.  Warps never wait on one another: they share the bound
+// Work decomposition: a work item is one (row, vocabulary slice), owned by one CTA (2 warps for
+// bf16 rows, 8 for fp32); per iteration a lane takes 16 consecutive tokens (one 32-byte load of
+// bf16, two of fp32), a warp 512 and the CTA 1024 or 4096 contiguous tokens.  Warps never wait on one another: they share the bound
 // m through one tagged shared-memory word, each warp writes its own partial result, and the
 // split-V reduction merges them.  The batched evaluation is called from an outer loop so that
 // the hot loop contains no call.  A fused variant (MULTI) races one row under several noise

@@ -295,8 +295,9 @@ sweep4_kernel(const __grid_constant__ SweepArgs A) {
       philox4x32<ROUNDS>(A.rk, A.rounds, s4_call_index(g0), c1s, pos, seq, cw);
     };
 
-    // ---- warm start: evaluate, per lane, the most promising group of the first step ------------
-    if (n_steps > 0) {
+    // ---- warm start: evaluate, per lane, the most promising group of the first step; skipped
+    //      when an earlier slice of the row has already published a bound ---------------------
+    if (n_steps > 0 && m_enc == 0u) {
       G g[kS4LaneGroups];
       uint32_t cw[4];
       load_step(g, 0);
@@ -324,9 +325,9 @@ sweep4_kernel(const __grid_constant__ SweepArgs A) {
         const uint32_t e = s4_flush<DT, ROUNDS, MULTI>(A.rounds, 0, nb, filter_offset(dec_ordered(m_enc)));
         if (e > m_enc) m_enc = e;
       }
-      if (lane == 0 && m_enc > 0u)
-        atomicMax((unsigned long long*)&sh.m_tag, ((unsigned long long)tag << 32) | m_enc);
     }
+    if (kWarps > 1 && lane == 0 && m_enc > 0u)
+      atomicMax((unsigned long long*)&sh.m_tag, ((unsigned long long)tag << 32) | m_enc);
     float nm4 = filter_offset(dec_ordered(m_enc)) + 4.0f;
 
     // one group: candidate iff coarse_lower(w) <= 2^(amax c2 + nm + 4)   (false for NaN)
@@ -339,6 +340,7 @@ sweep4_kernel(const __grid_constant__ SweepArgs A) {
       }
     };
     auto poll_bound = [&]() {
+      if (kWarps == 1) return;
       const unsigned long long mt = *m_tag;  // bound published by the other warps of the CTA
       const uint32_t m_new = ((uint32_t)(mt >> 32) == tag) ? (uint32_t)mt : 0u;
       if (m_new > m_enc) {
@@ -350,11 +352,17 @@ sweep4_kernel(const __grid_constant__ SweepArgs A) {
       __syncwarp();
       const int nb = min(qn, 32);
       qn -= nb;
-      const uint32_t e = s4_flush<DT, ROUNDS, MULTI>(A.rounds, qn, nb, nm4 - 4.0f);
+      uint32_t e = s4_flush<DT, ROUNDS, MULTI>(A.rounds, qn, nb, nm4 - 4.0f);
+      // the slices of a row trade their bounds through the row's hint word at batch time
+      if (A.splits > 1) {
+        uint32_t h = 0u;
+        if (lane == 0) h = e > m_enc ? atomicMax(A.hints + row, e) : __ldcg(A.hints + row);
+        e = max(e, __shfl_sync(0xffffffffu, h, 0));
+      }
       if (e > m_enc) {
         m_enc = e;
         nm4 = filter_offset(dec_ordered(m_enc)) + 4.0f;
-        if (lane == 0)
+        if (kWarps > 1 && lane == 0)
           atomicMax((unsigned long long*)&sh.m_tag, ((unsigned long long)tag << 32) | e);
       }
     };
