@@ -172,12 +172,15 @@ __device__ __forceinline__ RowResult finalize_row(const SweepArgs& A, int row, i
   r.idx = -1;
   r.score = -CUDART_INF;
   r.lse = -CUDART_INF;
-  if (lane != 0) return r;
-  r.lse = (with_lse && lsum > 0.0) ? (double)lm * (double)inv_t + log(lsum)
-                                   : -CUDART_INF;
-  if (best.i1 < 0) {
-    if (dev_status) atomicOr(dev_status, GLS_DEV_EMPTY_SUPPORT);
-  } else {
+  // Three independent fp64 chains run side by side: lane 0 re-scores the leader, lane 1 the
+  // runner-up if it is closer than the fp32 error bound, lane 2 takes the logarithm of the sum.
+  const float window = 2.0f * 0x1p-17f * (36.0f + fabsf(best.s1));
+  const int code = lane == 0 ? best.i1 : best.i2;
+  const bool want = (lane == 0 && best.i1 >= 0) ||
+                    (lane == 1 && best.i1 >= 0 && best.i2 >= 0 && best.s1 - best.s2 <= window);
+  double ex = -CUDART_INF;
+  int tok = -1;
+  if (want) {
     const char* rowp = (const char*)A.data + (b * A.sb + k * A.sk + j * A.sj) * ES;
     StreamKey sk;
     sk.c1 = ((uint32_t)k & A.kmask) | (A.domain << 16);
@@ -185,30 +188,30 @@ __device__ __forceinline__ RowResult finalize_row(const SweepArgs& A, int row, i
     sk.seq = A.seq_ids ? A.seq_ids[b] : A.seq_base + (uint32_t)b;
     // In the fused multi-stream race a candidate is (token << 3) | stream; ordering by that
     // code is "lowest token, then lowest stream", the tie rule.
-    const bool multi = A.multi_k > 0;
-    StreamKey sk1 = sk, sk2 = sk;
-    int t1 = best.i1, t2 = best.i2;
-    if (multi) {
-      sk1.c1 = sk.c1 + ((uint32_t)best.i1 & 7u);
-      t1 = (int)((uint32_t)best.i1 >> 3);
-      if (best.i2 >= 0) {
-        sk2.c1 = sk.c1 + ((uint32_t)best.i2 & 7u);
-        t2 = (int)((uint32_t)best.i2 >> 3);
-      }
+    tok = code;
+    if (A.multi_k > 0) {
+      sk.c1 += (uint32_t)code & 7u;
+      tok = (int)((uint32_t)code >> 3);
     }
-    double e1 = exact_score<DT, SPEC, ROUNDS>(A, rowp, sk1, t1, inv_t);
-    int code = best.i1, idx = t1;
-    // a runner-up closer than the fp32 error bound is re-scored too
-    const float window = 2.0f * 0x1p-17f * (36.0f + fabsf(best.s1));
-    if (best.i2 >= 0 && best.s1 - best.s2 <= window) {
-      const double e2 = exact_score<DT, SPEC, ROUNDS>(A, rowp, sk2, t2, inv_t);
-      if (e2 > e1 || (e2 == e1 && best.i2 < code)) {
-        e1 = e2;
-        idx = t2;
-      }
+    ex = exact_score<DT, SPEC, ROUNDS>(A, rowp, sk, tok, inv_t);
+  }
+  double lse = -CUDART_INF;
+  if (lane == 2 && with_lse && lsum > 0.0) lse = (double)lm * (double)inv_t + log(lsum);
+  lse = __shfl_sync(0xffffffffu, lse, 2);
+  const double e2 = __shfl_sync(0xffffffffu, ex, 1);
+  const int tok2 = __shfl_sync(0xffffffffu, tok, 1);
+  const bool want2 = __shfl_sync(0xffffffffu, (int)want, 1) != 0;
+  if (lane != 0) return r;
+  r.lse = lse;
+  if (best.i1 < 0) {
+    if (dev_status) atomicOr(dev_status, GLS_DEV_EMPTY_SUPPORT);
+  } else {
+    r.idx = tok;
+    r.score = ex;
+    if (want2 && (e2 > ex || (e2 == ex && best.i2 < best.i1))) {
+      r.idx = tok2;
+      r.score = e2;
     }
-    r.idx = idx;
-    r.score = e1;
   }
   return r;
 }
@@ -549,7 +552,9 @@ static int run_rows(SweepArgs& A, int dtype, int spec, const Plan& P, void* work
   A.hints = (uint32_t*)(ws + P.off_hints);
   A.partials = (Partial*)(ws + P.off_partials);
   RowResult* rowres = (RowResult*)(ws + P.off_rows);
-  if (cudaMemsetAsync(A.hints, 0, (size_t)P.rows * sizeof(uint32_t), st) != cudaSuccess)
+  // the noise_spec 4 sweep touches the hint words only when rows are cut into slices
+  if ((spec != 4 || P.splits > 1) &&
+      cudaMemsetAsync(A.hints, 0, (size_t)P.rows * sizeof(uint32_t), st) != cudaSuccess)
     return GLS_ERR_CUDA;
   cudaError_t err;
   const bool r10 = A.rounds == 10;

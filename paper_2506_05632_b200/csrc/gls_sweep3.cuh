@@ -82,6 +82,11 @@ __device__ __forceinline__ unsigned long long fma_f32x2(unsigned long long a, un
   asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
   return d;
 }
+__device__ __forceinline__ unsigned long long mul_f32x2(unsigned long long a, unsigned long long b) {
+  unsigned long long d;
+  asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
 __device__ __forceinline__ unsigned long long add_f32x2(unsigned long long a, unsigned long long b) {
   unsigned long long d;
   asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
@@ -179,12 +184,15 @@ __device__ __forceinline__ void lse16(const Group16<DT>& g, float amax, float c2
       lm = amax;
     }
   }
-  const float nl = -lm * c2;
-  const unsigned long long c22 = pack_f32x2(c2, c2), nl2 = pack_f32x2(nl, nl);
+  // (a - lm) first, then the scale: the difference is exact (or rounded at 2^-24 of itself), so
+  // the exponent is good to 1e-7 of its own size however large the logits are; a * c2 - lm * c2
+  // would carry the rounding of the two large products
+  const unsigned long long c22 = pack_f32x2(c2, c2), nlm2 = pack_f32x2(-lm, -lm);
 #pragma unroll
   for (int t = 0; t < 16; t += 2) {
     float e0, e1;
-    unpack_f32x2(fma_f32x2(pack_f32x2(group16_get<DT>(g, t), group16_get<DT>(g, t + 1)), c22, nl2), e0, e1);
+    const unsigned long long d2 = add_f32x2(pack_f32x2(group16_get<DT>(g, t), group16_get<DT>(g, t + 1)), nlm2);
+    unpack_f32x2(mul_f32x2(d2, c22), e0, e1);
     ls2 = add_f32x2(ls2, pack_f32x2(ex2_approx(e0), ex2_approx(e1)));
   }
 }

@@ -272,7 +272,8 @@ sweep4_kernel(const __grid_constant__ SweepArgs A) {
     const int n_full = (aligned && span >= kS4WarpTokens) ? (span - kS4WarpTokens) / kCtaTokens + 1 : 0;
     const int tok0 = base_w + lane * 16;  // the lane's first group; its others follow at +512 tokens
 
-    uint32_t m_enc = __ldcg(A.hints + row);  // bound published by earlier slices of the row
+    // bound published by earlier slices of the row (the hint words are cleared only when rows are cut)
+    uint32_t m_enc = A.splits > 1 ? __ldcg(A.hints + row) : 0u;
     float lm = kS3LseFloor;
     unsigned long long ls2 = 0ull;
     int qn = 0;

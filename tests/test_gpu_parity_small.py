@@ -257,6 +257,30 @@ def test_flat_and_peaked_rows(gls, oracle, dtype):
         parity.check_verify(parity.to_np(out), refv, name + " verify")
 
 
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("spec", [3, 4])
+def test_orderings_that_defeat_the_filter(gls, oracle, dtype, spec):
+    """Rows on which the running bound never settles: steeply ascending logits make every later
+    group of tokens a candidate (the per-warp candidate queue fills at its maximum rate and the
+    log-sum-exp moves its reference point every few groups); descending rows are decided by
+    their first group; constant rows leave the decision to the noise alone."""
+    B, K, V = 2, 2, 2048 * 9 + 700
+    i = torch.arange(V, device="cuda", dtype=torch.float32)
+    rows = torch.stack([1.0 * i, 0.3 * i, -1.0 * i, torch.zeros_like(i), 0.02 * i,
+                        (i % 4096) * 2.0])                      # [6, V]
+    logits = rows.view(1, 1, 6, V).expand(B, K, 6, V).contiguous().to(dtype)
+    for it in (1.0, 0.25):
+        kw = dict(seed=SEED + 5, spec=spec, inv_temp=it)
+        tok, sc, ref = _draft_both(gls, oracle, logits, **kw)
+        parity.check_draft(tok, sc, ref, "orderings draft %s T=1/%g" % (dtype, it))
+        dt = torch.from_numpy(ref["tokens"][:, :, :5].copy()).cuda()
+        out = gls.target_sample_verify(logits, dt, **kw)
+        refv = oracle.target_sample_verify(synth.to_numpy_rows(logits), ref["tokens"][:, :, :5], **kw)
+        parity.check_verify(parity.to_np(out), refv, "orderings verify %s T=1/%g" % (dtype, it))
+        # same logits on both sides: every draft is accepted at every position
+        assert (parity.to_np(out)["tau"] == 6).all()
+
+
 def test_host_detectable_errors(gls):
     x = torch.zeros(2, 2, 2, 64, device="cuda")
     tok = torch.zeros(2, 2, 1, dtype=torch.int32, device="cuda")
