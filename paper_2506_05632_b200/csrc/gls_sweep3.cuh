@@ -152,6 +152,23 @@ __device__ __forceinline__ float group16_get<kF32>(const Group16<kF32>& g, int t
   return __uint_as_float(t < 8 ? g.a.w[t] : g.b.w[t - 8]);
 }
 
+// (logit t - lm, logit t+1 - lm) as an fp32 pair, t even.  bf16: the mixed-precision add takes
+// the 16-bit halves of the word as they are (bf16 + fp32 -> fp32, rounded once), so the pair is
+// never unpacked.
+__device__ __forceinline__ unsigned long long group16_diff2(const Group16<kBF16>& g, int t, float nlm,
+                                                            unsigned long long) {
+  unsigned short lo, hi;
+  asm("mov.b32 {%0,%1}, %2;" : "=h"(lo), "=h"(hi) : "r"(g.a.w[t >> 1]));
+  float d0, d1;
+  asm("add.rn.f32.bf16 %0, %1, %2;" : "=f"(d0) : "h"(lo), "f"(nlm));
+  asm("add.rn.f32.bf16 %0, %1, %2;" : "=f"(d1) : "h"(hi), "f"(nlm));
+  return pack_f32x2(d0, d1);
+}
+__device__ __forceinline__ unsigned long long group16_diff2(const Group16<kF32>& g, int t, float,
+                                                            unsigned long long nlm2) {
+  return add_f32x2(pack_f32x2(group16_get<kF32>(g, t), group16_get<kF32>(g, t + 1)), nlm2);
+}
+
 // the group as loaded, to 16-byte aligned shared memory
 __device__ __forceinline__ void store_group16(uint32_t* dst, const Group16<kBF16>& g) {
   reinterpret_cast<uint4*>(dst)[0] = make_uint4(g.a.w[0], g.a.w[1], g.a.w[2], g.a.w[3]);
@@ -191,8 +208,7 @@ __device__ __forceinline__ void lse16(const Group16<DT>& g, float amax, float c2
 #pragma unroll
   for (int t = 0; t < 16; t += 2) {
     float e0, e1;
-    const unsigned long long d2 = add_f32x2(pack_f32x2(group16_get<DT>(g, t), group16_get<DT>(g, t + 1)), nlm2);
-    unpack_f32x2(mul_f32x2(d2, c22), e0, e1);
+    unpack_f32x2(mul_f32x2(group16_diff2(g, t, -lm, nlm2), c22), e0, e1);
     ls2 = add_f32x2(ls2, pack_f32x2(ex2_approx(e0), ex2_approx(e1)));
   }
 }
