@@ -97,6 +97,24 @@ __device__ __forceinline__ float coarse_lower(uint32_t w) {
   return __uint_as_float(0x3f800000u | (w >> 9)) - 1.0f;
 }
 
+// An upper bound on 2^x without the special-function unit (which the log-sum-exp keeps busy):
+// with xs = sat(x / 126 + 1) in [0, 1], i.e. x clamped to [-126, 0], the integer
+// round(32768 (x clamped)) is placed in the low mantissa bits of a float by a magic-number
+// multiply-add and moved into exponent and mantissa position by one integer multiply-add: the
+// result is 2^floor(x) (1 + frac(x)) >= 2^x (the chord of a convex function), at most 6.2 % above
+// it.  The caller passes x / 126 + 1 with x already raised by 2^-9 to cover the roundings (of
+// c2 / 126, 2^-24 * 126 in xs, half a unit of 2^-15 in the integer).  NaN gives 2^-126.
+__device__ __forceinline__ float exp2_upper_from_scaled(float amax, float c2s, float nms) {
+  float xs;
+  asm("fma.rn.sat.f32 %0, %1, %2, %3;" : "=f"(xs) : "f"(amax), "f"(c2s), "f"(nms));
+  const float t = fmaf(xs, 4128768.0f, 12582912.0f - 4128768.0f);  // 126 * 32768; 1.5 * 2^23
+  return __uint_as_float(__float_as_uint(t) * 256u + 0xff800000u);
+}
+// the second and third argument of exp2_upper_from_scaled for x = amax * c2 + nm4
+__device__ __forceinline__ float scaled_offset(float nm4) {
+  return fmaf(nm4 + 0x1p-9f, 1.0f / 126.0f, 1.0f + 0x1p-22f);
+}
+
 // generator call that serves group g (and g + 32, g + 64, g + 96 when g mod 128 < 32)
 __device__ __forceinline__ uint32_t s4_call_index(uint32_t g) { return ((g >> 7) << 5) | (g & 31u); }
 
@@ -330,10 +348,12 @@ sweep4_kernel(const __grid_constant__ SweepArgs A) {
     if (kWarps > 1 && lane == 0 && m_enc > 0u)
       atomicMax((unsigned long long*)&sh.m_tag, ((unsigned long long)tag << 32) | m_enc);
     float nm4 = filter_offset(dec_ordered(m_enc)) + 4.0f;
+    const float c2s = c2 * (1.0f / 126.0f);
+    float nms = scaled_offset(nm4);
 
-    // one group: candidate iff coarse_lower(w) <= 2^(amax c2 + nm + 4)   (false for NaN)
+    // one group: candidate iff coarse_lower(w) <= (an upper bound on) 2^(amax c2 + nm + 4)
     auto test_group = [&](float amax, uint32_t w, uint32_t gidx) {
-      const bool pass = coarse_lower(w) <= ex2_approx(fmaf(amax, c2, nm4));
+      const bool pass = coarse_lower(w) <= exp2_upper_from_scaled(amax, c2s, nms);
       const unsigned bal = __ballot_sync(0xffffffffu, pass);
       if (bal != 0u) {
         if (pass) queue[qn + __popc(bal & ((1u << lane) - 1u))] = make_uint2(w, gidx);
@@ -347,6 +367,7 @@ sweep4_kernel(const __grid_constant__ SweepArgs A) {
       if (m_new > m_enc) {
         m_enc = m_new;
         nm4 = filter_offset(dec_ordered(m_enc)) + 4.0f;
+        nms = scaled_offset(nm4);
       }
     };
     auto flush_batch = [&]() {
@@ -363,6 +384,7 @@ sweep4_kernel(const __grid_constant__ SweepArgs A) {
       if (e > m_enc) {
         m_enc = e;
         nm4 = filter_offset(dec_ordered(m_enc)) + 4.0f;
+        nms = scaled_offset(nm4);
         if (kWarps > 1 && lane == 0)
           atomicMax((unsigned long long*)&sh.m_tag, ((unsigned long long)tag << 32) | e);
       }
