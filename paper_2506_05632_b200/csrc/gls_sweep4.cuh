@@ -9,8 +9,9 @@
 // resource of this path on sm_100a -- runs once per 64 tokens, and
 //     S_i >= M_g = -log1p(-v0) / 16 >= v0 / 16 >= w * 2^-36        for every token of the group.
 // With m a lower bound on the row's best score, a token can only matter if S_i <= exp(a_i - m)
-// (a_i = logit_i / T), hence a group only if  w * 2^-32 <= 16 * exp(max a - m): one fused
-// multiply-add, one ex2 and one compare per 16 tokens.  A few dozen groups per row pass.  They
+// (a_i = logit_i / T), hence a group only if  w * 2^-32 <= 16 * exp(max a - m): a group maximum,
+// two multiply-adds, an integer multiply-add and one compare per 16 tokens (the right-hand side
+// is replaced by an upper bound that needs no ex2).  A few dozen groups per row pass.  They
 // are not examined on the spot: the lane pushes (w, g) on a small per-warp queue in shared
 // memory and the sweep goes on; when 32 groups are queued the warp evaluates them together, one
 // group per lane (the 16 refinement bits and the position of the minimum from a second
@@ -52,8 +53,8 @@ constexpr int kS4QueueCap = 32 + kS4WarpGroups;
 // Launch shape per element type, chosen by measurement.  A lane holds its four groups in
 // registers (32 for bf16, 64 for fp32).  bf16 rows: the next step's loads are issued before the
 // current step is used (32 more registers), one warp per CTA and 16 CTAs per SM (128 registers);
-// config 4 draft / target: 6.48 / 4.90 TB/s against 6.05 / 4.75 TB/s for 2 warps x 10 CTAs
-// without the prefetch.  fp32 rows: 8 warps x 2 CTAs (128 registers), no prefetch.
+// at the time of the choice config 4 draft / target ran at 6.48 / 4.90 TB/s against 6.05 / 4.75
+// TB/s for 2 warps x 10 CTAs without the prefetch.  fp32 rows: 8 warps x 2 CTAs (128 registers), no prefetch.
 template <int DT>
 struct S4Cfg {
   static constexpr int kWarps = DT == kBF16 ? GLS_S4_BF16_WARPS : GLS_S4_F32_WARPS;
