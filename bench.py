@@ -246,8 +246,32 @@ def run_ours(args):
     clocks = sampler.stop(t_begin, t_end) if rank == 0 else None
     draft_ms = statistics.mean(m[0].elapsed_time(m[1]) for m in marks)
     verify_ms = statistics.mean(m[1].elapsed_time(m[2]) for m in marks)
+    l2_warm = None
     if flush is not None:  # the flush writes are inside the wall bracket: use the per-call sums
         total_ms = (draft_ms + verify_ms) * args.steps
+        # the same steps again without the flush: inputs that fit the L2 stay there
+        _, wm = _time_calls(step, args.steps, 0, None)
+        l2_warm = {"draft_ms": statistics.mean(m[0].elapsed_time(m[1]) for m in wm),
+                   "verify_ms": statistics.mean(m[1].elapsed_time(m[2]) for m in wm)}
+    graphed = None
+    if flush is not None:
+        # small batches are bound by the host issuing the launches: the same step as a replayed
+        # CUDA graph (L2 flushed between replays, each replay in its own event pair)
+        gs = pipeline.GraphedStep(w.draft_logits, w.target_logits, buf, inv_temp=w.inv_temp,
+                                  seed=w.noise_seed, seq_base=seq_base, spec=args.spec)
+        for _ in range(3):
+            gs.replay()
+        gm = []
+        for _ in range(args.steps):
+            flush.add_(1)
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            gs.replay()
+            b.record()
+            gm.append((a, b))
+        torch.cuda.synchronize()
+        g_ms = statistics.mean(a.elapsed_time(b) for a, b in gm)
+        graphed = {"ms_per_step": g_ms, "value": world * B * L / (g_ms * 1e-3), "unit": UNIT}
     t = torch.tensor([total_ms], dtype=torch.float64, device="cuda")
     if dist is not None:
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
@@ -311,12 +335,17 @@ def run_ours(args):
     cpu = None
     if not args.no_cpu:
         cpu, _, _ = _cpu_baseline(args.workload, {"cfg2": 8, "cfg3": 32, "cfg4": 16}[args.workload])
+        # the same oracle on one thread, on a sample an all-core pass handles in about a second
+        one, _, _ = _cpu_baseline(args.workload, {"cfg2": 2, "cfg3": 2, "cfg4": 1}[args.workload],
+                                  threads=1)
+        cpu["one_thread"] = {"value": one["value"], "sample": one["sample"]}
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
             "config": {"workload": WORKLOAD_DESC[args.workload] + (" (B overridden to %d)" % B if args.batch else ""),
                        "noise_spec": args.spec,
                        "philox_rounds": 10,
+                       "l2_warm": l2_warm, "cuda_graph_replay": graphed,
                        "l2": "flushed between steps" if flush is not None
                        else "inputs (%.2f GB) larger than L2" % ((dbytes + tbytes) / 1e9),
                        "mean_tau": tau_mean},

@@ -50,6 +50,30 @@ def spec_step(draft_logits, target_logits, buf, inv_temp=1.0, seed=0, seq_base=0
     return buf.out
 
 
+class GraphedStep:
+    """`spec_step` on fixed tensors captured once into a CUDA graph and replayed.
+
+    A step is a handful of short launches; for small batches the host-side cost of issuing them
+    exceeds their run time, and a replayed graph removes it.  The logits are read from the
+    tensors given here (refill them in place between replays); results land in `buf.out`."""
+
+    def __init__(self, draft_logits, target_logits, buf, **kw):
+        self.buf = buf
+        self.graph = torch.cuda.CUDAGraph()
+        side = torch.cuda.Stream(device=draft_logits.device)
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):  # warm up outside capture (first-use initialisation)
+            spec_step(draft_logits, target_logits, buf, **kw)
+        torch.cuda.current_stream().wait_stream(side)
+        torch.cuda.synchronize()
+        with torch.cuda.graph(self.graph):
+            spec_step(draft_logits, target_logits, buf, **kw)
+
+    def replay(self):
+        self.graph.replay()
+        return self.buf.out
+
+
 class HostStepper:
     """Hot path from HOST logits: chunked, double-buffered H2D copies overlapped with the sweeps."""
 
