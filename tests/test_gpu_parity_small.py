@@ -281,6 +281,28 @@ def test_orderings_that_defeat_the_filter(gls, oracle, dtype, spec):
         assert (parity.to_np(out)["tau"] == 6).all()
 
 
+def test_step_replayed_as_cuda_graph_matches_eager(gls):
+    """The library's calls can be captured: a replayed graph of one step gives the eager result,
+    also after the logits were refilled in place."""
+    from paper_2506_05632_b200 import pipeline
+    B, K, L, V = 3, 2, 3, 5000
+    d = _rand_logits(B, K, L, V, torch.bfloat16, 71)
+    t = _rand_logits(B, K, L + 1, V, torch.bfloat16, 72)
+    kw = dict(inv_temp=0.9, seed=SEED + 9, seq_base=4)
+    buf = pipeline.StepBuffers(B, K, L, V)
+    gs = pipeline.GraphedStep(d, t, buf, **kw)
+    for refill in (False, True):
+        if refill:
+            d.copy_(_rand_logits(B, K, L, V, torch.bfloat16, 73))
+            t[:, :, :L].copy_(d)
+        out = {k: v.clone() for k, v in gs.replay().items() if v is not None}
+        ref = pipeline.spec_step(d, t, pipeline.StepBuffers(B, K, L, V), **kw)
+        torch.cuda.synchronize()
+        for k in out:
+            assert torch.equal(out[k], ref[k]), k
+    assert (out["tau"] == L + 1).all()  # identical rows on both sides accept every position
+
+
 def test_host_detectable_errors(gls):
     x = torch.zeros(2, 2, 2, 64, device="cuda")
     tok = torch.zeros(2, 2, 1, dtype=torch.int32, device="cuda")
