@@ -267,6 +267,31 @@ int gls_target_sample_verify_sparse(const gls_sparse_rows_t* target_rows, int B,
                                     uint32_t* device_status, void* stream);
 
 /*
+ * Top-M truncation fused in front of the sparse-row races (Sec. 4.4, Appendix D.1: the paper's
+ * experiments sample from the M = 50 most likely tokens).  Every dense row [V] is reduced, in one
+ * pass, to its M largest logits (ties at the M-th value: lowest token index; NaN, +inf and -inf
+ * logits are never kept; a row with fewer than M finite logits keeps them all), then
+ * gls_draft_sample_sparse / gls_target_sample_verify_sparse run on the lists: probabilities are
+ * normalised over the kept tokens and the noise of a kept token is that of its vocabulary id.
+ * 1 <= M <= 256.  `workspace` (device, gls_topm_workspace_bytes) receives the lists: int32 ids
+ * [B,K,J,M] followed, 256-byte aligned, by fp32 logits [B,K,J,M], in index order, id -1 past the
+ * kept count; the caller may read them after the call.  Errors as for the dense entry points;
+ * K * (L + 1) must not exceed 1536 for the verify call.
+ */
+size_t gls_topm_workspace_bytes(int B, int K, int J, int M);
+int gls_draft_sample_topm(const gls_rows_t* draft_logits, int B, int K, int J, int64_t V, int M,
+                          float inv_temp, const float* inv_temp_per_draft_host,
+                          const gls_noise_t* noise, int32_t* out_tokens, float* out_scores,
+                          void* workspace, size_t workspace_bytes, uint32_t* device_status,
+                          void* stream);
+int gls_target_sample_verify_topm(const gls_rows_t* target_logits, int B, int K, int L, int64_t V,
+                                  int M, float inv_temp, const int32_t* draft_tokens,
+                                  const gls_noise_t* noise, uint32_t flags, int32_t* out_tokens,
+                                  int32_t* out_num_tokens, uint8_t* out_accept, float* out_scores,
+                                  void* workspace, size_t workspace_bytes, uint32_t* device_status,
+                                  void* stream);
+
+/*
  * Compression -- Sec. 5.1 and Appendix C.  Per batch row b (one source sample):
  *     encoder:   Y = argmin_i min_k S_i^(k) / lambda_q,i          lambda_q = softmax(enc_logw[b,:])
  *                M = bins[Y]                                      (the log2(L_max)-bit message)

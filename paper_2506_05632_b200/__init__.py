@@ -10,6 +10,7 @@ kernels of csrc/.  There is no CPU fallback: if libgls.so cannot be loaded the c
 """
 from .binding import (  # noqa: F401
     COMBINE_ACTIVE, COMBINE_ALL, NO_BONUS, NOISE_SHARED_ACROSS_K, DEV_EMPTY_SUPPORT, GlsError,
-    build, compress_select, draft_sample, draft_sample_sparse, draft_sample_static, lib_path, load,
+    build, compress_select, draft_sample, draft_sample_sparse, draft_sample_static,
+    draft_sample_topm, lib_path, load,
     static_scratch_bytes, status_string, target_sample_verify, target_sample_verify_sparse,
-    version, workspace_bytes)
+    target_sample_verify_topm, topm_workspace_bytes, version, workspace_bytes)

@@ -104,6 +104,18 @@ def load():
             C.POINTER(_Rows), C.c_int, C.c_int, C.c_int, C.c_int64, C.c_float, C.c_void_p,
             C.POINTER(_Noise), C.c_uint32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
             C.c_void_p, C.c_size_t, C.c_void_p, C.c_void_p]
+        L.gls_topm_workspace_bytes.restype = C.c_size_t
+        L.gls_topm_workspace_bytes.argtypes = [C.c_int, C.c_int, C.c_int, C.c_int]
+        L.gls_draft_sample_topm.restype = C.c_int
+        L.gls_draft_sample_topm.argtypes = [
+            C.POINTER(_Rows), C.c_int, C.c_int, C.c_int, C.c_int64, C.c_int, C.c_float, C.c_void_p,
+            C.POINTER(_Noise), C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p,
+            C.c_void_p]
+        L.gls_target_sample_verify_topm.restype = C.c_int
+        L.gls_target_sample_verify_topm.argtypes = [
+            C.POINTER(_Rows), C.c_int, C.c_int, C.c_int, C.c_int64, C.c_int, C.c_float, C.c_void_p,
+            C.POINTER(_Noise), C.c_uint32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
+            C.c_void_p, C.c_size_t, C.c_void_p, C.c_void_p]
         L.gls_compress_select.restype = C.c_int
         L.gls_compress_select.argtypes = [
             C.POINTER(_Rows), C.POINTER(_Rows), C.c_void_p, C.c_int64, C.c_int, C.c_int,
@@ -280,6 +292,71 @@ def target_sample_verify_sparse(token_ids, logits, draft_tokens, inv_temp=1.0, f
         C.byref(rows), B, K, Ld, float(inv_temp), _ptr(draft_tokens) if Ld > 0 else None,
         C.byref(nz), int(flags), _ptr(out["tokens"]), _ptr(out["tau"]),
         _ptr(out["accept"]) if Ld > 0 else None, _ptr(out.get("scores")), _ptr(status), _stream()))
+    return out
+
+
+def topm_workspace_bytes(B, K, J, M):
+    return int(load().gls_topm_workspace_bytes(int(B), int(K), int(J), int(M)))
+
+
+def _topm_lists(workspace, B, K, J, M):
+    """Views of the kept (ids int32, logits fp32) lists [B,K,J,M] a top-M call left in its workspace."""
+    n = B * K * J * M
+    off = (n * 4 + 255) // 256 * 256
+    ids = workspace[:n * 4].view(torch.int32).view(B, K, J, M)
+    lg = workspace[off:off + n * 4].view(torch.float32).view(B, K, J, M)
+    return ids, lg
+
+
+def draft_sample_topm(logits, M, inv_temp=1.0, inv_temp_per_draft=None, seed=0, seq_base=0,
+                      seq_ids=None, pos_base=0, spec=4, rounds=10, noise_flags=0, want_scores=True,
+                      workspace=None, status=None):
+    """Dense logits [B,K,J,V] truncated to their M largest per row, then draft_sample_sparse.
+
+    Returns (tokens int32 [B,K,J], scores | None, (kept ids, kept logits) views [B,K,J,M])."""
+    L = load()
+    B, K, J, V = logits.shape
+    dev = logits.device
+    rows = _rows(logits, 3)
+    nz = _noise(seed, seq_base, seq_ids, pos_base, spec, rounds, noise_flags)
+    out_tokens = torch.empty((B, K, J), dtype=torch.int32, device=dev)
+    out_scores = torch.empty((B, K, J), dtype=torch.float32, device=dev) if want_scores else None
+    workspace = _workspace(workspace, topm_workspace_bytes(B, K, J, M), dev)
+    itk = None
+    if inv_temp_per_draft is not None:
+        itk = (C.c_float * K)(*[float(x) for x in inv_temp_per_draft])
+    _check(L.gls_draft_sample_topm(C.byref(rows), B, K, J, V, int(M), float(inv_temp),
+                                   C.cast(itk, C.c_void_p) if itk is not None else None,
+                                   C.byref(nz), _ptr(out_tokens), _ptr(out_scores),
+                                   workspace.data_ptr(), workspace.numel(), _ptr(status), _stream()))
+    return out_tokens, out_scores, _topm_lists(workspace, B, K, J, M)
+
+
+def target_sample_verify_topm(logits, draft_tokens, M, inv_temp=1.0, flags=0, seed=0, seq_base=0,
+                              seq_ids=None, pos_base=0, spec=4, rounds=10, noise_flags=0,
+                              want_scores=True, workspace=None, status=None):
+    """Dense target logits [B,K,J,V] truncated to their M largest per row, then
+    target_sample_verify_sparse.  Returns dict(tokens, tau, accept, scores | None)."""
+    L = load()
+    B, K, J, V = logits.shape
+    Ld = J if (flags & NO_BONUS) else J - 1
+    dev = logits.device
+    rows = _rows(logits, 3)
+    nz = _noise(seed, seq_base, seq_ids, pos_base, spec, rounds, noise_flags)
+    if Ld > 0:
+        if draft_tokens.dtype != torch.int32 or not draft_tokens.is_contiguous():
+            raise GlsError("draft_tokens must be contiguous int32")
+        assert tuple(draft_tokens.shape) == (B, K, Ld)
+    out = dict(tokens=torch.empty((B, J), dtype=torch.int32, device=dev),
+               tau=torch.empty((B,), dtype=torch.int32, device=dev),
+               accept=torch.empty((B, K, Ld), dtype=torch.uint8, device=dev),
+               scores=torch.empty((B, J), dtype=torch.float32, device=dev) if want_scores else None)
+    workspace = _workspace(workspace, topm_workspace_bytes(B, K, J, M), dev)
+    _check(L.gls_target_sample_verify_topm(
+        C.byref(rows), B, K, Ld, V, int(M), float(inv_temp),
+        _ptr(draft_tokens) if Ld > 0 else None, C.byref(nz), int(flags), _ptr(out["tokens"]),
+        _ptr(out["tau"]), _ptr(out["accept"]) if Ld > 0 else None, _ptr(out.get("scores")),
+        workspace.data_ptr(), workspace.numel(), _ptr(status), _stream()))
     return out
 
 

@@ -14,6 +14,7 @@
 #include "gls_kernels.cuh"
 #include "gls_sweep3.cuh"
 #include "gls_sweep4.cuh"
+#include "gls_topm.cuh"
 
 namespace gls {
 
@@ -982,6 +983,90 @@ static int static_scratch_address(void** out) {
 extern "C" {
 
 size_t gls_static_scratch_bytes(void) { return (size_t)GLS_STATIC_SCRATCH_BYTES; }
+
+// ------------------------------------------------------------------------------------------
+// Dense rows truncated to their M largest logits, then the sparse-row races.
+// ------------------------------------------------------------------------------------------
+size_t gls_topm_workspace_bytes(int B, int K, int J, int M) {
+  if (B <= 0 || K <= 0 || J <= 0 || M <= 0 || M > gls::kTopmMaxM) return 0;
+  return gls::align_up((size_t)B * K * J * M * sizeof(int32_t), 256) +
+         gls::align_up((size_t)B * K * J * M * sizeof(float), 256);
+}
+
+namespace gls {
+// selects into the workspace and describes the result as sparse rows
+static int topm_select(const gls_rows_t* rows, int B, int K, int J, int64_t V, int M, void* workspace,
+                       size_t workspace_bytes, cudaStream_t st, gls_sparse_rows_t* out) {
+  if (M <= 0 || M > kTopmMaxM || !sizes_ok(B, K, J, V)) return GLS_ERR_INVALID_ARG;
+  const int rc = check_rows(rows);
+  if (rc != GLS_OK) return rc;
+  const size_t need = gls_topm_workspace_bytes(B, K, J, M);
+  if (!workspace || workspace_bytes < need) return GLS_ERR_WORKSPACE;
+  TopmArgs T;
+  T.data = rows->data;
+  T.sb = rows->stride_b;
+  T.sk = rows->stride_k;
+  T.sj = rows->stride_j;
+  T.K = K;
+  T.J = J;
+  T.V = (int)V;
+  T.M = M;
+  T.rows = (long long)B * K * J;
+  T.ids = (int32_t*)workspace;
+  T.logits = (float*)((char*)workspace + align_up((size_t)T.rows * M * sizeof(int32_t), 256));
+  const long long want = (T.rows + kTopmWarps - 1) / kTopmWarps;
+  const long long cap = (long long)kNumSMs * kTopmCtasPerSM;
+  const int grid = (int)(want < cap ? want : cap);
+  if (rows->dtype == GLS_BF16)
+    topm_select_kernel<kBF16><<<grid, kTopmWarps * 32, 0, st>>>(T);
+  else
+    topm_select_kernel<kF32><<<grid, kTopmWarps * 32, 0, st>>>(T);
+  if (cudaGetLastError() != cudaSuccess) return GLS_ERR_CUDA;
+  out->token_ids = T.ids;
+  out->logits = T.logits;
+  out->stride_b = (int64_t)K * J * M;
+  out->stride_k = (int64_t)J * M;
+  out->stride_j = M;
+  out->M = M;
+  return GLS_OK;
+}
+}  // namespace gls
+
+int gls_draft_sample_topm(const gls_rows_t* draft_logits, int B, int K, int J, int64_t V, int M,
+                          float inv_temp, const float* inv_temp_per_draft_host,
+                          const gls_noise_t* noise, int32_t* out_tokens, float* out_scores,
+                          void* workspace, size_t workspace_bytes, uint32_t* device_status,
+                          void* stream) {
+  if (!noise || !out_tokens) return GLS_ERR_INVALID_ARG;
+  gls_sparse_rows_t sp;
+  const int rc = gls::topm_select(draft_logits, B, K, J, V, M, workspace, workspace_bytes,
+                                  (cudaStream_t)stream, &sp);
+  if (rc != GLS_OK) return rc;
+  return gls_draft_sample_sparse(&sp, B, K, J, inv_temp, inv_temp_per_draft_host, noise, out_tokens,
+                                 out_scores, device_status, stream);
+}
+
+int gls_target_sample_verify_topm(const gls_rows_t* target_logits, int B, int K, int L, int64_t V,
+                                  int M, float inv_temp, const int32_t* draft_tokens,
+                                  const gls_noise_t* noise, uint32_t flags, int32_t* out_tokens,
+                                  int32_t* out_num_tokens, uint8_t* out_accept, float* out_scores,
+                                  void* workspace, size_t workspace_bytes, uint32_t* device_status,
+                                  void* stream) {
+  if (flags & ~(GLS_COMBINE_ALL | GLS_NO_BONUS)) return GLS_ERR_INVALID_ARG;
+  const int J = L + ((flags & GLS_NO_BONUS) ? 0 : 1);
+  if (!noise || !out_tokens || !out_num_tokens || L < 0) return GLS_ERR_INVALID_ARG;
+  if ((long long)K * J > 1536) return GLS_ERR_UNSUPPORTED;
+  gls_sparse_rows_t sp;
+  // rows shared by all drafts (stride_k == 0) are truncated once and stay shared
+  const int ksel = (target_logits && target_logits->stride_k == 0) ? 1 : K;
+  const int rc = gls::topm_select(target_logits, B, ksel, J, V, M, workspace, workspace_bytes,
+                                  (cudaStream_t)stream, &sp);
+  if (rc != GLS_OK) return rc;
+  if (ksel == 1) sp.stride_k = 0;
+  return gls_target_sample_verify_sparse(&sp, B, K, L, inv_temp, draft_tokens, noise, flags,
+                                         out_tokens, out_num_tokens, out_accept, out_scores,
+                                         device_status, stream);
+}
 
 int gls_draft_sample_static(const gls_rows_t* draft_logits, int B, int K, int J, int64_t V,
                             float inv_temp, const float* inv_temp_per_draft_host,

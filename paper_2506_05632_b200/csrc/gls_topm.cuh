@@ -1,0 +1,213 @@
+// gls_topm.cuh -- top-M truncation of dense rows in one pass (Sec. 4.4 / Appendix D.1 of arXiv
+// 2506.05632: the experiments sample from the M = 50 most likely tokens).
+//
+// A warp owns a row.  It streams the row once (the same 2048-token steps as the noise_spec 4
+// sweep: four 32-byte loads per lane, the next step's loads in flight) and keeps, in shared memory,
+// the tokens whose logit exceeds a threshold thr.  thr is -inf until the buffer first overflows;
+// from then on it is the M-th largest logit seen so far, so a later token can only enter the top M
+// if its logit is strictly larger (ties go to the lower index, and the row is read in index
+// order).  Whenever the buffer holds more than 512 entries the warp prunes it to the M largest
+// (an 8-bit radix select on the order-preserving integer code of the logits, then a stable
+// compaction) and raises thr.  After the first prune a token passes with probability M / (tokens
+// seen), so a row of 150k tokens is pruned about three times and the pass runs at the speed of
+// the loads.  Output: per row M (token id, logit) pairs in index order, id = -1 past the number of
+// finite logits.  NaN, +inf and -inf logits are never kept.
+#pragma once
+#include "gls_sweep4.cuh"
+
+namespace gls {
+
+constexpr int kTopmCap = 1024;   // buffer entries per warp: 512 kept at most + 512 from one group step
+constexpr int kTopmMaxM = 256;
+constexpr int kTopmWarps = 4;    // rows per CTA
+constexpr int kTopmCtasPerSM = 4;
+
+struct TopmArgs {
+  const void* data;       // rows [B][K][J][V]
+  long long sb, sk, sj;   // element strides
+  int K, J, V, M;
+  long long rows;
+  int32_t* ids;           // [rows][M]
+  float* logits;          // [rows][M]
+};
+
+struct TopmWarpBuf {
+  uint32_t key[kTopmCap];  // order-preserving code of the logit
+  int idx[kTopmCap];
+  uint32_t hist[256];
+};
+
+// Keeps the M largest of the n buffered entries (ties: first come, i.e. lowest index), in their
+// order of arrival; returns the new count and the code of the M-th largest.  Requires n > M.
+__device__ __noinline__ int topm_prune(TopmWarpBuf* wb, int n, int M, uint32_t* kth_out) {
+  const int lane = threadIdx.x & 31;
+  const uint32_t lt = (1u << lane) - 1u;
+  uint32_t prefix = 0u;
+  int remaining = M;  // rank still to find among the entries that share `prefix`
+#pragma unroll 1
+  for (int pass = 3; pass >= 0; --pass) {
+    for (int i = lane; i < 256; i += 32) wb->hist[i] = 0u;
+    __syncwarp();
+    const int shift = 8 * pass;
+    for (int i = lane; i < n; i += 32) {
+      const uint32_t k = wb->key[i];
+      if (pass == 3 || (k >> (shift + 8)) == prefix) atomicAdd(&wb->hist[(k >> shift) & 255u], 1u);
+    }
+    __syncwarp();
+    // lane l owns bins 255 - 8l .. 248 - 8l, scanned from the top
+    uint32_t c[8];
+    uint32_t mine = 0u;
+#pragma unroll
+    for (int t = 0; t < 8; ++t) {
+      c[t] = wb->hist[255 - 8 * lane - t];
+      mine += c[t];
+    }
+    uint32_t above = mine;  // inclusive scan over lanes, then made exclusive
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+      const uint32_t o = __shfl_up_sync(0xffffffffu, above, d);
+      if (lane >= d) above += o;
+    }
+    above -= mine;
+    int bin = -1, rem_new = 0;
+    uint32_t run = above;
+#pragma unroll
+    for (int t = 0; t < 8; ++t) {
+      if (bin < 0 && run + c[t] >= (uint32_t)remaining) {
+        bin = 255 - 8 * lane - t;
+        rem_new = remaining - (int)run;
+      }
+      run += c[t];
+    }
+    // the first lane (highest bins) whose range reaches the rank holds the answer
+    const unsigned found = __ballot_sync(0xffffffffu, bin >= 0);
+    const int src = __ffs(found) - 1;
+    bin = __shfl_sync(0xffffffffu, bin, src);
+    remaining = __shfl_sync(0xffffffffu, rem_new, src);
+    prefix = (prefix << 8) | (uint32_t)bin;
+    __syncwarp();
+  }
+  const uint32_t kth = prefix;
+  int out = 0, ties_seen = 0;
+#pragma unroll 1
+  for (int base = 0; base < n; base += 32) {
+    const int i = base + lane;
+    const bool valid = i < n;
+    const uint32_t k = valid ? wb->key[i] : 0u;
+    const int id = valid ? wb->idx[i] : 0;
+    const bool eq = valid && k == kth;
+    const unsigned eqb = __ballot_sync(0xffffffffu, eq);
+    const bool keep = (valid && k > kth) || (eq && ties_seen + __popc(eqb & lt) < remaining);
+    const unsigned kb = __ballot_sync(0xffffffffu, keep);
+    __syncwarp();  // every lane holds its entry before anything is moved down
+    if (keep) {
+      const int pos = out + __popc(kb & lt);
+      wb->key[pos] = k;
+      wb->idx[pos] = id;
+    }
+    out += __popc(kb);
+    ties_seen += __popc(eqb);
+    __syncwarp();
+  }
+  *kth_out = kth;
+  return out;
+}
+
+template <int DT>
+__global__ void __launch_bounds__(kTopmWarps * 32, kTopmCtasPerSM)
+topm_select_kernel(const TopmArgs T) {
+  __shared__ TopmWarpBuf bufs[kTopmWarps];
+  const int lane = threadIdx.x & 31;
+  const int warp = threadIdx.x >> 5;
+  const uint32_t lt = (1u << lane) - 1u;
+  constexpr int ES = DT == kBF16 ? 2 : 4;
+  typedef Group16<DT> G;
+  TopmWarpBuf* const wb = &bufs[warp];
+
+  for (long long row = (long long)blockIdx.x * kTopmWarps + warp; row < T.rows;
+       row += (long long)gridDim.x * kTopmWarps) {
+    const int j = (int)(row % T.J);
+    const long long bk = row / T.J;
+    const int k = (int)(bk % T.K);
+    const long long b = bk / T.K;
+    const char* rowp = (const char*)T.data + (b * T.sb + k * T.sk + j * T.sj) * ES;
+    const bool aligned = (((uintptr_t)rowp) & 31) == 0;
+    const int n_steps = (T.V + kS4WarpTokens - 1) / kS4WarpTokens;
+    const int n_full = aligned ? T.V / kS4WarpTokens : 0;
+    const int tok0 = lane * 16;
+
+    auto load_step = [&](G (&g)[kS4LaneGroups], int s) {
+      const int tok = tok0 + s * kS4WarpTokens;
+      if (s < n_full) {
+        const char* p = rowp + (size_t)tok * ES;
+#pragma unroll
+        for (int q = 0; q < kS4LaneGroups; ++q) load16_vec(g[q], p + q * 512 * ES);
+      } else {
+#pragma unroll
+        for (int q = 0; q < kS4LaneGroups; ++q) load16_scalar(g[q], rowp, tok + q * 512, T.V);
+      }
+    };
+
+    float thr = -CUDART_INF_F;
+    int n = 0;
+    __syncwarp();  // the previous row's output loop is done with the buffer
+    G nxt[kS4LaneGroups];
+    if (n_steps > 0) load_step(nxt, 0);
+#pragma unroll 1
+    for (int s = 0; s < n_steps; ++s) {
+      G g[kS4LaneGroups];
+#pragma unroll
+      for (int q = 0; q < kS4LaneGroups; ++q) g[q] = nxt[q];
+      if (s + 1 < n_steps) load_step(nxt, s + 1);
+#pragma unroll
+      for (int q = 0; q < kS4LaneGroups; ++q) {
+        const float gmax = group16_max(g[q]);
+        if (__any_sync(0xffffffffu, gmax > thr)) {  // false for NaN
+          const int tok = tok0 + s * kS4WarpTokens + q * 512;
+          uint32_t m = 0u;
+#pragma unroll
+          for (int t = 0; t < 16; ++t) {
+            const float a = group16_get<DT>(g[q], t);
+            if (a > thr && a < CUDART_INF_F && tok + t < T.V) m |= 1u << t;
+          }
+          // the lanes' tokens are appended in index order
+          const int cnt = __popc(m);
+          int incl = cnt;
+#pragma unroll
+          for (int d = 1; d < 32; d <<= 1) {
+            const int o = __shfl_up_sync(0xffffffffu, incl, d);
+            if (lane >= d) incl += o;
+          }
+          int pos = n + incl - cnt;
+#pragma unroll
+          for (int t = 0; t < 16; ++t) {
+            if ((m >> t) & 1u) {
+              wb->key[pos] = enc_ordered(group16_get<DT>(g[q], t));
+              wb->idx[pos] = tok + t;
+              ++pos;
+            }
+          }
+          n += __shfl_sync(0xffffffffu, incl, 31);
+          __syncwarp();
+          if (n > kTopmCap - 512) {
+            uint32_t kth;
+            n = topm_prune(wb, n, T.M, &kth);
+            thr = dec_ordered(kth);
+          }
+        }
+      }
+    }
+    if (n > T.M) {
+      uint32_t kth;
+      n = topm_prune(wb, n, T.M, &kth);
+    }
+    __syncwarp();
+    for (int i = lane; i < T.M; i += 32) {
+      T.ids[row * T.M + i] = i < n ? wb->idx[i] : -1;
+      T.logits[row * T.M + i] = i < n ? dec_ordered(wb->key[i]) : -CUDART_INF_F;
+    }
+  }
+  (void)lt;
+}
+
+}  // namespace gls
