@@ -6,18 +6,20 @@
 // the tokens whose logit exceeds a threshold thr.  thr is -inf until the buffer first overflows;
 // from then on it is the M-th largest logit seen so far, so a later token can only enter the top M
 // if its logit is strictly larger (ties go to the lower index, and the row is read in index
-// order).  Whenever the buffer holds more than 512 entries the warp prunes it to the M largest
-// (an 8-bit radix select on the order-preserving integer code of the logits, then a stable
-// compaction) and raises thr.  After the first prune a token passes with probability M / (tokens
-// seen), so a row of 150k tokens is pruned about three times and the pass runs at the speed of
-// the loads.  Output: per row M (token id, logit) pairs in index order, id = -1 past the number of
+// order).  The sweep itself only compares each group's maximum with thr and queues the groups
+// that exceed it; queued groups are examined 32 at a time (one per lane, their logits read again
+// from L2), their tokens above thr appended to the buffer, and whenever the buffer holds more
+// than M + 64 entries the warp prunes it to the M largest (an 8-bit radix select on the
+// order-preserving integer code of the logits, then a stable compaction) and raises thr.  A
+// token passes with probability about M / (tokens seen), so a row of 150k tokens appends a few
+// hundred tokens and is pruned about ten times.  Output: per row M (token id, logit) pairs in index order, id = -1 past the number of
 // finite logits.  NaN, +inf and -inf logits are never kept.
 #pragma once
 #include "gls_sweep4.cuh"
 
 namespace gls {
 
-constexpr int kTopmCap = 1024;   // buffer entries per warp: 512 kept at most + 512 from one group step
+constexpr int kTopmCap = 1024;   // buffer entries per warp: at most M + 64 kept + 512 from one batch
 constexpr int kTopmMaxM = 256;
 constexpr int kTopmWarps = 4;    // rows per CTA
 constexpr int kTopmCtasPerSM = 4;
@@ -113,16 +115,64 @@ __device__ __noinline__ int topm_prune(TopmWarpBuf* wb, int n, int M, uint32_t* 
   return out;
 }
 
+// Batched examination of queued groups: lane l < nb takes group queue[first + l], reads its 16
+// logits again (L2 hits) and appends the tokens above the current threshold to the token buffer,
+// in index order (the queue is in index order, lanes append in lane order).  Then the buffer is
+// pruned if it has grown past M + 64.  Returns the new count; *thr is raised by a prune.
+template <int DT>
+__device__ __noinline__ int topm_expand(TopmWarpBuf* wb, const int* queue, const char* rowp, int V,
+                                        int first, int nb, int n, int M, float* thr_io) {
+  const int lane = threadIdx.x & 31;
+  const float thr = *thr_io;
+  float a[16];
+  uint32_t m = 0u;
+  int tok = 0;
+  if (lane < nb) {
+    tok = queue[first + lane] << 4;
+#pragma unroll
+    for (int t = 0; t < 16; ++t) a[t] = tok + t < V ? load_logit<DT>(rowp, tok + t) : -CUDART_INF_F;
+#pragma unroll
+    for (int t = 0; t < 16; ++t)
+      if (a[t] > thr && a[t] < CUDART_INF_F) m |= 1u << t;  // false for NaN
+  }
+  const int cnt = __popc(m);
+  int incl = cnt;
+#pragma unroll
+  for (int d = 1; d < 32; d <<= 1) {
+    const int o = __shfl_up_sync(0xffffffffu, incl, d);
+    if (lane >= d) incl += o;
+  }
+  int pos = n + incl - cnt;
+#pragma unroll
+  for (int t = 0; t < 16; ++t) {
+    if ((m >> t) & 1u) {
+      wb->key[pos] = enc_ordered(a[t]);
+      wb->idx[pos] = tok + t;
+      ++pos;
+    }
+  }
+  n += __shfl_sync(0xffffffffu, incl, 31);
+  __syncwarp();
+  if (n > M + 64) {
+    uint32_t kth;
+    n = topm_prune(wb, n, M, &kth);
+    *thr_io = dec_ordered(kth);
+  }
+  return n;
+}
+
 template <int DT>
 __global__ void __launch_bounds__(kTopmWarps * 32, kTopmCtasPerSM)
 topm_select_kernel(const TopmArgs T) {
   __shared__ TopmWarpBuf bufs[kTopmWarps];
+  __shared__ int queues[kTopmWarps][kS4QueueCap];  // group indices awaiting examination
   const int lane = threadIdx.x & 31;
   const int warp = threadIdx.x >> 5;
   const uint32_t lt = (1u << lane) - 1u;
   constexpr int ES = DT == kBF16 ? 2 : 4;
   typedef Group16<DT> G;
   TopmWarpBuf* const wb = &bufs[warp];
+  int* const queue = queues[warp];
 
   for (long long row = (long long)blockIdx.x * kTopmWarps + warp; row < T.rows;
        row += (long long)gridDim.x * kTopmWarps) {
@@ -149,53 +199,36 @@ topm_select_kernel(const TopmArgs T) {
     };
 
     float thr = -CUDART_INF_F;
-    int n = 0;
+    int n = 0, qn = 0, s = 0;
     __syncwarp();  // the previous row's output loop is done with the buffer
     G nxt[kS4LaneGroups];
     if (n_steps > 0) load_step(nxt, 0);
+    for (;;) {
+      // the sweep: a group whose maximum exceeds the threshold is queued (in index order); the
+      // examination is called from the outer loop so that this loop carries no call
 #pragma unroll 1
-    for (int s = 0; s < n_steps; ++s) {
-      G g[kS4LaneGroups];
+      for (; s < n_steps && qn < 32; ++s) {
+        G g[kS4LaneGroups];
 #pragma unroll
-      for (int q = 0; q < kS4LaneGroups; ++q) g[q] = nxt[q];
-      if (s + 1 < n_steps) load_step(nxt, s + 1);
+        for (int q = 0; q < kS4LaneGroups; ++q) g[q] = nxt[q];
+        if (s + 1 < n_steps) load_step(nxt, s + 1);
+        const int g0 = (tok0 + s * kS4WarpTokens) >> 4;
 #pragma unroll
-      for (int q = 0; q < kS4LaneGroups; ++q) {
-        const float gmax = group16_max(g[q]);
-        if (__any_sync(0xffffffffu, gmax > thr)) {  // false for NaN
-          const int tok = tok0 + s * kS4WarpTokens + q * 512;
-          uint32_t m = 0u;
-#pragma unroll
-          for (int t = 0; t < 16; ++t) {
-            const float a = group16_get<DT>(g[q], t);
-            if (a > thr && a < CUDART_INF_F && tok + t < T.V) m |= 1u << t;
-          }
-          // the lanes' tokens are appended in index order
-          const int cnt = __popc(m);
-          int incl = cnt;
-#pragma unroll
-          for (int d = 1; d < 32; d <<= 1) {
-            const int o = __shfl_up_sync(0xffffffffu, incl, d);
-            if (lane >= d) incl += o;
-          }
-          int pos = n + incl - cnt;
-#pragma unroll
-          for (int t = 0; t < 16; ++t) {
-            if ((m >> t) & 1u) {
-              wb->key[pos] = enc_ordered(group16_get<DT>(g[q], t));
-              wb->idx[pos] = tok + t;
-              ++pos;
-            }
-          }
-          n += __shfl_sync(0xffffffffu, incl, 31);
-          __syncwarp();
-          if (n > kTopmCap - 512) {
-            uint32_t kth;
-            n = topm_prune(wb, n, T.M, &kth);
-            thr = dec_ordered(kth);
+        for (int q = 0; q < kS4LaneGroups; ++q) {
+          const bool hit = group16_max(g[q]) > thr;  // false for NaN
+          const unsigned bal = __ballot_sync(0xffffffffu, hit);
+          if (bal != 0u) {
+            if (hit) queue[qn + __popc(bal & lt)] = g0 + 32 * q;
+            qn += __popc(bal);
           }
         }
       }
+      if (qn == 0 && s >= n_steps) break;
+      __syncwarp();
+      for (int first = 0; first < qn; first += 32)
+        n = topm_expand<DT>(wb, queue, rowp, T.V, first, min(32, qn - first), n, T.M, &thr);
+      qn = 0;
+      if (s >= n_steps) break;
     }
     if (n > T.M) {
       uint32_t kth;
@@ -207,7 +240,6 @@ topm_select_kernel(const TopmArgs T) {
       T.logits[row * T.M + i] = i < n ? dec_ordered(wb->key[i]) : -CUDART_INF_F;
     }
   }
-  (void)lt;
 }
 
 }  // namespace gls
