@@ -245,3 +245,24 @@ def compress_select(enc_logw, dec_logw=None, bins=None, seed=0, seq_base=0, seq_
         raise ValueError("oracle compress_select: invalid arguments")
     return dict(enc_index=enc_index, message=message, dec_index=dec_index, match=match,
                 scores=scores, gaps=gaps)
+
+
+def top_m_rows(logits, M):
+    """Top-M truncation of dense rows (Sec. 4.4 / Appendix D.1: sampling from the M most likely
+    tokens): per row keep the M largest finite logits, ties at the M-th value going to the lower
+    token index, and set every other entry to -inf (a masked token).  NaN, +inf and -inf entries are
+    never kept; a row with fewer than M finite entries keeps them all.
+
+    logits: float array [..., V].  Returns (float32 array of the same shape, list of kept index
+    arrays in ascending order, one per row in C order).  Plain sort per row: slow and obvious."""
+    x = np.asarray(logits, dtype=np.float32)
+    flat = x.reshape(-1, x.shape[-1])
+    out = np.full_like(flat, -np.inf)
+    kept = []
+    for r in range(flat.shape[0]):
+        cand = [(-float(v), i) for i, v in enumerate(flat[r]) if np.isfinite(v)]
+        cand.sort()  # by logit descending, then index ascending
+        k = np.array(sorted(i for _, i in cand[:M]), dtype=np.int64)
+        out[r, k] = flat[r, k]
+        kept.append(k)
+    return out.reshape(x.shape), kept

@@ -12,25 +12,10 @@ pytestmark = pytest.mark.gpu
 SEED = synth.NOISE_SEED + 505
 
 
-def _select_cpu(row, M):
-    """Indices of the M largest finite entries of a 1-D float array (ties: lowest index), ascending."""
-    idx = np.arange(row.size)
-    ok = np.isfinite(row)
-    order = np.lexsort((idx[ok], -row[ok].astype(np.float64)))[:M]
-    return np.sort(idx[ok][order])
-
-
 def _masked(dense, M):
-    """dense [..., V] torch (any float dtype) -> (fp32 numpy rows with -inf outside the top M, kept ids)."""
-    x = dense.float().cpu().numpy()
-    flat = x.reshape(-1, x.shape[-1])
-    out = np.full_like(flat, -np.inf)
-    kept = []
-    for r in range(flat.shape[0]):
-        k = _select_cpu(flat[r], M)
-        out[r, k] = flat[r, k]
-        kept.append(k)
-    return out.reshape(x.shape), kept
+    """dense [..., V] torch (any float dtype) -> the oracle's truncated fp32 rows and kept ids."""
+    from oracle import gls_oracle
+    return gls_oracle.top_m_rows(dense.float().cpu().numpy(), M)
 
 
 def _check_lists(lists, dense, M, what):

@@ -297,3 +297,47 @@ def test_excluded_and_empty_rows(oracle):
     assert (r["tokens"] == -1).all()
     v = oracle.target_sample_verify(e, np.zeros((3, 2, 1), np.int32), seed=SEED)
     assert (v["tokens"][:, 0] == -1).all() and (v["tau"] == 1).all() and not v["accept"].any()
+
+
+def test_top_m_truncation_of_the_oracle(oracle):
+    """Sec. 4.4 truncation as the oracle defines it, against numpy's stable sort and by its
+    properties: size, dominance, ties to the lower index, special values never kept."""
+    rng = np.random.default_rng(12)
+    for V, M in [(1, 1), (5, 10), (40, 7), (300, 50), (2000, 256)]:
+        x = np.round(rng.normal(size=(3, 2, V)) * 4) / 4  # many ties
+        x[0, 0, rng.integers(0, V)] = np.nan
+        x[1, 1, rng.integers(0, V)] = np.inf
+        x[2, 0, rng.integers(0, V)] = -np.inf
+        out, kept = oracle.top_m_rows(x, M)
+        flat, oflat = x.reshape(-1, V).astype(np.float32), out.reshape(-1, V)
+        for r in range(flat.shape[0]):
+            fin = np.isfinite(flat[r])
+            k = kept[r]
+            assert len(k) == min(M, int(fin.sum())) and np.all(np.diff(k) > 0)
+            assert np.array_equal(oflat[r, k], flat[r, k])
+            rest = np.setdiff1d(np.arange(V), k)
+            assert np.all(np.isneginf(oflat[r, rest]))
+            # second route: stable argsort of the negated finite values
+            idx = np.flatnonzero(fin)
+            want = np.sort(idx[np.argsort(-flat[r, idx], kind="stable")[:M]])
+            assert np.array_equal(k, want)
+            if len(k) and len(rest):
+                lo = flat[r, k].min()
+                dropped = flat[r, rest][np.isfinite(flat[r, rest])]
+                assert np.all(dropped <= lo)
+                # a dropped token that ties with the smallest kept one has a higher index than every kept tie
+                ties_kept = k[flat[r, k] == lo]
+                ties_dropped = rest[flat[r, rest] == lo]
+                assert ties_dropped.size == 0 or ties_dropped.min() > ties_kept.max()
+    # truncation then the race: the token drawn is always a kept one, and follows the renormalised law
+    V, M, n = 12, 4, 40000
+    logits = rng.normal(size=V).astype(np.float32) * 1.5
+    out, kept = oracle.top_m_rows(logits[None, :], M)
+    rows = np.broadcast_to(out.reshape(1, 1, 1, V), (n, 1, 1, V))
+    tok = oracle.draft_sample(rows, seed=SEED + 31)["tokens"].reshape(-1)
+    assert set(np.unique(tok)) <= set(kept[0].tolist())
+    lk = logits[kept[0]].astype(np.float64)
+    p = np.exp(lk - lk.max())
+    p /= p.sum()
+    counts = np.array([(tok == i).sum() for i in kept[0]])
+    assert stats.chisquare(counts, p * n).pvalue > 1e-4
