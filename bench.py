@@ -215,8 +215,23 @@ def run_ours(args):
     small = dbytes + tbytes < 512e6  # fits the 126 MB L2 several times over? then flush
     flush = torch.zeros(64 << 20, dtype=torch.float32, device="cuda") if small else None
 
+    topm_ws = None
+    if args.topm:
+        # extra workload: every row truncated to its top-M logits in front of the races
+        args.no_e2e = args.no_cpu = True
+        topm_ws = torch.empty(pkg.topm_workspace_bytes(B, K, L + 1, args.topm), dtype=torch.uint8,
+                              device="cuda")
+
     def step(marks):
         _mark(marks)
+        if args.topm:
+            dtok = pkg.draft_sample_topm(w.draft_logits, args.topm, workspace=topm_ws,
+                                         status=buf.status, **kw)[0]
+            _mark(marks)
+            buf.out = pkg.target_sample_verify_topm(w.target_logits, dtok, args.topm,
+                                                    workspace=topm_ws, status=buf.status, **kw)
+            _mark(marks)
+            return
         pkg.draft_sample(w.draft_logits, out_tokens=buf.draft_tokens, out_scores=buf.draft_scores,
                          workspace=buf.workspace, status=buf.status, **kw)
         _mark(marks)
@@ -254,7 +269,7 @@ def run_ours(args):
         l2_warm = {"draft_ms": statistics.mean(m[0].elapsed_time(m[1]) for m in wm),
                    "verify_ms": statistics.mean(m[1].elapsed_time(m[2]) for m in wm)}
     graphed = None
-    if flush is not None:
+    if flush is not None and not args.topm:
         # small batches are bound by the host issuing the launches: the same step as a replayed
         # CUDA graph (L2 flushed between replays, each replay in its own event pair)
         gs = pipeline.GraphedStep(w.draft_logits, w.target_logits, buf, inv_temp=w.inv_temp,
@@ -319,12 +334,18 @@ def run_ours(args):
     achieved = tbytes / (verify_ms * 1e-3) / 1e9
     kname = {4: "sweep4_kernel", 3: "sweep3_kernel"}.get(args.spec, "sweep_kernel") + "<%s, lse>" % (
         "bf16" if w.target_logits.dtype == torch.bfloat16 else "f32")
-    roofline = {"bound": "hbm", "kernel": kname + " (target side: the dominant kernel; the event bracket "
-                "is the whole call, which also runs finalize_verify_kernel, ~4 % of it, so the "
-                "kernel alone is slightly faster than reported)",
+    if args.topm:
+        kname = "topm_select_kernel<%s> + sparse_verify_kernel" % (
+            "bf16" if w.target_logits.dtype == torch.bfloat16 else "f32")
+    kdesc = (" (target side: selection of the top-M tokens of every row, then the race on the lists; "
+             "the event bracket is the whole call)") if args.topm else (
+        " (target side: the dominant kernel; the event bracket "
+        "is the whole call, which also runs finalize_verify_kernel, ~4 % of it, so the "
+        "kernel alone is slightly faster than reported)")
+    roofline = {"bound": "hbm", "kernel": kname + kdesc,
                 "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                 "peak_source": "of " + which,
-                "traffic": (TRAFFIC_RATIO * tbytes) if (TRAFFIC_RATIO and args.spec == 4) else None,
+                "traffic": (TRAFFIC_RATIO * tbytes) if (TRAFFIC_RATIO and args.spec == 4 and not args.topm) else None,
                 "algorithmic_bytes": tbytes, "ms": verify_ms,
                 "draft_side": {"achieved": dbytes / (draft_ms * 1e-3) / 1e9, "ms": draft_ms,
                                "frac": dbytes / (draft_ms * 1e-3) / 1e9 / peak},
@@ -343,7 +364,7 @@ def run_ours(args):
             "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
             "config": {"workload": WORKLOAD_DESC[args.workload] + (" (B overridden to %d)" % B if args.batch else ""),
-                       "noise_spec": args.spec,
+                       "noise_spec": args.spec, "top_m": args.topm or None,
                        "philox_rounds": 10,
                        "l2_warm": l2_warm, "cuda_graph_replay": graphed,
                        "l2": "flushed between steps" if flush is not None
@@ -433,6 +454,8 @@ def main():
     ap.add_argument("--batch", type=int, default=None,
                     help="override B (reduced copy of the workload, e.g. for an ncu capture)")
     ap.add_argument("--spec", type=int, default=4, choices=[1, 2, 3, 4], help="noise_spec")
+    ap.add_argument("--topm", type=int, default=0,
+                    help="extra workload: truncate every row to its top-M logits first (Sec. 4.4)")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle baseline leg")
     args = ap.parse_args()
