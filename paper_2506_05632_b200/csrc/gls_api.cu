@@ -993,6 +993,8 @@ size_t gls_topm_workspace_bytes(int B, int K, int J, int M) {
          gls::align_up((size_t)B * K * J * M * sizeof(float), 256);
 }
 
+}  // extern "C"
+
 namespace gls {
 // selects into the workspace and describes the result as sparse rows
 static int topm_select(const gls_rows_t* rows, int B, int K, int J, int64_t V, int M, void* workspace,
@@ -1031,6 +1033,8 @@ static int topm_select(const gls_rows_t* rows, int B, int K, int J, int64_t V, i
   return GLS_OK;
 }
 }  // namespace gls
+
+extern "C" {
 
 int gls_draft_sample_topm(const gls_rows_t* draft_logits, int B, int K, int J, int64_t V, int M,
                           float inv_temp, const float* inv_temp_per_draft_host,
