@@ -222,6 +222,7 @@ __global__ void __launch_bounds__(128)
 finalize_rows_kernel(const __grid_constant__ SweepArgs A, int rows, int with_lse,
                      RowResult* __restrict__ rowres, int32_t* __restrict__ out_tokens,
                      float* __restrict__ out_scores, uint32_t* __restrict__ dev_status) {
+  asm volatile("griddepcontrol.wait;" ::: "memory");  // the sweep before this launch is complete
   const int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
   if (row >= rows) return;
   const RowResult r = finalize_row<DT, SPEC, ROUNDS>(A, row, with_lse, dev_status);
@@ -311,6 +312,7 @@ constexpr size_t kFusedVerifyMaxSmem = 48 * 1024;
 template <int DT, int SPEC, int ROUNDS>
 __global__ void __launch_bounds__(kFusedVerifyMaxWarps * 32)
 finalize_verify_kernel(const __grid_constant__ SweepArgs A, const VerifyArgs va) {
+  asm volatile("griddepcontrol.wait;" ::: "memory");  // the sweep before this launch is complete
   RowResult* srows = reinterpret_cast<RowResult*>(s3_smem_raw);
   const int b = blockIdx.x;
   const int nrows = va.K * va.J;
@@ -518,14 +520,32 @@ static cudaError_t launch_sweep_t(const SweepArgs& A, bool lse, int grid, cudaSt
   return cudaGetLastError();
 }
 
+// The reduction kernels are launched as programmatic dependents of the sweep before them in the
+// stream: their blocks may be scheduled while the sweep drains (the sweep signals that its
+// block is done), and wait at their first instruction until the whole sweep has completed and its
+// writes are visible.  This hides the launch latency between the two kernels of a call.
+static cudaLaunchAttribute g_dependent_attr[1];
+static cudaLaunchConfig_t dependent_launch(int grid, int block, size_t smem, cudaStream_t st) {
+  g_dependent_attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  g_dependent_attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)grid);
+  cfg.blockDim = dim3((unsigned)block);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cfg.attrs = g_dependent_attr;
+  cfg.numAttrs = 1;
+  return cfg;
+}
+
 template <int DT, int SPEC, int ROUNDS>
 static cudaError_t launch_finalize_t(const SweepArgs& A, int rows, bool lse, RowResult* rowres,
                                      int32_t* out_tokens, float* out_scores, uint32_t* status,
                                      cudaStream_t st) {
   const int wpb = 4;
-  finalize_rows_kernel<DT, SPEC, ROUNDS><<<(rows + wpb - 1) / wpb, wpb * 32, 0, st>>>(
-      A, rows, lse ? 1 : 0, rowres, out_tokens, out_scores, status);
-  return cudaGetLastError();
+  cudaLaunchConfig_t cfg = dependent_launch((rows + wpb - 1) / wpb, wpb * 32, 0, st);
+  return cudaLaunchKernelEx(&cfg, finalize_rows_kernel<DT, SPEC, ROUNDS>, A, rows, lse ? 1 : 0, rowres,
+                            out_tokens, out_scores, status);
 }
 
 // sweep + split reduction of one batch of rows
@@ -534,8 +554,8 @@ static cudaError_t launch_fused_verify_t(const SweepArgs& A, const VerifyArgs& v
   const size_t smem = (size_t)va.K * va.J * sizeof(RowResult);
   const int nrows = va.K * va.J;
   const int warps = nrows < kFusedVerifyMaxWarps ? nrows : kFusedVerifyMaxWarps;
-  finalize_verify_kernel<DT, SPEC, ROUNDS><<<va.B, warps * 32, smem, st>>>(A, va);
-  return cudaGetLastError();
+  cudaLaunchConfig_t cfg = dependent_launch(va.B, warps * 32, smem, st);
+  return cudaLaunchKernelEx(&cfg, finalize_verify_kernel<DT, SPEC, ROUNDS>, A, va);
 }
 
 // sweep + split reduction of one batch of rows.  With `va` (verification) and a sequence's

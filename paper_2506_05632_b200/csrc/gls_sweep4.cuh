@@ -492,6 +492,8 @@ sweep4_kernel(const __grid_constant__ SweepArgs A) {
       if (A.splits > 1 && m_enc > 0u) atomicMax(A.hints + row, m_enc);
     }
   }
+  // this block has no more work: a dependent launch (the reduction) may start to be scheduled
+  asm volatile("griddepcontrol.launch_dependents;");
 }
 
 }  // namespace gls
