@@ -96,12 +96,12 @@ static Plan make_plan3(long long rows, long long V, int dtype) {
 #define GLS_S4_WASTE 0.15
 #define GLS_S4_MIN_STEPS 4
 #endif
-template <int DT>
+template <int SH>
 static Plan make_plan4_t(long long rows, long long V) {
   Plan p;
-  constexpr int kCtaTok = S4Cfg<DT>::kCtaTokens;
+  constexpr int kCtaTok = S4Cfg<SH>::kCtaTokens;
   constexpr int kMinChunk = GLS_S4_MIN_STEPS * kCtaTok;
-  const long long grid = (long long)kNumSMs * S4Cfg<DT>::kCtasPerSM;
+  const long long grid = (long long)kNumSMs * S4Cfg<SH>::kCtasPerSM;
   long long max_splits = (V + kMinChunk - 1) / kMinChunk;
   if (rows * max_splits < 2 * grid) max_splits = (V + kCtaTok - 1) / kCtaTok;
   long long splits = 1;
@@ -115,17 +115,25 @@ static Plan make_plan4_t(long long rows, long long V) {
   chunk = (chunk + kCtaTok - 1) / kCtaTok * kCtaTok;
   p.chunk = (int)chunk;
   p.splits = (int)((V + chunk - 1) / chunk);
-  p.parts = p.splits * S4Cfg<DT>::kWarps;
+  p.parts = p.splits * S4Cfg<SH>::kWarps;
   p.rows = rows;
   plan_layout(p);
   return p;
 }
-static Plan make_plan4(long long rows, long long V, int dtype) {
-  return dtype == GLS_BF16 ? make_plan4_t<kBF16>(rows, V) : make_plan4_t<kF32>(rows, V);
+// the sweep's launch shape for rows of V elements (multi: the fused multi-stream race)
+static int s4_shape(int dtype, long long V, bool multi) {
+  if (dtype == GLS_BF16) return kS4ShapeBf16;
+  return (multi || V < kS4WideMinTokens) ? kS4ShapeF32Narrow : kS4ShapeF32Wide;
+}
+static Plan make_plan4(long long rows, long long V, int dtype, bool multi) {
+  const int sh = s4_shape(dtype, V, multi);
+  return sh == kS4ShapeBf16 ? make_plan4_t<kS4ShapeBf16>(rows, V)
+         : sh == kS4ShapeF32Wide ? make_plan4_t<kS4ShapeF32Wide>(rows, V)
+                                 : make_plan4_t<kS4ShapeF32Narrow>(rows, V);
 }
 
-static Plan make_plan(long long rows, long long V, int spec, int dtype) {
-  return spec == 4 ? make_plan4(rows, V, dtype)
+static Plan make_plan(long long rows, long long V, int spec, int dtype, bool multi = false) {
+  return spec == 4 ? make_plan4(rows, V, dtype, multi)
                    : spec == 3 ? make_plan3(rows, V, dtype) : make_plan12(rows, V);
 }
 
@@ -581,20 +589,22 @@ static int run_rows(SweepArgs& A, int dtype, int spec, const Plan& P, void* work
   const bool r10 = A.rounds == 10;
   const bool bf = dtype == GLS_BF16;
   if (spec == 4) {
-    const long long cap = (long long)kNumSMs * (bf ? S4Cfg<kBF16>::kCtasPerSM : S4Cfg<kF32>::kCtasPerSM);
-    const int grid = (int)(P.n_items < cap ? P.n_items : cap);
-#define SWEEP4(DT, R)                                                                       \
+    const int sh = s4_shape(dtype, A.V, A.multi_k > 0);
+#define SWEEP4(SH, R)                                                                       \
   do {                                                                                      \
-    const size_t smem = sizeof(S4Shared<DT>);                                               \
+    const long long cap = (long long)kNumSMs * S4Cfg<SH>::kCtasPerSM;                       \
+    const int grid = (int)(P.n_items < cap ? P.n_items : cap);                              \
+    const size_t smem = sizeof(S4Shared<SH>);                                               \
     if (A.multi_k > 0)                                                                      \
-      sweep4_kernel<DT, true, R, true><<<grid, S4Cfg<DT>::kWarps * 32, smem, st>>>(A);      \
+      sweep4_kernel<SH, true, R, true><<<grid, S4Cfg<SH>::kWarps * 32, smem, st>>>(A);      \
     else if (lse)                                                                           \
-      sweep4_kernel<DT, true, R><<<grid, S4Cfg<DT>::kWarps * 32, smem, st>>>(A);            \
+      sweep4_kernel<SH, true, R><<<grid, S4Cfg<SH>::kWarps * 32, smem, st>>>(A);            \
     else                                                                                    \
-      sweep4_kernel<DT, false, R><<<grid, S4Cfg<DT>::kWarps * 32, smem, st>>>(A);           \
+      sweep4_kernel<SH, false, R><<<grid, S4Cfg<SH>::kWarps * 32, smem, st>>>(A);           \
   } while (0)
-    if (bf) { if (r10) SWEEP4(kBF16, 10); else SWEEP4(kBF16, 0); }
-    else { if (r10) SWEEP4(kF32, 10); else SWEEP4(kF32, 0); }
+    if (sh == kS4ShapeBf16) { if (r10) SWEEP4(kS4ShapeBf16, 10); else SWEEP4(kS4ShapeBf16, 0); }
+    else if (sh == kS4ShapeF32Wide) { if (r10) SWEEP4(kS4ShapeF32Wide, 10); else SWEEP4(kS4ShapeF32Wide, 0); }
+    else { if (r10) SWEEP4(kS4ShapeF32Narrow, 10); else SWEEP4(kS4ShapeF32Narrow, 0); }
 #undef SWEEP4
     err = cudaGetLastError();
   } else if (spec == 3) {
@@ -696,8 +706,8 @@ size_t gls_workspace_bytes(int B, int K, int J, int64_t V) {
     const size_t c = make_plan3((long long)B * J, V, dt).total;  // fused multi-stream encoder
     if (b > need) need = b;
     if (c > need) need = c;
-    const size_t d = make_plan4((long long)B * K * J, V, dt).total;
-    const size_t e = make_plan4((long long)B * J, V, dt).total;
+    const size_t d = make_plan4((long long)B * K * J, V, dt, false).total;
+    const size_t e = make_plan4((long long)B * J, V, dt, true).total;
     if (d > need) need = d;
     if (e > need) need = e;
   }
@@ -925,7 +935,7 @@ int gls_compress_select(const gls_rows_t* enc_logw, const gls_rows_t* dec_logw, 
   // its own and the epilogue takes the best of the K winners.
   const bool fused_enc = spec >= 3 && K <= 8 && N < (1LL << 28);
   if (fused_enc) {
-    const Plan PE = make_plan((long long)B, N, spec, enc_logw->dtype);
+    const Plan PE = make_plan((long long)B, N, spec, enc_logw->dtype, true);
     if (workspace_bytes < PE.total) return GLS_ERR_WORKSPACE;
     A.K = 1;
     A.multi_k = K;

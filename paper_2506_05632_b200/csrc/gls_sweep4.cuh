@@ -50,18 +50,28 @@ constexpr int kS4WarpTokens = 16 * kS4WarpGroups;               // 2048
 // Groups per warp queue: a batch is taken at 32 queued groups, and one step can add 128 more.
 constexpr int kS4QueueCap = 32 + kS4WarpGroups;
 
-// Launch shape per element type, chosen by measurement.  A lane holds its four groups in
-// registers (32 for bf16, 64 for fp32).  bf16 rows: the next step's loads are issued before the
-// current step is used (32 more registers), one warp per CTA and 16 CTAs per SM (128 registers);
-// at the time of the choice config 4 draft / target ran at 6.48 / 4.90 TB/s against 6.05 / 4.75
-// TB/s for 2 warps x 10 CTAs without the prefetch.  fp32 rows: 8 warps x 2 CTAs (128 registers), no prefetch.
-template <int DT>
+// Launch shapes, chosen by measurement.  A lane holds its four groups in registers (32 for bf16,
+// 64 for fp32); every shape runs under a 128-register budget.
+//   shape 1, bf16 rows: the next step's loads are issued before the current step is used (32 more
+//     registers), one warp per CTA and 16 CTAs per SM (at the time of the choice config 4 ran at
+//     6.48 / 4.90 TB/s against 6.05 / 4.75 TB/s for 2 warps x 10 CTAs without the prefetch);
+//   shape 0, fp32 rows of at least 2^19 tokens: 8 warps x 2 CTAs, no prefetch (config 5 decoders
+//     6.58 TB/s against 5.96 TB/s for 1 x 16);
+//   shape 2, shorter fp32 rows and the fused multi-stream race: 1 warp x 16 CTAs, so that a warp's
+//     share of a row stays tens of steps long (rows of 128k tokens: 5.14 / 5.01 TB/s per draft /
+//     target call against 4.62 / 4.24 TB/s for 8 x 2).
+constexpr int kS4ShapeF32Wide = 0, kS4ShapeBf16 = 1, kS4ShapeF32Narrow = 2;
+constexpr long long kS4WideMinTokens = 1LL << 19;
+template <int SH>
 struct S4Cfg {
-  static constexpr int kWarps = DT == kBF16 ? GLS_S4_BF16_WARPS : GLS_S4_F32_WARPS;
-  static constexpr int kCtasPerSM = DT == kBF16 ? GLS_S4_BF16_CTAS : GLS_S4_F32_CTAS;
+  static constexpr int kDT = SH == kS4ShapeBf16 ? kBF16 : kF32;
+  static constexpr int kWarps =
+      SH == kS4ShapeBf16 ? GLS_S4_BF16_WARPS : SH == kS4ShapeF32Wide ? GLS_S4_F32_WARPS : 1;
+  static constexpr int kCtasPerSM =
+      SH == kS4ShapeBf16 ? GLS_S4_BF16_CTAS : SH == kS4ShapeF32Wide ? GLS_S4_F32_CTAS : 16;
   static constexpr int kCtaTokens = kWarps * kS4WarpTokens;
   // the next step's loads are issued before the current step is used (bf16: 32 more registers)
-  static constexpr bool kPrefetch = DT == kBF16 ? (GLS_S4_BF16_PREFETCH != 0) : false;
+  static constexpr bool kPrefetch = SH == kS4ShapeBf16 ? (GLS_S4_BF16_PREFETCH != 0) : false;
 };
 constexpr int kS4MaxCtaTokens = 8 * kS4WarpTokens;
 
@@ -73,16 +83,16 @@ struct S4WarpCtx {  // what the batched path needs to know about the warp's curr
   float inv_t;
   int msg, tok_end;
 };
-template <int DT>
+template <int SH>
 struct S4Shared {
   unsigned long long m_tag;  // (item tag << 32) | ordered code of the CTA-wide bound on the best score
-  S4WarpCtx ctx[S4Cfg<DT>::kWarps];
-  Top2 best[S4Cfg<DT>::kWarps * 32];
-  uint2 queue[S4Cfg<DT>::kWarps][kS4QueueCap];  // (coarse word, group | stream << 28)
+  S4WarpCtx ctx[S4Cfg<SH>::kWarps];
+  Top2 best[S4Cfg<SH>::kWarps * 32];
+  uint2 queue[S4Cfg<SH>::kWarps][kS4QueueCap];  // (coarse word, group | stream << 28)
 };
-template <int DT>
-__device__ __forceinline__ S4Shared<DT>& s4_shared() {
-  return *reinterpret_cast<S4Shared<DT>*>(s3_smem_raw);
+template <int SH>
+__device__ __forceinline__ S4Shared<SH>& s4_shared() {
+  return *reinterpret_cast<S4Shared<SH>*>(s3_smem_raw);
 }
 
 // Exp(1) from the uniform v = (word + frac) * 2^-32, frac in (0, 1) standing for further bits
@@ -126,9 +136,10 @@ __device__ __forceinline__ uint32_t s4_call_index(uint32_t g) { return ((g >> 7)
 // per round, drawing the token's own exponential unless it is the group's minimum.  Returns the
 // best lower bound found (ordered code, 0 if none).
 // ------------------------------------------------------------------------------------------
-template <int DT, int ROUNDS, bool MULTI>
+template <int SH, int ROUNDS, bool MULTI>
 __device__ __noinline__ uint32_t s4_flush(int rounds_rt, int first, int n, float nm) {
-  S4Shared<DT>& sh = s4_shared<DT>();
+  constexpr int DT = S4Cfg<SH>::kDT;
+  S4Shared<SH>& sh = s4_shared<SH>();
   const int lane = threadIdx.x & 31;
   const int warp = threadIdx.x >> 5;
   const S4WarpCtx cx = sh.ctx[warp];
@@ -205,13 +216,14 @@ __device__ __noinline__ uint32_t s4_flush(int rounds_rt, int first, int n, float
 
 // The lane's share of a work item again for the softmax sum, token by token, leaving out NaN and
 // +inf logits (they cannot define a probability).  Rare: only rows that hold such values.
-template <int DT>
+template <int SH>
 __device__ __noinline__ void lse4_redo_careful(const char* rowp, int tok0, int n_steps, int tok_end,
                                                float c2, float* lm_out, float* ls_out) {
+  constexpr int DT = S4Cfg<SH>::kDT;
   float lm = kS3LseFloor, ls = 0.f;
   for (int s = 0; s < n_steps; ++s) {
     for (int j = 0; j < kS4LaneGroups; ++j) {
-      const int tok = tok0 + s * S4Cfg<DT>::kCtaTokens + j * 512;
+      const int tok = tok0 + s * S4Cfg<SH>::kCtaTokens + j * 512;
       for (int t = 0; t < 16; ++t) {
         if (tok + t >= tok_end) break;
         const float a = load_logit<DT>(rowp, tok + t);
@@ -231,15 +243,16 @@ __device__ __noinline__ void lse4_redo_careful(const char* rowp, int tok0, int n
 // ------------------------------------------------------------------------------------------
 // The kernel
 // ------------------------------------------------------------------------------------------
-template <int DT, bool LSE, int ROUNDS, bool MULTI = false>
-__global__ void __launch_bounds__(S4Cfg<DT>::kWarps * 32, S4Cfg<DT>::kCtasPerSM)
+template <int SH, bool LSE, int ROUNDS, bool MULTI = false>
+__global__ void __launch_bounds__(S4Cfg<SH>::kWarps * 32, S4Cfg<SH>::kCtasPerSM)
 sweep4_kernel(const __grid_constant__ SweepArgs A) {
-  S4Shared<DT>& sh = s4_shared<DT>();
+  constexpr int DT = S4Cfg<SH>::kDT;
+  S4Shared<SH>& sh = s4_shared<SH>();
   const int lane = threadIdx.x & 31;
   const int warp = threadIdx.x >> 5;
   constexpr int ES = DT == kBF16 ? 2 : 4;
-  constexpr int kWarps = S4Cfg<DT>::kWarps;
-  constexpr int kCtaTokens = S4Cfg<DT>::kCtaTokens;
+  constexpr int kWarps = S4Cfg<SH>::kWarps;
+  constexpr int kCtaTokens = S4Cfg<SH>::kCtaTokens;
   typedef Group16<DT> G;
   uint2* const queue = sh.queue[warp];
   volatile unsigned long long* const m_tag = &sh.m_tag;
@@ -342,7 +355,7 @@ sweep4_kernel(const __grid_constant__ SweepArgs A) {
       const int nb = __popc(bal);
       __syncwarp();
       if (nb > 0) {
-        const uint32_t e = s4_flush<DT, ROUNDS, MULTI>(A.rounds, 0, nb, filter_offset(dec_ordered(m_enc)));
+        const uint32_t e = s4_flush<SH, ROUNDS, MULTI>(A.rounds, 0, nb, filter_offset(dec_ordered(m_enc)));
         if (e > m_enc) m_enc = e;
       }
     }
@@ -375,7 +388,7 @@ sweep4_kernel(const __grid_constant__ SweepArgs A) {
       __syncwarp();
       const int nb = min(qn, 32);
       qn -= nb;
-      uint32_t e = s4_flush<DT, ROUNDS, MULTI>(A.rounds, qn, nb, nm4 - 4.0f);
+      uint32_t e = s4_flush<SH, ROUNDS, MULTI>(A.rounds, qn, nb, nm4 - 4.0f);
       // the slices of a row trade their bounds through the row's hint word at batch time
       if (A.splits > 1) {
         uint32_t h = 0u;
@@ -430,7 +443,7 @@ sweep4_kernel(const __grid_constant__ SweepArgs A) {
       // ---- the sweep.  The inner loop runs until 32 groups are queued; the batched evaluation
       //      is called from the outer loop so that the inner loop carries no call.
       int s = 0;
-      constexpr bool PREFETCH = S4Cfg<DT>::kPrefetch;
+      constexpr bool PREFETCH = S4Cfg<SH>::kPrefetch;
       G nxt[PREFETCH ? kS4LaneGroups : 1];
       if (PREFETCH && n_steps > 0) load_step(nxt, 0);
       for (;;) {
@@ -471,7 +484,7 @@ sweep4_kernel(const __grid_constant__ SweepArgs A) {
       unpack_f32x2(ls2, s0, s1);
       if (__any_sync(0xffffffffu, !(s0 + s1 < CUDART_INF_F))) {  // NaN or +inf logits in the slice
         float rl, rs;
-        lse4_redo_careful<DT>(rowp, tok0, n_steps, tok_end, c2, &rl, &rs);
+        lse4_redo_careful<SH>(rowp, tok0, n_steps, tok_end, c2, &rl, &rs);
         lm = rl;
         s0 = rs;
         s1 = 0.f;
