@@ -436,8 +436,8 @@ def run_compress(args):
                          "frac": db / (dec_ms * 1e-3) / 1e9 / peak, "peak_source": "of " + which,
                          "traffic": None, "algorithmic_bytes": db, "ms": dec_ms,
                          "encoder": {"ms": ms_enc, "achieved": eb / (ms_enc * 1e-3) / 1e9,
-                                     "note": "fused race over tokens and K noise streams; bound by "
-                                             "instruction issue (K generator calls per group)"},
+                                     "note": "fused race over tokens and K noise streams: the log-sum-exp "
+                                             "plus K generator calls per 64 elements"},
                          "step": {"achieved": (eb + db) / (ms_all * 1e-3) / 1e9}},
             "cpu_baseline": None}
     assert int(status.item()) == 0
