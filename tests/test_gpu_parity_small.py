@@ -281,6 +281,19 @@ def test_orderings_that_defeat_the_filter(gls, oracle, dtype, spec):
         assert (parity.to_np(out)["tau"] == 6).all()
 
 
+def test_fp32_rows_around_the_launch_shape_switch(gls, oracle):
+    """fp32 rows shorter than 2^19 tokens take a one-warp launch shape, longer ones an eight-warp
+    shape: the same data on both sides of the switch, draft and verify."""
+    for V in ((1 << 19) - 16, 1 << 19, (1 << 19) + 2048 * 3 + 5):
+        logits = _rand_logits(1, 2, 2, V, torch.float32, 91, scale=2.0)
+        kw = dict(seed=SEED + 11, inv_temp=1.1)
+        tok, sc, ref = _draft_both(gls, oracle, logits[:, :, :1], **kw)
+        parity.check_draft(tok, sc, ref, "draft V=%d" % V)
+        out = gls.target_sample_verify(logits, torch.from_numpy(ref["tokens"]).cuda(), **kw)
+        refv = oracle.target_sample_verify(synth.to_numpy_rows(logits), ref["tokens"], **kw)
+        parity.check_verify(parity.to_np(out), refv, "verify V=%d" % V)
+
+
 def test_step_replayed_as_cuda_graph_matches_eager(gls):
     """The library's calls can be captured: a replayed graph of one step gives the eager result,
     also after the logits were refilled in place."""
