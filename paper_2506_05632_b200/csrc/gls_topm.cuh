@@ -146,7 +146,7 @@ __device__ __noinline__ int topm_expand(TopmWarpBuf* wb, const int* queue, const
 #pragma unroll
   for (int t = 0; t < 16; ++t) {
     if ((m >> t) & 1u) {
-      wb->key[pos] = enc_ordered(a[t]);
+      wb->key[pos] = enc_ordered(a[t] + 0.0f);  // -0 and +0 are the same logit: one code
       wb->idx[pos] = tok + t;
       ++pos;
     }

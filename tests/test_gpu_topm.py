@@ -43,6 +43,7 @@ def test_selection_is_exact(gls, dtype):
     V, M = 2048 * 5 + 100, 50
     i = torch.arange(V, device="cuda", dtype=torch.float32)
     rows = torch.stack([i, -i, torch.zeros_like(i), (i % 7), -(i % 5), 0.001 * i])
+    rows[2, ::3] = -0.0                    # -0 and +0 are the same logit: ties go by index
     rows[3, 100] = float("nan")
     rows[3, 101] = float("inf")
     rows[4, :] = float("-inf")
