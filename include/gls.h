@@ -29,15 +29,6 @@
  *               4 / 5 the per-token streams of 0 / 1 (noise_spec 4)
  *
  *   noise_spec 1:  block = i >> 2, w = out[i & 3],                v = (w + 0.5) * 2^-32
- *   noise_spec 2:  coarse  block = i >> 3 in `domain`:   h = 16-bit field (i & 7) of the 128 output
- *                  bits, i.e. (out[(i & 7) >> 1] >> (16 * (i & 1))) & 0xffff;
- *                  refine  block = i >> 2 in `domain + 2`: r = out[i & 3];
- *                                                               v = (h * 2^32 + r + 0.5) * 2^-48
- *   noise_spec 3:  coarse  block = i >> 4 in `domain`:   h = byte (i & 15) of the 128 output bits,
- *                  i.e. (out[(i & 15) >> 2] >> (8 * (i & 3))) & 0xff;
- *                  refine  block = i >> 1 in `domain + 2`: x = the low 40 bits of the 64-bit half
- *                  (i & 1), i.e. ((out[2 (i & 1) + 1] & 0xff) << 32) | out[2 (i & 1)];
- *                                                               v = (h * 2^40 + x + 0.5) * 2^-48
  *   S = -log1p(-v)   (v is strictly inside (0,1), so S is finite and positive; this is the paper's
  *                     S = -ln U with U = 1 - v)
  *
@@ -54,13 +45,13 @@
  *                  S_i = M - log1p(-(u + 0.5) 2^-32) otherwise
  *
  * A draft call and a verify call that describe the same (seed, sequence, position, k, i) therefore
- * see the same S -- that is the coupling.  All four specs are exact definitions of i.i.d. Exp(1)
- * noise.  Specs 2 and 3 let a kernel decide most tokens from the coarse bits alone (16 bits for 8
- * tokens per generator call, or 8 bits for 16 tokens per call) and generate the refinement bits
- * only for the few tokens that can still win.  Spec 4 goes further: one generator call covers 64
- * tokens, and a whole group is settled by the bound S_i >= M >= w * 2^-36 (a few dozen groups
- * per row need a closer look).  Spec 4 is the default and the fastest: the generator's
- * 32x32->64-bit multiplies are the scarcest resource of the sweep on sm_100a.
+ * see the same S -- that is the coupling.  Both specs are exact definitions of i.i.d. Exp(1) noise.
+ * Spec 1 is the literal reading, one uniform per token.  Under spec 4 one generator call covers
+ * 64 tokens, and a whole group is settled by the bound S_i >= M >= w * 2^-36 (a few dozen groups
+ * per row need a closer look).  Spec 4 is the default and about three times faster: the
+ * generator's 32x32->64-bit multiplies are the scarcest resource of the sweep on sm_100a.
+ * (Values 2 and 3 named two intermediate layouts that split a 48-bit uniform into coarse and
+ * refinement bits; they are retired and return GLS_ERR_UNSUPPORTED.)
  *
  * CONVENTIONS
  *   - Token / candidate indices are 0-based (the paper counts from 1).
@@ -69,7 +60,7 @@
  *     on the caller's stream and returns without synchronising.
  *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).
  *   - Rows: the token dimension is contiguous; strides are in ELEMENTS and may be 0 (broadcast).
- *     Rows whose first element is 32-byte aligned (16-byte for noise_spec 1 and 2) take the
+ *     Rows whose first element is 32-byte aligned (16-byte for noise_spec 1) take the
  *     vectorised path; others are still handled (slower scalar loads).
  *   - A logit of -inf is a legal "masked" token (top-K truncation, Sec. 4.4).  NaN and +inf
  *     logits never win a race and are excluded from the log-sum-exp.
@@ -127,7 +118,7 @@ typedef struct {
   uint32_t seq_base;       /* sequence id of batch row b is seq_base + b ...                   */
   const uint32_t* seq_ids; /* ... unless this optional DEVICE array [B] is given               */
   uint32_t pos_base;       /* position id of index j is pos_base + j                           */
-  uint32_t noise_spec;     /* 1, 2, 3 or 4 (see above); 0 selects 4                            */
+  uint32_t noise_spec;     /* 1 or 4 (see above); 0 selects 4                                  */
   uint32_t rounds;         /* Philox rounds, 0 selects 10; 7..16 accepted                      */
   uint32_t flags;          /* GLS_NOISE_*                                                      */
 } gls_noise_t;
@@ -203,8 +194,8 @@ int gls_draft_sample_static(const gls_rows_t* draft_logits, int B, int K, int J,
                             uint32_t* device_status, void* stream);
 
 /*
- * Target side and verification -- Sec. 3 step 1, Algorithm 2 from "Let the set of active drafts"
- * to the end.  With S = {0..K-1} initially, for j = 0..L-1:
+ * Target side and verification -- Sec. 3 step 1 and the verification phase of Algorithm 2 (from
+ * the initialisation of the active set to the end).  With S = {0..K-1} initially, for j = 0..L-1:
  *     Y_j = i-component of argmin_{i, k in S} S_i^(j,k) / q_i^(j,k),
  *           q^(j,k) = softmax(target_logits[b,k,j,:] * inv_temp)
  *     accept[b,k,j] = (k in S and draft_tokens[b,k,j] == Y_j);  S <- {k in S : accept}
@@ -232,8 +223,8 @@ int gls_target_sample_verify(const gls_rows_t* target_logits, int B, int K, int 
                              size_t workspace_bytes, uint32_t* device_status, void* stream);
 
 /*
- * Sparse rows -- Sec. 4.4 ("enabling top-K sampling ... allows us to throw away all but M << N
- * high-probability tokens") and Appendix D.1 (the experiments keep the top 50 tokens).  A row is a
+ * Sparse rows -- Sec. 4.4 (top-K truncation: only M << N high-probability tokens are kept) and
+ * Appendix D.1 (the experiments keep the top 50 tokens).  A row is a
  * list of M kept tokens: their ids in the full vocabulary and their logits; every other token has
  * probability zero.  The races are those of the dense entry points on the row with -inf outside
  * the list, with the noise of each kept token keyed by its ORIGINAL id, so a sparse call and a

@@ -356,7 +356,7 @@ int glso_draft_sample(const void* logits, int dtype, int64_t sb, int64_t sk, int
 }
 
 /* ------------------------------------------------------------------------------------------ */
-/* Target side + verification: Algorithm 2 from "Let the set of active drafts be S".            */
+/* Target side + verification: Algorithm 2, verification phase (active set to the end).         */
 /*   tokens[B,J] (-1 beyond tau), tau[B], accept[B,K,L], scores[B,J], gaps[B,J],                 */
 /*   row_lse[B,K,J] (NaN for rows the algorithm never evaluates)                                 */
 /*   J = L + 1, or L with GLSO_NO_BONUS.                                                         */

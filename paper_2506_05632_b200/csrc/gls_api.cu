@@ -6,19 +6,39 @@
 // translation unit, so the draft-side, target-side and compression entry points see bit-identical
 // shared randomness (the paper's analysis assumes identical floating-point behaviour on both
 // sides of the coupling, Sec. 5.3).
+#include <atomic>
 #include <cmath>
 #include <cstring>
 #include <mutex>
 
 #include "../../include/gls.h"
 #include "gls_kernels.cuh"
-#include "gls_sweep3.cuh"
+#include "gls_group16.cuh"
 #include "gls_sweep4.cuh"
 #include "gls_topm.cuh"
 
 namespace gls {
 
-constexpr int kNumSMs = 148;  // B200
+// Number of SMs of the current device (grids and slice plans are sized from it); looked up once
+// per device.  148 on B200; that value is also the answer when no device can be queried, so that
+// gls_workspace_bytes() stays callable without one.
+static int num_sms() {
+  constexpr int kMaxDev = 64;
+  static std::atomic<int> cache[kMaxDev];
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDev) {
+    (void)cudaGetLastError();
+    return 148;
+  }
+  int n = cache[dev].load(std::memory_order_relaxed);
+  if (n > 0) return n;
+  if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) {
+    (void)cudaGetLastError();
+    return 148;
+  }
+  cache[dev].store(n, std::memory_order_relaxed);
+  return n;
+}
 constexpr int kMinChunk = 2048;
 constexpr int kMaxChunk = 16384;
 
@@ -38,12 +58,12 @@ static void plan_layout(Plan& p) {
   p.total = p.off_rows + align_up((size_t)p.rows * sizeof(RowResult), 256);
 }
 
-// noise_spec 1 and 2 (a warp per work item).  Slice size: aim at ~8 work items per resident warp
+// noise_spec 1 (a warp per work item).  Slice size: aim at ~8 work items per resident warp
 // so that the static round-robin over warps balances, but keep slices long enough to amortise
 // the per-item reduction.
-static Plan make_plan12(long long rows, long long V) {
+static Plan make_plan1(long long rows, long long V) {
   Plan p;
-  const long long target_items = 8LL * kNumSMs * 32;
+  const long long target_items = 8LL * num_sms() * 32;
   long long chunk = (rows * V + target_items - 1) / target_items;
   chunk = (chunk + kWarpTokens - 1) / kWarpTokens * kWarpTokens;
   if (chunk < kMinChunk) chunk = kMinChunk;
@@ -58,40 +78,11 @@ static Plan make_plan12(long long rows, long long V) {
   return p;
 }
 
-// noise_spec 3 (a CTA per work item, one partial per warp).  Every item costs a fixed set-up and
+// noise_spec 4 (a CTA per work item, one partial per warp).  Every item costs a fixed set-up and
 // merge, so rows are cut into as few slices as keep the static round-robin over the resident
 // CTAs balanced: the fewest slices for which the last round of items wastes at most 15 % of the
-// machine, or that give every CTA at least 12 items.  Slices are whole CTA iterations and at
-// least four of them long, except that small problems may go down to one CTA iteration.
-template <int DT>
-static Plan make_plan3_t(long long rows, long long V) {
-  Plan p;
-  constexpr int kCtaTok = S3Cfg<DT>::kCtaTokens;
-  constexpr int kMinChunk = 4 * kCtaTok;
-  const long long grid = (long long)kNumSMs * S3Cfg<DT>::kCtasPerSM;
-  long long max_splits = (V + kMinChunk - 1) / kMinChunk;
-  if (rows * max_splits < 2 * grid) max_splits = (V + kCtaTok - 1) / kCtaTok;
-  long long splits = 1;
-  for (; splits < max_splits; ++splits) {
-    const long long items = rows * splits;
-    if (items >= 12 * grid) break;
-    const long long rounds = (items + grid - 1) / grid;
-    if (items >= grid && (double)(rounds * grid - items) <= 0.15 * (double)(rounds * grid)) break;
-  }
-  long long chunk = (V + splits - 1) / splits;
-  chunk = (chunk + kCtaTok - 1) / kCtaTok * kCtaTok;
-  p.chunk = (int)chunk;
-  p.splits = (int)((V + chunk - 1) / chunk);
-  p.parts = p.splits * S3Cfg<DT>::kWarps;
-  p.rows = rows;
-  plan_layout(p);
-  return p;
-}
-static Plan make_plan3(long long rows, long long V, int dtype) {
-  return dtype == GLS_BF16 ? make_plan3_t<kBF16>(rows, V) : make_plan3_t<kF32>(rows, V);
-}
-
-// noise_spec 4: the same rule with that sweep's CTA shape (a warp step is 2048 tokens).
+// machine, or that give every CTA at least 12 items.  Slices are whole CTA steps and at least four
+// of them long, except that small problems may go down to one CTA step (2048 tokens per warp).
 #ifndef GLS_S4_WASTE
 #define GLS_S4_WASTE 0.15
 #define GLS_S4_MIN_STEPS 4
@@ -101,7 +92,7 @@ static Plan make_plan4_t(long long rows, long long V) {
   Plan p;
   constexpr int kCtaTok = S4Cfg<SH>::kCtaTokens;
   constexpr int kMinChunk = GLS_S4_MIN_STEPS * kCtaTok;
-  const long long grid = (long long)kNumSMs * S4Cfg<SH>::kCtasPerSM;
+  const long long grid = (long long)num_sms() * S4Cfg<SH>::kCtasPerSM;
   long long max_splits = (V + kMinChunk - 1) / kMinChunk;
   if (rows * max_splits < 2 * grid) max_splits = (V + kCtaTok - 1) / kCtaTok;
   long long splits = 1;
@@ -133,8 +124,7 @@ static Plan make_plan4(long long rows, long long V, int dtype, bool multi) {
 }
 
 static Plan make_plan(long long rows, long long V, int spec, int dtype, bool multi = false) {
-  return spec == 4 ? make_plan4(rows, V, dtype, multi)
-                   : spec == 3 ? make_plan3(rows, V, dtype) : make_plan12(rows, V);
+  return spec == 4 ? make_plan4(rows, V, dtype, multi) : make_plan1(rows, V);
 }
 
 // ------------------------------------------------------------------------------------------
@@ -241,7 +231,7 @@ finalize_rows_kernel(const __grid_constant__ SweepArgs A, int rows, int with_lse
 }
 
 // ------------------------------------------------------------------------------------------
-// Algorithm 2, from "Let the set of active drafts be S" to the end; one thread per sequence.
+// Algorithm 2, verification phase (active-set initialisation to the end); one thread per sequence.
 // rows[(b*K + k)*J + j] holds the winner of row (b,k,j) under its own noise stream.
 // ------------------------------------------------------------------------------------------
 // `rows` points at the K x J results of sequence b: rows[k * J + j].
@@ -321,7 +311,7 @@ template <int DT, int SPEC, int ROUNDS>
 __global__ void __launch_bounds__(kFusedVerifyMaxWarps * 32)
 finalize_verify_kernel(const __grid_constant__ SweepArgs A, const VerifyArgs va) {
   asm volatile("griddepcontrol.wait;" ::: "memory");  // the sweep before this launch is complete
-  RowResult* srows = reinterpret_cast<RowResult*>(s3_smem_raw);
+  RowResult* srows = reinterpret_cast<RowResult*>(gls_smem_raw);
   const int b = blockIdx.x;
   const int nrows = va.K * va.J;
   for (int r = threadIdx.x >> 5; r < nrows; r += (int)(blockDim.x >> 5)) {
@@ -470,7 +460,7 @@ sparse_draft_kernel(const __grid_constant__ SweepArgs A, const SparseArgs S, int
 template <int SPEC, int ROUNDS>
 __global__ void __launch_bounds__(kFusedVerifyMaxWarps * 32)
 sparse_verify_kernel(const __grid_constant__ SweepArgs A, const SparseArgs S, const VerifyArgs va) {
-  RowResult* srows = reinterpret_cast<RowResult*>(s3_smem_raw);
+  RowResult* srows = reinterpret_cast<RowResult*>(gls_smem_raw);
   const int b = blockIdx.x;
   const int nrows = va.K * va.J;
   for (int r = threadIdx.x >> 5; r < nrows; r += (int)(blockDim.x >> 5)) {
@@ -493,6 +483,7 @@ static int fill_noise(SweepArgs& A, const gls_noise_t* nz, uint32_t domain, int*
   if (rounds < 7 || rounds > 16) return GLS_ERR_INVALID_ARG;
   const int spec = nz->noise_spec ? (int)nz->noise_spec : 4;
   if (spec < 1 || spec > 4) return GLS_ERR_INVALID_ARG;
+  if (spec == 2 || spec == 3) return GLS_ERR_UNSUPPORTED;  // retired bit-splitting layouts
   if (nz->flags & ~GLS_NOISE_SHARED_ACROSS_K) return GLS_ERR_INVALID_ARG;
   uint32_t k0 = (uint32_t)(nz->seed & 0xffffffffu), k1 = (uint32_t)(nz->seed >> 32);
   for (int r = 0; r < 16; ++r) {
@@ -519,12 +510,12 @@ static int check_rows(const gls_rows_t* r) {
   return GLS_OK;
 }
 
-template <int DT, int SPEC, int ROUNDS>
+template <int DT, int ROUNDS>
 static cudaError_t launch_sweep_t(const SweepArgs& A, bool lse, int grid, cudaStream_t st) {
   if (lse)
-    sweep_kernel<DT, SPEC, true, ROUNDS><<<grid, kSweepThreads, 0, st>>>(A);
+    sweep_kernel<DT, true, ROUNDS><<<grid, kSweepThreads, 0, st>>>(A);
   else
-    sweep_kernel<DT, SPEC, false, ROUNDS><<<grid, kSweepThreads, 0, st>>>(A);
+    sweep_kernel<DT, false, ROUNDS><<<grid, kSweepThreads, 0, st>>>(A);
   return cudaGetLastError();
 }
 
@@ -532,16 +523,16 @@ static cudaError_t launch_sweep_t(const SweepArgs& A, bool lse, int grid, cudaSt
 // stream: their blocks may be scheduled while the sweep drains (the sweep signals that its
 // block is done), and wait at their first instruction until the whole sweep has completed and its
 // writes are visible.  This hides the launch latency between the two kernels of a call.
-static cudaLaunchAttribute g_dependent_attr[1];
-static cudaLaunchConfig_t dependent_launch(int grid, int block, size_t smem, cudaStream_t st) {
-  g_dependent_attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-  g_dependent_attr[0].val.programmaticStreamSerializationAllowed = 1;
+static cudaLaunchConfig_t dependent_launch(cudaLaunchAttribute* attr, int grid, int block,
+                                           size_t smem, cudaStream_t st) {
+  attr->id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr->val.programmaticStreamSerializationAllowed = 1;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3((unsigned)grid);
   cfg.blockDim = dim3((unsigned)block);
   cfg.dynamicSmemBytes = smem;
   cfg.stream = st;
-  cfg.attrs = g_dependent_attr;
+  cfg.attrs = attr;
   cfg.numAttrs = 1;
   return cfg;
 }
@@ -551,7 +542,8 @@ static cudaError_t launch_finalize_t(const SweepArgs& A, int rows, bool lse, Row
                                      int32_t* out_tokens, float* out_scores, uint32_t* status,
                                      cudaStream_t st) {
   const int wpb = 4;
-  cudaLaunchConfig_t cfg = dependent_launch((rows + wpb - 1) / wpb, wpb * 32, 0, st);
+  cudaLaunchAttribute attr;
+  cudaLaunchConfig_t cfg = dependent_launch(&attr, (rows + wpb - 1) / wpb, wpb * 32, 0, st);
   return cudaLaunchKernelEx(&cfg, finalize_rows_kernel<DT, SPEC, ROUNDS>, A, rows, lse ? 1 : 0, rowres,
                             out_tokens, out_scores, status);
 }
@@ -562,7 +554,8 @@ static cudaError_t launch_fused_verify_t(const SweepArgs& A, const VerifyArgs& v
   const size_t smem = (size_t)va.K * va.J * sizeof(RowResult);
   const int nrows = va.K * va.J;
   const int warps = nrows < kFusedVerifyMaxWarps ? nrows : kFusedVerifyMaxWarps;
-  cudaLaunchConfig_t cfg = dependent_launch(va.B, warps * 32, smem, st);
+  cudaLaunchAttribute attr;
+  cudaLaunchConfig_t cfg = dependent_launch(&attr, va.B, warps * 32, smem, st);
   return cudaLaunchKernelEx(&cfg, finalize_verify_kernel<DT, SPEC, ROUNDS>, A, va);
 }
 
@@ -592,7 +585,7 @@ static int run_rows(SweepArgs& A, int dtype, int spec, const Plan& P, void* work
     const int sh = s4_shape(dtype, A.V, A.multi_k > 0);
 #define SWEEP4(SH, R)                                                                       \
   do {                                                                                      \
-    const long long cap = (long long)kNumSMs * S4Cfg<SH>::kCtasPerSM;                       \
+    const long long cap = (long long)num_sms() * S4Cfg<SH>::kCtasPerSM;                       \
     const int grid = (int)(P.n_items < cap ? P.n_items : cap);                              \
     const size_t smem = sizeof(S4Shared<SH>);                                               \
     if (A.multi_k > 0)                                                                      \
@@ -607,41 +600,12 @@ static int run_rows(SweepArgs& A, int dtype, int spec, const Plan& P, void* work
     else { if (r10) SWEEP4(kS4ShapeF32Narrow, 10); else SWEEP4(kS4ShapeF32Narrow, 0); }
 #undef SWEEP4
     err = cudaGetLastError();
-  } else if (spec == 3) {
-    const long long cap = (long long)kNumSMs * (bf ? S3Cfg<kBF16>::kCtasPerSM : S3Cfg<kF32>::kCtasPerSM);
-    const int grid = (int)(P.n_items < cap ? P.n_items : cap);
-#define SWEEP3(DT, R)                                                                       \
-  do {                                                                                      \
-    const size_t smem = sizeof(S3Shared<DT>);                                               \
-    if (A.multi_k > 0) {                                                                    \
-      cudaFuncSetAttribute(sweep3_kernel<DT, true, R, true>,                                \
-                           cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);         \
-      sweep3_kernel<DT, true, R, true><<<grid, S3Cfg<DT>::kWarps * 32, smem, st>>>(A);           \
-    } else if (lse) {                                                                       \
-      cudaFuncSetAttribute(sweep3_kernel<DT, true, R>,                                      \
-                           cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);         \
-      sweep3_kernel<DT, true, R><<<grid, S3Cfg<DT>::kWarps * 32, smem, st>>>(A);                 \
-    } else {                                                                                \
-      cudaFuncSetAttribute(sweep3_kernel<DT, false, R>,                                     \
-                           cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);         \
-      sweep3_kernel<DT, false, R><<<grid, S3Cfg<DT>::kWarps * 32, smem, st>>>(A);                \
-    }                                                                                       \
-  } while (0)
-    if (bf) { if (r10) SWEEP3(kBF16, 10); else SWEEP3(kBF16, 0); }
-    else { if (r10) SWEEP3(kF32, 10); else SWEEP3(kF32, 0); }
-#undef SWEEP3
-    err = cudaGetLastError();
   } else {
     const long long want = (P.n_items + kSweepThreads / 32 - 1) / (kSweepThreads / 32);
-    const int grid = (int)(want < (long long)kNumSMs * 4 ? want : (long long)kNumSMs * 4);
+    const int grid = (int)(want < (long long)num_sms() * 4 ? want : (long long)num_sms() * 4);
 #define SWEEP_CALL(...) launch_sweep_t<__VA_ARGS__>(A, lse, grid, st)
-    if (bf) {
-      if (spec == 1) err = r10 ? SWEEP_CALL(kBF16, 1, 10) : SWEEP_CALL(kBF16, 1, 0);
-      else err = r10 ? SWEEP_CALL(kBF16, 2, 10) : SWEEP_CALL(kBF16, 2, 0);
-    } else {
-      if (spec == 1) err = r10 ? SWEEP_CALL(kF32, 1, 10) : SWEEP_CALL(kF32, 1, 0);
-      else err = r10 ? SWEEP_CALL(kF32, 2, 10) : SWEEP_CALL(kF32, 2, 0);
-    }
+    if (bf) err = r10 ? SWEEP_CALL(kBF16, 10) : SWEEP_CALL(kBF16, 0);
+    else err = r10 ? SWEEP_CALL(kF32, 10) : SWEEP_CALL(kF32, 0);
 #undef SWEEP_CALL
   }
   if (err != cudaSuccess) return GLS_ERR_CUDA;
@@ -654,13 +618,9 @@ static int run_rows(SweepArgs& A, int dtype, int spec, const Plan& P, void* work
                                          status, st))
   if (bf) {
     if (spec == 1) err = r10 ? FIN_CALL(kBF16, 1, 10) : FIN_CALL(kBF16, 1, 0);
-    else if (spec == 2) err = r10 ? FIN_CALL(kBF16, 2, 10) : FIN_CALL(kBF16, 2, 0);
-    else if (spec == 3) err = r10 ? FIN_CALL(kBF16, 3, 10) : FIN_CALL(kBF16, 3, 0);
     else err = r10 ? FIN_CALL(kBF16, 4, 10) : FIN_CALL(kBF16, 4, 0);
   } else {
     if (spec == 1) err = r10 ? FIN_CALL(kF32, 1, 10) : FIN_CALL(kF32, 1, 0);
-    else if (spec == 2) err = r10 ? FIN_CALL(kF32, 2, 10) : FIN_CALL(kF32, 2, 0);
-    else if (spec == 3) err = r10 ? FIN_CALL(kF32, 3, 10) : FIN_CALL(kF32, 3, 0);
     else err = r10 ? FIN_CALL(kF32, 4, 10) : FIN_CALL(kF32, 4, 0);
   }
 #undef FIN_CALL
@@ -700,14 +660,10 @@ const char* gls_status_string(int status) {
 size_t gls_workspace_bytes(int B, int K, int J, int64_t V) {
   if (!sizes_ok(B, K, J, V)) return 0;
   // the largest need over the noise layouts and element types (the call may use any of them)
-  size_t need = make_plan12((long long)B * K * J, V).total;
+  size_t need = make_plan1((long long)B * K * J, V).total;
   for (int dt = 0; dt < 2; ++dt) {
-    const size_t b = make_plan3((long long)B * K * J, V, dt).total;
-    const size_t c = make_plan3((long long)B * J, V, dt).total;  // fused multi-stream encoder
-    if (b > need) need = b;
-    if (c > need) need = c;
     const size_t d = make_plan4((long long)B * K * J, V, dt, false).total;
-    const size_t e = make_plan4((long long)B * J, V, dt, true).total;
+    const size_t e = make_plan4((long long)B * J, V, dt, true).total;  // fused multi-stream encoder
     if (d > need) need = d;
     if (e > need) need = e;
   }
@@ -838,8 +794,6 @@ int gls_draft_sample_sparse(const gls_sparse_rows_t* draft_rows, int B, int K, i
   sparse_draft_kernel<SPEC, R><<<grid, wpb * 32, 0, st>>>(A, S, rows, out_tokens, out_scores, device_status)
   const bool r10 = A.rounds == 10;
   if (spec == 1) { if (r10) SPARSE_DRAFT(1, 10); else SPARSE_DRAFT(1, 0); }
-  else if (spec == 2) { if (r10) SPARSE_DRAFT(2, 10); else SPARSE_DRAFT(2, 0); }
-  else if (spec == 3) { if (r10) SPARSE_DRAFT(3, 10); else SPARSE_DRAFT(3, 0); }
   else { if (r10) SPARSE_DRAFT(4, 10); else SPARSE_DRAFT(4, 0); }
 #undef SPARSE_DRAFT
   return cudaGetLastError() == cudaSuccess ? GLS_OK : GLS_ERR_CUDA;
@@ -891,8 +845,6 @@ int gls_target_sample_verify_sparse(const gls_sparse_rows_t* target_rows, int B,
 #define SPARSE_VERIFY(SPEC, R) sparse_verify_kernel<SPEC, R><<<B, warps * 32, smem, st>>>(A, S, va)
   const bool r10 = A.rounds == 10;
   if (spec == 1) { if (r10) SPARSE_VERIFY(1, 10); else SPARSE_VERIFY(1, 0); }
-  else if (spec == 2) { if (r10) SPARSE_VERIFY(2, 10); else SPARSE_VERIFY(2, 0); }
-  else if (spec == 3) { if (r10) SPARSE_VERIFY(3, 10); else SPARSE_VERIFY(3, 0); }
   else { if (r10) SPARSE_VERIFY(4, 10); else SPARSE_VERIFY(4, 0); }
 #undef SPARSE_VERIFY
   return cudaGetLastError() == cudaSuccess ? GLS_OK : GLS_ERR_CUDA;
@@ -933,7 +885,7 @@ int gls_compress_select(const gls_rows_t* enc_logw, const gls_rows_t* dec_logw, 
   // With the default noise layout, up to 8 streams and N < 2^28 it runs fused: each row is read
   // and summed once and the K streams share one bound; otherwise every stream sweeps the row on
   // its own and the epilogue takes the best of the K winners.
-  const bool fused_enc = spec >= 3 && K <= 8 && N < (1LL << 28);
+  const bool fused_enc = spec == 4 && K <= 8 && N < (1LL << 28);
   if (fused_enc) {
     const Plan PE = make_plan((long long)B, N, spec, enc_logw->dtype, true);
     if (workspace_bytes < PE.total) return GLS_ERR_WORKSPACE;
@@ -1047,7 +999,7 @@ static int topm_select(const gls_rows_t* rows, int B, int K, int J, int64_t V, i
   T.ids = (int32_t*)workspace;
   T.logits = (float*)((char*)workspace + align_up((size_t)T.rows * M * sizeof(int32_t), 256));
   const long long want = (T.rows + kTopmWarps - 1) / kTopmWarps;
-  const long long cap = (long long)kNumSMs * kTopmCtasPerSM;
+  const long long cap = (long long)num_sms() * kTopmCtasPerSM;
   const int grid = (int)(want < cap ? want : cap);
   if (rows->dtype == GLS_BF16)
     topm_select_kernel<kBF16><<<grid, kTopmWarps * 32, 0, st>>>(T);

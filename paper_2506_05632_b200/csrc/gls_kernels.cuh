@@ -1,18 +1,21 @@
-// gls_kernels.cuh -- device code of libgls: fused noise + score + argmax sweep for sm_100a.
+// gls_kernels.cuh -- device code shared by every kernel of libgls (Philox4x32, the exact fp64
+// noise and score, the top-2 tracker, the filter's margins) and the sweep for noise_spec 1, the
+// literal "one uniform per token" reading of Sec. 3 of arXiv 2506.05632.
 //
 // One pass over each row of logits computes, per (row, vocabulary slice):
 //   - the two best candidates of the Gumbel-max race  argmax_i (logit_i / T - ln S_i)
-//     (Sec. 3 step 2 / Algorithm 1 of arXiv 2506.05632, log domain), with S_i generated in
-//     registers from the counter-based generator described in include/gls.h;
+//     (Sec. 3 step 2 / Algorithm 1, log domain), with S_i generated in registers from the
+//     counter-based generator described in include/gls.h;
 //   - optionally the running (max, sum) of the row's softmax normaliser, needed where rows
 //     with different normalisers meet in the min over k (Algorithm 2, the Y_j line).
 //
 // The sweep never evaluates a logarithm for a token that cannot win.  With m a lower bound on
 // the row's final best score, token i can only matter if  S_i <= exp(logit_i/T - m), and
-// S_i = -log1p(-v_i) >= v_i >= (coarse bits of v_i).  So per group of 8 consecutive tokens one
-// test "min coarse bits < 2^(max logit * c - m')" decides, and only groups that pass look at
-// their tokens one by one (fp32 score from the full-precision uniform).  The filter has no false
-// negatives (margins below), so the result equals a full evaluation.
+// S_i = -log1p(-v_i) >= v_i.  So per group of 8 consecutive tokens one test
+// "min word < 2^(max logit * c - m')" decides, and only groups that pass look at their tokens one
+// by one (fp32 score from the full word).  The filter has no false negatives (margins below), so
+// the result equals a full evaluation.  (The default layout, noise_spec 4, has its own sweep in
+// gls_sweep4.cuh.)
 #pragma once
 #include <cuda_runtime.h>
 #include <math_constants.h>
@@ -85,11 +88,6 @@ __device__ __forceinline__ float ex2_approx(float x) {
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
 }
-__device__ __forceinline__ uint32_t min_u16x2(uint32_t a, uint32_t b) {
-  uint32_t d;
-  asm("min.u16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
-  return d;
-}
 __device__ __forceinline__ uint32_t max_bf16x2(uint32_t a, uint32_t b) {
   uint32_t d;
   asm("max.bf16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));  // a NaN operand is ignored
@@ -150,35 +148,23 @@ struct StreamKey {
   uint32_t seq;
 };
 
-// The uniform of token i under noise_spec SPEC, as the 48-bit (or 32-bit) integer numerator and
-// the scale 2^-bits: v = (num + 0.5) * 2^-bits.
-template <int SPEC, int ROUNDS>
+// The uniform of token i under noise_spec 1: v = (word + 0.5) * 2^-32.
+template <int ROUNDS>
 __device__ __forceinline__ double uniform_exact(const SweepArgs& A, const StreamKey& sk, int i) {
   uint32_t o[4];
-  if (SPEC == 1) {
-    philox4x32<ROUNDS>(A.rk, A.rounds, (uint32_t)i >> 2, sk.c1, sk.pos, sk.seq, o);
-    return ((double)o[i & 3] + 0.5) * 0x1p-32;
-  } else if (SPEC == 3) {
-    philox4x32<ROUNDS>(A.rk, A.rounds, (uint32_t)i >> 4, sk.c1, sk.pos, sk.seq, o);
-    const uint32_t h = (o[(i & 15) >> 2] >> (8 * (i & 3))) & 0xffu;
-    philox4x32<ROUNDS>(A.rk, A.rounds, (uint32_t)i >> 1, sk.c1 + (2u << 16), sk.pos, sk.seq, o);
-    const uint32_t lo = (i & 1) ? o[2] : o[0], hi = ((i & 1) ? o[3] : o[1]) & 0xffu;
-    return ((double)h * 1099511627776.0 + (double)hi * 4294967296.0 + (double)lo + 0.5) * 0x1p-48;
-  } else {
-    philox4x32<ROUNDS>(A.rk, A.rounds, (uint32_t)i >> 3, sk.c1, sk.pos, sk.seq, o);
-    const uint32_t h = (o[(i & 7) >> 1] >> (16 * (i & 1))) & 0xffffu;
-    philox4x32<ROUNDS>(A.rk, A.rounds, (uint32_t)i >> 2, sk.c1 + (2u << 16), sk.pos, sk.seq, o);
-    return ((double)h * 4294967296.0 + (double)o[i & 3] + 0.5) * 0x1p-48;
-  }
+  philox4x32<ROUNDS>(A.rk, A.rounds, (uint32_t)i >> 2, sk.c1, sk.pos, sk.seq, o);
+  const uint32_t t = (uint32_t)i & 3u;
+  const uint32_t w = t == 0 ? o[0] : t == 1 ? o[1] : t == 2 ? o[2] : o[3];
+  return ((double)w + 0.5) * 0x1p-32;
 }
 
-// The exponential S_i of token i in fp64.  noise_spec 1-3: S = -log1p(-v) (Sec. 3: S = -ln U,
+// The exponential S_i of token i in fp64.  noise_spec 1: S = -log1p(-v) (Sec. 3: S = -ln U,
 // U = 1 - v).  noise_spec 4: the group of 16 is built from its minimum M = -log1p(-v0) / 16,
 // v0 = (w * 2^16 + r + 0.5) * 2^-48: S = M at position loc of the group, M - log1p(-v_i) at the
 // others, v_i = (u_i + 0.5) * 2^-32 (an exact sampler of 16 i.i.d. Exp(1) values).
 template <int SPEC, int ROUNDS>
 __device__ __forceinline__ double noise_exact(const SweepArgs& A, const StreamKey& sk, int i) {
-  if (SPEC != 4) return -log1p(-uniform_exact<SPEC, ROUNDS>(A, sk, i));
+  if (SPEC != 4) return -log1p(-uniform_exact<ROUNDS>(A, sk, i));
   uint32_t o[4];
   const uint32_t g = (uint32_t)i >> 4;
   philox4x32<ROUNDS>(A.rk, A.rounds, ((g >> 7) << 5) | (g & 31u), sk.c1, sk.pos, sk.seq, o);
@@ -208,10 +194,17 @@ __device__ __noinline__ double exact_score(const SweepArgs& A, const void* row,
   return a - log(noise_exact<SPEC, ROUNDS>(A, sk, i));
 }
 
-// fp32 score from the full uniform; |error| is well below score_slack().
-__device__ __forceinline__ float score_f32(float a, float inv_t, float v, float* ln_s) {
-  const float s = -log1pf(-v);
-  const float l = logf(s);
+// Exp(1) from the uniform v = (word + frac) * 2^-32, frac in (0, 1) standing for further bits
+// and the half-step offset: -log1p(-v), through the complement 1 - v = (~word + 1 - frac) * 2^-32
+// when v > 1/2, so that the conversion of the word to fp32 can never round v up to 1.
+__device__ __forceinline__ float exp1_from_word(uint32_t word, float frac) {
+  if (word & 0x80000000u) return -logf(fmaf((float)(~word), 0x1p-32f, (1.0f - frac) * 0x1p-32f));
+  return -log1pf(-fmaf((float)word, 0x1p-32f, frac * 0x1p-32f));
+}
+
+// fp32 score from the exponential; |error| is well below score_slack().
+__device__ __forceinline__ float score_f32(float a, float inv_t, float s_noise, float* ln_s) {
+  const float l = logf(s_noise);
   *ln_s = l;
   return fmaf(a, inv_t, -l);
 }
@@ -274,41 +267,24 @@ __device__ __forceinline__ void top2_warp_merge(Top2& t) {
 // ------------------------------------------------------------------------------------------
 // Per-token examination of one lane's group of 8 tokens (rare path).
 //   a[8]   logits (excluded / out-of-range tokens hold -inf)
-//   w[]    coarse generator output of the group: SPEC 2: 4 words = 8 halfwords, SPEC 1: 8 words
+//   w[8]   the tokens' generator words
 // ------------------------------------------------------------------------------------------
-template <int SPEC, int ROUNDS>
-__device__ __noinline__ void examine_group(const SweepArgs& A, const StreamKey sk, int tok0,
-                                           const float (&a)[8], const uint32_t* w, float inv_t,
-                                           float c2, float m, const uint8_t* bins, int msg,
-                                           Top2& best) {
+template <int ROUNDS>
+__device__ __noinline__ void examine_group(int tok0, const float (&a)[8], const uint32_t* w,
+                                           float inv_t, float c2, float m, const uint8_t* bins,
+                                           int msg, Top2& best) {
   float nm = filter_offset(m);
-  uint32_t fine[4];
-  int fine_block = -1;
 #pragma unroll 1
   for (int t = 0; t < 8; ++t) {
     const float at = a[t];
     if (!(at < CUDART_INF_F)) continue;  // NaN and +inf never win
     const float thr = ex2_approx(fmaf(at, c2, nm));
-    float v;
-    if (SPEC == 1) {
-      const uint32_t wt = w[t];
-      if (!(__uint2float_rd(wt) < thr * 4294967296.0f)) continue;
-      v = ((float)wt + 0.5f) * 0x1p-32f;
-    } else {
-      const uint32_t h = (w[t >> 1] >> (16 * (t & 1))) & 0xffffu;
-      if (!((float)h < thr * 65536.0f)) continue;
-      const int blk = (tok0 + t) >> 2;
-      if (blk != fine_block) {
-        philox4x32<ROUNDS>(A.rk, A.rounds, (uint32_t)blk, sk.c1 + (2u << 16), sk.pos, sk.seq, fine);
-        fine_block = blk;
-      }
-      const uint32_t r = fine[(tok0 + t) & 3];
-      v = fmaf((float)h, 0x1p-16f, fmaf((float)r, 0x1p-48f, 0x1p-49f));
-    }
+    const uint32_t wt = w[t];
+    if (!(__uint2float_rd(wt) < thr * 4294967296.0f)) continue;
     const int i = tok0 + t;
     if (bins != nullptr && (int)__ldg(bins + i) != msg) continue;
     float ln_s;
-    const float s = score_f32(at, inv_t, v, &ln_s);
+    const float s = score_f32(at, inv_t, exp1_from_word(wt, 0.5f), &ln_s);
     top2_offer(best, s, i);
     const float lower = s - score_slack(s, ln_s);
     if (lower > m) {
@@ -441,7 +417,7 @@ __device__ __forceinline__ void lse_group(const float (&a)[8], float amax, float
 
 constexpr float kLseFloor = -3.0e38f;  // finite stand-in for "no finite logit seen yet"
 
-template <int DT, int SPEC, bool LSE, int ROUNDS>
+template <int DT, bool LSE, int ROUNDS>
 __global__ void __launch_bounds__(kSweepThreads, 4)
 sweep_kernel(const __grid_constant__ SweepArgs A) {
   const int lane = threadIdx.x & 31;
@@ -486,27 +462,20 @@ sweep_kernel(const __grid_constant__ SweepArgs A) {
       if (!full) cur = load_group_scalar<DT>(rowp, tok, tok_end);
       if (it + 1 < n_full) nxt = load_group_vec<DT>(rowp, tok + kWarpTokens);
 
-      // coarse noise of the group and its smallest value
-      uint32_t w[SPEC == 1 ? 8 : 4];
-      float vlow;  // lower bound on min_t v_t, scaled by 2^16 (SPEC 2) or 2^32 (SPEC 1)
-      if (SPEC == 1) {
+      // the group's eight generator words and the smallest of them
+      uint32_t w[8];
+      {
         uint32_t o[4];
         philox4x32<ROUNDS>(A.rk, A.rounds, (uint32_t)tok >> 2, sk.c1, sk.pos, sk.seq, o);
         w[0] = o[0]; w[1] = o[1]; w[2] = o[2]; w[3] = o[3];
         philox4x32<ROUNDS>(A.rk, A.rounds, ((uint32_t)tok >> 2) + 1u, sk.c1, sk.pos, sk.seq, o);
         w[4] = o[0]; w[5] = o[1]; w[6] = o[2]; w[7] = o[3];
-        const uint32_t wm = min(min(min(w[0], w[1]), min(w[2], w[3])),
-                                min(min(w[4], w[5]), min(w[6], w[7])));
-        vlow = __uint2float_rd(wm);
-      } else {
-        uint32_t o[4];
-        philox4x32<ROUNDS>(A.rk, A.rounds, (uint32_t)tok >> 3, sk.c1, sk.pos, sk.seq, o);
-        w[0] = o[0]; w[1] = o[1]; w[2] = o[2]; w[3] = o[3];
-        const uint32_t mm = min_u16x2(min_u16x2(w[0], w[1]), min_u16x2(w[2], w[3]));
-        vlow = (float)min(mm & 0xffffu, mm >> 16);
       }
+      const uint32_t wm = min(min(min(w[0], w[1]), min(w[2], w[3])),
+                              min(min(w[4], w[5]), min(w[6], w[7])));
+      const float vlow = __uint2float_rd(wm);  // lower bound on 2^32 min_t v_t
       const float amax = group_max<DT>(cur);
-      const float thr = ex2_approx(fmaf(amax, c2, nm)) * (SPEC == 1 ? 4294967296.0f : 65536.0f);
+      const float thr = ex2_approx(fmaf(amax, c2, nm)) * 4294967296.0f;
       const bool pass = vlow < thr;
 
       if (LSE) {
@@ -519,7 +488,7 @@ sweep_kernel(const __grid_constant__ SweepArgs A) {
         if (pass) {
           float a[8];
           unpack_group<DT>(cur, a);
-          examine_group<SPEC, ROUNDS>(A, sk, tok, a, w, inv_t, c2, m, bins, msg, best);
+          examine_group<ROUNDS>(tok, a, w, inv_t, c2, m, bins, msg, best);
         }
         // share the improved bound with the warp and with the other slices of the row
         float mb = lane_bound(best);

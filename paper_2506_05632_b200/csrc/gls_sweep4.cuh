@@ -29,7 +29,7 @@
 // loop so that the hot loop contains no call.  A fused variant (MULTI) races one row under
 // several noise streams at once for the compression encoder of Sec. 5.1.
 #pragma once
-#include "gls_sweep3.cuh"
+#include "gls_group16.cuh"
 
 namespace gls {
 
@@ -92,15 +92,7 @@ struct S4Shared {
 };
 template <int SH>
 __device__ __forceinline__ S4Shared<SH>& s4_shared() {
-  return *reinterpret_cast<S4Shared<SH>*>(s3_smem_raw);
-}
-
-// Exp(1) from the uniform v = (word + frac) * 2^-32, frac in (0, 1) standing for further bits
-// and the half-step offset: -log1p(-v), through the complement 1 - v = (~word + 1 - frac) * 2^-32
-// when v > 1/2, so that the conversion of the word to fp32 can never round v up to 1.
-__device__ __forceinline__ float exp1_from_word(uint32_t word, float frac) {
-  if (word & 0x80000000u) return -logf(fmaf((float)(~word), 0x1p-32f, (1.0f - frac) * 0x1p-32f));
-  return -log1pf(-fmaf((float)word, 0x1p-32f, frac * 0x1p-32f));
+  return *reinterpret_cast<S4Shared<SH>*>(gls_smem_raw);
 }
 
 // lower bound on word * 2^-32 from its top 23 bits, without an integer-to-float conversion
@@ -220,7 +212,7 @@ template <int SH>
 __device__ __noinline__ void lse4_redo_careful(const char* rowp, int tok0, int n_steps, int tok_end,
                                                float c2, float* lm_out, float* ls_out) {
   constexpr int DT = S4Cfg<SH>::kDT;
-  float lm = kS3LseFloor, ls = 0.f;
+  float lm = kGroupLseFloor, ls = 0.f;
   for (int s = 0; s < n_steps; ++s) {
     for (int j = 0; j < kS4LaneGroups; ++j) {
       const int tok = tok0 + s * S4Cfg<SH>::kCtaTokens + j * 512;
@@ -306,7 +298,7 @@ sweep4_kernel(const __grid_constant__ SweepArgs A) {
 
     // bound published by earlier slices of the row (the hint words are cleared only when rows are cut)
     uint32_t m_enc = A.splits > 1 ? __ldcg(A.hints + row) : 0u;
-    float lm = kS3LseFloor;
+    float lm = kGroupLseFloor;
     unsigned long long ls2 = 0ull;
     int qn = 0;
 

@@ -34,8 +34,31 @@ def check_scores(gpu, ref, mask, what):
         what, bad.sum(), np.abs(gpu - ref)[bad].max(), tol[bad].min())
 
 
-def check_draft(gpu_tokens, gpu_scores, ref, what="draft"):
-    """gpu_* numpy arrays [B,K,J]; ref = oracle.draft_sample(...) dict.  Returns mismatch count."""
+class Tally:
+    """Counts over several comparisons of one workload: decisions, near-ties among them (oracle's
+    top-2 gap below the threshold) and mismatches; `check()` applies the rule to the totals."""
+
+    def __init__(self, what):
+        self.what, self.decisions, self.near_ties, self.mismatches = what, 0, 0, 0
+
+    def add(self, decisions, near_ties, mismatches):
+        self.decisions += int(decisions)
+        self.near_ties += int(near_ties)
+        self.mismatches += int(mismatches)
+
+    def check(self):
+        assert self.mismatches <= self.near_ties, self.as_dict()
+        assert self.mismatches <= _budget(self.decisions), "%s: %d mismatches of %d decisions" % (
+            self.what, self.mismatches, self.decisions)
+
+    def as_dict(self):
+        return dict(what=self.what, decisions=self.decisions, near_ties=self.near_ties,
+                    mismatches=self.mismatches)
+
+
+def check_draft(gpu_tokens, gpu_scores, ref, what="draft", tally=None):
+    """gpu_* numpy arrays [B,K,J]; ref = oracle.draft_sample(...) dict.  Returns mismatch count.
+    With `tally` the mismatch budget is left to the tally's totals."""
     gt = np.asarray(gpu_tokens)
     rt = ref["tokens"]
     assert gt.shape == rt.shape
@@ -43,14 +66,18 @@ def check_draft(gpu_tokens, gpu_scores, ref, what="draft"):
     near = _near_tie(ref["gaps"], ref["scores"])
     assert not (mism & ~near).any(), "%s: %d token mismatches outside near-ties, first at %s" % (
         what, (mism & ~near).sum(), np.argwhere(mism & ~near)[:5].tolist())
-    assert mism.sum() <= _budget(mism.size), "%s: %d mismatches of %d" % (what, mism.sum(), mism.size)
+    if tally is None:
+        assert mism.sum() <= _budget(mism.size), "%s: %d mismatches of %d" % (what, mism.sum(), mism.size)
+    else:
+        tally.add(mism.size, (near & (rt >= 0)).sum(), mism.sum())
     if gpu_scores is not None:
         check_scores(gpu_scores, ref["scores"], ~mism & (rt >= 0), what)
     return int(mism.sum())
 
 
-def check_verify(gpu, ref, what="verify"):
-    """gpu: dict of numpy arrays (tokens [B,J], tau [B], accept [B,K,L], scores); ref: oracle dict."""
+def check_verify(gpu, ref, what="verify", tally=None):
+    """gpu: dict of numpy arrays (tokens [B,J], tau [B], accept [B,K,L], scores); ref: oracle dict.
+    Decisions are the positions the oracle emitted; a sequence that differs counts once."""
     rt, rtau = ref["tokens"], ref["tau"]
     B, J = rt.shape
     near = _near_tie(ref["gaps"], ref["scores"]) & (rt >= 0)
@@ -70,14 +97,17 @@ def check_verify(gpu, ref, what="verify"):
         # everything before the near-tie position must still agree
         assert np.array_equal(gpu["tokens"][b, :f], rt[b, :f]), (what, b)
         assert np.array_equal(gpu["accept"][b][:, :f], ref["accept"][b][:, :f]), (what, b)
-    assert n_mism <= _budget(B * J), "%s: %d of %d sequences differ" % (what, n_mism, B)
+    if tally is None:
+        assert n_mism <= _budget(B * J), "%s: %d of %d sequences differ" % (what, n_mism, B)
+    else:
+        tally.add(emitted.sum(), (near & emitted).sum(), n_mism)
     if gpu.get("scores") is not None:
         agree = (gpu["tokens"] == rt) & emitted & (rt >= 0)
         check_scores(gpu["scores"], ref["scores"], agree, what)
     return n_mism
 
 
-def check_compress(gpu, ref, what="compress"):
+def check_compress(gpu, ref, what="compress", tally=None):
     B = len(ref["enc_index"])
     near = _near_tie(ref["gaps"], ref["scores"])
     n_mism = 0
@@ -94,8 +124,11 @@ def check_compress(gpu, ref, what="compress"):
             assert gpu["message"][b] == ref["message"][b]
             d = gpu["dec_index"][b] != ref["dec_index"][b]
             assert not (d & ~near[b, 1:]).any(), "%s: decoder index of sample %d" % (what, b)
-    assert n_mism <= _budget(B * (1 + ref["dec_index"].shape[1])), \
-        "%s: %d of %d samples differ" % (what, n_mism, B)
+    if tally is None:
+        assert n_mism <= _budget(B * (1 + ref["dec_index"].shape[1])), \
+            "%s: %d of %d samples differ" % (what, n_mism, B)
+    else:
+        tally.add(near.size, (near & np.isfinite(ref["scores"])).sum(), n_mism)
     if gpu.get("scores") is not None:
         agree = np.concatenate([(gpu["enc_index"] == ref["enc_index"])[:, None],
                                 gpu["dec_index"] == ref["dec_index"]], axis=1)

@@ -24,7 +24,7 @@ def _draft_both(gls, oracle, logits, **kw):
 
 
 @pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
-@pytest.mark.parametrize("spec", [1, 2, 3, 4])
+@pytest.mark.parametrize("spec", [1, 4])
 def test_draft_shapes(gls, oracle, dtype, spec):
     """Ragged vocabularies around every tile boundary: one lane group (8 or 16 tokens), one warp
     iteration (256 or 512), one CTA iteration (2048 or 4096), one slice and several slices."""
@@ -109,7 +109,7 @@ def test_masked_nan_inf_and_empty_rows(gls, oracle):
 
 
 @pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
-@pytest.mark.parametrize("spec", [1, 2, 3, 4])
+@pytest.mark.parametrize("spec", [1, 4])
 def test_verify_small(gls, oracle, dtype, spec):
     """Algorithm 2 end to end on reduced copies of the verify workloads, several shapes."""
     for cfg, B, K, L, V in ((2, 16, 4, 4, 3000), (3, 8, 8, 5, 5001), (4, 6, 8, 8, 2500),
@@ -194,7 +194,7 @@ def test_config1_statistics_on_gpu(gls, oracle):
     assert acc >= theory.lml_bound(p, q, K) - 4 * np.sqrt(acc * (1 - acc) / n)
 
 
-@pytest.mark.parametrize("spec", [1, 2, 3, 4])
+@pytest.mark.parametrize("spec", [1, 4])
 def test_compress_small(gls, oracle, spec):
     for B, K, N, lmax in ((12, 1, 50, 1), (10, 4, 3000, 4), (6, 3, 70001, 16), (5, 2, 257, 2)):
         w = synth.compress_workload("cuda", B=B, K=K, N=N, D=4, l_max=lmax, seed=40 + N)
@@ -258,7 +258,7 @@ def test_flat_and_peaked_rows(gls, oracle, dtype):
 
 
 @pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
-@pytest.mark.parametrize("spec", [3, 4])
+@pytest.mark.parametrize("spec", [1, 4])
 def test_orderings_that_defeat_the_filter(gls, oracle, dtype, spec):
     """Rows on which the running bound never settles: steeply ascending logits make every later
     group of tokens a candidate (the per-warp candidate queue fills at its maximum rate and the
@@ -279,6 +279,29 @@ def test_orderings_that_defeat_the_filter(gls, oracle, dtype, spec):
         parity.check_verify(parity.to_np(out), refv, "orderings verify %s T=1/%g" % (dtype, it))
         # same logits on both sides: every draft is accepted at every position
         assert (parity.to_np(out)["tau"] == 6).all()
+
+
+def test_spec1_word_next_to_two_pow_32(gls, oracle):
+    """noise_spec 1, a uniform within 128 * 2^-32 of one: S = -ln(1 - v) is about 19 and must be
+    formed from the complement of the generator word (an fp32 v would round to exactly 1 and the
+    token would drop out of the race).  The two tokens below carry such words under the test seed
+    (found by a search over the oracle's noise); each is made the row's peak so that it wins."""
+    seed = 0x5EED250605632001
+    for tok_star in (1889245, 2165634):
+        V = tok_star + 1000
+        S = oracle.exp_noise_row(seed, seq=10, pos=0, k=0, V=V, spec=1)
+        assert S[tok_star] > -np.log(128 * 2.0**-32) and S.argmax() == tok_star
+        for dtype in (torch.float32, torch.bfloat16):
+            x = torch.zeros(1, 1, 1, V, device="cuda", dtype=dtype)
+            x[..., tok_star] = 40.0
+            kw = dict(seed=seed, seq_base=10, spec=1)
+            tok, sc, ref = _draft_both(gls, oracle, x, **kw)
+            assert ref["tokens"].item() == tok_star
+            parity.check_draft(tok, sc, ref, "spec 1 complement %s" % dtype)
+            out = gls.target_sample_verify(x, torch.from_numpy(ref["tokens"]).cuda(),
+                                           flags=gls.NO_BONUS, **kw)
+            refv = oracle.target_sample_verify(synth.to_numpy_rows(x), ref["tokens"], flags=2, **kw)
+            parity.check_verify(parity.to_np(out), refv, "spec 1 complement verify %s" % dtype)
 
 
 def test_fp32_rows_around_the_launch_shape_switch(gls, oracle):
@@ -325,6 +348,9 @@ def test_host_detectable_errors(gls):
         gls.draft_sample(x, inv_temp=float("nan"))
     with pytest.raises(gls.GlsError):
         gls.draft_sample(x, spec=5)
+    for retired in (2, 3):  # the bit-splitting layouts are no longer implemented
+        with pytest.raises(gls.GlsError):
+            gls.draft_sample(x, spec=retired)
     with pytest.raises(gls.GlsError):
         gls.draft_sample(x, rounds=3)
     with pytest.raises(gls.GlsError):

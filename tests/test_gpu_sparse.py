@@ -26,7 +26,7 @@ def _topk_case(B, K, J, V, M, seed, pad=0, shuffle=True):
     return ids.contiguous(), vals.contiguous(), masked
 
 
-@pytest.mark.parametrize("spec", [1, 2, 3, 4])
+@pytest.mark.parametrize("spec", [1, 4])
 def test_sparse_draft_matches_oracle_on_masked_dense_rows(gls, oracle, spec):
     for n, (B, K, J, V, M, pad) in enumerate([(3, 2, 2, 5000, 50, 0), (2, 3, 1, 152064, 50, 14),
                                               (4, 1, 2, 300, 7, 1), (2, 2, 1, 40, 40, 0)]):

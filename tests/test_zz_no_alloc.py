@@ -70,3 +70,22 @@ def test_problem_beyond_the_static_limit_is_refused(gls):
         gls.draft_sample_static(one, tok, None, seed=SEED)
     torch.cuda.synchronize()
     assert int(tok.item()) == -5  # nothing was enqueued
+
+
+def test_static_calls_leave_device_memory_as_it_is(gls):
+    """The point of the entry point: once the first call on the device has resolved the built-in
+    buffer's address, further calls obtain no device memory from the driver (free memory as the
+    driver reports it is unchanged) nor from torch's allocator."""
+    logits = _logits(4, 2, 2, 20000, torch.bfloat16, 5)
+    tok = torch.empty((4, 2, 2), dtype=torch.int32, device="cuda")
+    sc = torch.empty((4, 2, 2), dtype=torch.float32, device="cuda")
+    gls.draft_sample_static(logits, tok, sc, seed=SEED)  # first use on this device
+    torch.cuda.synchronize()
+    free0, _ = torch.cuda.mem_get_info()
+    held0, reserved0 = torch.cuda.memory_allocated(), torch.cuda.memory_reserved()
+    for i in range(5):
+        gls.draft_sample_static(logits, tok, sc, seed=SEED + i)
+    torch.cuda.synchronize()
+    free1, _ = torch.cuda.mem_get_info()
+    assert free1 == free0
+    assert torch.cuda.memory_allocated() == held0 and torch.cuda.memory_reserved() == reserved0
