@@ -175,3 +175,44 @@ def test_l0_is_plain_target_sampling(oracle):
     o = oracle.target_sample_verify(tl, np.zeros((n, 2, 0), np.int32), seed=SEED)
     assert (o["tau"] == 1).all()
     assert _chi2_p(np.bincount(o["tokens"][:, 0], minlength=V), Mb[START]) > 1e-3
+
+
+def test_appendix_b_acceptance_with_j_of_k_active(oracle):
+    """Appendix B, last part: with J of K drafts active, the strongly invariant variant accepts
+    with probability at least sum_j J / sum_i [max(q_i/q_j, p_i/p_j) + (K-1) q_i/q_j], while the
+    printed algorithm (min over the active set) has the bound with K replaced by J.  Context-free
+    toy: the same p and q at both positions, so position 1 given |S| = J after position 0 is one
+    draw of that setting.  Checked two-sided against the exact probabilities (quadrature) and
+    one-sided against the bounds; target rows are given per draft (equal in content)."""
+    from tests import theory
+
+    p = np.array([0.1, 0.2, 0.3, 0.4])
+    q = np.array([0.35, 0.3, 0.2, 0.15])
+    K, L, n = 3, 2, 150_000
+    d = np.ascontiguousarray(np.broadcast_to(np.log(p).astype(np.float32), (n, K, L, V)))
+    t = np.ascontiguousarray(np.broadcast_to(np.log(q).astype(np.float32), (n, K, L, V)))
+    X = oracle.draft_sample(d, seed=SEED + 7)["tokens"]
+    for flags, label in ((NO_BONUS | COMBINE_ALL, "all"), (NO_BONUS, "active")):
+        o = oracle.target_sample_verify(t, X, flags=flags, seed=SEED + 7)
+        acc = o["accept"].astype(bool)
+        n_active = acc[:, :, 0].sum(axis=1)
+        hit = acc[:, :, 1].any(axis=1)
+        for J in (1, 2, 3):
+            sel = n_active == J
+            m = int(sel.sum())
+            assert m > 2000
+            rate = hit[sel].mean()
+            if label == "all":
+                exact = theory.exact_acceptance_active(p, q, K, J)
+                bound = theory.lml_bound_active(p, q, K, J)
+            else:
+                exact = theory.exact_acceptance(p, q, J)
+                bound = theory.lml_bound(p, q, J)
+            sd = np.sqrt(exact * (1 - exact) / m)
+            assert abs(rate - exact) < 4 * sd, (label, J, rate, exact)
+            assert exact >= bound - 1e-9
+        # with every draft active the two variants coincide
+    assert abs(theory.exact_acceptance_active(p, q, K, K) - theory.exact_acceptance(p, q, K)) < 1e-7
+    # fewer active drafts of the same K: the strongly invariant variant accepts less often than
+    # the printed algorithm would with those J drafts alone
+    assert theory.exact_acceptance_active(p, q, K, 1) < theory.exact_acceptance(p, q, 1)

@@ -88,3 +88,47 @@ def exact_acceptance(p, q, K):
         val, _ = integrate.quad(outer, 0.0, np.inf, epsabs=1e-10, epsrel=1e-9)
         total += K * q[j] * val
     return total
+
+
+def lml_bound_active(p, q, K, J):
+    """Appendix B: with J of the K coupled drafts still active, the probability that the target
+    token (min over ALL K streams) matches an active draft is at least
+    sum_j J / sum_i [max(q_i/q_j, p_i/p_j) + (K-1) q_i/q_j]."""
+    return lml_bound(p, q, K) * J / K
+
+
+def exact_acceptance_active(p, q, K, J):
+    """Exact Pr[Y in {X^(1..J)}] when Y is the target race over all K streams and only J of the
+    K proposals count (Appendix B's setting), by the same conditioning as exact_acceptance():
+    given the winning pair (token j, value t), the winning stream is one of the J active ones
+    with probability J/K -- then the match fails only if that stream misses j (1 - e^{-t D_j})
+    and so do the other J-1 active ones -- or one of the K-J inactive ones, where all J active
+    streams must miss:
+      Pr = sum_j q_j int_0^inf e^{-K t} [ J (1 - (1 - e^{-t D_j}) (1 - a_j)^{J-1})
+                                          + (K - J) (1 - (1 - a_j)^J) ] dt."""
+    p = np.asarray(p, float)
+    q = np.asarray(q, float)
+    n = len(p)
+    total = 0.0
+    for j in range(n):
+        c = p * q[j] / p[j] - q
+        d = p / p[j]
+        Dj = np.sum(np.maximum(0.0, c))
+        others = [i for i in range(n) if i != j]
+
+        def a_j(t):
+            def inner(r):
+                return np.exp(-r - sum(max(0.0, t * c[i] + r * d[i]) for i in others))
+
+            val, _ = integrate.quad(inner, 0.0, np.inf, epsabs=1e-11, epsrel=1e-10)
+            return val
+
+        def outer(t):
+            a = a_j(t)
+            win_active = 1.0 - (1.0 - np.exp(-t * Dj)) * (1.0 - a) ** (J - 1)
+            win_inactive = 1.0 - (1.0 - a) ** J
+            return np.exp(-K * t) * (J * win_active + (K - J) * win_inactive)
+
+        val, _ = integrate.quad(outer, 0.0, np.inf, epsabs=1e-10, epsrel=1e-9)
+        total += q[j] * val
+    return total
