@@ -203,9 +203,12 @@ int gls_draft_sample_static(const gls_rows_t* draft_logits, int B, int K, int J,
  * If all L positions leave S non-empty, the bonus token Y_L is drawn the same way from the rows at
  * position L and tau = L + 1 (with GLS_NO_BONUS: no such rows, tau = L).
  * GLS_COMBINE_ALL is Appendix B: Y_j = argmin_i min over ALL k of S_i^(j,k) / q_i with q the target
- * distribution of the accepted prefix, while S still records the survivors.  It is implemented for
- * target rows shared by all k (stride_k = 0, where each stream's race over the shared row is that
- * quantity); per-draft target rows return GLS_ERR_UNSUPPORTED.
+ * distribution of the accepted prefix, while S still records the survivors.  With target rows
+ * shared by all k (stride_k = 0) each stream's race over the shared row is that quantity.  With a
+ * row per draft, q is the row of the lowest-numbered active draft (active drafts share the
+ * accepted prefix): every row is raced under all K streams at once and the epilogue reads that
+ * row; this needs the default noise layout, K <= 8 and V < 2^28 (GLS_ERR_UNSUPPORTED otherwise)
+ * and costs K times the noise arithmetic of a plain call.
  * Algorithm 1 is the case L = 1 with GLS_NO_BONUS: accept iff some accept[b,k,0] is 1.
  *
  *   target_logits   [B,K,J,V] rows, J = L + 1 (J = L with GLS_NO_BONUS)

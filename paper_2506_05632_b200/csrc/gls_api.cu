@@ -189,7 +189,7 @@ __device__ __forceinline__ RowResult finalize_row(const SweepArgs& A, int row, i
     // code is "lowest token, then lowest stream", the tie rule.
     tok = code;
     if (A.multi_k > 0) {
-      sk.c1 += (uint32_t)code & 7u;
+      sk.c1 = (A.domain << 16) + ((uint32_t)code & 7u);
       tok = (int)((uint32_t)code >> 3);
     }
     ex = exact_score<DT, SPEC, ROUNDS>(A, rowp, sk, tok, inv_t);
@@ -236,7 +236,7 @@ finalize_rows_kernel(const __grid_constant__ SweepArgs A, int rows, int with_lse
 // ------------------------------------------------------------------------------------------
 // `rows` points at the K x J results of sequence b: rows[k * J + j].
 __device__ void verify_sequence(const RowResult* rows, int b, int K, int L, int J, uint32_t flags,
-                                const int32_t* __restrict__ draft_tokens,
+                                bool multi_rows, const int32_t* __restrict__ draft_tokens,
                                 int32_t* __restrict__ out_tokens, int32_t* __restrict__ out_num,
                                 uint8_t* __restrict__ accept, float* __restrict__ out_scores,
                                 uint32_t* __restrict__ dev_status) {
@@ -252,8 +252,11 @@ __device__ void verify_sequence(const RowResult* rows, int b, int K, int L, int 
     // subtracting each row's log-sum-exp; ties: lowest token, then lowest k
     double bs = 0.0;
     int bi = -1;
+    // Appendix B on rows raced under all K streams at once: the target distribution of the
+    // accepted prefix is the row of any draft that is still active; take the lowest such k
+    const int kref = multi_rows ? __ffsll((long long)active) - 1 : -1;
     for (int k = 0; k < K; ++k) {
-      if (!((active >> k) & 1ull) && !(flags & GLS_COMBINE_ALL)) continue;
+      if (multi_rows ? (k != kref) : (!((active >> k) & 1ull) && !(flags & GLS_COMBINE_ALL))) continue;
       const RowResult r = rows[(long long)k * J + j];
       if (r.idx < 0) continue;
       const double sc = r.score - r.lse;
@@ -281,7 +284,7 @@ __device__ void verify_sequence(const RowResult* rows, int b, int K, int L, int 
 }
 
 __global__ void verify_epilogue_kernel(const RowResult* __restrict__ rows, int B, int K, int L,
-                                       int J, uint32_t flags,
+                                       int J, uint32_t flags, bool multi_rows,
                                        const int32_t* __restrict__ draft_tokens,
                                        int32_t* __restrict__ out_tokens,
                                        int32_t* __restrict__ out_num, uint8_t* __restrict__ accept,
@@ -289,8 +292,8 @@ __global__ void verify_epilogue_kernel(const RowResult* __restrict__ rows, int B
                                        uint32_t* __restrict__ dev_status) {
   const int b = blockIdx.x * blockDim.x + threadIdx.x;
   if (b >= B) return;
-  verify_sequence(rows + (long long)b * K * J, b, K, L, J, flags, draft_tokens, out_tokens, out_num,
-                  accept, out_scores, dev_status);
+  verify_sequence(rows + (long long)b * K * J, b, K, L, J, flags, multi_rows, draft_tokens, out_tokens,
+                  out_num, accept, out_scores, dev_status);
 }
 
 // Split-V reduction and Algorithm 2's loop in one launch: a CTA per sequence finalises the
@@ -298,6 +301,7 @@ __global__ void verify_epilogue_kernel(const RowResult* __restrict__ rows, int B
 struct VerifyArgs {
   int B, K, L, J;
   uint32_t flags;
+  bool multi_rows;  // every row result is the best over all K noise streams (Appendix B)
   const int32_t* draft_tokens;
   int32_t* out_tokens;
   int32_t* out_num;
@@ -320,8 +324,8 @@ finalize_verify_kernel(const __grid_constant__ SweepArgs A, const VerifyArgs va)
   }
   __syncthreads();
   if (threadIdx.x == 0)
-    verify_sequence(srows, b, va.K, va.L, va.J, va.flags, va.draft_tokens, va.out_tokens, va.out_num,
-                    va.accept, va.out_scores, va.dev_status);
+    verify_sequence(srows, b, va.K, va.L, va.J, va.flags, va.multi_rows, va.draft_tokens, va.out_tokens,
+                    va.out_num, va.accept, va.out_scores, va.dev_status);
 }
 
 // Sec. 5.1 encoder bookkeeping: Y = best over the K streams of the encoder row, M = l_Y.
@@ -402,16 +406,22 @@ __device__ __forceinline__ RowResult sparse_row(const SweepArgs& A, const Sparse
   sk.seq = A.seq_ids ? A.seq_ids[b] : A.seq_base + (uint32_t)b;
   double best = -CUDART_INF, amax = -CUDART_INF;
   int bid = -1;
+  // multi_k > 0: the list is raced under the streams 0 .. multi_k-1 together (Appendix B); a
+  // token that ties with itself under two streams is one token, so only the score matters
+  const int n_streams = A.multi_k > 0 ? A.multi_k : 1;
   for (int m = lane; m < S.M; m += 32) {
     const int id = __ldg(S.ids + base + m);
     const float a = __ldg(S.logits + base + m);
     if (!sparse_keep(id, a)) continue;
     const double al = (double)a * inv_t;
     amax = fmax(amax, al);
-    const double sc = al - log(noise_exact<SPEC, ROUNDS>(A, sk, id));
-    if (bid < 0 || sc > best || (sc == best && id < bid)) {
-      best = sc;
-      bid = id;
+    for (int ks = 0; ks < n_streams; ++ks) {
+      if (A.multi_k > 0) sk.c1 = ((uint32_t)ks & A.kmask) | (A.domain << 16);
+      const double sc = al - log(noise_exact<SPEC, ROUNDS>(A, sk, id));
+      if (bid < 0 || sc > best || (sc == best && id < bid)) {
+        best = sc;
+        bid = id;
+      }
     }
   }
 #pragma unroll
@@ -469,8 +479,8 @@ sparse_verify_kernel(const __grid_constant__ SweepArgs A, const SparseArgs S, co
   }
   __syncthreads();
   if (threadIdx.x == 0)
-    verify_sequence(srows, b, va.K, va.L, va.J, va.flags, va.draft_tokens, va.out_tokens, va.out_num,
-                    va.accept, va.out_scores, va.dev_status);
+    verify_sequence(srows, b, va.K, va.L, va.J, va.flags, va.multi_rows, va.draft_tokens, va.out_tokens,
+                    va.out_num, va.accept, va.out_scores, va.dev_status);
 }
 
 // ------------------------------------------------------------------------------------------
@@ -664,8 +674,10 @@ size_t gls_workspace_bytes(int B, int K, int J, int64_t V) {
   for (int dt = 0; dt < 2; ++dt) {
     const size_t d = make_plan4((long long)B * K * J, V, dt, false).total;
     const size_t e = make_plan4((long long)B * J, V, dt, true).total;  // fused multi-stream encoder
+    const size_t f = make_plan4((long long)B * K * J, V, dt, true).total;  // Appendix B, row per draft
     if (d > need) need = d;
     if (e > need) need = e;
+    if (f > need) need = f;
   }
   return need;
 }
@@ -713,18 +725,21 @@ int gls_target_sample_verify(const gls_rows_t* target_logits, int B, int K, int 
   if (!finite_pos(inv_temp)) return GLS_ERR_INVALID_ARG;
   int rc = check_rows(target_logits);
   if (rc != GLS_OK) return rc;
-  // Appendix B couples every stream to the accepted prefix's distribution.  When all k share one
-  // target row per position (stride_k = 0) the rows' own winners already are that race.
-  if ((flags & GLS_COMBINE_ALL) && target_logits->stride_k != 0 && K > 1)
-    return GLS_ERR_UNSUPPORTED;
   SweepArgs A;
   std::memset(&A, 0, sizeof(A));
   for (int k = 0; k < K; ++k) A.inv_t[k] = inv_temp;
   int spec;
   rc = fill_noise(A, noise, 0u, &spec);
   if (rc != GLS_OK) return rc;
-  const Plan P = make_plan((long long)B * K * J, V, spec, target_logits->dtype);
+  // Appendix B couples every stream to the accepted prefix's distribution.  When all k share one
+  // target row per position (stride_k = 0) the rows' own winners already are that race.  With a
+  // row per draft, every row is raced under all K streams at once (the fused multi-stream race)
+  // and the epilogue reads the row of the lowest active draft.
+  const bool multi = (flags & GLS_COMBINE_ALL) && target_logits->stride_k != 0 && K > 1;
+  if (multi && (spec != 4 || K > 8 || V >= (1LL << 28))) return GLS_ERR_UNSUPPORTED;
+  const Plan P = make_plan((long long)B * K * J, V, spec, target_logits->dtype, multi);
   if (!workspace || workspace_bytes < P.total) return GLS_ERR_WORKSPACE;
+  if (multi) A.multi_k = K;
   A.data = target_logits->data;
   A.sb = target_logits->stride_b;
   A.sk = target_logits->stride_k;
@@ -736,6 +751,7 @@ int gls_target_sample_verify(const gls_rows_t* target_logits, int B, int K, int 
   VerifyArgs va;
   va.B = B; va.K = K; va.L = L; va.J = J;
   va.flags = flags;
+  va.multi_rows = multi;
   va.draft_tokens = draft_tokens;
   va.out_tokens = out_tokens;
   va.out_num = out_num_tokens;
@@ -748,7 +764,7 @@ int gls_target_sample_verify(const gls_rows_t* target_logits, int B, int K, int 
   if (rc != GLS_OK) return rc;
   if (fused) return GLS_OK;
   const RowResult* rowres = (const RowResult*)((char*)workspace + P.off_rows);
-  verify_epilogue_kernel<<<(B + 127) / 128, 128, 0, st>>>(rowres, B, K, L, J, flags, draft_tokens,
+  verify_epilogue_kernel<<<(B + 127) / 128, 128, 0, st>>>(rowres, B, K, L, J, flags, multi, draft_tokens,
                                                          out_tokens, out_num_tokens, out_accept,
                                                          out_scores, device_status);
   return cudaGetLastError() == cudaSuccess ? GLS_OK : GLS_ERR_CUDA;
@@ -812,7 +828,8 @@ int gls_target_sample_verify_sparse(const gls_sparse_rows_t* target_rows, int B,
   if (!finite_pos(inv_temp)) return GLS_ERR_INVALID_ARG;
   int rc = check_sparse(target_rows);
   if (rc != GLS_OK) return rc;
-  if ((flags & GLS_COMBINE_ALL) && target_rows->stride_k != 0 && K > 1) return GLS_ERR_UNSUPPORTED;
+  // Appendix B with a list per draft: every list is raced under all K streams (see sparse_row)
+  const bool multi = (flags & GLS_COMBINE_ALL) && target_rows->stride_k != 0 && K > 1;
   const size_t smem = (size_t)K * J * sizeof(RowResult);
   if (smem > kFusedVerifyMaxSmem) return GLS_ERR_UNSUPPORTED;
   SweepArgs A;
@@ -823,6 +840,7 @@ int gls_target_sample_verify_sparse(const gls_sparse_rows_t* target_rows, int B,
   if (rc != GLS_OK) return rc;
   A.K = K;
   A.J = J;
+  if (multi) A.multi_k = K;
   SparseArgs S;
   S.ids = target_rows->token_ids;
   S.logits = target_rows->logits;
@@ -833,6 +851,7 @@ int gls_target_sample_verify_sparse(const gls_sparse_rows_t* target_rows, int B,
   VerifyArgs va;
   va.B = B; va.K = K; va.L = L; va.J = J;
   va.flags = flags;
+  va.multi_rows = multi;
   va.draft_tokens = draft_tokens;
   va.out_tokens = out_tokens;
   va.out_num = out_num_tokens;

@@ -268,7 +268,8 @@ sweep4_kernel(const __grid_constant__ SweepArgs A) {
       const int k = bk % A.K;
       const int b = bk / A.K;
       rowp = (const char*)A.data + (b * A.sb + k * A.sk + j * A.sj) * ES;
-      c1 = ((uint32_t)k & A.kmask) | (A.domain << 16);
+      // the fused multi-stream race enumerates the streams itself, whatever the row's k
+      c1 = (MULTI ? 0u : ((uint32_t)k & A.kmask)) | (A.domain << 16);
       pos = A.pos_base + (uint32_t)j;
       seq = A.seq_ids ? __ldg(A.seq_ids + b) : A.seq_base + (uint32_t)b;
       const float inv_t = A.inv_t[k];

@@ -45,7 +45,8 @@ def test_random_shapes(gls, oracle, seed):
             decisions += refd["tokens"].size
         else:
             dtok = torch.zeros(B, K, 0, dtype=torch.int32, device="cuda")
-        flags = gls.COMBINE_ALL if (shared and rng.random() < 0.5) else 0
+        # Appendix B: on shared rows under either layout; on a row per draft under the default one
+        flags = gls.COMBINE_ALL if ((shared or spec == 4) and rng.random() < 0.4) else 0
         out = gls.target_sample_verify(t, dtok, flags=flags, **kw)
         refv = oracle.target_sample_verify(synth.to_numpy_rows(t.contiguous()), dtok.cpu().numpy(),
                                            flags=flags, **kw)

@@ -149,8 +149,11 @@ def test_verify_shared_target_row_and_combine_all(gls, oracle):
         ref = oracle.target_sample_verify(t.contiguous().cpu().numpy(), tok.cpu().numpy(),
                                           flags=flags, seed=SEED)
         parity.check_verify(parity.to_np(out), ref, "flags=%d" % flags)
-    with pytest.raises(gls.GlsError):  # per-draft rows with COMBINE_ALL are not implemented
-        gls.target_sample_verify(t.contiguous(), tok, flags=gls.COMBINE_ALL, seed=SEED)
+    # the same rows given per draft (contiguous copy): Appendix B runs as a multi-stream race per row
+    out = gls.target_sample_verify(t.contiguous(), tok, flags=gls.COMBINE_ALL, seed=SEED)
+    parity.check_verify(parity.to_np(out), ref, "Appendix B, row per draft")
+    with pytest.raises(gls.GlsError):  # ... which is built for the default noise layout only
+        gls.target_sample_verify(t.contiguous(), tok, flags=gls.COMBINE_ALL, seed=SEED, spec=1)
 
 
 def test_identical_rows_accept_everything(gls):
@@ -279,6 +282,46 @@ def test_orderings_that_defeat_the_filter(gls, oracle, dtype, spec):
         parity.check_verify(parity.to_np(out), refv, "orderings verify %s T=1/%g" % (dtype, it))
         # same logits on both sides: every draft is accepted at every position
         assert (parity.to_np(out)["tau"] == 6).all()
+
+
+@pytest.mark.parametrize("cfg", [2, 3, 4])
+def test_appendix_b_on_a_row_per_draft(gls, oracle, cfg):
+    """GLS_COMBINE_ALL (Appendix B: min over all K streams) with a target row per draft: every row
+    is raced under all K streams and the epilogue reads the row of the lowest active draft.
+    Reduced copies of the verify configurations, dense, as sparse lists and through the top-M
+    front end."""
+    B, K, L, V = {2: (6, 4, 4, 32000), 3: (4, 8, 3, 20000 + 77), 4: (3, 8, 4, 2048 * 11 + 5)}[cfg]
+    w = synth.verify_workload(cfg, "cuda", B=B, K=K, L=L, V=V)
+    kw = dict(seed=w.noise_seed, inv_temp=w.inv_temp, seq_base=5, pos_base=2)
+    tok, sc, ref = _draft_both(gls, oracle, w.draft_logits, **kw)
+    dt = torch.from_numpy(ref["tokens"]).cuda()
+    t_h = synth.to_numpy_rows(w.target_logits)
+    for flags in (gls.COMBINE_ALL, gls.COMBINE_ALL | gls.NO_BONUS):
+        t = w.target_logits if not (flags & gls.NO_BONUS) else w.target_logits[:, :, :L]
+        th = t_h if not (flags & gls.NO_BONUS) else np.ascontiguousarray(t_h[:, :, :L])
+        out = gls.target_sample_verify(t, dt, flags=flags, **kw)
+        refv = oracle.target_sample_verify(th, ref["tokens"], flags=flags, **kw)
+        parity.check_verify(parity.to_np(out), refv, "cfg%d Appendix B flags %d" % (cfg, flags))
+    # the strongly invariant output does not depend on the draft tokens beyond the stopping time:
+    # other draft tokens, same noise -> the emitted tokens agree on the common length
+    other = torch.roll(dt, 1, dims=1)
+    o1 = parity.to_np(gls.target_sample_verify(w.target_logits[:, :1].expand(B, K, L + 1, V), dt,
+                                               flags=gls.COMBINE_ALL, **kw))
+    o2 = parity.to_np(gls.target_sample_verify(w.target_logits[:, :1].expand(B, K, L + 1, V), other,
+                                               flags=gls.COMBINE_ALL, **kw))
+    common = np.minimum(o1["tau"], o2["tau"])
+    for b in range(B):
+        assert np.array_equal(o1["tokens"][b, :common[b]], o2["tokens"][b, :common[b]])
+    # sparse lists with a list per draft, and the top-M front end (M = 50, Appendix D.1)
+    M = 50
+    masked, kept = oracle.top_m_rows(w.target_logits.float().cpu().numpy(), M)
+    refs = oracle.target_sample_verify(masked, ref["tokens"], flags=gls.COMBINE_ALL, **kw)
+    outm = gls.target_sample_verify_topm(w.target_logits, dt, M, flags=gls.COMBINE_ALL, **kw)
+    parity.check_verify(parity.to_np(outm), refs, "cfg%d Appendix B top-M" % cfg)
+    ids = torch.tensor(np.stack(kept).reshape(B, K, L + 1, M), dtype=torch.int32, device="cuda")
+    lg = torch.gather(w.target_logits.float(), 3, ids.long())
+    outs = gls.target_sample_verify_sparse(ids, lg, dt, flags=gls.COMBINE_ALL, **kw)
+    parity.check_verify(parity.to_np(outs), refs, "cfg%d Appendix B sparse" % cfg)
 
 
 def test_spec1_word_next_to_two_pow_32(gls, oracle):
