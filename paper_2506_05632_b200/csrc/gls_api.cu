@@ -283,6 +283,72 @@ __device__ void verify_sequence(const RowResult* rows, int b, int K, int L, int 
   out_num[b] = n_out;
 }
 
+// The same loop run by one warp: lane l looks after drafts l and l + 32, so the list combine is a
+// warp argmax, the pruning a ballot, and the outputs are written in parallel; only the walk over
+// the positions is sequential.  `dtok` holds the sequence's draft tokens [K][L] (shared memory).
+// Result identical to verify_sequence().
+__device__ void verify_sequence_warp(const RowResult* rows, int b, int K, int L, int J, uint32_t flags,
+                                     bool multi_rows, const int32_t* dtok,
+                                     int32_t* __restrict__ out_tokens, int32_t* __restrict__ out_num,
+                                     uint8_t* __restrict__ accept, float* __restrict__ out_scores,
+                                     uint32_t* __restrict__ dev_status) {
+  const int lane = threadIdx.x & 31;
+  unsigned long long active = K >= 64 ? ~0ull : ((1ull << K) - 1ull);
+  int n_out = 0;
+  for (int j = 0; j < J; ++j) {
+    const int kref = multi_rows ? __ffsll((long long)active) - 1 : -1;
+    double bs = -CUDART_INF;
+    int bi = -1;
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+      const int k = lane + 32 * h;
+      if (k >= K) continue;
+      if (multi_rows ? (k != kref) : (!((active >> k) & 1ull) && !(flags & GLS_COMBINE_ALL))) continue;
+      const RowResult r = rows[(long long)k * J + j];
+      if (r.idx < 0) continue;
+      const double sc = r.score - r.lse;
+      if (bi < 0 || sc > bs || (sc == bs && r.idx < bi)) {
+        bs = sc;
+        bi = r.idx;
+      }
+    }
+#pragma unroll
+    for (int d = 16; d > 0; d >>= 1) {
+      const double os = __shfl_xor_sync(0xffffffffu, bs, d);
+      const int oi = __shfl_xor_sync(0xffffffffu, bi, d);
+      if (oi >= 0 && (bi < 0 || os > bs || (os == bs && oi < bi))) {
+        bs = os;
+        bi = oi;
+      }
+    }
+    if (lane == 0) {
+      out_tokens[(long long)b * J + j] = bi;
+      if (out_scores) out_scores[(long long)b * J + j] = bi >= 0 ? (float)bs : CUDART_NAN_F;
+      if (bi < 0 && dev_status) atomicOr(dev_status, GLS_DEV_EMPTY_SUPPORT);
+    }
+    n_out = j + 1;
+    if (j == L) break;  // bonus token
+    unsigned long long next = 0ull;
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+      const int k = lane + 32 * h;
+      const bool ok = k < K && ((active >> k) & 1ull) && bi >= 0 && dtok[k * L + j] == bi;
+      if (k < K) accept[((long long)b * K + k) * L + j] = ok ? 1 : 0;
+      next |= (unsigned long long)__ballot_sync(0xffffffffu, ok) << (32 * h);
+    }
+    active = next;
+    if (active == 0ull) break;
+  }
+  // what lies beyond the stopping time: token -1, score 0, not accepted
+  for (int j = n_out + lane; j < J; j += 32) {
+    out_tokens[(long long)b * J + j] = -1;
+    if (out_scores) out_scores[(long long)b * J + j] = 0.f;
+  }
+  for (int t = lane; t < K * L; t += 32)
+    if (t % L >= n_out) accept[(long long)b * K * L + t] = 0;
+  if (lane == 0) out_num[b] = n_out;
+}
+
 __global__ void verify_epilogue_kernel(const RowResult* __restrict__ rows, int B, int K, int L,
                                        int J, uint32_t flags, bool multi_rows,
                                        const int32_t* __restrict__ draft_tokens,
@@ -311,21 +377,30 @@ struct VerifyArgs {
 };
 constexpr int kFusedVerifyMaxWarps = 32;  // one warp per row result, up to a full CTA
 constexpr size_t kFusedVerifyMaxSmem = 48 * 1024;
+// a sequence's K x J row results and its K x L draft tokens
+static size_t fused_verify_smem(int K, int L, int J) {
+  return (size_t)K * J * sizeof(RowResult) + (size_t)K * (L > 0 ? L : 1) * sizeof(int32_t);
+}
 template <int DT, int SPEC, int ROUNDS>
 __global__ void __launch_bounds__(kFusedVerifyMaxWarps * 32)
 finalize_verify_kernel(const __grid_constant__ SweepArgs A, const VerifyArgs va) {
-  asm volatile("griddepcontrol.wait;" ::: "memory");  // the sweep before this launch is complete
   RowResult* srows = reinterpret_cast<RowResult*>(gls_smem_raw);
   const int b = blockIdx.x;
   const int nrows = va.K * va.J;
+  // the sequence's draft tokens, fetched while the sweep is still draining (they were written
+  // by work that completed before the sweep started)
+  int32_t* dtok = reinterpret_cast<int32_t*>(srows + nrows);
+  for (int t = threadIdx.x; t < va.K * va.L; t += (int)blockDim.x)
+    dtok[t] = va.draft_tokens[(long long)b * va.K * va.L + t];
+  asm volatile("griddepcontrol.wait;" ::: "memory");  // the sweep before this launch is complete
   for (int r = threadIdx.x >> 5; r < nrows; r += (int)(blockDim.x >> 5)) {
     const RowResult rr = finalize_row<DT, SPEC, ROUNDS>(A, b * nrows + r, 1, nullptr);
     if ((threadIdx.x & 31) == 0) srows[r] = rr;
   }
   __syncthreads();
-  if (threadIdx.x == 0)
-    verify_sequence(srows, b, va.K, va.L, va.J, va.flags, va.multi_rows, va.draft_tokens, va.out_tokens,
-                    va.out_num, va.accept, va.out_scores, va.dev_status);
+  if (threadIdx.x < 32)
+    verify_sequence_warp(srows, b, va.K, va.L, va.J, va.flags, va.multi_rows, dtok, va.out_tokens,
+                         va.out_num, va.accept, va.out_scores, va.dev_status);
 }
 
 // Sec. 5.1 encoder bookkeeping: Y = best over the K streams of the encoder row, M = l_Y.
@@ -477,10 +552,13 @@ sparse_verify_kernel(const __grid_constant__ SweepArgs A, const SparseArgs S, co
     const RowResult rr = sparse_row<SPEC, ROUNDS>(A, S, b * nrows + r, nullptr);
     if ((threadIdx.x & 31) == 0) srows[r] = rr;
   }
+  int32_t* dtok = reinterpret_cast<int32_t*>(srows + nrows);
+  for (int t = threadIdx.x; t < va.K * va.L; t += (int)blockDim.x)
+    dtok[t] = va.draft_tokens[(long long)b * va.K * va.L + t];
   __syncthreads();
-  if (threadIdx.x == 0)
-    verify_sequence(srows, b, va.K, va.L, va.J, va.flags, va.multi_rows, va.draft_tokens, va.out_tokens,
-                    va.out_num, va.accept, va.out_scores, va.dev_status);
+  if (threadIdx.x < 32)
+    verify_sequence_warp(srows, b, va.K, va.L, va.J, va.flags, va.multi_rows, dtok, va.out_tokens,
+                         va.out_num, va.accept, va.out_scores, va.dev_status);
 }
 
 // ------------------------------------------------------------------------------------------
@@ -561,7 +639,7 @@ static cudaError_t launch_finalize_t(const SweepArgs& A, int rows, bool lse, Row
 // sweep + split reduction of one batch of rows
 template <int DT, int SPEC, int ROUNDS>
 static cudaError_t launch_fused_verify_t(const SweepArgs& A, const VerifyArgs& va, cudaStream_t st) {
-  const size_t smem = (size_t)va.K * va.J * sizeof(RowResult);
+  const size_t smem = fused_verify_smem(va.K, va.L, va.J);
   const int nrows = va.K * va.J;
   const int warps = nrows < kFusedVerifyMaxWarps ? nrows : kFusedVerifyMaxWarps;
   cudaLaunchAttribute attr;
@@ -619,8 +697,7 @@ static int run_rows(SweepArgs& A, int dtype, int spec, const Plan& P, void* work
 #undef SWEEP_CALL
   }
   if (err != cudaSuccess) return GLS_ERR_CUDA;
-  const bool fuse = va != nullptr &&
-                    (size_t)va->K * va->J * sizeof(RowResult) <= kFusedVerifyMaxSmem;
+  const bool fuse = va != nullptr && fused_verify_smem(va->K, va->L, va->J) <= kFusedVerifyMaxSmem;
   if (fused) *fused = fuse;
 #define FIN_CALL(...)                                                                          \
   (fuse ? launch_fused_verify_t<__VA_ARGS__>(A, *va, st)                                       \
@@ -830,7 +907,7 @@ int gls_target_sample_verify_sparse(const gls_sparse_rows_t* target_rows, int B,
   if (rc != GLS_OK) return rc;
   // Appendix B with a list per draft: every list is raced under all K streams (see sparse_row)
   const bool multi = (flags & GLS_COMBINE_ALL) && target_rows->stride_k != 0 && K > 1;
-  const size_t smem = (size_t)K * J * sizeof(RowResult);
+  const size_t smem = fused_verify_smem(K, L, J);
   if (smem > kFusedVerifyMaxSmem) return GLS_ERR_UNSUPPORTED;
   SweepArgs A;
   std::memset(&A, 0, sizeof(A));
