@@ -232,6 +232,13 @@ def run_ours(args):
                                                     workspace=topm_ws, status=buf.status, **kw)
             _mark(marks)
             return
+        if args.fused:
+            _mark(marks)
+            pkg.draft_verify(w.draft_logits, w.target_logits, out_draft_tokens=buf.draft_tokens,
+                             out_draft_scores=buf.draft_scores, out=buf.out, workspace=buf.workspace,
+                             status=buf.status, **kw)
+            _mark(marks)
+            return
         pkg.draft_sample(w.draft_logits, out_tokens=buf.draft_tokens, out_scores=buf.draft_scores,
                          workspace=buf.workspace, status=buf.status, **kw)
         _mark(marks)
@@ -273,7 +280,8 @@ def run_ours(args):
         # small batches are bound by the host issuing the launches: the same step as a replayed
         # CUDA graph (L2 flushed between replays, each replay in its own event pair)
         gs = pipeline.GraphedStep(w.draft_logits, w.target_logits, buf, inv_temp=w.inv_temp,
-                                  seed=w.noise_seed, seq_base=seq_base, spec=args.spec)
+                                  seed=w.noise_seed, seq_base=seq_base, spec=args.spec,
+                                  fused=args.fused)
         for _ in range(3):
             gs.replay()
         gm = []
@@ -456,6 +464,7 @@ def main():
     ap.add_argument("--spec", type=int, default=4, choices=[1, 2, 3, 4], help="noise_spec")
     ap.add_argument("--topm", type=int, default=0,
                     help="extra workload: truncate every row to its top-M logits first (Sec. 4.4)")
+    ap.add_argument("--fused", action="store_true", help="one gls_draft_verify call per step")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle baseline leg")
     args = ap.parse_args()

@@ -226,6 +226,34 @@ int gls_target_sample_verify(const gls_rows_t* target_logits, int B, int K, int 
                              size_t workspace_bytes, uint32_t* device_status, void* stream);
 
 /*
+ * Draft phase and verification in one call -- Algorithm 2 from its draft loop to its end, for the
+ * case where both sets of logits are resident (all L draft positions are known, e.g. a drafter
+ * that is not autoregressive in the tokens sampled here, a replayed or re-scored step, or the
+ * last position of an autoregressive loop together with its verification).  Equivalent to
+ * gls_draft_sample(draft_logits, J = L) followed by gls_target_sample_verify(target_logits, the
+ * tokens just drawn), bit for bit, but one sweep launch covers both sets of rows and one
+ * reduction launch finalises the draft rows, the target rows and Algorithm 2's loop, which halves
+ * the number of launches of a step (what bounds small batches).
+ *
+ *   draft_logits       [B,K,L,V] rows, temperature inv_temp_draft (or per draft, host array [K])
+ *   target_logits      [B,K,J,V] rows, J = L + 1 (J = L with GLS_NO_BONUS), temperature
+ *                      inv_temp_target; same dtype as draft_logits
+ *   out_draft_tokens   [B,K,L] int32, out_draft_scores NULL or [B,K,L] fp32 (as gls_draft_sample)
+ *   out_tokens, out_num_tokens, out_accept, out_scores: as gls_target_sample_verify
+ *   workspace          at least gls_draft_verify_workspace_bytes(B, K, L, J, V) bytes
+ * L >= 1.  Default noise layout only; GLS_COMBINE_ALL only with target rows shared by all k; K, L
+ * such that K * (32 J + 4 L) bytes fit in 48 KB (GLS_ERR_UNSUPPORTED otherwise: use the two calls).
+ */
+size_t gls_draft_verify_workspace_bytes(int B, int K, int L, int J, int64_t V);
+int gls_draft_verify(const gls_rows_t* draft_logits, const gls_rows_t* target_logits, int B, int K,
+                     int L, int64_t V, float inv_temp_draft, const float* inv_temp_per_draft_host,
+                     float inv_temp_target, const gls_noise_t* noise, uint32_t flags,
+                     int32_t* out_draft_tokens, float* out_draft_scores, int32_t* out_tokens,
+                     int32_t* out_num_tokens, uint8_t* out_accept, float* out_scores,
+                     void* workspace, size_t workspace_bytes, uint32_t* device_status,
+                     void* stream);
+
+/*
  * Sparse rows -- Sec. 4.4 (top-K truncation: only M << N high-probability tokens are kept) and
  * Appendix D.1 (the experiments keep the top 50 tokens).  A row is a
  * list of M kept tokens: their ids in the full vocabulary and their logits; every other token has

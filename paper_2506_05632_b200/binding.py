@@ -104,6 +104,13 @@ def load():
             C.POINTER(_Rows), C.c_int, C.c_int, C.c_int, C.c_int64, C.c_float, C.c_void_p,
             C.POINTER(_Noise), C.c_uint32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
             C.c_void_p, C.c_size_t, C.c_void_p, C.c_void_p]
+        L.gls_draft_verify_workspace_bytes.restype = C.c_size_t
+        L.gls_draft_verify_workspace_bytes.argtypes = [C.c_int, C.c_int, C.c_int, C.c_int, C.c_int64]
+        L.gls_draft_verify.restype = C.c_int
+        L.gls_draft_verify.argtypes = [
+            C.POINTER(_Rows), C.POINTER(_Rows), C.c_int, C.c_int, C.c_int, C.c_int64, C.c_float,
+            C.c_void_p, C.c_float, C.POINTER(_Noise), C.c_uint32, C.c_void_p, C.c_void_p, C.c_void_p,
+            C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p, C.c_void_p]
         L.gls_topm_workspace_bytes.restype = C.c_size_t
         L.gls_topm_workspace_bytes.argtypes = [C.c_int, C.c_int, C.c_int, C.c_int]
         L.gls_draft_sample_topm.restype = C.c_int
@@ -390,6 +397,48 @@ def target_sample_verify(logits, draft_tokens, inv_temp=1.0, flags=0, seed=0, se
         _ptr(out["accept"]) if Ld > 0 else None, _ptr(out.get("scores")), workspace.data_ptr(),
         workspace.numel(), _ptr(status), _stream()))
     return out
+
+
+def draft_verify_workspace_bytes(B, K, L, J, V):
+    return int(load().gls_draft_verify_workspace_bytes(int(B), int(K), int(L), int(J), int(V)))
+
+
+def draft_verify(draft_logits, target_logits, inv_temp=1.0, inv_temp_per_draft=None,
+                 inv_temp_target=None, flags=0, seed=0, seq_base=0, seq_ids=None, pos_base=0,
+                 spec=4, rounds=10, noise_flags=0, want_scores=True, workspace=None, status=None,
+                 out_draft_tokens=None, out_draft_scores=None, out=None):
+    """gls_draft_verify: draft_logits [B,K,L,V] and target_logits [B,K,J,V] (J = L+1, or L with
+    NO_BONUS) in one call.  Returns (draft tokens [B,K,L], draft scores | None, dict(tokens, tau,
+    accept, scores | None)) -- what draft_sample followed by target_sample_verify return."""
+    L_ = load()
+    B, K, L, V = draft_logits.shape
+    J = target_logits.shape[2]
+    assert tuple(target_logits.shape) == (B, K, J, V) and J == (L if (flags & NO_BONUS) else L + 1)
+    dev = draft_logits.device
+    drows, trows = _rows(draft_logits, 3), _rows(target_logits, 3)
+    nz = _noise(seed, seq_base, seq_ids, pos_base, spec, rounds, noise_flags)
+    if out_draft_tokens is None:
+        out_draft_tokens = torch.empty((B, K, L), dtype=torch.int32, device=dev)
+    if out_draft_scores is None and want_scores:
+        out_draft_scores = torch.empty((B, K, L), dtype=torch.float32, device=dev)
+    if out is None:
+        out = dict(tokens=torch.empty((B, J), dtype=torch.int32, device=dev),
+                   tau=torch.empty((B,), dtype=torch.int32, device=dev),
+                   accept=torch.empty((B, K, L), dtype=torch.uint8, device=dev),
+                   scores=torch.empty((B, J), dtype=torch.float32, device=dev)
+                   if want_scores else None)
+    workspace = _workspace(workspace, draft_verify_workspace_bytes(B, K, L, J, V), dev)
+    itk = None
+    if inv_temp_per_draft is not None:
+        itk = (C.c_float * K)(*[float(x) for x in inv_temp_per_draft])
+    _check(L_.gls_draft_verify(
+        C.byref(drows), C.byref(trows), B, K, L, V, float(inv_temp),
+        C.cast(itk, C.c_void_p) if itk is not None else None,
+        float(inv_temp if inv_temp_target is None else inv_temp_target), C.byref(nz), int(flags),
+        _ptr(out_draft_tokens), _ptr(out_draft_scores), _ptr(out["tokens"]), _ptr(out["tau"]),
+        _ptr(out["accept"]), _ptr(out.get("scores")), workspace.data_ptr(), workspace.numel(),
+        _ptr(status), _stream()))
+    return out_draft_tokens, out_draft_scores, out
 
 
 def compress_select(enc_logw, dec_logw=None, bins=None, K=None, seed=0, seq_base=0, seq_ids=None,

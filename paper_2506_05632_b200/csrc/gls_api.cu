@@ -44,6 +44,9 @@ constexpr int kMaxChunk = 16384;
 
 struct Plan {
   int chunk, splits, parts;
+  int chunk1, splits1, chunk2, splits2;  // two sets of rows swept by one launch each
+  bool two_launches;
+  int per_slice;  // partial results per slice (warps per CTA)
   long long rows, n_items;
   size_t off_hints, off_partials, off_rows, total;
 };
@@ -62,7 +65,7 @@ static void plan_layout(Plan& p) {
 // so that the static round-robin over warps balances, but keep slices long enough to amortise
 // the per-item reduction.
 static Plan make_plan1(long long rows, long long V) {
-  Plan p;
+  Plan p = Plan();
   const long long target_items = 8LL * num_sms() * 32;
   long long chunk = (rows * V + target_items - 1) / target_items;
   chunk = (chunk + kWarpTokens - 1) / kWarpTokens * kWarpTokens;
@@ -89,7 +92,7 @@ static Plan make_plan1(long long rows, long long V) {
 #endif
 template <int SH>
 static Plan make_plan4_t(long long rows, long long V) {
-  Plan p;
+  Plan p = Plan();
   constexpr int kCtaTok = S4Cfg<SH>::kCtaTokens;
   constexpr int kMinChunk = GLS_S4_MIN_STEPS * kCtaTok;
   const long long grid = (long long)num_sms() * S4Cfg<SH>::kCtasPerSM;
@@ -123,6 +126,31 @@ static Plan make_plan4(long long rows, long long V, int dtype, bool multi) {
                                  : make_plan4_t<kS4ShapeF32Narrow>(rows, V);
 }
 
+// The fused draft + verify call (noise_spec 4): one launch over both sets while the input is small
+// (the launches are what a small step costs), else one launch per set, each sliced for its own
+// number of rows (the kernel specialised for its set is faster where the sweep is what a step costs).
+static Plan make_plan_step(long long rows1, long long rows2, long long V, int dtype) {
+  Plan p = make_plan4(rows1 + rows2, V, dtype, false);
+  p.two_launches = (double)(rows1 + rows2) * (double)V * (dtype == GLS_BF16 ? 2.0 : 4.0) > 128e6;
+  p.chunk1 = p.chunk2 = p.chunk;
+  p.splits1 = p.splits2 = p.splits;
+  if (p.two_launches) {
+    const Plan a = make_plan4(rows1, V, dtype, false), b = make_plan4(rows2, V, dtype, false);
+    p.per_slice = p.parts / p.splits;  // warps per CTA
+    p.chunk1 = a.chunk;
+    p.splits1 = a.splits;
+    p.chunk2 = b.chunk;
+    p.splits2 = b.splits;
+    // first set: slots = its own slicing; the slot stride serves both sets
+    p.splits = a.splits;
+    p.chunk = a.chunk;
+    p.parts = (a.splits > b.splits ? a.splits : b.splits) * p.per_slice;
+    plan_layout(p);
+    p.n_items = 0;
+  }
+  return p;
+}
+
 static Plan make_plan(long long rows, long long V, int spec, int dtype, bool multi = false) {
   return spec == 4 ? make_plan4(rows, V, dtype, multi) : make_plan1(rows, V);
 }
@@ -138,17 +166,17 @@ __device__ __forceinline__ RowResult finalize_row(const SweepArgs& A, int row, i
                                                   uint32_t* __restrict__ dev_status) {
   const int lane = threadIdx.x & 31;
   constexpr int ES = DT == kBF16 ? 2 : 4;
-  const int j = row % A.J;
-  const int bk = row / A.J;
-  const int k = bk % A.K;
-  const int b = bk / A.K;
-  const float inv_t = A.inv_t[k];
+  const RowLoc rl = locate_row<ES>(A, row);
+  const int j = rl.j, k = rl.k, b = rl.b;
+  const float inv_t = rl.inv_t;
   const float c2 = inv_t * kLog2e;
 
+  const int used = rl.second ? A.parts2 : A.parts1;
+  const int n_parts = used > 0 ? used : A.parts;  // slots in use
   Top2 best;
   top2_init(best);
   float lm = kLseFloor;
-  for (int s = lane; s < A.parts; s += 32) {
+  for (int s = lane; s < n_parts; s += 32) {
     const Partial p = A.partials[(long long)row * A.parts + s];
     top2_offer(best, p.s1, p.i1);
     top2_offer(best, p.s2, p.i2);
@@ -159,7 +187,7 @@ __device__ __forceinline__ RowResult finalize_row(const SweepArgs& A, int row, i
   for (int d = 16; d > 0; d >>= 1) lm = fmaxf(lm, __shfl_xor_sync(0xffffffffu, lm, d));
   double lsum = 0.0;
   if (with_lse) {
-    for (int s = lane; s < A.parts; s += 32) {
+    for (int s = lane; s < n_parts; s += 32) {
       const Partial p = A.partials[(long long)row * A.parts + s];
       if (p.ls > 0.f) lsum += (double)p.ls * exp2((double)(p.lm - lm) * (double)c2);
     }
@@ -180,7 +208,7 @@ __device__ __forceinline__ RowResult finalize_row(const SweepArgs& A, int row, i
   double ex = -CUDART_INF;
   int tok = -1;
   if (want) {
-    const char* rowp = (const char*)A.data + (b * A.sb + k * A.sk + j * A.sj) * ES;
+    const char* rowp = rl.rowp;
     StreamKey sk;
     sk.c1 = ((uint32_t)k & A.kmask) | (A.domain << 16);
     sk.pos = A.pos_base + (uint32_t)j;
@@ -396,6 +424,38 @@ finalize_verify_kernel(const __grid_constant__ SweepArgs A, const VerifyArgs va)
   for (int r = threadIdx.x >> 5; r < nrows; r += (int)(blockDim.x >> 5)) {
     const RowResult rr = finalize_row<DT, SPEC, ROUNDS>(A, b * nrows + r, 1, nullptr);
     if ((threadIdx.x & 31) == 0) srows[r] = rr;
+  }
+  __syncthreads();
+  if (threadIdx.x < 32)
+    verify_sequence_warp(srows, b, va.K, va.L, va.J, va.flags, va.multi_rows, dtok, va.out_tokens,
+                         va.out_num, va.accept, va.out_scores, va.dev_status);
+}
+
+// The fused draft + verify call: a CTA per sequence finalises the sequence's K x L draft rows
+// (tokens and scores go to the caller and into shared memory) and its K x J target rows, then a
+// warp runs Algorithm 2's loop on them.
+template <int DT, int SPEC, int ROUNDS>
+__global__ void __launch_bounds__(kFusedVerifyMaxWarps * 32)
+finalize_step_kernel(const __grid_constant__ SweepArgs A, const VerifyArgs va,
+                     int32_t* __restrict__ out_draft_tokens, float* __restrict__ out_draft_scores) {
+  asm volatile("griddepcontrol.wait;" ::: "memory");  // the sweep before this launch is complete
+  RowResult* srows = reinterpret_cast<RowResult*>(gls_smem_raw);
+  const int b = blockIdx.x;
+  const int nd = va.K * va.L, nt = va.K * va.J;
+  int32_t* dtok = reinterpret_cast<int32_t*>(srows + nt);
+  for (int r = threadIdx.x >> 5; r < nd + nt; r += (int)(blockDim.x >> 5)) {
+    if (r < nd) {
+      const RowResult rr = finalize_row<DT, SPEC, ROUNDS>(A, b * nd + r, 0, va.dev_status);
+      if ((threadIdx.x & 31) == 0) {
+        dtok[r] = rr.idx;
+        out_draft_tokens[(long long)b * nd + r] = rr.idx;
+        if (out_draft_scores)
+          out_draft_scores[(long long)b * nd + r] = rr.idx >= 0 ? (float)rr.score : CUDART_NAN_F;
+      }
+    } else {
+      const RowResult rr = finalize_row<DT, SPEC, ROUNDS>(A, A.rows1 + b * nt + (r - nd), 1, nullptr);
+      if ((threadIdx.x & 31) == 0) srows[r - nd] = rr;
+    }
   }
   __syncthreads();
   if (threadIdx.x < 32)
@@ -647,23 +707,44 @@ static cudaError_t launch_fused_verify_t(const SweepArgs& A, const VerifyArgs& v
   return cudaLaunchKernelEx(&cfg, finalize_verify_kernel<DT, SPEC, ROUNDS>, A, va);
 }
 
+struct StepOut {  // the draft-side outputs of the fused draft + verify call
+  int32_t* draft_tokens;
+  float* draft_scores;
+};
+template <int DT, int SPEC, int ROUNDS>
+static cudaError_t launch_step_t(const SweepArgs& A, const VerifyArgs& va, const StepOut& so,
+                                 cudaStream_t st) {
+  const size_t smem = fused_verify_smem(va.K, va.L, va.J);
+  const int nrows = va.K * (va.L + va.J);
+  const int warps = nrows < kFusedVerifyMaxWarps ? nrows : kFusedVerifyMaxWarps;
+  cudaLaunchAttribute attr;
+  cudaLaunchConfig_t cfg = dependent_launch(&attr, va.B, warps * 32, smem, st);
+  return cudaLaunchKernelEx(&cfg, finalize_step_kernel<DT, SPEC, ROUNDS>, A, va, so.draft_tokens,
+                            so.draft_scores);
+}
+
 // sweep + split reduction of one batch of rows.  With `va` (verification) and a sequence's
 // K x J row results fitting in shared memory, the reduction and Algorithm 2's loop run as one
 // launch and *fused is set; otherwise the rows' results are left in the workspace.
 static int run_rows(SweepArgs& A, int dtype, int spec, const Plan& P, void* workspace, bool lse,
                     int32_t* out_tokens, float* out_scores, uint32_t* status, cudaStream_t st,
-                    const VerifyArgs* va = nullptr, bool* fused = nullptr) {
+                    const VerifyArgs* va = nullptr, bool* fused = nullptr,
+                    const StepOut* step = nullptr) {
   char* ws = (char*)workspace;
   A.chunk = P.chunk;
   A.splits = P.splits;
   A.parts = P.parts;
   A.rows = (int)P.rows;
   A.n_items = P.n_items;
+  A.row_begin = 0;
+  A.row_count = (int)P.rows;
+  A.parts1 = P.two_launches ? P.splits1 * P.per_slice : 0;
+  A.parts2 = P.two_launches ? P.splits2 * P.per_slice : 0;
   A.hints = (uint32_t*)(ws + P.off_hints);
   A.partials = (Partial*)(ws + P.off_partials);
   RowResult* rowres = (RowResult*)(ws + P.off_rows);
   // the noise_spec 4 sweep touches the hint words only when rows are cut into slices
-  if ((spec != 4 || P.splits > 1) &&
+  if ((spec != 4 || P.splits > 1 || (P.two_launches && (P.splits1 > 1 || P.splits2 > 1))) &&
       cudaMemsetAsync(A.hints, 0, (size_t)P.rows * sizeof(uint32_t), st) != cudaSuccess)
     return GLS_ERR_CUDA;
   cudaError_t err;
@@ -671,17 +752,39 @@ static int run_rows(SweepArgs& A, int dtype, int spec, const Plan& P, void* work
   const bool bf = dtype == GLS_BF16;
   if (spec == 4) {
     const int sh = s4_shape(dtype, A.V, A.multi_k > 0);
+    // Two sets of rows: one launch with both variants of the sweep while the input is small (the
+    // launches are what a small step costs), otherwise one launch per set (the kernel
+    // specialised for its set is faster where the sweep itself is what a step costs).
+    const bool small_step = !P.two_launches;
 #define SWEEP4(SH, R)                                                                       \
   do {                                                                                      \
     const long long cap = (long long)num_sms() * S4Cfg<SH>::kCtasPerSM;                       \
     const int grid = (int)(P.n_items < cap ? P.n_items : cap);                              \
     const size_t smem = sizeof(S4Shared<SH>);                                               \
     if (A.multi_k > 0)                                                                      \
-      sweep4_kernel<SH, true, R, true><<<grid, S4Cfg<SH>::kWarps * 32, smem, st>>>(A);      \
+      sweep4_kernel<SH, 1, R, true><<<grid, S4Cfg<SH>::kWarps * 32, smem, st>>>(A);         \
+    else if (A.data2 != nullptr && small_step)                                              \
+      sweep4_kernel<SH, 2, R><<<grid, S4Cfg<SH>::kWarps * 32, smem, st>>>(A);               \
+    else if (A.data2 != nullptr) {                                                          \
+      SweepArgs A1 = A, A2 = A;                                                             \
+      A1.row_count = A.rows1;                                                               \
+      A1.chunk = P.chunk1;                                                                  \
+      A1.splits = P.splits1;                                                                \
+      A1.n_items = (long long)A.rows1 * P.splits1;                                          \
+      A2.row_begin = A.rows1;                                                               \
+      A2.row_count = A.rows - A.rows1;                                                      \
+      A2.chunk = P.chunk2;                                                                  \
+      A2.splits = P.splits2;                                                                \
+      A2.n_items = (long long)A2.row_count * P.splits2;                                     \
+      const int g1 = (int)(A1.n_items < cap ? A1.n_items : cap);                            \
+      const int g2 = (int)(A2.n_items < cap ? A2.n_items : cap);                            \
+      sweep4_kernel<SH, 0, R><<<g1, S4Cfg<SH>::kWarps * 32, smem, st>>>(A1);                \
+      sweep4_kernel<SH, 1, R><<<g2, S4Cfg<SH>::kWarps * 32, smem, st>>>(A2);                \
+    }                                                                                       \
     else if (lse)                                                                           \
-      sweep4_kernel<SH, true, R><<<grid, S4Cfg<SH>::kWarps * 32, smem, st>>>(A);            \
+      sweep4_kernel<SH, 1, R><<<grid, S4Cfg<SH>::kWarps * 32, smem, st>>>(A);               \
     else                                                                                    \
-      sweep4_kernel<SH, false, R><<<grid, S4Cfg<SH>::kWarps * 32, smem, st>>>(A);           \
+      sweep4_kernel<SH, 0, R><<<grid, S4Cfg<SH>::kWarps * 32, smem, st>>>(A);               \
   } while (0)
     if (sh == kS4ShapeBf16) { if (r10) SWEEP4(kS4ShapeBf16, 10); else SWEEP4(kS4ShapeBf16, 0); }
     else if (sh == kS4ShapeF32Wide) { if (r10) SWEEP4(kS4ShapeF32Wide, 10); else SWEEP4(kS4ShapeF32Wide, 0); }
@@ -699,6 +802,11 @@ static int run_rows(SweepArgs& A, int dtype, int spec, const Plan& P, void* work
   if (err != cudaSuccess) return GLS_ERR_CUDA;
   const bool fuse = va != nullptr && fused_verify_smem(va->K, va->L, va->J) <= kFusedVerifyMaxSmem;
   if (fused) *fused = fuse;
+  if (step != nullptr) {  // two sets of rows (noise_spec 4 only): draft results, then Algorithm 2
+    if (bf) err = r10 ? launch_step_t<kBF16, 4, 10>(A, *va, *step, st) : launch_step_t<kBF16, 4, 0>(A, *va, *step, st);
+    else err = r10 ? launch_step_t<kF32, 4, 10>(A, *va, *step, st) : launch_step_t<kF32, 4, 0>(A, *va, *step, st);
+    return err == cudaSuccess ? GLS_OK : GLS_ERR_CUDA;
+  }
 #define FIN_CALL(...)                                                                          \
   (fuse ? launch_fused_verify_t<__VA_ARGS__>(A, *va, st)                                       \
         : launch_finalize_t<__VA_ARGS__>(A, (int)P.rows, lse, rowres, out_tokens, out_scores, \
@@ -755,6 +863,16 @@ size_t gls_workspace_bytes(int B, int K, int J, int64_t V) {
     if (d > need) need = d;
     if (e > need) need = e;
     if (f > need) need = f;
+  }
+  return need;
+}
+
+size_t gls_draft_verify_workspace_bytes(int B, int K, int L, int J, int64_t V) {
+  if (L < 1 || J < L || J > L + 1 || !sizes_ok(B, K, L + J, V)) return 0;
+  size_t need = 0;
+  for (int dt = 0; dt < 2; ++dt) {
+    const size_t t = make_plan_step((long long)B * K * L, (long long)B * K * J, V, dt).total;
+    if (t > need) need = t;
   }
   return need;
 }
@@ -845,6 +963,74 @@ int gls_target_sample_verify(const gls_rows_t* target_logits, int B, int K, int 
                                                          out_tokens, out_num_tokens, out_accept,
                                                          out_scores, device_status);
   return cudaGetLastError() == cudaSuccess ? GLS_OK : GLS_ERR_CUDA;
+}
+
+int gls_draft_verify(const gls_rows_t* draft_logits, const gls_rows_t* target_logits, int B, int K,
+                     int L, int64_t V, float inv_temp_draft, const float* inv_temp_per_draft_host,
+                     float inv_temp_target, const gls_noise_t* noise, uint32_t flags,
+                     int32_t* out_draft_tokens, float* out_draft_scores, int32_t* out_tokens,
+                     int32_t* out_num_tokens, uint8_t* out_accept, float* out_scores,
+                     void* workspace, size_t workspace_bytes, uint32_t* device_status,
+                     void* stream) {
+  if (flags & ~(GLS_COMBINE_ALL | GLS_NO_BONUS)) return GLS_ERR_INVALID_ARG;
+  const int J = L + ((flags & GLS_NO_BONUS) ? 0 : 1);
+  if (!noise || !out_draft_tokens || !out_tokens || !out_num_tokens || !out_accept || L < 1 ||
+      !sizes_ok(B, K, L + J, V))
+    return GLS_ERR_INVALID_ARG;
+  if (!finite_pos(inv_temp_target)) return GLS_ERR_INVALID_ARG;
+  int rc = check_rows(draft_logits);
+  if (rc != GLS_OK) return rc;
+  rc = check_rows(target_logits);
+  if (rc != GLS_OK) return rc;
+  if (draft_logits->dtype != target_logits->dtype) return GLS_ERR_UNSUPPORTED;
+  SweepArgs A;
+  std::memset(&A, 0, sizeof(A));
+  for (int k = 0; k < K; ++k) {
+    const float it = inv_temp_per_draft_host ? inv_temp_per_draft_host[k] : inv_temp_draft;
+    if (!finite_pos(it)) return GLS_ERR_INVALID_ARG;
+    A.inv_t[k] = it;
+  }
+  int spec;
+  rc = fill_noise(A, noise, 0u, &spec);
+  if (rc != GLS_OK) return rc;
+  // one launch sweeps both sets of rows under the default noise layout; Appendix B with a target
+  // row per draft and sequences whose row results exceed the epilogue's shared memory take the
+  // two separate calls
+  if (spec != 4) return GLS_ERR_UNSUPPORTED;
+  if ((flags & GLS_COMBINE_ALL) && target_logits->stride_k != 0 && K > 1) return GLS_ERR_UNSUPPORTED;
+  if (fused_verify_smem(K, L, J) > kFusedVerifyMaxSmem) return GLS_ERR_UNSUPPORTED;
+  const long long rows_d = (long long)B * K * L, rows_t = (long long)B * K * J;
+  const Plan P = make_plan_step(rows_d, rows_t, V, draft_logits->dtype);
+  if (!workspace || workspace_bytes < P.total) return GLS_ERR_WORKSPACE;
+  A.data = draft_logits->data;
+  A.sb = draft_logits->stride_b;
+  A.sk = draft_logits->stride_k;
+  A.sj = draft_logits->stride_j;
+  A.K = K;
+  A.J = L;
+  A.V = (int)V;
+  A.data2 = target_logits->data;
+  A.sb2 = target_logits->stride_b;
+  A.sk2 = target_logits->stride_k;
+  A.sj2 = target_logits->stride_j;
+  A.J2 = J;
+  A.rows1 = (int)rows_d;
+  A.inv_t2 = inv_temp_target;
+  VerifyArgs va;
+  va.B = B; va.K = K; va.L = L; va.J = J;
+  va.flags = flags;
+  va.multi_rows = false;
+  va.draft_tokens = nullptr;  // taken from the draft rows of this very call
+  va.out_tokens = out_tokens;
+  va.out_num = out_num_tokens;
+  va.accept = out_accept;
+  va.out_scores = out_scores;
+  va.dev_status = device_status;
+  StepOut so;
+  so.draft_tokens = out_draft_tokens;
+  so.draft_scores = out_draft_scores;
+  return run_rows(A, draft_logits->dtype, spec, P, workspace, true, nullptr, nullptr, nullptr,
+                  (cudaStream_t)stream, &va, nullptr, &so);
 }
 
 static int check_sparse(const gls_sparse_rows_t* r) {

@@ -59,12 +59,21 @@ struct SweepArgs {
   const void* data;       // rows [B][K][J][V]
   long long sb, sk, sj;   // element strides
   int K, J, V;
+  // Optional second set of rows (the fused draft + verify call): rows [rows1, rows) of the call
+  // are rows [b][k][j] of `data2` with J2 positions per (b, k) and the temperature inv_t2; rows
+  // [0, rows1) are those of `data`.  data2 == NULL: one set, rows1 == rows.
+  const void* data2;
+  long long sb2, sk2, sj2;
+  int J2, rows1;
+  float inv_t2;
   int chunk;              // tokens per slice
   int splits;             // slices per row
-  int parts;              // partial results per row (slices x producers per slice)
+  int parts;              // partial-result slots per row (slices x producers per slice)
+  int parts1, parts2;     // slots in use per row of the first / second set (0: all of them)
   int rows;               // B * K * J
   int multi_k;            // > 0: one race per row over this many noise streams (fused encoder)
-  long long n_items;      // rows * splits
+  long long n_items;      // row_count * splits
+  int row_begin, row_count;  // the rows this launch sweeps: [row_begin, row_begin + row_count)
   float inv_t[kMaxK];     // 1/T per k
   uint32_t rk[32];        // Philox round keys: rk[2r], rk[2r+1]
   int rounds;
@@ -178,6 +187,33 @@ __device__ __forceinline__ double noise_exact(const SweepArgs& A, const StreamKe
   const uint32_t t = (uint32_t)i & 3u;
   const uint32_t u = t == 0 ? o[0] : t == 1 ? o[1] : t == 2 ? o[2] : o[3];
   return m + (-log1p(-((double)u + 0.5) * 0x1p-32));
+}
+
+// Where row `row` of the call lives and which (b, k, j) it is.
+struct RowLoc {
+  const char* rowp;
+  int b, k, j;
+  float inv_t;
+  bool second;
+};
+template <int ES>
+__device__ __forceinline__ RowLoc locate_row(const SweepArgs& A, int row) {
+  RowLoc r;
+  r.second = A.data2 != nullptr && row >= A.rows1;
+  const int rr = r.second ? row - A.rows1 : row;
+  const int J = r.second ? A.J2 : A.J;
+  r.j = rr % J;
+  const int bk = rr / J;
+  r.k = bk % A.K;
+  r.b = bk / A.K;
+  if (r.second) {
+    r.rowp = (const char*)A.data2 + (r.b * A.sb2 + r.k * A.sk2 + r.j * A.sj2) * ES;
+    r.inv_t = A.inv_t2;
+  } else {
+    r.rowp = (const char*)A.data + (r.b * A.sb + r.k * A.sk + r.j * A.sj) * ES;
+    r.inv_t = A.inv_t[r.k];
+  }
+  return r;
 }
 
 template <int DT>

@@ -235,9 +235,9 @@ __device__ __noinline__ void lse4_redo_careful(const char* rowp, int tok0, int n
 // ------------------------------------------------------------------------------------------
 // The kernel
 // ------------------------------------------------------------------------------------------
-template <int SH, bool LSE, int ROUNDS, bool MULTI = false>
-__global__ void __launch_bounds__(S4Cfg<SH>::kWarps * 32, S4Cfg<SH>::kCtasPerSM)
-sweep4_kernel(const __grid_constant__ SweepArgs A) {
+// One work item: slice `split` of row `row`, swept by the calling CTA.
+template <int SH, bool LSE, int ROUNDS, bool MULTI>
+__device__ __forceinline__ void s4_item(const SweepArgs& A, int row, int split, uint32_t tag) {
   constexpr int DT = S4Cfg<SH>::kDT;
   S4Shared<SH>& sh = s4_shared<SH>();
   const int lane = threadIdx.x & 31;
@@ -248,31 +248,21 @@ sweep4_kernel(const __grid_constant__ SweepArgs A) {
   typedef Group16<DT> G;
   uint2* const queue = sh.queue[warp];
   volatile unsigned long long* const m_tag = &sh.m_tag;
-
-  if (threadIdx.x == 0) sh.m_tag = 0ull;
-  __syncthreads();
-
-  uint32_t tag = 0u;
-  for (long long item = blockIdx.x; item < A.n_items; item += gridDim.x) {
-    ++tag;
-    const int split = (int)(item / A.rows);
-    const int row = (int)(item - (long long)split * A.rows);
+  {
     const int tok_begin = split * A.chunk;  // a multiple of 2048
     const int tok_end = min(A.V, tok_begin + A.chunk);
     uint32_t c1, pos, seq;
     const char* rowp;
     float c2;
     {
-      const int j = row % A.J;
-      const int bk = row / A.J;
-      const int k = bk % A.K;
-      const int b = bk / A.K;
-      rowp = (const char*)A.data + (b * A.sb + k * A.sk + j * A.sj) * ES;
+      const RowLoc rl = locate_row<ES>(A, row);
+      const int j = rl.j, k = rl.k, b = rl.b;
+      rowp = rl.rowp;
       // the fused multi-stream race enumerates the streams itself, whatever the row's k
       c1 = (MULTI ? 0u : ((uint32_t)k & A.kmask)) | (A.domain << 16);
       pos = A.pos_base + (uint32_t)j;
       seq = A.seq_ids ? __ldg(A.seq_ids + b) : A.seq_base + (uint32_t)b;
-      const float inv_t = A.inv_t[k];
+      const float inv_t = rl.inv_t;
       c2 = inv_t * kLog2e;
       __syncwarp();  // the previous item's batched path is done with the context
       if (lane == 0) {
@@ -494,8 +484,39 @@ sweep4_kernel(const __grid_constant__ SweepArgs A) {
       Partial pr;
       pr.s1 = t2.s1; pr.i1 = t2.i1; pr.s2 = t2.s2; pr.i2 = t2.i2;
       pr.lm = lm; pr.ls = ls; pr.pad0 = 0; pr.pad1 = 0;
-      A.partials[((long long)row * A.splits + split) * kWarps + warp] = pr;
+      A.partials[(long long)row * A.parts + split * kWarps + warp] = pr;
       if (A.splits > 1 && m_enc > 0u) atomicMax(A.hints + row, m_enc);
+    }
+  }
+}
+
+// the same out of line, so that two variants in one kernel are each compiled on their own
+template <int SH, bool LSE, int ROUNDS>
+__device__ __noinline__ void s4_item_call(const SweepArgs& A, int row, int split, uint32_t tag) {
+  s4_item<SH, LSE, ROUNDS, false>(A, row, split, tag);
+}
+
+// LSEMODE 0: races only (draft side, decoders); 1: races and the rows' log-sum-exp (target side,
+// encoder); 2: two sets of rows in one launch, the first without and the second with the
+// log-sum-exp (the fused draft + verify call).
+template <int SH, int LSEMODE, int ROUNDS, bool MULTI = false>
+__global__ void __launch_bounds__(S4Cfg<SH>::kWarps * 32, S4Cfg<SH>::kCtasPerSM)
+sweep4_kernel(const __grid_constant__ SweepArgs A) {
+  S4Shared<SH>& sh = s4_shared<SH>();
+  if (threadIdx.x == 0) sh.m_tag = 0ull;
+  __syncthreads();
+  uint32_t tag = 0u;
+  for (long long item = blockIdx.x; item < A.n_items; item += gridDim.x) {
+    ++tag;
+    const int split = (int)(item / A.row_count);
+    const int row = A.row_begin + (int)(item - (long long)split * A.row_count);
+    if constexpr (LSEMODE == 2) {
+      if (row >= A.rows1)
+        s4_item_call<SH, true, ROUNDS>(A, row, split, tag);
+      else
+        s4_item_call<SH, false, ROUNDS>(A, row, split, tag);
+    } else {
+      s4_item<SH, LSEMODE == 1, ROUNDS, MULTI>(A, row, split, tag);
     }
   }
   // this block has no more work: a dependent launch (the reduction) may start to be scheduled

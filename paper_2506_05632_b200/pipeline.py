@@ -33,16 +33,22 @@ class StepBuffers:
                         accept=torch.empty((B, K, L), dtype=torch.uint8, device=device),
                         scores=torch.empty((B, L + 1), dtype=torch.float32, device=device))
         need = max(binding.workspace_bytes(B, K, max(L, 1), V),
-                   binding.workspace_bytes(B, K, L + 1, V))
+                   binding.workspace_bytes(B, K, L + 1, V),
+                   binding.draft_verify_workspace_bytes(B, K, L, L + 1, V) if L > 0 else 0)
         self.workspace = torch.empty(need, dtype=torch.uint8, device=device)
         self.status = torch.zeros(1, dtype=torch.int32, device=device)
 
 
 def spec_step(draft_logits, target_logits, buf, inv_temp=1.0, seed=0, seq_base=0, pos_base=0,
-              spec=4, rounds=10):
-    """draft_logits [B,K,L,V], target_logits [B,K,L+1,V] on the device -> buf.out (device)."""
+              spec=4, rounds=10, fused=False):
+    """draft_logits [B,K,L,V], target_logits [B,K,L+1,V] on the device -> buf.out (device).
+    fused: one gls_draft_verify call instead of a draft call followed by a verify call."""
     kw = dict(inv_temp=inv_temp, seed=seed, seq_base=seq_base, pos_base=pos_base, spec=spec,
               rounds=rounds, workspace=buf.workspace, status=buf.status)
+    if fused and draft_logits.shape[2] > 0:
+        binding.draft_verify(draft_logits, target_logits, out_draft_tokens=buf.draft_tokens,
+                             out_draft_scores=buf.draft_scores, out=buf.out, **kw)
+        return buf.out
     if draft_logits.shape[2] > 0:
         binding.draft_sample(draft_logits, out_tokens=buf.draft_tokens,
                              out_scores=buf.draft_scores, **kw)

@@ -135,3 +135,18 @@ def test_autoregressive_draft_shape(gls, oracle):
     sel = torch.from_numpy(idx).cuda()
     ref = oracle.draft_sample(synth.to_numpy_rows(w.draft_logits[sel]), seq_ids=idx, **kw)
     assert np.array_equal(tok.cpu().numpy()[idx], ref["tokens"])
+
+
+def test_config3_one_call_equals_two_calls(gls):
+    """gls_draft_verify at full size (one sweep launch per set of rows, each sliced for its own
+    row count, one reduction launch): bit-identical to the draft call followed by the verify call."""
+    w = synth.verify_workload(3, "cuda")
+    kw = dict(seed=w.noise_seed, inv_temp=w.inv_temp)
+    tok, sc = gls.draft_sample(w.draft_logits, **kw)
+    out = gls.target_sample_verify(w.target_logits, tok, **kw)
+    dtok, dsc, fout = gls.draft_verify(w.draft_logits, w.target_logits, **kw)
+    torch.cuda.synchronize()
+    assert torch.equal(dtok, tok) and torch.equal(dsc, sc)
+    for key in ("tokens", "tau", "accept"):
+        assert torch.equal(fout[key], out[key]), key
+    assert torch.equal(fout["scores"].nan_to_num(7.0), out["scores"].nan_to_num(7.0))

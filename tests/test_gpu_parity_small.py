@@ -410,3 +410,38 @@ def test_host_detectable_errors(gls):
     t, _ = gls.draft_sample(x)
     torch.cuda.synchronize()
     assert t.shape == (2, 2, 2)
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+def test_draft_verify_in_one_call(gls, oracle, dtype):
+    """gls_draft_verify (both sets of rows in one sweep launch, one reduction launch) against the
+    oracle and, bit for bit, against the two separate calls: ragged vocabularies, rows cut into
+    several slices, per-draft temperatures, no bonus position, shared target rows with Appendix B."""
+    for (B, K, L, V) in ((3, 2, 1, 517), (5, 4, 3, 40001), (2, 8, 4, 2048 * 9 + 700), (9, 3, 2, 16385)):
+        d = _rand_logits(B, K, L, V, dtype, 300 + V % 97, scale=2.5)
+        t = _rand_logits(B, K, L + 1, V, dtype, 301 + V % 97, scale=2.5)
+        t[:, :, :L] = (d.float() + 0.5 * _rand_logits(B, K, L, V, torch.float32, 302, 1.0)).to(dtype)
+        its = [0.7 + 0.3 * k for k in range(K)]
+        for flags, tt, kw in (
+                (0, t, dict(seed=SEED + 21, inv_temp=0.9, seq_base=3, pos_base=1)),
+                (gls.NO_BONUS, t[:, :, :L], dict(seed=SEED + 22, inv_temp_per_draft=its, inv_temp=1.3)),
+                (gls.COMBINE_ALL, t[:, :1].expand(B, K, L + 1, V), dict(seed=SEED + 23, inv_temp=1.0))):
+            dtok, dsc, out = gls.draft_verify(d, tt, flags=flags, **kw)
+            tok2, sc2 = gls.draft_sample(d, **kw)
+            vkw = {k: v for k, v in kw.items() if k != "inv_temp_per_draft"}
+            out2 = gls.target_sample_verify(tt, tok2, flags=flags, **vkw)
+            torch.cuda.synchronize()
+            assert torch.equal(dtok, tok2) and torch.equal(dsc, sc2)
+            for key in ("tokens", "tau", "accept"):
+                assert torch.equal(out[key], out2[key]), key
+            assert torch.equal(out["scores"].nan_to_num(7.0), out2["scores"].nan_to_num(7.0))
+            ref = oracle.draft_sample(synth.to_numpy_rows(d), **kw)
+            parity.check_draft(dtok.cpu().numpy(), dsc.cpu().numpy(), ref, "fused draft V=%d" % V)
+            refv = oracle.target_sample_verify(synth.to_numpy_rows(tt.contiguous()), ref["tokens"],
+                                               flags=flags, **vkw)
+            parity.check_verify(parity.to_np(out), refv, "fused verify V=%d flags=%d" % (V, flags))
+    x = _rand_logits(1, 2, 2, 100, torch.float32, 5)
+    with pytest.raises(gls.GlsError):  # the literal noise layout takes the two separate calls
+        gls.draft_verify(x, x[:, :, :2].repeat(1, 1, 2, 1)[:, :, :3], spec=1)
+    with pytest.raises(gls.GlsError):  # both sets must have one element type
+        gls.draft_verify(x, x[:, :, :2].repeat(1, 1, 2, 1)[:, :, :3].to(torch.bfloat16))
