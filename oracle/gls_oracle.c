@@ -13,7 +13,9 @@
  *                            early stop when S is empty, bonus token Y_{L+1}.
  *   - Appendix B:            min over all k instead of k in S (strong drafter invariance).
  *   - Sec. 5.1 / Appendix C: encoder index Y, message M = l_Y, decoder indices X^(k) restricted
- *                            to candidates with l_i = M, over (importance) weights.
+ *                            to candidates with l_i = M, over (importance) weights; with the
+ *                            Gaussian model of Sec. 5.2 / Appendix D.3 also the weights themselves,
+ *                            the decoder outputs and the MMSE reconstruction.
  *
  * Races are evaluated in the log domain, argmin_i S_i/p_i = argmax_i (ln p_i - ln S_i), with
  * ln p_i = logit_i / T - lse and lse = ln sum_i exp(logit_i / T) computed by the two-pass
@@ -47,6 +49,7 @@
 
 #define GLSO_F32 0
 #define GLSO_BF16 1
+#define GLSO_F64 2 /* rows the oracle computes itself (Gaussian importance log-weights) */
 #define GLSO_NOISE_SHARED_ACROSS_K 1u
 #define GLSO_COMBINE_ALL 1u
 #define GLSO_NO_BONUS 2u
@@ -200,6 +203,7 @@ void glso_exp_noise_batch(uint64_t seed, int rounds, int spec, uint32_t domain, 
 /* ------------------------------------------------------------------------------------------ */
 static double load_elem(const void* base, int dtype, int64_t idx) {
   if (dtype == GLSO_F32) return (double)((const float*)base)[idx];
+  if (dtype == GLSO_F64) return ((const double*)base)[idx];
   uint32_t bits = (uint32_t)((const uint16_t*)base)[idx] << 16; /* bf16 = top half of an fp32 */
   float f;
   memcpy(&f, &bits, 4);
@@ -327,7 +331,7 @@ static glso_key_t make_key(const glso_noise_t* nz, uint32_t domain, int b, int j
 static const void* row_ptr(const void* data, int dtype, int64_t sb, int64_t sk, int64_t sj, int b,
                            int k, int j) {
   int64_t off = sb * b + sk * k + sj * j;
-  return (const char*)data + off * (dtype == GLSO_F32 ? 4 : 2);
+  return (const char*)data + off * (dtype == GLSO_F32 ? 4 : dtype == GLSO_F64 ? 8 : 2);
 }
 
 /* ------------------------------------------------------------------------------------------ */
@@ -487,6 +491,111 @@ int glso_compress_select(const void* enc_logw, int enc_dtype, int64_t enc_sb, co
     match[b] = (uint8_t)hit;
   }
   return 0;
+}
+
+/* ------------------------------------------------------------------------------------------ */
+/* Compression from the source: Appendix C (importance sampling) with the Gaussian model of     */
+/* Sec. 5.2 / Appendix D.3, applied per dimension to D-dimensional vectors.                     */
+/*   candidates u_i (i < N, D floats each) drawn by the caller from the proposal N(0, s2_prior) */
+/*   source a_b, side information t_bk = a_b + zeta                                             */
+/*   encoder log-weight  ln p_{W|A}(u_i | a_b) - ln prop(u_i),  p_{W|A}(.|a) = N(a, s2_eta)     */
+/*   decoder log-weight  ln p_{W|T}(u_i | t_bk) - ln prop(u_i),                                 */
+/*                       p_{W|T}(.|t) = N(t / s2_T, s2_W - 1 / s2_T), s2_T = 1 + s2_zeta,       */
+/*                       s2_W = 1 + s2_eta                                                      */
+/*   (additive terms common to a row are dropped: they cannot change an argmin and cancel in    */
+/*   the normalised score; the factor L_max of Appendix C's decoder weight is such a term)      */
+/* then the selection of Sec. 5.1 on these weights, the decoder outputs W_k = u_{X^(k)}, the    */
+/* MMSE reconstruction g(w, t) = (s2_zeta w + s2_eta t) / (s2_eta + s2_zeta + s2_eta s2_zeta)   */
+/* and its squared error per dimension.                                                          */
+/*   logw_out: NULL or [B, 1 + K, N] doubles (the weights as computed, for the pins)            */
+/*   recon [B,K,D], sqerr [B,K] (mean over the D dimensions); the rest as glso_compress_select  */
+/* ------------------------------------------------------------------------------------------ */
+static void gaussian_logw_row(const float* u, int64_t N, int D, const double* mean, double var,
+                              double s2_prior, double* out) {
+  for (int64_t i = 0; i < N; ++i) {
+    double acc = 0.0;
+    for (int d = 0; d < D; ++d) {
+      double x = (double)u[i * D + d];
+      double diff = x - mean[d];
+      acc += -(diff * diff) / (2.0 * var) + (x * x) / (2.0 * s2_prior);
+    }
+    out[i] = acc;
+  }
+}
+
+int glso_compress_gaussian(const float* u, const float* a, const float* t, const uint8_t* bins,
+                           int64_t bins_sb, int B, int K, int64_t N, int D, double s2_eta,
+                           double s2_zeta, double s2_prior, const glso_noise_t* nz,
+                           int32_t* enc_index, uint8_t* message, int32_t* dec_index,
+                           uint8_t* match, double* scores, double* gaps, double* recon,
+                           double* sqerr, double* logw_out) {
+  if (!u || !a || !t || !nz || !enc_index || !message || !dec_index || !match || B <= 0 ||
+      K <= 0 || K > GLSO_MAX_K || N <= 0 || D <= 0 || D > 64)
+    return 1;
+  if (!(s2_eta > 0.0) || !(s2_zeta > 0.0) || !(s2_prior > 0.0)) return 1;
+  const double s2T = 1.0 + s2_zeta, s2W = 1.0 + s2_eta;
+  const double var_dec = s2W - 1.0 / s2T;
+  const double denom = s2_eta + s2_zeta + s2_eta * s2_zeta;
+  int failed = 0;
+#pragma omp parallel for schedule(dynamic, 1)
+  for (int b = 0; b < B; ++b) {
+    double* w = (double*)malloc(sizeof(double) * (size_t)N);
+    if (!w) {
+      failed = 1;
+      continue;
+    }
+    double mean[64];
+    const uint8_t* lab = bins ? bins + bins_sb * b : NULL;
+    /* encoder: Y = argmin_i min_k S_i^(k) / lambda_q,i */
+    for (int d = 0; d < D; ++d) mean[d] = (double)a[(int64_t)b * D + d];
+    gaussian_logw_row(u, N, D, mean, s2_eta, s2_prior, w);
+    if (logw_out) memcpy(logw_out + (int64_t)b * (1 + K) * N, w, sizeof(double) * (size_t)N);
+    double lse = row_lse(w, GLSO_F64, N, 1.0, NULL, 0);
+    race_t rc;
+    race_init(&rc);
+    if (lse != -INFINITY)
+      for (int k = 0; k < K; ++k) {
+        glso_key_t nk = make_key(nz, 1u, b, 0, k);
+        race_row(&rc, w, GLSO_F64, N, 1.0, lse, &nk, NULL, 0, k);
+      }
+    enc_index[b] = (int32_t)rc.i1;
+    int msg = (lab && rc.i1 >= 0) ? (int)lab[rc.i1] : 0;
+    message[b] = (uint8_t)msg;
+    if (scores) scores[(int64_t)b * (1 + K)] = rc.i1 >= 0 ? rc.s1 : NAN;
+    if (gaps) gaps[(int64_t)b * (1 + K)] = gap_of(&rc);
+    /* decoder k: X^(k) over the candidates labelled M, W_k = u_{X^(k)}, reconstruction g(W_k, t_k) */
+    int hit = 0;
+    for (int k = 0; k < K; ++k) {
+      const float* tk = t + ((int64_t)b * K + k) * D;
+      for (int d = 0; d < D; ++d) mean[d] = (double)tk[d] / s2T;
+      gaussian_logw_row(u, N, D, mean, var_dec, s2_prior, w);
+      if (logw_out)
+        memcpy(logw_out + ((int64_t)b * (1 + K) + 1 + k) * N, w, sizeof(double) * (size_t)N);
+      glso_key_t nk = make_key(nz, 1u, b, 0, k);
+      race_t rd;
+      race_init(&rd);
+      race_row(&rd, w, GLSO_F64, N, 1.0, 0.0, &nk, lab, msg, k);
+      dec_index[(int64_t)b * K + k] = (int32_t)rd.i1;
+      if (scores) scores[(int64_t)b * (1 + K) + 1 + k] = rd.i1 >= 0 ? rd.s1 : NAN;
+      if (gaps) gaps[(int64_t)b * (1 + K) + 1 + k] = gap_of(&rd);
+      if (rd.i1 >= 0 && rd.i1 == rc.i1) hit = 1;
+      double se = 0.0;
+      for (int d = 0; d < D; ++d) {
+        double g = NAN;
+        if (rd.i1 >= 0) {
+          double wk = (double)u[rd.i1 * D + d];
+          g = (s2_zeta * wk + s2_eta * (double)tk[d]) / denom;
+          double e = g - (double)a[(int64_t)b * D + d];
+          se += e * e;
+        }
+        if (recon) recon[((int64_t)b * K + k) * D + d] = g;
+      }
+      if (sqerr) sqerr[(int64_t)b * K + k] = rd.i1 >= 0 ? se / D : NAN;
+    }
+    match[b] = (uint8_t)hit;
+    free(w);
+  }
+  return failed;
 }
 
 void glso_set_threads(int n) {

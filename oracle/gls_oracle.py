@@ -23,7 +23,7 @@ _LIB = os.path.join(_HERE, "libgls_oracle.so")
 _lock = threading.Lock()
 _lib = None
 
-F32, BF16 = 0, 1
+F32, BF16, F64 = 0, 1, 2
 NOISE_SHARED_ACROSS_K = 1
 COMBINE_ALL = 1
 NO_BONUS = 2
@@ -129,6 +129,8 @@ def _as_rows(a):
         return a, F32
     if a.dtype == np.uint16:
         return a, BF16
+    if a.dtype == np.float64:
+        return a, F64
     raise TypeError("logits must be float32 or uint16 (bf16 bit patterns), got %s" % a.dtype)
 
 
@@ -245,6 +247,49 @@ def compress_select(enc_logw, dec_logw=None, bins=None, seed=0, seq_base=0, seq_
         raise ValueError("oracle compress_select: invalid arguments")
     return dict(enc_index=enc_index, message=message, dec_index=dec_index, match=match,
                 scores=scores, gaps=gaps)
+
+
+def compress_gaussian(u, a, t, bins=None, s2_eta=0.5, s2_zeta=0.25, s2_prior=1.0, seed=0,
+                      seq_base=0, seq_ids=None, pos_base=0, spec=4, rounds=10, noise_flags=0,
+                      want_logw=False):
+    """Appendix C with the Gaussian model of Sec. 5.2 / Appendix D.3 (per dimension).
+
+    u [N,D] candidates drawn from N(0, s2_prior I); a [B,D] sources; t [B,K,D] side information.
+    Returns compress_select's dict plus recon [B,K,D], sqerr [B,K] (mean squared error per
+    dimension of each decoder's reconstruction) and, on request, logw [B,1+K,N]."""
+    u = np.ascontiguousarray(u, dtype=np.float32)
+    a = np.ascontiguousarray(a, dtype=np.float32)
+    t = np.ascontiguousarray(t, dtype=np.float32)
+    N, D = u.shape
+    B, K, _ = t.shape
+    assert a.shape == (B, D) and t.shape == (B, K, D)
+    bptr, bsb = None, 0
+    if bins is not None:
+        bins = np.ascontiguousarray(bins, dtype=np.uint8)
+        bptr = bins.ctypes.data
+        bsb = 0 if bins.ndim == 1 else N
+        assert bins.shape[-1] == N
+    nz, keep = _noise(seed, seq_base, seq_ids, pos_base, spec, rounds, noise_flags)
+    out = dict(enc_index=np.empty((B,), np.int32), message=np.empty((B,), np.uint8),
+               dec_index=np.full((B, K), -1, np.int32), match=np.zeros((B,), np.uint8),
+               scores=np.full((B, 1 + K), np.nan), gaps=np.full((B, 1 + K), np.nan),
+               recon=np.empty((B, K, D)), sqerr=np.empty((B, K)))
+    logw = np.empty((B, 1 + K, N)) if want_logw else None
+    f = lib().glso_compress_gaussian
+    f.restype = C.c_int
+    rc = f(C.c_void_p(u.ctypes.data), C.c_void_p(a.ctypes.data), C.c_void_p(t.ctypes.data),
+           C.c_void_p(bptr), C.c_int64(bsb), C.c_int(B), C.c_int(K), C.c_int64(N), C.c_int(D),
+           C.c_double(s2_eta), C.c_double(s2_zeta), C.c_double(s2_prior), C.byref(nz),
+           C.c_void_p(out["enc_index"].ctypes.data), C.c_void_p(out["message"].ctypes.data),
+           C.c_void_p(out["dec_index"].ctypes.data), C.c_void_p(out["match"].ctypes.data),
+           C.c_void_p(out["scores"].ctypes.data), C.c_void_p(out["gaps"].ctypes.data),
+           C.c_void_p(out["recon"].ctypes.data), C.c_void_p(out["sqerr"].ctypes.data),
+           C.c_void_p(logw.ctypes.data if want_logw else None))
+    if rc != 0:
+        raise ValueError("oracle compress_gaussian: invalid arguments")
+    if want_logw:
+        out["logw"] = logw
+    return out
 
 
 def top_m_rows(logits, M):
