@@ -159,6 +159,39 @@ int gls_draft_sample(const gls_rows_t* draft_logits, int B, int K, int J, int64_
                      size_t workspace_bytes, uint32_t* device_status, void* stream);
 
 /*
+ * Compression from the source -- Appendix C (importance sampling: candidates U_i drawn from a
+ * proposal, unnormalised weights p_{W|A}(U_i | a) / prop(U_i) at the encoder and
+ * p_{W|T}(U_i | t_k) 1{l_i = M} / prop(U_i) at decoder k) with the Gaussian model of Sec. 5.2 /
+ * Appendix D.3 applied per dimension: p_{W|A}(. | a) = N(a, s2_eta), T_k = A + N(0, s2_zeta),
+ * p_{W|T}(. | t) = N(t / s2_T, s2_W - 1 / s2_T) with s2_T = 1 + s2_zeta, s2_W = 1 + s2_eta, proposal
+ * N(0, s2_prior).  The log-weights
+ *     encoder  sum_d -(u_id - a_bd)^2 / (2 s2_eta) + u_id^2 / (2 s2_prior)
+ *     decoder  sum_d -(u_id - t_bkd / s2_T)^2 / (2 (s2_W - 1 / s2_T)) + u_id^2 / (2 s2_prior)
+ * (terms common to a row dropped) are computed inside the kernels from the D coordinates of each
+ * candidate -- nothing of size B x N is read or written -- and raced as in gls_compress_select,
+ * whose outputs this call reproduces for those weights; the winners' weights are recomputed in
+ * fp64.  Then, per decoder, W_k = U_{X^(k)}, the MMSE reconstruction
+ *     g(w, t) = (s2_zeta w + s2_eta t) / (s2_eta + s2_zeta + s2_eta s2_zeta)      (Appendix D.3)
+ * and its squared error against the source, averaged over the D dimensions.
+ *
+ *   candidates  [N,D] fp32, source [B,D] fp32, side_info [B,K,D] fp32 (all contiguous)
+ *   bins        NULL, [N] (bins_stride_b = 0) or [B,N] uint8
+ *   out_recon   NULL or [B,K,D] fp32;  out_sqerr NULL or [B,K] fp32;  the rest as
+ *               gls_compress_select
+ *   workspace   gls_compress_gaussian_workspace_bytes(B, K, N) bytes
+ * Default noise layout only; D <= 16, K <= 8, N < 2^28 (GLS_ERR_UNSUPPORTED otherwise: compute
+ * the weights and call gls_compress_select).
+ */
+size_t gls_compress_gaussian_workspace_bytes(int B, int K, int64_t N);
+int gls_compress_gaussian(const float* candidates, const float* source, const float* side_info,
+                          const uint8_t* bins, int64_t bins_stride_b, int B, int K, int64_t N, int D,
+                          double s2_eta, double s2_zeta, double s2_prior, const gls_noise_t* noise,
+                          int32_t* out_enc_index, uint8_t* out_message, int32_t* out_dec_index,
+                          uint8_t* out_match, float* out_scores, float* out_recon, float* out_sqerr,
+                          void* workspace, size_t workspace_bytes, uint32_t* device_status,
+                          void* stream);
+
+/*
  * Draft-side sampling for callers that cannot allocate device memory.  The paper has no counterpart
  * to this call; it exists for deployment only and computes exactly what gls_draft_sample computes.
  *

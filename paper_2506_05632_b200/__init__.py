@@ -8,10 +8,11 @@ kernels of csrc/.  There is no CPU fallback: if libgls.so cannot be loaded the c
     target_sample_verify(logits, tokens, ...) Algorithm 2 verification
     draft_verify(draft, target, ...)          both of the above in one call (one sweep launch)
     compress_select(enc, dec, bins, ...)      Sec. 5.1 encoder / decoder index selection
+    compress_gaussian(u, a, t, bins, ...)     the same from the source: Appendix C weights computed in the kernels
 """
 from .binding import (  # noqa: F401
     COMBINE_ACTIVE, COMBINE_ALL, NO_BONUS, NOISE_SHARED_ACROSS_K, DEV_EMPTY_SUPPORT, GlsError,
-    build, compress_select, draft_sample, draft_sample_sparse, draft_sample_static,
+    build, compress_gaussian, compress_gaussian_workspace_bytes, compress_select, draft_sample, draft_sample_sparse, draft_sample_static,
     draft_sample_topm, draft_verify, draft_verify_workspace_bytes, lib_path, load,
     static_scratch_bytes, status_string, target_sample_verify, target_sample_verify_sparse,
     target_sample_verify_topm, topm_workspace_bytes, version, workspace_bytes)

@@ -123,6 +123,14 @@ def load():
             C.POINTER(_Rows), C.c_int, C.c_int, C.c_int, C.c_int64, C.c_int, C.c_float, C.c_void_p,
             C.POINTER(_Noise), C.c_uint32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
             C.c_void_p, C.c_size_t, C.c_void_p, C.c_void_p]
+        L.gls_compress_gaussian_workspace_bytes.restype = C.c_size_t
+        L.gls_compress_gaussian_workspace_bytes.argtypes = [C.c_int, C.c_int, C.c_int64]
+        L.gls_compress_gaussian.restype = C.c_int
+        L.gls_compress_gaussian.argtypes = [
+            C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64, C.c_int, C.c_int, C.c_int64,
+            C.c_int, C.c_double, C.c_double, C.c_double, C.POINTER(_Noise), C.c_void_p, C.c_void_p,
+            C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t,
+            C.c_void_p, C.c_void_p]
         L.gls_compress_select.restype = C.c_int
         L.gls_compress_select.argtypes = [
             C.POINTER(_Rows), C.POINTER(_Rows), C.c_void_p, C.c_int64, C.c_int, C.c_int,
@@ -476,5 +484,48 @@ def compress_select(enc_logw, dec_logw=None, bins=None, K=None, seed=0, seq_base
         C.byref(erows), C.byref(drows) if drows is not None else None, _ptr(bins), bsb, B, K, N,
         C.byref(nz), _ptr(out["enc_index"]), _ptr(out["message"]), _ptr(out["dec_index"]),
         _ptr(out["match"]), _ptr(out.get("scores")), workspace.data_ptr(), workspace.numel(),
+        _ptr(status), _stream()))
+    return out
+
+
+def compress_gaussian_workspace_bytes(B, K, N):
+    return int(load().gls_compress_gaussian_workspace_bytes(int(B), int(K), int(N)))
+
+
+def compress_gaussian(candidates, source, side_info, bins=None, s2_eta=0.5, s2_zeta=0.25,
+                      s2_prior=1.0, seed=0, seq_base=0, seq_ids=None, pos_base=0, spec=4, rounds=10,
+                      noise_flags=0, want_scores=True, workspace=None, status=None, out=None):
+    """gls_compress_gaussian: candidates [N,D], source [B,D], side_info [B,K,D] (fp32, device).
+
+    Returns compress_select's dict plus recon [B,K,D] and sqerr [B,K]."""
+    L = load()
+    N, D = candidates.shape
+    B, K, _ = side_info.shape
+    for x in (candidates, source, side_info):
+        if not x.is_cuda or x.dtype != torch.float32 or not x.is_contiguous():
+            raise GlsError("candidates, source and side_info must be contiguous float32 device tensors")
+    assert tuple(source.shape) == (B, D) and tuple(side_info.shape) == (B, K, D)
+    dev = candidates.device
+    bsb = 0
+    if bins is not None:
+        if bins.dtype != torch.uint8 or not bins.is_contiguous():
+            raise GlsError("bins must be contiguous uint8")
+        bsb = 0 if bins.dim() == 1 else N
+    nz = _noise(seed, seq_base, seq_ids, pos_base, spec, rounds, noise_flags)
+    if out is None:
+        out = dict(enc_index=torch.empty((B,), dtype=torch.int32, device=dev),
+                   message=torch.empty((B,), dtype=torch.uint8, device=dev),
+                   dec_index=torch.full((B, K), -1, dtype=torch.int32, device=dev),
+                   match=torch.zeros((B,), dtype=torch.uint8, device=dev),
+                   scores=torch.full((B, 1 + K), float("nan"), dtype=torch.float32, device=dev)
+                   if want_scores else None,
+                   recon=torch.empty((B, K, D), dtype=torch.float32, device=dev),
+                   sqerr=torch.empty((B, K), dtype=torch.float32, device=dev))
+    workspace = _workspace(workspace, compress_gaussian_workspace_bytes(B, K, N), dev)
+    _check(L.gls_compress_gaussian(
+        candidates.data_ptr(), source.data_ptr(), side_info.data_ptr(), _ptr(bins), bsb, B, K, N, D,
+        float(s2_eta), float(s2_zeta), float(s2_prior), C.byref(nz), _ptr(out["enc_index"]),
+        _ptr(out["message"]), _ptr(out["dec_index"]), _ptr(out["match"]), _ptr(out.get("scores")),
+        _ptr(out.get("recon")), _ptr(out.get("sqerr")), workspace.data_ptr(), workspace.numel(),
         _ptr(status), _stream()))
     return out

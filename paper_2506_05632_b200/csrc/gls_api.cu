@@ -16,6 +16,7 @@
 #include "gls_group16.cuh"
 #include "gls_sweep4.cuh"
 #include "gls_topm.cuh"
+#include "gls_gauss.cuh"
 
 namespace gls {
 
@@ -220,7 +221,7 @@ __device__ __forceinline__ RowResult finalize_row(const SweepArgs& A, int row, i
       sk.c1 = (A.domain << 16) + ((uint32_t)code & 7u);
       tok = (int)((uint32_t)code >> 3);
     }
-    ex = exact_score<DT, SPEC, ROUNDS>(A, rowp, sk, tok, inv_t);
+    ex = exact_score<DT, SPEC, ROUNDS>(A, rowp, sk, tok, inv_t, b, k);
   }
   double lse = -CUDART_INF;
   if (lane == 2 && with_lse && lsum > 0.0) lse = (double)lm * (double)inv_t + log(lsum);
@@ -1207,6 +1208,176 @@ int gls_compress_select(const gls_rows_t* enc_logw, const gls_rows_t* dec_logw, 
   decoder_epilogue_kernel<<<(B + 127) / 128, 128, 0, st>>>(rowres_d, B, K, out_enc_index,
                                                           out_dec_index, out_match, out_scores);
   return cudaGetLastError() == cudaSuccess ? GLS_OK : GLS_ERR_CUDA;
+}
+
+}  // extern "C"
+
+// ------------------------------------------------------------------------------------------
+// Compression from the source (Appendix C with the Gaussian model of Appendix D.3).
+// ------------------------------------------------------------------------------------------
+namespace gls {
+
+// W_k = u_{X^(k)}, the MMSE reconstruction g(w, t) = (s2_zeta w + s2_eta t) / (s2_eta + s2_zeta +
+// s2_eta s2_zeta) per dimension, and its mean squared error against the source; a thread per (b, k).
+__global__ void gauss_recon_kernel(const float* __restrict__ u, const float* __restrict__ a,
+                                   const float* __restrict__ t, const int32_t* __restrict__ dec_index,
+                                   int BK, int K, int D, double s2_eta, double s2_zeta,
+                                   float* __restrict__ recon, float* __restrict__ sqerr) {
+  const int r = blockIdx.x * blockDim.x + threadIdx.x;
+  if (r >= BK) return;
+  const int b = r / K;
+  const int x = dec_index[r];
+  const double den = s2_eta + s2_zeta + s2_eta * s2_zeta;
+  double se = 0.0;
+  for (int d = 0; d < D; ++d) {
+    float g = CUDART_NAN_F;
+    if (x >= 0) {
+      const double w = (double)u[(long long)x * D + d];
+      const double gd = (s2_zeta * w + s2_eta * (double)t[(long long)r * D + d]) / den;
+      const double e = gd - (double)a[(long long)b * D + d];
+      se += e * e;
+      g = (float)gd;
+    }
+    if (recon) recon[(long long)r * D + d] = g;
+  }
+  if (sqerr) sqerr[r] = x >= 0 ? (float)(se / D) : CUDART_NAN_F;
+}
+
+struct GaussPlan {
+  int tiles, n_ranges, rows_per_range_enc, rows_per_range_dec;
+  size_t off_hints, off_partials, off_rows, total;
+};
+static GaussPlan make_gauss_plan(int B, int K, long long N) {
+  GaussPlan p;
+  p.tiles = (int)((N + kGTile - 1) / kGTile);
+  // enough CTAs for several waves over the machine, each with whole blocks of rows
+  long long want = (4LL * num_sms() + p.tiles - 1) / p.tiles;
+  if (want < 1) want = 1;
+  auto per_range = [&](long long rows) {
+    long long n = want;
+    const long long blocks = (rows + kGRows - 1) / kGRows;
+    if (n > blocks) n = blocks;
+    return (int)(((blocks + n - 1) / n) * kGRows);
+  };
+  p.rows_per_range_enc = per_range(B);
+  p.rows_per_range_dec = per_range((long long)B * K);
+  p.n_ranges = 0;  // set per pass by the caller
+  const size_t rows = (size_t)B * K;
+  p.off_hints = 0;
+  p.off_partials = align_up(rows * sizeof(uint32_t), 256);
+  p.off_rows = p.off_partials + align_up(rows * p.tiles * sizeof(Partial), 256);
+  p.total = p.off_rows + align_up(rows * sizeof(RowResult), 256);
+  return p;
+}
+
+}  // namespace gls
+
+extern "C" {
+
+size_t gls_compress_gaussian_workspace_bytes(int B, int K, int64_t N) {
+  if (B <= 0 || K <= 0 || K > gls::kGMaxK || N <= 0 || N >= (1LL << 28)) return 0;
+  return gls::make_gauss_plan(B, K, N).total;
+}
+
+int gls_compress_gaussian(const float* candidates, const float* source, const float* side_info,
+                          const uint8_t* bins, int64_t bins_stride_b, int B, int K, int64_t N, int D,
+                          double s2_eta, double s2_zeta, double s2_prior, const gls_noise_t* noise,
+                          int32_t* out_enc_index, uint8_t* out_message, int32_t* out_dec_index,
+                          uint8_t* out_match, float* out_scores, float* out_recon, float* out_sqerr,
+                          void* workspace, size_t workspace_bytes, uint32_t* device_status,
+                          void* stream) {
+  if (!candidates || !source || !side_info || !noise || !out_enc_index || !out_message ||
+      !out_dec_index || !out_match || B <= 0 || K <= 0 || N <= 0 || D <= 0)
+    return GLS_ERR_INVALID_ARG;
+  if (!(s2_eta > 0.0) || !(s2_zeta > 0.0) || !(s2_prior > 0.0) || !std::isfinite(s2_eta) ||
+      !std::isfinite(s2_zeta) || !std::isfinite(s2_prior))
+    return GLS_ERR_INVALID_ARG;
+  if (bins_stride_b != 0 && bins_stride_b < N) return GLS_ERR_INVALID_ARG;
+  if (K > kGMaxK || D > kGMaxD || N >= (1LL << 28) || (long long)B * K >= (1LL << 24))
+    return GLS_ERR_UNSUPPORTED;
+  if (((uintptr_t)candidates | (uintptr_t)source | (uintptr_t)side_info) % 4) return GLS_ERR_MISALIGNED;
+  SweepArgs A;
+  std::memset(&A, 0, sizeof(A));
+  for (int k = 0; k < K; ++k) A.inv_t[k] = 1.0f;
+  int spec;
+  int rc = fill_noise(A, noise, 1u, &spec);
+  if (rc != GLS_OK) return rc;
+  if (spec != 4) return GLS_ERR_UNSUPPORTED;
+  GaussPlan P = make_gauss_plan(B, K, N);
+  if (!workspace || workspace_bytes < P.total) return GLS_ERR_WORKSPACE;
+  cudaStream_t st = (cudaStream_t)stream;
+  char* ws = (char*)workspace;
+  A.gu = candidates;
+  A.ga = source;
+  A.gt = side_info;
+  A.gD = D;
+  A.g_s2_eta = s2_eta;
+  A.g_s2_zeta = s2_zeta;
+  A.g_s2_prior = s2_prior;
+  A.V = (int)N;
+  A.J = 1;
+  A.splits = 1;
+  A.parts = P.tiles;
+  A.hints = (uint32_t*)(ws + P.off_hints);
+  A.partials = (Partial*)(ws + P.off_partials);
+  RowResult* rowres = (RowResult*)(ws + P.off_rows);
+  const size_t smem = gauss_smem_bytes(D);
+  const bool r10 = A.rounds == 10;
+  const double var_dec = (1.0 + s2_eta) - 1.0 / (1.0 + s2_zeta);
+#define GAUSS_SWEEP(ENC, rows_, per_range_, scale_)                                              \
+  do {                                                                                           \
+    const int n_ranges = ((rows_) + (per_range_) - 1) / (per_range_);                            \
+    if (cudaMemsetAsync(A.hints, 0, (size_t)(rows_) * sizeof(uint32_t), st) != cudaSuccess ||    \
+        cudaMemsetAsync(A.partials, 0xff, (size_t)(rows_) * P.tiles * sizeof(Partial), st) !=    \
+            cudaSuccess)                                                                         \
+      return GLS_ERR_CUDA;                                                                       \
+    if (r10) {                                                                                   \
+      cudaFuncSetAttribute(gauss_sweep_kernel<10, ENC>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem); \
+      gauss_sweep_kernel<10, ENC><<<P.tiles * n_ranges, kGWarps * 32, smem, st>>>(               \
+          A, n_ranges, (per_range_), (long long)N, (float)(scale_));                             \
+    } else {                                                                                     \
+      cudaFuncSetAttribute(gauss_sweep_kernel<0, ENC>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem); \
+      gauss_sweep_kernel<0, ENC><<<P.tiles * n_ranges, kGWarps * 32, smem, st>>>(                \
+          A, n_ranges, (per_range_), (long long)N, (float)(scale_));                             \
+    }                                                                                            \
+    if (cudaGetLastError() != cudaSuccess) return GLS_ERR_CUDA;                                  \
+  } while (0)
+  // encoder: one race per source sample over candidates and the K streams, with the log-sum-exp
+  A.K = 1;
+  A.multi_k = K;
+  A.rows = B;
+  A.g_dec = 0;
+  GAUSS_SWEEP(true, B, P.rows_per_range_enc, 1.0 / std::sqrt(2.0 * s2_eta));
+  cudaError_t err = r10 ? launch_finalize_t<kF32, 4, 10>(A, B, true, rowres, nullptr, nullptr, nullptr, st)
+                        : launch_finalize_t<kF32, 4, 0>(A, B, true, rowres, nullptr, nullptr, nullptr, st);
+  if (err != cudaSuccess) return GLS_ERR_CUDA;
+  encoder_epilogue_kernel<<<(B + 127) / 128, 128, 0, st>>>(rowres, B, 1, bins, bins_stride_b,
+                                                          out_enc_index, out_message, out_scores,
+                                                          device_status, 1 + K);
+  if (cudaGetLastError() != cudaSuccess) return GLS_ERR_CUDA;
+  // decoders: row (b, k) under stream k, restricted to the candidates labelled M
+  A.K = K;
+  A.multi_k = 0;
+  A.rows = B * K;
+  A.g_dec = 1;
+  A.bins = bins;
+  A.bins_sb = bins_stride_b;
+  A.msg = out_message;
+  GAUSS_SWEEP(false, B * K, P.rows_per_range_dec, 1.0 / std::sqrt(2.0 * var_dec));
+#undef GAUSS_SWEEP
+  err = r10 ? launch_finalize_t<kF32, 4, 10>(A, B * K, false, rowres, nullptr, nullptr, device_status, st)
+            : launch_finalize_t<kF32, 4, 0>(A, B * K, false, rowres, nullptr, nullptr, device_status, st);
+  if (err != cudaSuccess) return GLS_ERR_CUDA;
+  decoder_epilogue_kernel<<<(B + 127) / 128, 128, 0, st>>>(rowres, B, K, out_enc_index, out_dec_index,
+                                                          out_match, out_scores);
+  if (cudaGetLastError() != cudaSuccess) return GLS_ERR_CUDA;
+  if (out_recon || out_sqerr) {
+    gauss_recon_kernel<<<(B * K + 127) / 128, 128, 0, st>>>(candidates, source, side_info, out_dec_index,
+                                                           B * K, K, D, s2_eta, s2_zeta, out_recon,
+                                                           out_sqerr);
+    if (cudaGetLastError() != cudaSuccess) return GLS_ERR_CUDA;
+  }
+  return GLS_OK;
 }
 
 }  // extern "C"

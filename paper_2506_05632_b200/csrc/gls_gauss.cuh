@@ -1,0 +1,397 @@
+// gls_gauss.cuh -- compression from the source: the races of Sec. 5.1 over importance weights
+// that are computed on the fly (Appendix C of arXiv 2506.05632 with the Gaussian model of
+// Sec. 5.2 / Appendix D.3, applied per dimension), instead of being streamed from memory.
+//
+// The log-weight of candidate u_i for a row with mean mu and variance v is
+//     sum_d -(u_id - mu_d)^2 / (2 v) + u_id^2 / (2 s2_prior)
+// (encoder row b: mu = a_b, v = s2_eta; decoder row (b, k): mu = t_bk / s2_T, v = s2_W - 1 / s2_T).
+// Streaming precomputed weights reads 4 bytes per (row, candidate); computing them needs the
+// D coordinates of the candidate, which are the same for every row.  So the loop nest is turned
+// around: a CTA takes a tile of 2048 candidates (the 128 noise groups that 32 generator calls
+// serve), keeps its coordinates in shared memory, pre-scaled by 1 / sqrt(2 v), and walks over the
+// rows, four at a time.  Per row block a lane computes the 4 x 16 weights of its group of 16
+// candidates in two-wide fp32 arithmetic (one add and one multiply-add per coordinate and pair),
+// then the group test of the sweep (gls_sweep4.cuh) decides from the coarse word of the group's
+// minimum whether any of the 16 can still win; candidate groups are examined in batches, exactly
+// as in the sweep, and the leaders are re-scored in fp64 by the reduction kernel, which
+// recomputes their weights from the source in fp64.  Per (row, tile) one partial result is
+// written (only if the tile produced a candidate, or carries a share of the log-sum-exp).
+#pragma once
+#include "gls_sweep4.cuh"
+
+namespace gls {
+
+constexpr int kGTile = 2048;        // candidates per tile = 128 groups of 16
+constexpr int kGWarps = 4;          // warp w owns groups 32 w .. 32 w + 31 of the tile
+constexpr int kGRows = 4;           // rows per block
+constexpr int kGPad = 20;           // floats per group in shared memory (16 + 4: no bank conflicts)
+constexpr int kGMaxD = 16;
+constexpr int kGMaxK = 8;
+constexpr int kGQueue = 32 + kGRows * kGMaxK;  // a block adds at most rows x streams entries per lane group
+
+struct GaussRowCtx {  // one row of the current block
+  uint32_t c1, pos, seq;  // noise stream (c1 without the stream number in the encoder pass)
+  uint32_t m_enc;         // ordered code of the row's bound
+  int row, b;             // row number (-1: past the end), source sample
+  int msg;                // label a candidate must carry (decoder pass with labels)
+};
+struct __align__(16) GaussEntry {  // a queued group: coarse word, group | stream << 28, row slot, weights
+  uint32_t w, g, slot, pad;
+  float a[16];
+};
+struct __align__(16) GaussShared {
+  float mu[kGMaxD][kGRows];                       // scaled means of the block's rows
+  GaussRowCtx ctx[kGRows];
+  uint32_t xw[kGRows * kGMaxK][4][32];            // coarse words: [stream-row][word][lane]
+  Top2 best[kGWarps][kGRows];                     // per warp and row slot
+  float lse_m[kGWarps][kGRows], lse_s[kGWarps][kGRows];
+  GaussEntry queue[kGWarps][kGQueue];
+  float us[1];                                    // [(D + 1)][128 * kGPad], D-th plane: |u|^2 / (2 s2_prior)
+};
+__host__ __device__ inline size_t gauss_smem_bytes(int D) {
+  return sizeof(GaussShared) + (size_t)(D + 1) * 128 * kGPad * sizeof(float);
+}
+
+// Batched evaluation of queued groups (cf. s4_flush): lane l < n takes entry first + l.  Entries
+// may belong to different rows of the block; each lane works under its own row's key and bound.
+// The lanes' results are merged per row slot into sh.best[warp][slot]; improved bounds go to the
+// row's context and to its hint word.
+template <int ROUNDS, bool ENC>
+__device__ __noinline__ void gauss_flush(const SweepArgs& A, GaussShared& sh, int first, int n) {
+  const int lane = threadIdx.x & 31;
+  const int warp = threadIdx.x >> 5;
+  constexpr float c2 = kLog2e;
+  uint32_t msk = 0u, g = 0u, ks = 0u;
+  int loc = -1, slot = 0;
+  float M = 1.f, lg2M = 0.f, nm = CUDART_INF_F;
+  const GaussEntry& e = sh.queue[warp][first + (lane < n ? lane : 0)];
+  Top2 b;
+  top2_init(b);
+  float lower = -CUDART_INF_F;
+  const uint8_t* bins = nullptr;
+  GaussRowCtx cx = sh.ctx[0];
+  if (lane < n) {
+    slot = (int)e.slot;
+    cx = sh.ctx[slot];
+    bins = A.bins ? A.bins + A.bins_sb * cx.b : nullptr;
+    g = e.g;
+    ks = g >> 28;
+    g &= 0x0fffffffu;
+    uint32_t f[4];
+    philox4x32<ROUNDS>(A.rk, A.rounds, g, cx.c1 + ks + (2u << 16), cx.pos, cx.seq, f);
+    loc = (int)((f[0] >> 16) & 15u);
+    M = exp1_from_word(e.w, ((float)(f[0] & 0xffffu) + 0.5f) * 0x1p-16f) * 0.0625f;
+    lg2M = lg2_approx(M);
+    nm = filter_offset(dec_ordered(cx.m_enc));
+    // the candidate at the minimum has S = M exactly: its score bounds the row's best at once
+    const long long il = ((long long)g << 4) + loc;
+    const float a = e.a[loc];
+    if (a > -CUDART_INF_F && a < CUDART_INF_F &&
+        (ENC || bins == nullptr || (int)__ldg(bins + il) == cx.msg)) {
+      const float ln_s = logf(M);
+      const float s = a - ln_s;
+      nm = fminf(nm, filter_offset(s - score_slack(s, ln_s)));
+    }
+    const float nmM = nm - lg2M + 0x1p-10f;
+#pragma unroll
+    for (int t = 0; t < 16; ++t) {
+      const float at = e.a[t];
+      if (at < CUDART_INF_F && fmaf(at, c2, nmM) >= 0.f) msk |= 1u << t;  // false for NaN
+    }
+  }
+  while (__any_sync(0xffffffffu, msk != 0u)) {
+    if (msk != 0u) {
+      const int t = __ffs(msk) - 1;
+      msk &= msk - 1u;
+      const long long i = ((long long)g << 4) + t;
+      const float a = e.a[t];
+      if (fmaf(a, c2, nm - lg2M + 0x1p-10f) >= 0.f &&
+          (ENC || bins == nullptr || (int)__ldg(bins + i) == cx.msg)) {
+        float s_noise = M;
+        if (t != loc) {
+          uint32_t f[4];
+          philox4x32<ROUNDS>(A.rk, A.rounds, (uint32_t)(i >> 2), cx.c1 + ks + (4u << 16), cx.pos,
+                             cx.seq, f);
+          const uint32_t u = (i & 2) ? ((i & 1) ? f[3] : f[2]) : ((i & 1) ? f[1] : f[0]);
+          s_noise = M + exp1_from_word(u, 0.5f);
+        }
+        const float ln_s = logf(s_noise);
+        const float s = a - ln_s;
+        // encoder pass: the candidate is (token, stream), ordered by token first
+        top2_offer(b, s, ENC ? (int)(((uint32_t)i << 3) | ks) : (int)i);
+        const float lo = s - score_slack(s, ln_s);
+        lower = fmaxf(lower, lo);
+        nm = fminf(nm, filter_offset(lo));
+      }
+    }
+  }
+  // merge the lanes' results per row slot
+#pragma unroll
+  for (int r = 0; r < kGRows; ++r) {
+    Top2 m = b;
+    float lo = lower;
+    if (!(lane < n && slot == r)) {
+      top2_init(m);
+      lo = -CUDART_INF_F;
+    }
+    if (!__any_sync(0xffffffffu, m.i1 >= 0)) continue;
+    top2_warp_merge(m);
+    const uint32_t enc = __reduce_max_sync(0xffffffffu, enc_ordered(lo));
+    if (lane == 0) {
+      Top2 cur = sh.best[warp][r];
+      top2_offer(cur, m.s1, m.i1);
+      top2_offer(cur, m.s2, m.i2);
+      sh.best[warp][r] = cur;
+      const uint32_t old = atomicMax(&sh.ctx[r].m_enc, enc);
+      if (enc > old) atomicMax(A.hints + sh.ctx[r].row, enc);
+    }
+  }
+  __syncwarp();
+}
+
+// ------------------------------------------------------------------------------------------
+// The kernel.  Grid: tiles x row ranges.  ENC: rows are source samples b, each raced under the
+// A.multi_k noise streams at once, with the log-sum-exp of the weights; otherwise rows are
+// decoder rows (b, k) under stream k, restricted to the candidates labelled A.msg[b].
+//   row range r of n_ranges covers rows [r * rows_per_range, ...); blockIdx.x = tile * n_ranges + r
+// ------------------------------------------------------------------------------------------
+template <int ROUNDS, bool ENC>
+__global__ void __launch_bounds__(kGWarps * 32, 1)
+gauss_sweep_kernel(const __grid_constant__ SweepArgs A, int n_ranges, int rows_per_range,
+                   long long N, float scale /* 1 / sqrt(2 v) of this pass */) {
+  GaussShared& sh = *reinterpret_cast<GaussShared*>(gls_smem_raw);
+  const int lane = threadIdx.x & 31;
+  const int warp = threadIdx.x >> 5;
+  const int D = A.gD;
+  const int K = A.K;
+  const int tile = blockIdx.x / n_ranges;
+  const int range = blockIdx.x - tile * n_ranges;
+  const int row_lo = range * rows_per_range;
+  const int row_hi = min(A.rows, row_lo + rows_per_range);
+  const long long cand0 = (long long)tile * kGTile;
+  const int n_streams = ENC ? A.multi_k : 1;
+  float* const us = sh.us;
+  constexpr int kPlane = 128 * kGPad;
+
+  // ---- the tile's coordinates, scaled, to shared memory; plane D holds |u|^2 / (2 s2_prior),
+  //      -inf for candidates past the end (their weights become -inf)
+  {
+    const float half_inv_prior = (float)(0.5 / A.g_s2_prior);
+    for (int c = threadIdx.x; c < kGTile; c += kGWarps * 32) {
+      const long long i = cand0 + c;
+      const int at = (c >> 4) * kGPad + (c & 15);
+      float nrm = 0.f;
+      for (int d = 0; d < D; ++d) {
+        const float x = i < N ? __ldg(A.gu + i * D + d) : 0.f;
+        nrm = fmaf(x, x, nrm);
+        us[d * kPlane + at] = x * scale;
+      }
+      us[D * kPlane + at] = i < N ? nrm * half_inv_prior : -CUDART_INF_F;
+    }
+  }
+  // what the next block needs: scaled means, contexts, coarse words
+  auto prepare = [&](int row0) {
+    for (int idx = threadIdx.x; idx < kGRows * D; idx += kGWarps * 32) {
+      const int r = idx / D, d = idx - r * D;
+      const int row = row0 + r;
+      float m = 0.f;
+      if (row < row_hi) {
+        if (ENC) m = __ldg(A.ga + (long long)row * D + d);
+        else m = __ldg(A.gt + (long long)row * D + d) / (float)(1.0 + A.g_s2_zeta);
+      }
+      sh.mu[d][r] = m * scale;
+    }
+    if (threadIdx.x < kGRows) {
+      const int r = threadIdx.x;
+      const int row = row0 + r;
+      GaussRowCtx cx;
+      cx.row = row < row_hi ? row : -1;
+      const int b = ENC ? row : row / K;
+      const int k = ENC ? 0 : row - b * K;
+      cx.b = b;
+      cx.c1 = ((uint32_t)k & A.kmask) | (A.domain << 16);
+      cx.pos = A.pos_base;
+      cx.seq = 0u;
+      cx.msg = 0;
+      cx.m_enc = 0u;
+      if (cx.row >= 0) {
+        cx.seq = A.seq_ids ? __ldg(A.seq_ids + b) : A.seq_base + (uint32_t)b;
+        cx.msg = (!ENC && A.bins && A.msg) ? (int)__ldg(A.msg + b) : 0;
+        cx.m_enc = __ldcg(A.hints + row);
+      }
+      sh.ctx[r] = cx;
+      top2_init(sh.best[0][r]);
+      top2_init(sh.best[1][r]);
+      top2_init(sh.best[2][r]);
+      top2_init(sh.best[3][r]);
+    }
+  };
+  // coarse words of the block's stream-rows: warp w computes stream-rows sr = w, w + 4, ...
+  auto coarse_words = [&](int row0) {
+    for (int sr = warp; sr < kGRows * n_streams; sr += kGWarps) {
+      const int r = sr / n_streams, ks = sr - r * n_streams;
+      const int row = row0 + r;
+      if (row >= row_hi) continue;
+      const int b = ENC ? row : row / K;
+      const int k = ENC ? 0 : row - b * K;
+      const uint32_t c1 = ((ENC ? (uint32_t)ks : (uint32_t)k) & A.kmask) | (A.domain << 16);
+      const uint32_t seq = A.seq_ids ? __ldg(A.seq_ids + b) : A.seq_base + (uint32_t)b;
+      uint32_t cw[4];
+      philox4x32<ROUNDS>(A.rk, A.rounds, ((uint32_t)tile << 5) | (uint32_t)lane, c1, A.pos_base, seq, cw);
+      sh.xw[sr][0][lane] = cw[0];
+      sh.xw[sr][1][lane] = cw[1];
+      sh.xw[sr][2][lane] = cw[2];
+      sh.xw[sr][3][lane] = cw[3];
+    }
+  };
+  prepare(row_lo);
+  coarse_words(row_lo);
+  __syncthreads();
+
+  const int gl = warp * 32 + lane;                      // the lane's group within the tile
+  const uint32_t gidx = (uint32_t)tile * 128u + (uint32_t)gl;  // ... and in the whole row
+  const float* const ug = us + gl * kGPad;
+  GaussEntry* const queue = sh.queue[warp];
+  const bool group_in_range = cand0 + (long long)gl * 16 < N;
+
+  for (int row0 = row_lo; row0 < row_hi; row0 += kGRows) {
+    // ---- weights of the lane's 16 candidates for the block's four rows -----------------------
+    unsigned long long acc[kGRows][8];
+#pragma unroll
+    for (int r = 0; r < kGRows; ++r)
+#pragma unroll
+      for (int p = 0; p < 8; ++p) acc[r][p] = 0ull;
+#pragma unroll 2
+    for (int d = 0; d < D; ++d) {
+      const float4 m4 = *reinterpret_cast<const float4*>(&sh.mu[d][0]);
+      unsigned long long up[8];
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        const float4 v = *reinterpret_cast<const float4*>(ug + d * kPlane + 4 * q);
+        up[2 * q] = pack_f32x2(v.x, v.y);
+        up[2 * q + 1] = pack_f32x2(v.z, v.w);
+      }
+      const float mr[kGRows] = {m4.x, m4.y, m4.z, m4.w};
+#pragma unroll
+      for (int r = 0; r < kGRows; ++r) {
+        const unsigned long long nm2 = pack_f32x2(-mr[r], -mr[r]);
+#pragma unroll
+        for (int p = 0; p < 8; ++p) {
+          const unsigned long long diff = add_f32x2(up[p], nm2);
+          acc[r][p] = fma_f32x2(diff, diff, acc[r][p]);
+        }
+      }
+    }
+    float pn[16];
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      const float4 v = *reinterpret_cast<const float4*>(ug + D * kPlane + 4 * q);
+      pn[4 * q] = v.x; pn[4 * q + 1] = v.y; pn[4 * q + 2] = v.z; pn[4 * q + 3] = v.w;
+    }
+    // ---- per row: group maximum, log-sum-exp (encoder), group test per stream ------------------
+    int qn = 0;
+#pragma unroll
+    for (int r = 0; r < kGRows; ++r) {
+      const GaussRowCtx cx = sh.ctx[r];
+      if (cx.row < 0) continue;  // uniform over the CTA
+      float wgt[16];
+      float amax = -CUDART_INF_F;
+#pragma unroll
+      for (int p = 0; p < 8; ++p) {
+        float s0, s1;
+        unpack_f32x2(acc[r][p], s0, s1);
+        wgt[2 * p] = pn[2 * p] - s0;
+        wgt[2 * p + 1] = pn[2 * p + 1] - s1;
+        amax = fmaxf(amax, fmaxf(wgt[2 * p], wgt[2 * p + 1]));
+      }
+      if (ENC) {
+        // the lane's share of sum_i exp(weight_i), relative to its own maximum; lanes are merged
+        // with the usual rescaling
+        float lm = amax, ls = 0.f;
+        if (amax > -CUDART_INF_F) {
+#pragma unroll
+          for (int t = 0; t < 16; ++t) ls += ex2_approx((wgt[t] - amax) * kLog2e);
+        } else {
+          lm = kGroupLseFloor;
+        }
+        float wm = lm;
+#pragma unroll
+        for (int dd = 16; dd > 0; dd >>= 1) wm = fmaxf(wm, __shfl_xor_sync(0xffffffffu, wm, dd));
+        ls *= ex2_approx((lm - wm) * kLog2e);
+#pragma unroll
+        for (int dd = 16; dd > 0; dd >>= 1) ls += __shfl_xor_sync(0xffffffffu, ls, dd);
+        if (lane == 0) {
+          sh.lse_m[warp][r] = wm;
+          sh.lse_s[warp][r] = ls;
+        }
+      }
+      const float nm4 = filter_offset(dec_ordered(cx.m_enc)) + 4.0f;
+      const float nms = scaled_offset(nm4);
+      const float thr = exp2_upper_from_scaled(amax, kLog2e * (1.0f / 126.0f), nms);
+      for (int ks = 0; ks < n_streams; ++ks) {
+        const uint32_t w = sh.xw[r * n_streams + ks][warp][lane];
+        const bool pass = group_in_range && coarse_lower(w) <= thr;
+        const unsigned bal = __ballot_sync(0xffffffffu, pass);
+        if (bal != 0u) {
+          if (pass) {
+            GaussEntry& e = queue[qn + __popc(bal & ((1u << lane) - 1u))];
+            e.w = w;
+            e.g = gidx | (((uint32_t)ks & A.kmask) << 28);
+            e.slot = (uint32_t)r;
+#pragma unroll
+            for (int t = 0; t < 16; ++t) e.a[t] = wgt[t];
+          }
+          qn += __popc(bal);
+          if (qn >= 32) {  // a full batch: evaluate it now (rare after the first rows)
+            __syncwarp();
+            qn -= 32;
+            gauss_flush<ROUNDS, ENC>(A, sh, qn, 32);
+          }
+        }
+      }
+    }
+    while (qn > 0) {
+      __syncwarp();
+      const int nb = min(qn, 32);
+      qn -= nb;
+      gauss_flush<ROUNDS, ENC>(A, sh, qn, nb);
+    }
+    __syncthreads();  // every warp's results for this block are in shared memory
+    // ---- warp r merges row slot r and writes its partial result; then the next block is set up
+    {
+      const int r = warp;
+      const int row = row0 + r;
+      if (row < row_hi && lane == 0) {
+        Top2 m = sh.best[0][r];
+        float lm = kGroupLseFloor, ls = 0.f;
+#pragma unroll
+        for (int w2 = 1; w2 < kGWarps; ++w2) {
+          top2_offer(m, sh.best[w2][r].s1, sh.best[w2][r].i1);
+          top2_offer(m, sh.best[w2][r].s2, sh.best[w2][r].i2);
+        }
+        if (ENC) {
+#pragma unroll
+          for (int w2 = 0; w2 < kGWarps; ++w2) lm = fmaxf(lm, sh.lse_m[w2][r]);
+#pragma unroll
+          for (int w2 = 0; w2 < kGWarps; ++w2)
+            ls += sh.lse_s[w2][r] * ex2_approx((sh.lse_m[w2][r] - lm) * kLog2e);
+        }
+        if (m.i1 >= 0 || (ENC && ls > 0.f)) {
+          Partial pr;
+          pr.s1 = m.s1; pr.i1 = m.i1; pr.s2 = m.s2; pr.i2 = m.i2;
+          pr.lm = lm; pr.ls = ls; pr.pad0 = 0; pr.pad1 = 0;
+          A.partials[(long long)row * A.parts + tile] = pr;
+        }
+      }
+    }
+    __syncthreads();  // the merge has read the block's results
+    if (row0 + kGRows < row_hi) {
+      prepare(row0 + kGRows);
+      coarse_words(row0 + kGRows);
+    }
+    __syncthreads();
+  }
+  asm volatile("griddepcontrol.launch_dependents;");
+}
+
+}  // namespace gls

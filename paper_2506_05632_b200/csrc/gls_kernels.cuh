@@ -85,6 +85,15 @@ struct SweepArgs {
   const uint8_t* bins;    // NULL, or candidate labels
   long long bins_sb;
   const uint8_t* msg;     // [B] label a candidate must carry (decoder side)
+  // Rows that are computed, not read (compression from the source, Appendix C with the Gaussian
+  // model of Appendix D.3): candidates gu [N][gD], sources ga [B][gD], side information
+  // gt [B][K][gD]; gu == NULL otherwise.  g_dec: the rows are decoder rows (b, k), else encoder
+  // rows b.
+  const float* gu;
+  const float* ga;
+  const float* gt;
+  int gD, g_dec;
+  double g_s2_eta, g_s2_zeta, g_s2_prior;
   uint32_t* hints;        // [rows] ordered-int encoding of a lower bound on the row's best score
   Partial* partials;      // [n_items]
 };
@@ -222,11 +231,32 @@ __device__ __forceinline__ float load_logit(const void* row, long long i) {
   return __uint_as_float((uint32_t)__ldg((const unsigned short*)row + i) << 16);
 }
 
+// Importance log-weight of candidate i for source sample b (decoder k if A.g_dec) in fp64
+// (Appendix C; Gaussian model of Appendix D.3 per dimension; terms common to a row dropped):
+//   encoder  sum_d -(u - a)^2 / (2 s2_eta) + u^2 / (2 s2_prior)
+//   decoder  sum_d -(u - t / s2_T)^2 / (2 (s2_W - 1 / s2_T)) + u^2 / (2 s2_prior)
+__device__ __forceinline__ double gauss_logw64(const SweepArgs& A, int b, int k, long long i) {
+  const double s2T = 1.0 + A.g_s2_zeta, s2W = 1.0 + A.g_s2_eta;
+  const double var = A.g_dec ? s2W - 1.0 / s2T : A.g_s2_eta;
+  const float* mu = A.g_dec ? A.gt + ((long long)b * A.K + k) * A.gD : A.ga + (long long)b * A.gD;
+  const float* u = A.gu + i * A.gD;
+  double acc = 0.0;
+  for (int d = 0; d < A.gD; ++d) {
+    const double x = (double)__ldg(u + d);
+    const double m = A.g_dec ? (double)__ldg(mu + d) / s2T : (double)__ldg(mu + d);
+    const double diff = x - m;
+    acc += -(diff * diff) / (2.0 * var) + (x * x) / (2.0 * A.g_s2_prior);
+  }
+  return acc;
+}
+
 // Exact score of one token in fp64: logit/T - ln S, S = -log1p(-v)  (Sec. 3: S = -ln U, U = 1 - v).
+// (b, k) are only used for rows that are computed from the source.
 template <int DT, int SPEC, int ROUNDS>
 __device__ __noinline__ double exact_score(const SweepArgs& A, const void* row,
-                                           const StreamKey& sk, int i, float inv_t) {
-  const double a = (double)load_logit<DT>(row, i) * (double)inv_t;
+                                           const StreamKey& sk, int i, float inv_t, int b, int k) {
+  const double a = A.gu != nullptr ? gauss_logw64(A, b, k, i)
+                                   : (double)load_logit<DT>(row, i) * (double)inv_t;
   return a - log(noise_exact<SPEC, ROUNDS>(A, sk, i));
 }
 
