@@ -46,6 +46,7 @@ struct __align__(16) GaussShared {
   Top2 best[kGWarps][kGRows];                     // per warp and row slot
   float lse_m[kGWarps][kGRows], lse_s[kGWarps][kGRows];
   GaussEntry queue[kGWarps][kGQueue];
+  uint32_t labels[128][4];                        // the tile's bin labels, 16 bytes per group
   float us[1];                                    // [(D + 1)][128 * kGPad], D-th plane: |u|^2 / (2 s2_prior)
 };
 __host__ __device__ inline size_t gauss_smem_bytes(int D) {
@@ -189,9 +190,25 @@ gauss_sweep_kernel(const __grid_constant__ SweepArgs A, int n_ranges, int rows_p
       us[D * kPlane + at] = i < N ? nrm * half_inv_prior : -CUDART_INF_F;
     }
   }
-  // what the next block needs: scaled means, contexts, coarse words
-  auto prepare = [&](int row0) {
-    for (int idx = threadIdx.x; idx < kGRows * D; idx += kGWarps * 32) {
+  // decoder pass with one label array for all samples: the tile's labels, so that the group test
+  // can look at the eligible candidates only (with L_max labels the best eligible score lies about
+  // ln L_max below the best overall, and that many more groups would pass a test on all sixteen)
+  const bool use_labels = !ENC && A.bins != nullptr && A.bins_sb == 0;
+  if (use_labels) {
+    for (int c = threadIdx.x; c < kGTile; c += kGWarps * 32) {
+      const long long i = cand0 + c;
+      reinterpret_cast<uint8_t*>(&sh.labels[0][0])[c] = i < N ? __ldg(A.bins + i) : (uint8_t)0;
+    }
+  }
+  // What the next block needs: scaled means, contexts, coarse words.  The global loads are issued
+  // early (fetch, before the arithmetic of the current block) and their values parked in a few
+  // registers; commit writes them to shared memory once the current block is done with it.
+  float pf_mu[1] = {0.f};  // kGRows * D <= 64 values, one per thread
+  uint32_t pf_seq = 0u, pf_hint = 0u;
+  int pf_msg = 0;
+  auto fetch = [&](int row0) {
+    const int idx = threadIdx.x;
+    if (idx < kGRows * D) {
       const int r = idx / D, d = idx - r * D;
       const int row = row0 + r;
       float m = 0.f;
@@ -199,7 +216,23 @@ gauss_sweep_kernel(const __grid_constant__ SweepArgs A, int n_ranges, int rows_p
         if (ENC) m = __ldg(A.ga + (long long)row * D + d);
         else m = __ldg(A.gt + (long long)row * D + d) / (float)(1.0 + A.g_s2_zeta);
       }
-      sh.mu[d][r] = m * scale;
+      pf_mu[0] = m * scale;
+    }
+    if (threadIdx.x < kGRows) {
+      const int row = row0 + threadIdx.x;
+      if (row < row_hi) {
+        const int b = ENC ? row : row / K;
+        pf_seq = A.seq_ids ? __ldg(A.seq_ids + b) : A.seq_base + (uint32_t)b;
+        pf_msg = (!ENC && A.bins && A.msg) ? (int)__ldg(A.msg + b) : 0;
+        pf_hint = __ldcg(A.hints + row);
+      }
+    }
+  };
+  auto commit = [&](int row0) {
+    const int idx = threadIdx.x;
+    if (idx < kGRows * D) {
+      const int r = idx / D, d = idx - r * D;
+      sh.mu[d][r] = pf_mu[0];
     }
     if (threadIdx.x < kGRows) {
       const int r = threadIdx.x;
@@ -211,14 +244,9 @@ gauss_sweep_kernel(const __grid_constant__ SweepArgs A, int n_ranges, int rows_p
       cx.b = b;
       cx.c1 = ((uint32_t)k & A.kmask) | (A.domain << 16);
       cx.pos = A.pos_base;
-      cx.seq = 0u;
-      cx.msg = 0;
-      cx.m_enc = 0u;
-      if (cx.row >= 0) {
-        cx.seq = A.seq_ids ? __ldg(A.seq_ids + b) : A.seq_base + (uint32_t)b;
-        cx.msg = (!ENC && A.bins && A.msg) ? (int)__ldg(A.msg + b) : 0;
-        cx.m_enc = __ldcg(A.hints + row);
-      }
+      cx.seq = pf_seq;
+      cx.msg = pf_msg;
+      cx.m_enc = cx.row >= 0 ? pf_hint : 0u;
       sh.ctx[r] = cx;
       top2_init(sh.best[0][r]);
       top2_init(sh.best[1][r]);
@@ -244,8 +272,17 @@ gauss_sweep_kernel(const __grid_constant__ SweepArgs A, int n_ranges, int rows_p
       sh.xw[sr][3][lane] = cw[3];
     }
   };
-  prepare(row_lo);
-  coarse_words(row_lo);
+  // The blocks of rows are walked in a rotated order that differs from tile to tile: CTAs that run
+  // at the same time then work on different rows, so that a row's bound, once some tile has found
+  // one and published it in the row's hint word, is there for (almost) every other tile.  In
+  // lockstep every CTA of the first wave would meet every row without a bound and examine all of
+  // its groups.
+  const int n_blocks = (row_hi - row_lo + kGRows - 1) / kGRows;
+  const int rot = (int)(((uint32_t)tile * 2654435761u >> 8) % (uint32_t)n_blocks);
+  auto block_row = [&](int it) { return row_lo + ((it + rot) % n_blocks) * kGRows; };
+  fetch(block_row(0));
+  commit(block_row(0));
+  coarse_words(block_row(0));
   __syncthreads();
 
   const int gl = warp * 32 + lane;                      // the lane's group within the tile
@@ -254,7 +291,9 @@ gauss_sweep_kernel(const __grid_constant__ SweepArgs A, int n_ranges, int rows_p
   GaussEntry* const queue = sh.queue[warp];
   const bool group_in_range = cand0 + (long long)gl * 16 < N;
 
-  for (int row0 = row_lo; row0 < row_hi; row0 += kGRows) {
+  for (int it = 0; it < n_blocks; ++it) {
+    const int row0 = block_row(it);
+    if (it + 1 < n_blocks) fetch(block_row(it + 1));
     // ---- weights of the lane's 16 candidates for the block's four rows -----------------------
     unsigned long long acc[kGRows][8];
 #pragma unroll
@@ -274,12 +313,14 @@ gauss_sweep_kernel(const __grid_constant__ SweepArgs A, int n_ranges, int rows_p
       const float mr[kGRows] = {m4.x, m4.y, m4.z, m4.w};
 #pragma unroll
       for (int r = 0; r < kGRows; ++r) {
+        // all differences first, then all multiply-adds: with one warp per scheduler a dependent
+        // pair issued back to back would stall on its own latency
         const unsigned long long nm2 = pack_f32x2(-mr[r], -mr[r]);
+        unsigned long long diff[8];
 #pragma unroll
-        for (int p = 0; p < 8; ++p) {
-          const unsigned long long diff = add_f32x2(up[p], nm2);
-          acc[r][p] = fma_f32x2(diff, diff, acc[r][p]);
-        }
+        for (int p = 0; p < 8; ++p) diff[p] = add_f32x2(up[p], nm2);
+#pragma unroll
+        for (int p = 0; p < 8; ++p) acc[r][p] = fma_f32x2(diff[p], diff[p], acc[r][p]);
       }
     }
     float pn[16];
@@ -290,6 +331,11 @@ gauss_sweep_kernel(const __grid_constant__ SweepArgs A, int n_ranges, int rows_p
     }
     // ---- per row: group maximum, log-sum-exp (encoder), group test per stream ------------------
     int qn = 0;
+    uint32_t lab[4] = {0u, 0u, 0u, 0u};
+    if (use_labels) {
+      const uint4 lv = *reinterpret_cast<const uint4*>(&sh.labels[gl][0]);
+      lab[0] = lv.x; lab[1] = lv.y; lab[2] = lv.z; lab[3] = lv.w;
+    }
 #pragma unroll
     for (int r = 0; r < kGRows; ++r) {
       const GaussRowCtx cx = sh.ctx[r];
@@ -303,6 +349,17 @@ gauss_sweep_kernel(const __grid_constant__ SweepArgs A, int n_ranges, int rows_p
         wgt[2 * p] = pn[2 * p] - s0;
         wgt[2 * p + 1] = pn[2 * p + 1] - s1;
         amax = fmaxf(amax, fmaxf(wgt[2 * p], wgt[2 * p + 1]));
+      }
+      if (use_labels) {  // maximum over the candidates that carry the transmitted label
+        const uint32_t m4 = (uint32_t)cx.msg * 0x01010101u;
+        amax = -CUDART_INF_F;
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          const uint32_t eq = __vcmpeq4(lab[q], m4);  // 0xff per matching byte
+#pragma unroll
+          for (int t = 0; t < 4; ++t)
+            if (eq & (1u << (8 * t))) amax = fmaxf(amax, wgt[4 * q + t]);
+        }
       }
       if (ENC) {
         // the lane's share of sum_i exp(weight_i), relative to its own maximum; lanes are merged
@@ -385,9 +442,9 @@ gauss_sweep_kernel(const __grid_constant__ SweepArgs A, int n_ranges, int rows_p
       }
     }
     __syncthreads();  // the merge has read the block's results
-    if (row0 + kGRows < row_hi) {
-      prepare(row0 + kGRows);
-      coarse_words(row0 + kGRows);
+    if (it + 1 < n_blocks) {
+      commit(block_row(it + 1));
+      coarse_words(block_row(it + 1));
     }
     __syncthreads();
   }
