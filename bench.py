@@ -159,6 +159,28 @@ def run_reference(args):
     print(json.dumps(line))
 
 
+def run_reference_compress(args):
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    n, secs = 8, []
+    for i in range(args.warmup + args.steps):
+        base, dt = _cpu_baseline_compress(n)
+        if i >= args.warmup:
+            secs.append(dt)
+    value = n * len(secs) / sum(secs)
+    base["value"] = value
+    print(json.dumps({"impl": "reference", "metric": "compressed_source_samples_per_s", "value": value,
+                      "unit": "samples/s", "n_gpus": args.gpus, "steps": args.steps,
+                      "warmup": args.warmup, "ms_per_step": 1e3 * sum(secs) / len(secs),
+                      "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+                      "data": "synthetic",
+                      "config": {"workload": WORKLOAD_DESC["cfg5"],
+                                 "sample": "each step = %d source samples of the workload" % n},
+                      "cpu_baseline": base,
+                      "e2e": {"value": value, "unit": "samples/s", "h2d_bytes_per_step": 0,
+                              "d2h_bytes_per_step": 0}}))
+
+
 def _time_calls(fn, steps, warmup, flush=None):
     """CUDA-event timing on the current stream: total ms and per-call event pairs."""
     import torch
@@ -185,6 +207,169 @@ def _mark(lst):
         e = torch.cuda.Event(enable_timing=True)
         e.record()
         lst.append(e)
+
+
+def _fracs(nbytes, ms, peak):
+    gbs = nbytes / (ms * 1e-3) / 1e9
+    return {"ms": ms, "gbs": gbs, "frac_of_measured": gbs / peak, "frac_of_nominal_8TBs": gbs / 8000.0}
+
+
+def _event_ms(fn, steps, flush=None, warmup=3):
+    """Mean CUDA-event time of fn() over `steps` calls, each call in its own event pair (so that
+    an L2 flush between calls stays outside the brackets)."""
+    import torch
+
+    for _ in range(warmup):
+        fn()
+    torch.cuda.synchronize()
+    ev = []
+    for _ in range(steps):
+        if flush is not None:
+            flush.add_(1)
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        fn()
+        b.record()
+        ev.append((a, b))
+    torch.cuda.synchronize()
+    return statistics.mean(a.elapsed_time(b) for a, b in ev)
+
+
+def _measure_verify(cfg_id, steps, peak, spec=4):
+    """One verification workload: draft call, verify call, the fused call and (small inputs) a
+    replayed CUDA graph, L2-cold; Appendix B's variant of the verify call."""
+    import torch
+
+    import paper_2506_05632_b200 as pkg
+    from paper_2506_05632_b200 import pipeline, synth
+
+    w = synth.verify_workload(cfg_id, "cuda")
+    B, K, L, V = w.shape
+    buf = pipeline.StepBuffers(B, K, L, V)
+    kw = dict(inv_temp=w.inv_temp, seed=w.noise_seed, spec=spec, workspace=buf.workspace,
+              status=buf.status)
+    db = w.draft_logits.numel() * w.draft_logits.element_size()
+    tb = w.target_logits.numel() * w.target_logits.element_size()
+    small = db + tb < 512e6
+    flush = torch.zeros(64 << 20, dtype=torch.float32, device="cuda") if small else None
+
+    def draft():
+        pkg.draft_sample(w.draft_logits, out_tokens=buf.draft_tokens, out_scores=buf.draft_scores, **kw)
+
+    def verify():
+        pkg.target_sample_verify(w.target_logits, buf.draft_tokens, out=buf.out, **kw)
+
+    def fused():
+        pkg.draft_verify(w.draft_logits, w.target_logits, out_draft_tokens=buf.draft_tokens,
+                         out_draft_scores=buf.draft_scores, out=buf.out, **kw)
+
+    def verify_all():
+        pkg.target_sample_verify(w.target_logits, buf.draft_tokens, out=buf.out,
+                                 flags=pkg.COMBINE_ALL, **kw)
+
+    res = {"workload": WORKLOAD_DESC["cfg%d" % cfg_id],
+           "l2": "flushed between calls" if small else "inputs larger than L2",
+           "draft_call": _fracs(db, _event_ms(draft, steps, flush), peak),
+           "verify_call": _fracs(tb, _event_ms(verify, steps, flush), peak),
+           "one_call": _fracs(db + tb, _event_ms(fused, steps, flush), peak)}
+    res["verified_positions_per_s"] = B * L / (res["one_call"]["ms"] * 1e-3)
+    res["verify_call_appendix_b"] = _fracs(tb, _event_ms(verify_all, max(3, steps // 4), flush), peak)
+    if small:
+        res["l2_warm"] = {"draft_call_ms": _event_ms(draft, steps), "verify_call_ms": _event_ms(verify, steps),
+                          "one_call_ms": _event_ms(fused, steps)}
+        gs = pipeline.GraphedStep(w.draft_logits, w.target_logits, buf, inv_temp=w.inv_temp,
+                                  seed=w.noise_seed, spec=spec, fused=True)
+        res["one_call_cuda_graph_ms"] = _event_ms(gs.replay, steps, flush)
+    assert int(buf.status.item()) == 0
+    return res
+
+
+def _measure_autoregressive(steps, peak):
+    """The draft phase as it is issued: one position per call on configuration 4's rows
+    (B * K = 2048 rows of 152 064 tokens, 623 MB), L2 flushed between calls."""
+    import torch
+
+    import paper_2506_05632_b200 as pkg
+    from paper_2506_05632_b200 import synth
+
+    w = synth.verify_workload(4, "cuda", L=1)
+    B, K, L, V = w.shape
+    ws = torch.empty(pkg.workspace_bytes(B, K, 1, V), dtype=torch.uint8, device="cuda")
+    tok = torch.empty((B, K, 1), dtype=torch.int32, device="cuda")
+    sc = torch.empty((B, K, 1), dtype=torch.float32, device="cuda")
+    flush = torch.zeros(64 << 20, dtype=torch.float32, device="cuda")
+    nb = w.draft_logits.numel() * 2
+    ms = _event_ms(lambda: pkg.draft_sample(w.draft_logits, out_tokens=tok, out_scores=sc, workspace=ws,
+                                            inv_temp=w.inv_temp, seed=w.noise_seed), steps, flush)
+    r = _fracs(nb, ms, peak)
+    r["workload"] = "autoregressive draft call: B=256 K=8 J=1 V=152064 bf16 (2048 rows)"
+    return r
+
+
+def _measure_compress(steps, peak, B=None):
+    """Configuration 5: selection over streamed log-weights (decoders, encoder, whole call) and
+    the same selection from the source (weights computed in the kernels)."""
+    import torch
+
+    import paper_2506_05632_b200 as pkg
+    from paper_2506_05632_b200 import synth
+
+    w = synth.compress_workload("cuda", B=B or 512)
+    B, K, N = w.dec_logw.shape
+    D = w.candidates.shape[1]
+    ws = torch.empty(max(pkg.workspace_bytes(B, K, 1, N), pkg.compress_gaussian_workspace_bytes(B, K, N)),
+                     dtype=torch.uint8, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    out = pkg.compress_select(w.enc_logw, w.dec_logw, w.bins, seed=w.noise_seed, workspace=ws, status=status)
+    gout = pkg.compress_gaussian(w.candidates, w.source, w.side, w.bins, s2_eta=0.5, s2_zeta=0.25,
+                                 s2_prior=1.0, seed=w.noise_seed, workspace=ws, status=status)
+    ms_all = _event_ms(lambda: pkg.compress_select(w.enc_logw, w.dec_logw, w.bins, seed=w.noise_seed,
+                                                   workspace=ws, status=status, out=out), steps)
+    ms_enc = _event_ms(lambda: pkg.compress_select(w.enc_logw, None, w.bins, K=K, seed=w.noise_seed,
+                                                   workspace=ws, status=status), steps)
+    ms_src = _event_ms(lambda: pkg.compress_gaussian(w.candidates, w.source, w.side, w.bins, s2_eta=0.5,
+                                                     s2_zeta=0.25, s2_prior=1.0, seed=w.noise_seed,
+                                                     workspace=ws, status=status, out=gout),
+                       max(3, steps // 5))
+    eb, db = w.enc_logw.numel() * 4, w.dec_logw.numel() * 4
+    agree = float((out["enc_index"] == gout["enc_index"]).float().mean().item())
+    # from the source the path is bound by fp32 arithmetic: (1 + K) rows per sample, N candidates,
+    # D coordinates, one two-wide add and one two-wide multiply-add per coordinate and PAIR of
+    # candidates; peak = SMs x 4 schedulers x 32 lanes x clock, one instruction per lane and clock
+    lane_instr = B * (1 + K) * N * D * 2 / 2
+    alu_peak = 148 * 4 * 32 * 1.965e9
+    assert int(status.item()) == 0
+    return {"workload": WORKLOAD_DESC["cfg5"],
+            "whole_call": dict(_fracs(eb + db, ms_all, peak), source_samples_per_s=B / (ms_all * 1e-3)),
+            "decoders": _fracs(db, ms_all - ms_enc, peak),
+            "encoder": _fracs(eb, ms_enc, peak),
+            "from_source": {"ms": ms_src, "source_samples_per_s": B / (ms_src * 1e-3),
+                            "bytes_read": int(w.candidates.numel() * 4 + w.source.numel() * 4 + w.side.numel() * 4 + N),
+                            "bound": "alu", "lane_instructions": lane_instr,
+                            "achieved_lane_instr_per_s": lane_instr / (ms_src * 1e-3),
+                            "peak_lane_instr_per_s": alu_peak,
+                            "frac": lane_instr / (ms_src * 1e-3) / alu_peak,
+                            "encoder_index_agrees_with_streamed": agree},
+            "match_rate": float(out["match"].float().mean().item())}
+
+
+def _cpu_baseline_compress(samples):
+    """The oracle's compress_select on `samples` source samples of configuration 5."""
+    import torch
+
+    from oracle import gls_oracle
+    from paper_2506_05632_b200 import synth
+
+    dev = "cuda" if torch.cuda.is_available() else "cpu"
+    w = synth.compress_workload(dev, B=samples)
+    enc, dec, bins = w.enc_logw.cpu().numpy(), w.dec_logw.cpu().numpy(), w.bins.cpu().numpy()
+    del w
+    t0 = time.perf_counter()
+    gls_oracle.compress_select(enc, dec, bins, seed=synth.NOISE_SEED + 5)
+    dt = time.perf_counter() - t0
+    return {"value": samples / dt, "unit": "samples/s", "cores": gls_oracle.max_threads(),
+            "kind": "oracle", "sample": "%d of the workload's 512 source samples, one pass, %.1f s wall"
+                                        % (samples, dt)}, dt
 
 
 def run_ours(args):
@@ -267,7 +452,24 @@ def run_ours(args):
         dist.barrier()
     clocks = sampler.stop(t_begin, t_end) if rank == 0 else None
     draft_ms = statistics.mean(m[0].elapsed_time(m[1]) for m in marks)
-    verify_ms = statistics.mean(m[1].elapsed_time(m[2]) for m in marks)
+    verify_ms = statistics.mean(m[-2].elapsed_time(m[-1]) for m in marks)
+    # the same step back to back for at least two seconds: the target-side sweep is bound by
+    # arithmetic and follows the SM clock, which settles under the power cap in a long run
+    sustained = None
+    if rank == 0 and world == 1 and not args.no_sustained and flush is None and not args.topm:
+        n_sus = max(args.steps, int(2000.0 / max(total_ms / args.steps, 1e-3)))
+        s2 = ClockSampler(local)
+        s2.start()
+        s2.wait_first()
+        tb0 = time.time()
+        sus_ms, sm = _time_calls(step, n_sus, 0, None)
+        tb1 = time.time()
+        sus_clocks = s2.stop(tb0, tb1)
+        sustained = {"steps": n_sus, "ms_per_step": sus_ms / n_sus,
+                     "value": B * L / (sus_ms / n_sus * 1e-3), "unit": UNIT,
+                     "draft_call_ms": statistics.mean(m[0].elapsed_time(m[1]) for m in sm),
+                     "verify_call_ms": statistics.mean(m[-2].elapsed_time(m[-1]) for m in sm),
+                     "clocks": sus_clocks}
     l2_warm = None
     if flush is not None:  # the flush writes are inside the wall bracket: use the per-call sums
         total_ms = (draft_ms + verify_ms) * args.steps
@@ -353,14 +555,38 @@ def run_ours(args):
     roofline = {"bound": "hbm", "kernel": kname + kdesc,
                 "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                 "peak_source": "of " + which,
+                "frac_of_nominal_8TBs": achieved / 8000.0,
                 "traffic": (TRAFFIC_RATIO * tbytes) if (TRAFFIC_RATIO and args.spec == 4 and not args.topm) else None,
                 "algorithmic_bytes": tbytes, "ms": verify_ms,
                 "draft_side": {"achieved": dbytes / (draft_ms * 1e-3) / 1e9, "ms": draft_ms,
-                               "frac": dbytes / (draft_ms * 1e-3) / 1e9 / peak},
+                               "frac": dbytes / (draft_ms * 1e-3) / 1e9 / peak,
+                               "frac_of_nominal_8TBs": dbytes / (draft_ms * 1e-3) / 8e12},
                 "step": {"achieved": (dbytes + tbytes) / (ms_per_step * 1e-3) / 1e9,
                          "frac_of_nominal_8TBs": (dbytes + tbytes) / (ms_per_step * 1e-3) / 8e12}}
+    if rank == 0 and world == 1 and not args.topm and not args.no_extras:
+        # Appendix B's variant of the verify call (every target row raced under all K streams)
+        ab_ms = _event_ms(lambda: pkg.target_sample_verify(
+            w.target_logits, buf.draft_tokens, out=buf.out, workspace=buf.workspace, status=buf.status,
+            flags=pkg.COMBINE_ALL, **kw), max(3, min(args.steps, 10)), flush)
+        roofline["verify_call_appendix_b"] = _fracs(tbytes, ab_ms, peak)
+    if sustained is not None:
+        sustained["verify_call"] = _fracs(tbytes, sustained["verify_call_ms"], peak)
+        sustained["draft_call"] = _fracs(dbytes, sustained["draft_call_ms"], peak)
+        sustained["step"] = _fracs(dbytes + tbytes, sustained["ms_per_step"], peak)
+        roofline["sustained"] = sustained
     del w, buf
     torch.cuda.empty_cache()
+    others = None
+    if world == 1 and args.workload == "cfg4" and not args.no_extras and not args.topm and not args.batch:
+        # the other configurations and shapes, in the same process (each frees its tensors)
+        n_o = max(20, min(args.steps, 100))
+        others = {}
+        for name, fn in (("cfg2", lambda: _measure_verify(2, n_o, peak, args.spec)),
+                         ("cfg3", lambda: _measure_verify(3, n_o, peak, args.spec)),
+                         ("cfg4_autoregressive_draft", lambda: _measure_autoregressive(n_o, peak)),
+                         ("cfg5", lambda: _measure_compress(n_o, peak))):
+            others[name] = fn()
+            torch.cuda.empty_cache()
     cpu = None
     if not args.no_cpu:
         cpu, _, _ = _cpu_baseline(args.workload, {"cfg2": 8, "cfg3": 32, "cfg4": 16}[args.workload])
@@ -368,6 +594,13 @@ def run_ours(args):
         one, _, _ = _cpu_baseline(args.workload, {"cfg2": 2, "cfg3": 2, "cfg4": 1}[args.workload],
                                   threads=1)
         cpu["one_thread"] = {"value": one["value"], "sample": one["sample"]}
+        from oracle import gls_oracle
+        gls_oracle.set_threads(cpu["cores"])  # back to all cores
+        if others is not None:  # the oracle on the other configurations (Sec. 8(d) of the plan)
+            c2, _, _ = _cpu_baseline("cfg2", 8)
+            c3, _, _ = _cpu_baseline("cfg3", 16)
+            c5, _ = _cpu_baseline_compress(48)
+            cpu["other_workloads"] = {"cfg2": c2, "cfg3": c3, "cfg5": c5}
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
@@ -377,7 +610,7 @@ def run_ours(args):
                        "l2_warm": l2_warm, "cuda_graph_replay": graphed,
                        "l2": "flushed between steps" if flush is not None
                        else "inputs (%.2f GB) larger than L2" % ((dbytes + tbytes) / 1e9),
-                       "mean_tau": tau_mean},
+                       "mean_tau": tau_mean, "other_workloads": others},
             "hbm_gbs": (dbytes + tbytes) / (ms_per_step * 1e-3) / 1e9,
             "clocks": clocks, "e2e": e2e, "gpu_launches": 4 * args.steps,
             "roofline": roofline, "cpu_baseline": cpu}
@@ -455,7 +688,7 @@ def run_compress(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=500)
+    ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="cfg4", choices=sorted(WORKLOAD_DESC))
@@ -465,13 +698,14 @@ def main():
     ap.add_argument("--topm", type=int, default=0,
                     help="extra workload: truncate every row to its top-M logits first (Sec. 4.4)")
     ap.add_argument("--fused", action="store_true", help="one gls_draft_verify call per step")
+    ap.add_argument("--no-sustained", action="store_true", help="skip the two-second back-to-back loop")
+    ap.add_argument("--no-extras", action="store_true", help="skip the other configurations")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle baseline leg")
     args = ap.parse_args()
     if args.workload == "cfg5":
         if args.impl == "reference":
-            print(json.dumps({"impl": "reference", "unavailable": "the reference arm times the "
-                              "verification workloads (cfg2-cfg4) only"}))
+            run_reference_compress(args)
         else:
             run_compress(args)
     elif args.impl == "reference":

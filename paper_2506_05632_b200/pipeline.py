@@ -92,6 +92,8 @@ class HostStepper:
                            ready=torch.cuda.Event(), free=torch.cuda.Event(),
                            buf=StepBuffers(self.chunk, K, L, V, device))
                       for _ in range(2)]
+        # a ragged last chunk has buffers of its own, allocated here and not inside step()
+        self.ragged = StepBuffers(B % self.chunk, K, L, V, device) if B % self.chunk else None
         self.h_tokens = torch.empty((B, L + 1), dtype=torch.int32).pin_memory()
         self.h_tau = torch.empty((B,), dtype=torch.int32).pin_memory()
         self.h_accept = torch.empty((B, K, L), dtype=torch.uint8).pin_memory()
@@ -119,7 +121,7 @@ class HostStepper:
                 d, t, bb = s["d"], s["t"], buf
             else:  # ragged last chunk
                 d, t = s["d"][:nb], s["t"][:nb]
-                bb = StepBuffers(nb, self.K, self.L, self.V, d.device)
+                bb = self.ragged
             out = spec_step(d, t, bb, inv_temp=inv_temp, seed=seed, seq_base=seq_base + b0,
                             spec=spec, rounds=rounds)
             self.h_tokens[b0:b1].copy_(out["tokens"], non_blocking=True)
