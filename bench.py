@@ -621,67 +621,41 @@ def run_ours(args):
 
 def run_compress(args):
     """Extra workload (not the headline metric): one step = gls_compress_select over the batch of
-    source samples, encoder and K decoders.  Unit: source samples per second."""
+    source samples, encoder and K decoders; also the same selection from the source
+    (gls_compress_gaussian).  Unit: source samples per second."""
     import torch
 
-    import paper_2506_05632_b200 as pkg
-    from paper_2506_05632_b200 import synth
-
     assert torch.cuda.is_available(), "bench.py needs a CUDA device (no CPU fallback)"
-    torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", "0")))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
     if int(os.environ.get("RANK", "0")) != 0:
         return
+    import paper_2506_05632_b200 as pkg
+
     pkg.load()
-    w = synth.compress_workload("cuda", B=args.batch or 512)
-    B, K, N = w.dec_logw.shape
-    ws = torch.empty(pkg.workspace_bytes(B, K, 1, N), dtype=torch.uint8, device="cuda")
-    status = torch.zeros(1, dtype=torch.int32, device="cuda")
-    out = pkg.compress_select(w.enc_logw, w.dec_logw, w.bins, seed=w.noise_seed, workspace=ws,
-                              status=status)
-
-    def timed(fn, steps):
-        for _ in range(max(args.warmup, 3)):
-            fn()
-        torch.cuda.synchronize()
-        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        a.record()
-        for _ in range(steps):
-            fn()
-        b.record()
-        torch.cuda.synchronize()
-        return a.elapsed_time(b) / steps
-
-    sampler = ClockSampler(int(os.environ.get("LOCAL_RANK", "0")))
+    peak, which = _peaks()
+    sampler = ClockSampler(local)
     sampler.start()
     sampler.wait_first()
     t0 = time.time()
-    ms_all = timed(lambda: pkg.compress_select(w.enc_logw, w.dec_logw, w.bins, seed=w.noise_seed,
-                                               workspace=ws, status=status, out=out), args.steps)
-    ms_enc = timed(lambda: pkg.compress_select(w.enc_logw, None, w.bins, K=K, seed=w.noise_seed,
-                                               workspace=ws, status=status), args.steps)
+    r = _measure_compress(args.steps, peak, B=args.batch)
     clocks = sampler.stop(t0, time.time())
-    eb, db = w.enc_logw.numel() * 4, w.dec_logw.numel() * 4
-    peak, which = _peaks()
-    dec_ms = ms_all - ms_enc
-    line = {"metric": "compressed_source_samples_per_s", "value": B / (ms_all * 1e-3),
+    whole, dec = r["whole_call"], r["decoders"]
+    line = {"metric": "compressed_source_samples_per_s", "value": whole["source_samples_per_s"],
             "unit": "samples/s", "n_gpus": 1, "steps": args.steps, "warmup": max(args.warmup, 3),
-            "ms_per_step": ms_all, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "ms_per_step": whole["ms"], "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "f32", "data": "synthetic",
-            "config": {"workload": WORKLOAD_DESC["cfg5"] + (" (B overridden to %d)" % B if args.batch else ""),
-                       "l2": "inputs (%.2f GB) larger than L2" % ((eb + db) / 1e9),
-                       "match_rate": float(out["match"].float().mean().item())},
+            "config": {"workload": WORKLOAD_DESC["cfg5"] + (" (B overridden to %d)" % args.batch if args.batch else ""),
+                       "l2": "inputs larger than L2", "match_rate": r["match_rate"],
+                       "from_source": r["from_source"]},
             "clocks": clocks, "e2e": None, "gpu_launches": 6 * args.steps,
             "roofline": {"bound": "hbm", "kernel": "sweep4_kernel<f32> (the K decoder sweeps: the "
                          "dominant kernel; time = whole call minus an encoder-only call)",
-                         "achieved": db / (dec_ms * 1e-3) / 1e9, "peak": peak, "unit": "GB/s",
-                         "frac": db / (dec_ms * 1e-3) / 1e9 / peak, "peak_source": "of " + which,
-                         "traffic": None, "algorithmic_bytes": db, "ms": dec_ms,
-                         "encoder": {"ms": ms_enc, "achieved": eb / (ms_enc * 1e-3) / 1e9,
-                                     "note": "fused race over tokens and K noise streams: the log-sum-exp "
-                                             "plus K generator calls per 64 elements"},
-                         "step": {"achieved": (eb + db) / (ms_all * 1e-3) / 1e9}},
+                         "achieved": dec["gbs"], "peak": peak, "unit": "GB/s",
+                         "frac": dec["frac_of_measured"], "peak_source": "of " + which,
+                         "frac_of_nominal_8TBs": dec["frac_of_nominal_8TBs"],
+                         "traffic": None, "ms": dec["ms"], "encoder": r["encoder"], "step": whole},
             "cpu_baseline": None}
-    assert int(status.item()) == 0
     print(json.dumps(line))
 
 
