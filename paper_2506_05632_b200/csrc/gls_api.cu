@@ -1321,23 +1321,28 @@ int gls_compress_gaussian(const float* candidates, const float* source, const fl
   A.hints = (uint32_t*)(ws + P.off_hints);
   A.partials = (Partial*)(ws + P.off_partials);
   RowResult* rowres = (RowResult*)(ws + P.off_rows);
-  const size_t smem = gauss_smem_bytes(D);
   const bool r10 = A.rounds == 10;
   const double var_dec = (1.0 + s2_eta) - 1.0 / (1.0 + s2_zeta);
+  // two quads of warps per CTA where the shared memory allows (more warps per scheduler), else one
+  constexpr size_t kSmemMax = 227 * 1024;
 #define GAUSS_SWEEP(ENC, rows_, per_range_, scale_)                                              \
   do {                                                                                           \
     const int n_ranges = ((rows_) + (per_range_) - 1) / (per_range_);                            \
+    const int streams = (ENC) ? K : 1;                                                           \
+    const int quads = gauss_smem_bytes(D, streams, kGMaxQuads) <= kSmemMax ? kGMaxQuads : 1;     \
+    const size_t smem = gauss_smem_bytes(D, streams, quads);                                     \
+    if (smem > kSmemMax) return GLS_ERR_UNSUPPORTED;                                             \
     if (cudaMemsetAsync(A.hints, 0, (size_t)(rows_) * sizeof(uint32_t), st) != cudaSuccess ||    \
         cudaMemsetAsync(A.partials, 0xff, (size_t)(rows_) * P.tiles * sizeof(Partial), st) !=    \
             cudaSuccess)                                                                         \
       return GLS_ERR_CUDA;                                                                       \
     if (r10) {                                                                                   \
       cudaFuncSetAttribute(gauss_sweep_kernel<10, ENC>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem); \
-      gauss_sweep_kernel<10, ENC><<<P.tiles * n_ranges, kGWarps * 32, smem, st>>>(               \
+      gauss_sweep_kernel<10, ENC><<<P.tiles * n_ranges, quads * kGWarps * 32, smem, st>>>(       \
           A, n_ranges, (per_range_), (long long)N, (float)(scale_));                             \
     } else {                                                                                     \
       cudaFuncSetAttribute(gauss_sweep_kernel<0, ENC>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem); \
-      gauss_sweep_kernel<0, ENC><<<P.tiles * n_ranges, kGWarps * 32, smem, st>>>(                \
+      gauss_sweep_kernel<0, ENC><<<P.tiles * n_ranges, quads * kGWarps * 32, smem, st>>>(        \
           A, n_ranges, (per_range_), (long long)N, (float)(scale_));                             \
     }                                                                                            \
     if (cudaGetLastError() != cudaSuccess) return GLS_ERR_CUDA;                                  \

@@ -27,30 +27,38 @@ constexpr int kGRows = 4;           // rows per block
 constexpr int kGPad = 20;           // floats per group in shared memory (16 + 4: no bank conflicts)
 constexpr int kGMaxD = 16;
 constexpr int kGMaxK = 8;
-constexpr int kGQueue = 32 + kGRows * kGMaxK;  // a block adds at most rows x streams entries per lane group
+constexpr int kGFlushAt = 16;                   // a batch is taken as soon as this many groups are queued
+constexpr int kGQueue = kGFlushAt + 32;         // one (row, stream) test adds at most 32 per warp
+constexpr int kGMaxQuads = 2;                   // warp quads per CTA, each walking its own row blocks
 
 struct GaussRowCtx {  // one row of the current block
   uint32_t c1, pos, seq;  // noise stream (c1 without the stream number in the encoder pass)
   uint32_t m_enc;         // ordered code of the row's bound
   int row, b;             // row number (-1: past the end), source sample
   int msg;                // label a candidate must carry (decoder pass with labels)
+  int pad;
 };
 struct __align__(16) GaussEntry {  // a queued group: coarse word, group | stream << 28, row slot, weights
   uint32_t w, g, slot, pad;
   float a[16];
 };
-struct __align__(16) GaussShared {
+// Shared memory of one warp quad (four warps that walk the same row blocks); the coarse words
+// [stream-row][word][lane] follow it, then the next quad's block.
+struct __align__(16) GaussQuad {
   float mu[kGMaxD][kGRows];                       // scaled means of the block's rows
   GaussRowCtx ctx[kGRows];
-  uint32_t xw[kGRows * kGMaxK][4][32];            // coarse words: [stream-row][word][lane]
   Top2 best[kGWarps][kGRows];                     // per warp and row slot
   float lse_m[kGWarps][kGRows], lse_s[kGWarps][kGRows];
   GaussEntry queue[kGWarps][kGQueue];
-  uint32_t labels[128][4];                        // the tile's bin labels, 16 bytes per group
-  float us[1];                                    // [(D + 1)][128 * kGPad], D-th plane: |u|^2 / (2 s2_prior)
 };
-__host__ __device__ inline size_t gauss_smem_bytes(int D) {
-  return sizeof(GaussShared) + (size_t)(D + 1) * 128 * kGPad * sizeof(float);
+// Layout: quads x (GaussQuad, coarse words [kGRows * streams][4][32]), labels [128][4], then the
+// tile [(D + 1)][128 * kGPad] floats, plane D holding |u|^2 / (2 s2_prior).
+__host__ __device__ inline size_t gauss_quad_bytes(int streams) {
+  return sizeof(GaussQuad) + (size_t)kGRows * streams * 4 * 32 * sizeof(uint32_t);
+}
+__host__ __device__ inline size_t gauss_smem_bytes(int D, int streams, int quads) {
+  return (size_t)quads * gauss_quad_bytes(streams) + 128 * 4 * sizeof(uint32_t) +
+         (size_t)(D + 1) * 128 * kGPad * sizeof(float);
 }
 
 // Batched evaluation of queued groups (cf. s4_flush): lane l < n takes entry first + l.  Entries
@@ -58,9 +66,9 @@ __host__ __device__ inline size_t gauss_smem_bytes(int D) {
 // The lanes' results are merged per row slot into sh.best[warp][slot]; improved bounds go to the
 // row's context and to its hint word.
 template <int ROUNDS, bool ENC>
-__device__ __noinline__ void gauss_flush(const SweepArgs& A, GaussShared& sh, int first, int n) {
+__device__ __noinline__ void gauss_flush(const SweepArgs& A, GaussQuad& sh, int first, int n) {
   const int lane = threadIdx.x & 31;
-  const int warp = threadIdx.x >> 5;
+  const int warp = (threadIdx.x >> 5) & (kGWarps - 1);
   constexpr float c2 = kLog2e;
   uint32_t msk = 0u, g = 0u, ks = 0u;
   int loc = -1, slot = 0;
@@ -157,12 +165,15 @@ __device__ __noinline__ void gauss_flush(const SweepArgs& A, GaussShared& sh, in
 //   row range r of n_ranges covers rows [r * rows_per_range, ...); blockIdx.x = tile * n_ranges + r
 // ------------------------------------------------------------------------------------------
 template <int ROUNDS, bool ENC>
-__global__ void __launch_bounds__(kGWarps * 32, 1)
+__global__ void __launch_bounds__(kGMaxQuads * kGWarps * 32, 1)
 gauss_sweep_kernel(const __grid_constant__ SweepArgs A, int n_ranges, int rows_per_range,
                    long long N, float scale /* 1 / sqrt(2 v) of this pass */) {
-  GaussShared& sh = *reinterpret_cast<GaussShared*>(gls_smem_raw);
+  // blockDim.x = quads * 128: every quad of warps walks its own row blocks over the shared tile
+  const int n_quads = (int)blockDim.x >> 7;
+  const int quad = (int)threadIdx.x >> 7;
+  const int tq = (int)threadIdx.x & 127;  // thread within the quad
   const int lane = threadIdx.x & 31;
-  const int warp = threadIdx.x >> 5;
+  const int warp = (threadIdx.x >> 5) & (kGWarps - 1);  // warp within the quad
   const int D = A.gD;
   const int K = A.K;
   const int tile = blockIdx.x / n_ranges;
@@ -171,14 +182,21 @@ gauss_sweep_kernel(const __grid_constant__ SweepArgs A, int n_ranges, int rows_p
   const int row_hi = min(A.rows, row_lo + rows_per_range);
   const long long cand0 = (long long)tile * kGTile;
   const int n_streams = ENC ? A.multi_k : 1;
-  float* const us = sh.us;
   constexpr int kPlane = 128 * kGPad;
+  const size_t quad_bytes = gauss_quad_bytes(n_streams);
+  GaussQuad& sh = *reinterpret_cast<GaussQuad*>(gls_smem_raw + (size_t)quad * quad_bytes);
+  uint32_t (*const xw)[4][32] =
+      reinterpret_cast<uint32_t(*)[4][32]>(gls_smem_raw + (size_t)quad * quad_bytes + sizeof(GaussQuad));
+  uint32_t (*const labels)[4] =
+      reinterpret_cast<uint32_t(*)[4]>(gls_smem_raw + (size_t)n_quads * quad_bytes);
+  float* const us = reinterpret_cast<float*>(gls_smem_raw + (size_t)n_quads * quad_bytes + 128 * 4 * sizeof(uint32_t));
+  auto quad_sync = [&]() { asm volatile("bar.sync %0, %1;" ::"r"(quad + 1), "r"(kGWarps * 32) : "memory"); };
 
   // ---- the tile's coordinates, scaled, to shared memory; plane D holds |u|^2 / (2 s2_prior),
   //      -inf for candidates past the end (their weights become -inf)
   {
     const float half_inv_prior = (float)(0.5 / A.g_s2_prior);
-    for (int c = threadIdx.x; c < kGTile; c += kGWarps * 32) {
+    for (int c = threadIdx.x; c < kGTile; c += (int)blockDim.x) {
       const long long i = cand0 + c;
       const int at = (c >> 4) * kGPad + (c & 15);
       float nrm = 0.f;
@@ -195,9 +213,9 @@ gauss_sweep_kernel(const __grid_constant__ SweepArgs A, int n_ranges, int rows_p
   // ln L_max below the best overall, and that many more groups would pass a test on all sixteen)
   const bool use_labels = !ENC && A.bins != nullptr && A.bins_sb == 0;
   if (use_labels) {
-    for (int c = threadIdx.x; c < kGTile; c += kGWarps * 32) {
+    for (int c = threadIdx.x; c < kGTile; c += (int)blockDim.x) {
       const long long i = cand0 + c;
-      reinterpret_cast<uint8_t*>(&sh.labels[0][0])[c] = i < N ? __ldg(A.bins + i) : (uint8_t)0;
+      reinterpret_cast<uint8_t*>(&labels[0][0])[c] = i < N ? __ldg(A.bins + i) : (uint8_t)0;
     }
   }
   // What the next block needs: scaled means, contexts, coarse words.  The global loads are issued
@@ -207,7 +225,7 @@ gauss_sweep_kernel(const __grid_constant__ SweepArgs A, int n_ranges, int rows_p
   uint32_t pf_seq = 0u, pf_hint = 0u;
   int pf_msg = 0;
   auto fetch = [&](int row0) {
-    const int idx = threadIdx.x;
+    const int idx = tq;
     if (idx < kGRows * D) {
       const int r = idx / D, d = idx - r * D;
       const int row = row0 + r;
@@ -218,8 +236,8 @@ gauss_sweep_kernel(const __grid_constant__ SweepArgs A, int n_ranges, int rows_p
       }
       pf_mu[0] = m * scale;
     }
-    if (threadIdx.x < kGRows) {
-      const int row = row0 + threadIdx.x;
+    if (tq < kGRows) {
+      const int row = row0 + tq;
       if (row < row_hi) {
         const int b = ENC ? row : row / K;
         pf_seq = A.seq_ids ? __ldg(A.seq_ids + b) : A.seq_base + (uint32_t)b;
@@ -229,15 +247,16 @@ gauss_sweep_kernel(const __grid_constant__ SweepArgs A, int n_ranges, int rows_p
     }
   };
   auto commit = [&](int row0) {
-    const int idx = threadIdx.x;
+    const int idx = tq;
     if (idx < kGRows * D) {
       const int r = idx / D, d = idx - r * D;
       sh.mu[d][r] = pf_mu[0];
     }
-    if (threadIdx.x < kGRows) {
-      const int r = threadIdx.x;
+    if (tq < kGRows) {
+      const int r = tq;
       const int row = row0 + r;
       GaussRowCtx cx;
+      cx.pad = 0;
       cx.row = row < row_hi ? row : -1;
       const int b = ENC ? row : row / K;
       const int k = ENC ? 0 : row - b * K;
@@ -266,10 +285,10 @@ gauss_sweep_kernel(const __grid_constant__ SweepArgs A, int n_ranges, int rows_p
       const uint32_t seq = A.seq_ids ? __ldg(A.seq_ids + b) : A.seq_base + (uint32_t)b;
       uint32_t cw[4];
       philox4x32<ROUNDS>(A.rk, A.rounds, ((uint32_t)tile << 5) | (uint32_t)lane, c1, A.pos_base, seq, cw);
-      sh.xw[sr][0][lane] = cw[0];
-      sh.xw[sr][1][lane] = cw[1];
-      sh.xw[sr][2][lane] = cw[2];
-      sh.xw[sr][3][lane] = cw[3];
+      xw[sr][0][lane] = cw[0];
+      xw[sr][1][lane] = cw[1];
+      xw[sr][2][lane] = cw[2];
+      xw[sr][3][lane] = cw[3];
     }
   };
   // The blocks of rows are walked in a rotated order that differs from tile to tile: CTAs that run
@@ -280,10 +299,13 @@ gauss_sweep_kernel(const __grid_constant__ SweepArgs A, int n_ranges, int rows_p
   const int n_blocks = (row_hi - row_lo + kGRows - 1) / kGRows;
   const int rot = (int)(((uint32_t)tile * 2654435761u >> 8) % (uint32_t)n_blocks);
   auto block_row = [&](int it) { return row_lo + ((it + rot) % n_blocks) * kGRows; };
-  fetch(block_row(0));
-  commit(block_row(0));
-  coarse_words(block_row(0));
-  __syncthreads();
+  __syncthreads();  // the tile is in shared memory
+  if (quad < n_blocks) {
+    fetch(block_row(quad));
+    commit(block_row(quad));
+    coarse_words(block_row(quad));
+  }
+  quad_sync();
 
   const int gl = warp * 32 + lane;                      // the lane's group within the tile
   const uint32_t gidx = (uint32_t)tile * 128u + (uint32_t)gl;  // ... and in the whole row
@@ -291,9 +313,9 @@ gauss_sweep_kernel(const __grid_constant__ SweepArgs A, int n_ranges, int rows_p
   GaussEntry* const queue = sh.queue[warp];
   const bool group_in_range = cand0 + (long long)gl * 16 < N;
 
-  for (int it = 0; it < n_blocks; ++it) {
+  for (int it = quad; it < n_blocks; it += n_quads) {
     const int row0 = block_row(it);
-    if (it + 1 < n_blocks) fetch(block_row(it + 1));
+    if (it + n_quads < n_blocks) fetch(block_row(it + n_quads));
     // ---- weights of the lane's 16 candidates for the block's four rows -----------------------
     unsigned long long acc[kGRows][8];
 #pragma unroll
@@ -333,7 +355,7 @@ gauss_sweep_kernel(const __grid_constant__ SweepArgs A, int n_ranges, int rows_p
     int qn = 0;
     uint32_t lab[4] = {0u, 0u, 0u, 0u};
     if (use_labels) {
-      const uint4 lv = *reinterpret_cast<const uint4*>(&sh.labels[gl][0]);
+      const uint4 lv = *reinterpret_cast<const uint4*>(&labels[gl][0]);
       lab[0] = lv.x; lab[1] = lv.y; lab[2] = lv.z; lab[3] = lv.w;
     }
 #pragma unroll
@@ -386,7 +408,7 @@ gauss_sweep_kernel(const __grid_constant__ SweepArgs A, int n_ranges, int rows_p
       const float nms = scaled_offset(nm4);
       const float thr = exp2_upper_from_scaled(amax, kLog2e * (1.0f / 126.0f), nms);
       for (int ks = 0; ks < n_streams; ++ks) {
-        const uint32_t w = sh.xw[r * n_streams + ks][warp][lane];
+        const uint32_t w = xw[r * n_streams + ks][warp][lane];
         const bool pass = group_in_range && coarse_lower(w) <= thr;
         const unsigned bal = __ballot_sync(0xffffffffu, pass);
         if (bal != 0u) {
@@ -399,10 +421,11 @@ gauss_sweep_kernel(const __grid_constant__ SweepArgs A, int n_ranges, int rows_p
             for (int t = 0; t < 16; ++t) e.a[t] = wgt[t];
           }
           qn += __popc(bal);
-          if (qn >= 32) {  // a full batch: evaluate it now (rare after the first rows)
+          while (qn >= kGFlushAt) {  // enough for a batch: evaluate it now (rare after the first rows)
             __syncwarp();
-            qn -= 32;
-            gauss_flush<ROUNDS, ENC>(A, sh, qn, 32);
+            const int nb = min(qn, 32);
+            qn -= nb;
+            gauss_flush<ROUNDS, ENC>(A, sh, qn, nb);
           }
         }
       }
@@ -413,7 +436,7 @@ gauss_sweep_kernel(const __grid_constant__ SweepArgs A, int n_ranges, int rows_p
       qn -= nb;
       gauss_flush<ROUNDS, ENC>(A, sh, qn, nb);
     }
-    __syncthreads();  // every warp's results for this block are in shared memory
+    quad_sync();  // every warp's results for this block are in shared memory
     // ---- warp r merges row slot r and writes its partial result; then the next block is set up
     {
       const int r = warp;
@@ -441,12 +464,12 @@ gauss_sweep_kernel(const __grid_constant__ SweepArgs A, int n_ranges, int rows_p
         }
       }
     }
-    __syncthreads();  // the merge has read the block's results
-    if (it + 1 < n_blocks) {
-      commit(block_row(it + 1));
-      coarse_words(block_row(it + 1));
+    quad_sync();  // the merge has read the block's results
+    if (it + n_quads < n_blocks) {
+      commit(block_row(it + n_quads));
+      coarse_words(block_row(it + n_quads));
     }
-    __syncthreads();
+    quad_sync();
   }
   asm volatile("griddepcontrol.launch_dependents;");
 }
