@@ -131,6 +131,16 @@ typedef struct {
 /* Library version, major * 10000 + minor * 100 + patch. */
 int gls_version(void);
 
+/*
+ * Self-check of the kernels' index arithmetic (no counterpart in the paper).  A library built with
+ * -DGLS_DEBUG_BOUNDS range-checks its own shared- and global-memory indices; a violation is counted,
+ * the first one recorded, and the access skipped (nothing traps).  Returns 1 and copies
+ * {count, site of the first violation, its value, its limit} of the current device to the HOST
+ * array (synchronising with the device) when the checks are compiled in, 0 (and zeros) when they
+ * are not, -1 if the copy failed.
+ */
+int gls_debug_bounds(uint32_t out_host[4]);
+
 /* Human-readable name of a status code (static storage, never NULL). */
 const char* gls_status_string(int status);
 

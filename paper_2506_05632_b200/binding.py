@@ -33,7 +33,7 @@ def _sources():
                   if f.endswith((".cu", ".cuh"))) + [os.path.join(_ROOT, "include", "gls.h")]
 
 
-def build(force=False, verbose=False):
+def build(force=False, verbose=False, debug_bounds=False):
     """Compile csrc/*.cu into libgls.so for sm_100a with nvcc (cross-compiles without a GPU)."""
     srcs = _sources()
     if (not force and os.path.exists(_LIB)
@@ -43,6 +43,8 @@ def build(force=False, verbose=False):
     tmp = _LIB + ".tmp%d" % os.getpid()
     cmd = ["nvcc", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
            "-shared", "-Xcompiler", "-fPIC", "-o", tmp] + cus
+    if debug_bounds or os.environ.get("GLS_DEBUG_BOUNDS") == "1":
+        cmd.insert(1, "-DGLS_DEBUG_BOUNDS")  # range checks of the kernels' own indices
     if verbose:
         cmd.insert(1, "-Xptxas=-v")
     subprocess.run(cmd, check=True)
@@ -138,6 +140,15 @@ def load():
             C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p, C.c_void_p]
         _lib = L
         return _lib
+
+
+def debug_bounds():
+    """(compiled in?, [count, first site, value, limit]) of the library's index self-check."""
+    out = (C.c_uint32 * 4)()
+    L = load()
+    L.gls_debug_bounds.restype = C.c_int
+    rc = int(L.gls_debug_bounds(out))
+    return rc, [int(x) for x in out]
 
 
 def version():

@@ -836,7 +836,18 @@ using namespace gls;
 
 extern "C" {
 
-int gls_version(void) { return 100; }
+int gls_version(void) { return 200; }
+
+int gls_debug_bounds(uint32_t out_host[4]) {
+#ifdef GLS_DEBUG_BOUNDS
+  if (!out_host) return 1;
+  if (cudaMemcpyFromSymbol(out_host, g_bounds_fault, 4 * sizeof(uint32_t)) != cudaSuccess) return -1;
+  return 1;
+#else
+  if (out_host) out_host[0] = out_host[1] = out_host[2] = out_host[3] = 0u;
+  return 0;
+#endif
+}
 
 const char* gls_status_string(int status) {
   switch (status) {

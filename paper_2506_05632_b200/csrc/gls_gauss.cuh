@@ -73,7 +73,8 @@ __device__ __noinline__ void gauss_flush(const SweepArgs& A, GaussQuad& sh, int 
   uint32_t msk = 0u, g = 0u, ks = 0u;
   int loc = -1, slot = 0;
   float M = 1.f, lg2M = 0.f, nm = CUDART_INF_F;
-  const GaussEntry& e = sh.queue[warp][first + (lane < n ? lane : 0)];
+  const GaussEntry& e =
+      sh.queue[warp][GLS_IN_RANGE(first + (lane < n ? lane : 0), 0, kGQueue, 33u) ? first + (lane < n ? lane : 0) : 0];
   Top2 b;
   top2_init(b);
   float lower = -CUDART_INF_F;
@@ -413,7 +414,8 @@ gauss_sweep_kernel(const __grid_constant__ SweepArgs A, int n_ranges, int rows_p
         const unsigned bal = __ballot_sync(0xffffffffu, pass);
         if (bal != 0u) {
           if (pass) {
-            GaussEntry& e = queue[qn + __popc(bal & ((1u << lane) - 1u))];
+            const int qi = qn + __popc(bal & ((1u << lane) - 1u));
+            GaussEntry& e = queue[GLS_IN_RANGE(qi, 0, kGQueue, 30u) ? qi : 0];
             e.w = w;
             e.g = gidx | (((uint32_t)ks & A.kmask) << 28);
             e.slot = (uint32_t)r;
@@ -460,7 +462,8 @@ gauss_sweep_kernel(const __grid_constant__ SweepArgs A, int n_ranges, int rows_p
           Partial pr;
           pr.s1 = m.s1; pr.i1 = m.i1; pr.s2 = m.s2; pr.i2 = m.i2;
           pr.lm = lm; pr.ls = ls; pr.pad0 = 0; pr.pad1 = 0;
-          A.partials[(long long)row * A.parts + tile] = pr;
+          if (GLS_IN_RANGE(tile, 0, A.parts, 31u) && GLS_IN_RANGE(row, 0, A.rows, 32u))
+            A.partials[(long long)row * A.parts + tile] = pr;
         }
       }
     }

@@ -23,6 +23,27 @@
 
 namespace gls {
 
+// Range checks of the kernels' own indices, compiled in with -DGLS_DEBUG_BOUNDS (the tests run
+// the small shapes once under it; the memory checker of the toolkit is not available on every
+// installation).  A violated check records (site, value, limit) in a device word array, counts it,
+// and the guarded access is skipped; nothing traps.  Without the option the macro only evaluates to
+// true and costs nothing.
+__device__ unsigned int g_bounds_fault[4];  // [0] count, [1] first site, [2] its value, [3] its limit
+#ifdef GLS_DEBUG_BOUNDS
+__device__ __forceinline__ bool bounds_ok(long long v, long long lo, long long hi, unsigned site) {
+  if (v >= lo && v < hi) return true;
+  if (atomicAdd(&g_bounds_fault[0], 1u) == 0u) {
+    g_bounds_fault[1] = site;
+    g_bounds_fault[2] = (unsigned)v;
+    g_bounds_fault[3] = (unsigned)hi;
+  }
+  return false;
+}
+#define GLS_IN_RANGE(v, lo, hi, site) (::gls::bounds_ok((long long)(v), (long long)(lo), (long long)(hi), (site)))
+#else
+#define GLS_IN_RANGE(v, lo, hi, site) (true)
+#endif
+
 constexpr int kMaxK = 64;
 constexpr int kWarpTokens = 256;  // tokens one warp consumes per iteration (8 per lane)
 constexpr float kLog2e = 1.4426950408889634f;
@@ -593,7 +614,7 @@ sweep_kernel(const __grid_constant__ SweepArgs A) {
       Partial p;
       p.s1 = best.s1; p.i1 = best.i1; p.s2 = best.s2; p.i2 = best.i2;
       p.lm = lm; p.ls = ls; p.pad0 = 0; p.pad1 = 0;
-      A.partials[item] = p;
+      if (GLS_IN_RANGE(item, 0, A.n_items, 10u)) A.partials[item] = p;
     }
   }
 }

@@ -141,7 +141,7 @@ __device__ __noinline__ uint32_t s4_flush(int rounds_rt, int first, int n, float
   float M = 1.f;
   float lb = -CUDART_INF_F;
   if (lane < n) {
-    const uint2 e = sh.queue[warp][first + lane];
+    const uint2 e = sh.queue[warp][GLS_IN_RANGE(first + lane, 0, kS4QueueCap, 25u) ? first + lane : 0];
     g = e.y;
     if (MULTI) {
       ks = g >> 28;
@@ -299,7 +299,8 @@ __device__ __forceinline__ void s4_item(const SweepArgs& A, int row, int split, 
       if (s < n_full) {
         const char* p = rowp + (size_t)tok * ES;
 #pragma unroll
-        for (int j = 0; j < kS4LaneGroups; ++j) load16_vec(g[j], p + j * 512 * ES);
+        for (int j = 0; j < kS4LaneGroups; ++j)
+          if (GLS_IN_RANGE(tok + j * 512 + 15, 0, tok_end, 22u)) load16_vec(g[j], p + j * 512 * ES);
       } else {
 #pragma unroll
         for (int j = 0; j < kS4LaneGroups; ++j) load16_scalar(g[j], rowp, tok + j * 512, tok_end);
@@ -333,7 +334,8 @@ __device__ __forceinline__ void s4_item(const SweepArgs& A, int row, int split, 
       const unsigned bal = __ballot_sync(0xffffffffu, pass);
       if (pass) {
         const uint32_t w = bj == 0 ? cw[0] : bj == 1 ? cw[1] : bj == 2 ? cw[2] : cw[3];
-        queue[__popc(bal & ((1u << lane) - 1u))] = make_uint2(w, ((uint32_t)tok0 >> 4) + 32u * bj);
+        const int qi = __popc(bal & ((1u << lane) - 1u));
+        if (GLS_IN_RANGE(qi, 0, kS4QueueCap, 20u)) queue[qi] = make_uint2(w, ((uint32_t)tok0 >> 4) + 32u * bj);
       }
       const int nb = __popc(bal);
       __syncwarp();
@@ -353,7 +355,10 @@ __device__ __forceinline__ void s4_item(const SweepArgs& A, int row, int split, 
       const bool pass = coarse_lower(w) <= exp2_upper_from_scaled(amax, c2s, nms);
       const unsigned bal = __ballot_sync(0xffffffffu, pass);
       if (bal != 0u) {
-        if (pass) queue[qn + __popc(bal & ((1u << lane) - 1u))] = make_uint2(w, gidx);
+        if (pass) {
+          const int qi = qn + __popc(bal & ((1u << lane) - 1u));
+          if (GLS_IN_RANGE(qi, 0, kS4QueueCap, 21u)) queue[qi] = make_uint2(w, gidx);
+        }
         qn += __popc(bal);
       }
     };
@@ -484,7 +489,8 @@ __device__ __forceinline__ void s4_item(const SweepArgs& A, int row, int split, 
       Partial pr;
       pr.s1 = t2.s1; pr.i1 = t2.i1; pr.s2 = t2.s2; pr.i2 = t2.i2;
       pr.lm = lm; pr.ls = ls; pr.pad0 = 0; pr.pad1 = 0;
-      A.partials[(long long)row * A.parts + split * kWarps + warp] = pr;
+      if (GLS_IN_RANGE(split * kWarps + warp, 0, A.parts, 23u) && GLS_IN_RANGE(row, 0, A.rows, 24u))
+        A.partials[(long long)row * A.parts + split * kWarps + warp] = pr;
       if (A.splits > 1 && m_enc > 0u) atomicMax(A.hints + row, m_enc);
     }
   }

@@ -146,8 +146,10 @@ __device__ __noinline__ int topm_expand(TopmWarpBuf* wb, const int* queue, const
 #pragma unroll
   for (int t = 0; t < 16; ++t) {
     if ((m >> t) & 1u) {
-      wb->key[pos] = enc_ordered(a[t] + 0.0f);  // -0 and +0 are the same logit: one code
-      wb->idx[pos] = tok + t;
+      if (GLS_IN_RANGE(pos, 0, kTopmCap, 41u)) {
+        wb->key[pos] = enc_ordered(a[t] + 0.0f);  // -0 and +0 are the same logit: one code
+        wb->idx[pos] = tok + t;
+      }
       ++pos;
     }
   }
@@ -218,7 +220,7 @@ topm_select_kernel(const TopmArgs T) {
           const bool hit = group16_max(g[q]) > thr;  // false for NaN
           const unsigned bal = __ballot_sync(0xffffffffu, hit);
           if (bal != 0u) {
-            if (hit) queue[qn + __popc(bal & lt)] = g0 + 32 * q;
+            if (hit && GLS_IN_RANGE(qn + __popc(bal & lt), 0, kS4QueueCap, 40u)) queue[qn + __popc(bal & lt)] = g0 + 32 * q;
             qn += __popc(bal);
           }
         }

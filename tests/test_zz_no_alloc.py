@@ -89,3 +89,12 @@ def test_static_calls_leave_device_memory_as_it_is(gls):
     free1, _ = torch.cuda.mem_get_info()
     assert free1 == free0
     assert torch.cuda.memory_allocated() == held0 and torch.cuda.memory_reserved() == reserved0
+
+
+def test_index_self_check_found_nothing(gls):
+    """When the library was built with its range checks (GLS_DEBUG_BOUNDS=1), no kernel that ran in
+    this process -- every GPU test before this one -- addressed anything outside its arrays.
+    Without the checks the entry point says so and the test has nothing to look at."""
+    compiled_in, words = gls.debug_bounds()
+    assert compiled_in in (0, 1)
+    assert words[0] == 0, "range check violated %d times; first: site %d value %d limit %d" % tuple(words)
