@@ -1334,13 +1334,14 @@ int gls_compress_gaussian(const float* candidates, const float* source, const fl
   RowResult* rowres = (RowResult*)(ws + P.off_rows);
   const bool r10 = A.rounds == 10;
   const double var_dec = (1.0 + s2_eta) - 1.0 / (1.0 + s2_zeta);
-  // two quads of warps per CTA where the shared memory allows (more warps per scheduler), else one
+  // as many quads of warps per CTA as the shared memory allows (more warps per scheduler)
   constexpr size_t kSmemMax = 227 * 1024;
 #define GAUSS_SWEEP(ENC, rows_, per_range_, scale_)                                              \
   do {                                                                                           \
     const int n_ranges = ((rows_) + (per_range_) - 1) / (per_range_);                            \
     const int streams = (ENC) ? K : 1;                                                           \
-    const int quads = gauss_smem_bytes(D, streams, kGMaxQuads) <= kSmemMax ? kGMaxQuads : 1;     \
+    int quads = kGMaxQuads;                                                                      \
+    while (quads > 1 && gauss_smem_bytes(D, streams, quads) > kSmemMax) --quads;                 \
     const size_t smem = gauss_smem_bytes(D, streams, quads);                                     \
     if (smem > kSmemMax) return GLS_ERR_UNSUPPORTED;                                             \
     if (cudaMemsetAsync(A.hints, 0, (size_t)(rows_) * sizeof(uint32_t), st) != cudaSuccess ||    \

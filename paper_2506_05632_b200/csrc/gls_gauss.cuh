@@ -23,13 +23,14 @@ namespace gls {
 
 constexpr int kGTile = 2048;        // candidates per tile = 128 groups of 16
 constexpr int kGWarps = 4;          // warp w owns groups 32 w .. 32 w + 31 of the tile
-constexpr int kGRows = 4;           // rows per block
-constexpr int kGPad = 20;           // floats per group in shared memory (16 + 4: no bank conflicts)
+constexpr int kGRows = 2;           // rows per block (2 x 16 weights per lane stay under 128 registers)
+constexpr int kGPad = 16;           // floats per group in shared memory; its four 16-byte chunks are
+                                    // stored XOR-swizzled by (group >> 1) & 3: conflict-free 128-bit reads
 constexpr int kGMaxD = 16;
 constexpr int kGMaxK = 8;
 constexpr int kGFlushAt = 16;                   // a batch is taken as soon as this many groups are queued
 constexpr int kGQueue = kGFlushAt + 32;         // one (row, stream) test adds at most 32 per warp
-constexpr int kGMaxQuads = 2;                   // warp quads per CTA, each walking its own row blocks
+constexpr int kGMaxQuads = 4;                   // warp quads per CTA, each walking its own row blocks
 
 struct GaussRowCtx {  // one row of the current block
   uint32_t c1, pos, seq;  // noise stream (c1 without the stream number in the encoder pass)
@@ -199,7 +200,8 @@ gauss_sweep_kernel(const __grid_constant__ SweepArgs A, int n_ranges, int rows_p
     const float half_inv_prior = (float)(0.5 / A.g_s2_prior);
     for (int c = threadIdx.x; c < kGTile; c += (int)blockDim.x) {
       const long long i = cand0 + c;
-      const int at = (c >> 4) * kGPad + (c & 15);
+      const int grp = c >> 4, t = c & 15;
+      const int at = grp * kGPad + 4 * ((t >> 2) ^ ((grp >> 1) & 3)) + (t & 3);
       float nrm = 0.f;
       for (int d = 0; d < D; ++d) {
         const float x = i < N ? __ldg(A.gu + i * D + d) : 0.f;
@@ -268,10 +270,8 @@ gauss_sweep_kernel(const __grid_constant__ SweepArgs A, int n_ranges, int rows_p
       cx.msg = pf_msg;
       cx.m_enc = cx.row >= 0 ? pf_hint : 0u;
       sh.ctx[r] = cx;
-      top2_init(sh.best[0][r]);
-      top2_init(sh.best[1][r]);
-      top2_init(sh.best[2][r]);
-      top2_init(sh.best[3][r]);
+#pragma unroll
+      for (int w2 = 0; w2 < kGWarps; ++w2) top2_init(sh.best[w2][r]);
     }
   };
   // coarse words of the block's stream-rows: warp w computes stream-rows sr = w, w + 4, ...
@@ -311,6 +311,7 @@ gauss_sweep_kernel(const __grid_constant__ SweepArgs A, int n_ranges, int rows_p
   const int gl = warp * 32 + lane;                      // the lane's group within the tile
   const uint32_t gidx = (uint32_t)tile * 128u + (uint32_t)gl;  // ... and in the whole row
   const float* const ug = us + gl * kGPad;
+  const int sw = (gl >> 1) & 3;  // chunk q of the group sits at position q ^ sw
   GaussEntry* const queue = sh.queue[warp];
   const bool group_in_range = cand0 + (long long)gl * 16 < N;
 
@@ -325,15 +326,15 @@ gauss_sweep_kernel(const __grid_constant__ SweepArgs A, int n_ranges, int rows_p
       for (int p = 0; p < 8; ++p) acc[r][p] = 0ull;
 #pragma unroll 2
     for (int d = 0; d < D; ++d) {
-      const float4 m4 = *reinterpret_cast<const float4*>(&sh.mu[d][0]);
+      const float2 m2 = *reinterpret_cast<const float2*>(&sh.mu[d][0]);
       unsigned long long up[8];
 #pragma unroll
       for (int q = 0; q < 4; ++q) {
-        const float4 v = *reinterpret_cast<const float4*>(ug + d * kPlane + 4 * q);
+        const float4 v = *reinterpret_cast<const float4*>(ug + d * kPlane + 4 * (q ^ sw));
         up[2 * q] = pack_f32x2(v.x, v.y);
         up[2 * q + 1] = pack_f32x2(v.z, v.w);
       }
-      const float mr[kGRows] = {m4.x, m4.y, m4.z, m4.w};
+      const float mr[kGRows] = {m2.x, m2.y};
 #pragma unroll
       for (int r = 0; r < kGRows; ++r) {
         // all differences first, then all multiply-adds: with one warp per scheduler a dependent
@@ -349,7 +350,7 @@ gauss_sweep_kernel(const __grid_constant__ SweepArgs A, int n_ranges, int rows_p
     float pn[16];
 #pragma unroll
     for (int q = 0; q < 4; ++q) {
-      const float4 v = *reinterpret_cast<const float4*>(ug + D * kPlane + 4 * q);
+      const float4 v = *reinterpret_cast<const float4*>(ug + D * kPlane + 4 * (q ^ sw));
       pn[4 * q] = v.x; pn[4 * q + 1] = v.y; pn[4 * q + 2] = v.z; pn[4 * q + 3] = v.w;
     }
     // ---- per row: group maximum, log-sum-exp (encoder), group test per stream ------------------
@@ -439,11 +440,12 @@ gauss_sweep_kernel(const __grid_constant__ SweepArgs A, int n_ranges, int rows_p
       gauss_flush<ROUNDS, ENC>(A, sh, qn, nb);
     }
     quad_sync();  // every warp's results for this block are in shared memory
-    // ---- warp r merges row slot r and writes its partial result; then the next block is set up
+    // ---- warp r (< rows per block) merges row slot r and writes its partial result; then the
+    //      next block is set up
     {
       const int r = warp;
       const int row = row0 + r;
-      if (row < row_hi && lane == 0) {
+      if (r < kGRows && row < row_hi && lane == 0) {
         Top2 m = sh.best[0][r];
         float lm = kGroupLseFloor, ls = 0.f;
 #pragma unroll
