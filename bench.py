@@ -596,7 +596,7 @@ def run_ours(args):
         cpu["one_thread"] = {"value": one["value"], "sample": one["sample"]}
         from oracle import gls_oracle
         gls_oracle.set_threads(cpu["cores"])  # back to all cores
-        if others is not None:  # the oracle on the other configurations (Sec. 8(d) of the plan)
+        if others is not None:  # the oracle on the other configurations
             c2, _, _ = _cpu_baseline("cfg2", 8)
             c3, _, _ = _cpu_baseline("cfg3", 16)
             c5, _ = _cpu_baseline_compress(48)

@@ -20,12 +20,13 @@ pytestmark = pytest.mark.gpu
 
 
 def _report(tally):
-    """One JSON line per workload into the scratch folder of a GPU run, when there is one."""
-    d = os.path.join(os.path.dirname(os.path.dirname(os.path.abspath(__file__))), "gpurun_out")
-    if os.path.isdir(d):
-        with open(os.path.join(d, "parity_counts.jsonl"), "a") as f:
-            f.write(json.dumps(tally.as_dict()) + "\n")
-    print(json.dumps(tally.as_dict()))
+    """One JSON line per workload, printed and, if GLS_PARITY_REPORT names a file, appended to it."""
+    line = json.dumps(tally.as_dict())
+    path = os.environ.get("GLS_PARITY_REPORT")
+    if path:
+        with open(path, "a") as f:
+            f.write(line + "\n")
+    print(line)
 
 
 def _verify_case(gls, oracle, cfg, chunk, **shape):
