@@ -132,7 +132,10 @@ static Plan make_plan4(long long rows, long long V, int dtype, bool multi) {
 // number of rows (the kernel specialised for its set is faster where the sweep is what a step costs).
 static Plan make_plan_step(long long rows1, long long rows2, long long V, int dtype) {
   Plan p = make_plan4(rows1 + rows2, V, dtype, false);
-  p.two_launches = (double)(rows1 + rows2) * (double)V * (dtype == GLS_BF16 ? 2.0 : 4.0) > 128e6;
+#ifndef GLS_STEP_ONE_LAUNCH_BYTES
+#define GLS_STEP_ONE_LAUNCH_BYTES 128e6
+#endif
+  p.two_launches = (double)(rows1 + rows2) * (double)V * (dtype == GLS_BF16 ? 2.0 : 4.0) > GLS_STEP_ONE_LAUNCH_BYTES;
   p.chunk1 = p.chunk2 = p.chunk;
   p.splits1 = p.splits2 = p.splits;
   if (p.two_launches) {

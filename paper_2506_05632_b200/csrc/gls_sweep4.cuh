@@ -496,12 +496,6 @@ __device__ __forceinline__ void s4_item(const SweepArgs& A, int row, int split, 
   }
 }
 
-// the same out of line, so that two variants in one kernel are each compiled on their own
-template <int SH, bool LSE, int ROUNDS>
-__device__ __noinline__ void s4_item_call(const SweepArgs& A, int row, int split, uint32_t tag) {
-  s4_item<SH, LSE, ROUNDS, false>(A, row, split, tag);
-}
-
 // LSEMODE 0: races only (draft side, decoders); 1: races and the rows' log-sum-exp (target side,
 // encoder); 2: two sets of rows in one launch, the first without and the second with the
 // log-sum-exp (the fused draft + verify call).
@@ -518,9 +512,9 @@ sweep4_kernel(const __grid_constant__ SweepArgs A) {
     const int row = A.row_begin + (int)(item - (long long)split * A.row_count);
     if constexpr (LSEMODE == 2) {
       if (row >= A.rows1)
-        s4_item_call<SH, true, ROUNDS>(A, row, split, tag);
+        s4_item<SH, true, ROUNDS, false>(A, row, split, tag);
       else
-        s4_item_call<SH, false, ROUNDS>(A, row, split, tag);
+        s4_item<SH, false, ROUNDS, false>(A, row, split, tag);
     } else {
       s4_item<SH, LSEMODE == 1, ROUNDS, MULTI>(A, row, split, tag);
     }
