@@ -372,13 +372,15 @@ __device__ __forceinline__ void s4_item(const SweepArgs& A, int row, int split, 
         nms = scaled_offset(nm4);
       }
     };
-    auto flush_batch = [&]() {
+    auto flush_batch = [&](bool last) {
       __syncwarp();
       const int nb = min(qn, 32);
       qn -= nb;
       uint32_t e = s4_flush<SH, ROUNDS, MULTI>(A.rounds, qn, nb, nm4 - 4.0f);
-      // the slices of a row trade their bounds through the row's hint word at batch time
-      if (A.splits > 1) {
+      // the slices of a row trade their bounds through the row's hint word at batch time (not
+      // after the item's last batch: nothing is left to filter, and the item publishes its bound
+      // when it ends)
+      if (A.splits > 1 && !last) {
         uint32_t h = 0u;
         if (lane == 0) h = e > m_enc ? atomicMax(A.hints + row, e) : __ldcg(A.hints + row);
         e = max(e, __shfl_sync(0xffffffffu, h, 0));
@@ -425,7 +427,7 @@ __device__ __forceinline__ void s4_item(const SweepArgs& A, int row, int split, 
           }
         }
         if (qn < 32) break;
-        flush_batch();
+        flush_batch(false);
       }
     } else {
       // ---- the sweep.  The inner loop runs until 32 groups are queued; the batched evaluation
@@ -457,11 +459,11 @@ __device__ __forceinline__ void s4_item(const SweepArgs& A, int row, int split, 
           poll_bound();
         }
         if (qn < 32) break;
-        flush_batch();
+        flush_batch(false);
       }
     }
     // ---- drain the queue ---------------------------------------------------------------------
-    while (qn > 0) flush_batch();
+    while (qn > 0) flush_batch(qn <= 32);
 
     // ---- combine the lanes; every warp writes its own partial result ---------------------------
     Top2 t2 = sh.best[threadIdx.x];
