@@ -28,7 +28,7 @@ constexpr int kGPad = 16;           // floats per group in shared memory; its fo
                                     // stored XOR-swizzled by (group >> 1) & 3: conflict-free 128-bit reads
 constexpr int kGMaxD = 16;
 constexpr int kGMaxK = 8;
-constexpr int kGFlushAt = 16;                   // a batch is taken as soon as this many groups are queued
+constexpr int kGFlushAt = 8;                    // a batch is taken as soon as this many groups are queued
 constexpr int kGQueue = kGFlushAt + 32;         // one (row, stream) test adds at most 32 per warp
 constexpr int kGMaxQuads = 4;                   // warp quads per CTA, each walking its own row blocks
 
@@ -37,7 +37,7 @@ struct GaussRowCtx {  // one row of the current block
   uint32_t m_enc;         // ordered code of the row's bound
   int row, b;             // row number (-1: past the end), source sample
   int msg;                // label a candidate must carry (decoder pass with labels)
-  int pad;
+  float nms;              // the group test's offset for the bound the row had when the block was set up
 };
 struct __align__(16) GaussEntry {  // a queued group: coarse word, group | stream << 28, row slot, weights
   uint32_t w, g, slot, pad;
@@ -46,16 +46,17 @@ struct __align__(16) GaussEntry {  // a queued group: coarse word, group | strea
 // Shared memory of one warp quad (four warps that walk the same row blocks); the coarse words
 // [stream-row][word][lane] follow it, then the next quad's block.
 struct __align__(16) GaussQuad {
-  float mu[kGMaxD][kGRows];                       // scaled means of the block's rows
-  GaussRowCtx ctx[kGRows];
-  Top2 best[kGWarps][kGRows];                     // per warp and row slot
-  float lse_m[kGWarps][kGRows], lse_s[kGWarps][kGRows];
+  // [2]: the block being worked on and the next one, which is set up meanwhile
+  float mu[2][kGMaxD][kGRows];                    // scaled means of the block's rows
+  GaussRowCtx ctx[2][kGRows];
+  Top2 best[2][kGWarps][kGRows];                  // per warp and row slot
+  float lse_m[2][kGWarps][kGRows], lse_s[2][kGWarps][kGRows];
   GaussEntry queue[kGWarps][kGQueue];
 };
-// Layout: quads x (GaussQuad, coarse words [kGRows * streams][4][32]), labels [128][4], then the
+// Layout: quads x (GaussQuad, coarse words [2][kGRows * streams][4][32]), labels [128][4], then the
 // tile [(D + 1)][128 * kGPad] floats, plane D holding |u|^2 / (2 s2_prior).
 __host__ __device__ inline size_t gauss_quad_bytes(int streams) {
-  return sizeof(GaussQuad) + (size_t)kGRows * streams * 4 * 32 * sizeof(uint32_t);
+  return sizeof(GaussQuad) + (size_t)2 * kGRows * streams * 4 * 32 * sizeof(uint32_t);
 }
 __host__ __device__ inline size_t gauss_smem_bytes(int D, int streams, int quads) {
   return (size_t)quads * gauss_quad_bytes(streams) + 128 * 4 * sizeof(uint32_t) +
@@ -67,7 +68,7 @@ __host__ __device__ inline size_t gauss_smem_bytes(int D, int streams, int quads
 // The lanes' results are merged per row slot into sh.best[warp][slot]; improved bounds go to the
 // row's context and to its hint word.
 template <int ROUNDS, bool ENC>
-__device__ __noinline__ void gauss_flush(const SweepArgs& A, GaussQuad& sh, int first, int n) {
+__device__ __noinline__ void gauss_flush(const SweepArgs& A, GaussQuad& sh, int buf, int first, int n) {
   const int lane = threadIdx.x & 31;
   const int warp = (threadIdx.x >> 5) & (kGWarps - 1);
   constexpr float c2 = kLog2e;
@@ -80,10 +81,10 @@ __device__ __noinline__ void gauss_flush(const SweepArgs& A, GaussQuad& sh, int 
   top2_init(b);
   float lower = -CUDART_INF_F;
   const uint8_t* bins = nullptr;
-  GaussRowCtx cx = sh.ctx[0];
+  GaussRowCtx cx = sh.ctx[buf][0];
   if (lane < n) {
     slot = (int)e.slot;
-    cx = sh.ctx[slot];
+    cx = sh.ctx[buf][slot];
     bins = A.bins ? A.bins + A.bins_sb * cx.b : nullptr;
     g = e.g;
     ks = g >> 28;
@@ -149,12 +150,12 @@ __device__ __noinline__ void gauss_flush(const SweepArgs& A, GaussQuad& sh, int 
     top2_warp_merge(m);
     const uint32_t enc = __reduce_max_sync(0xffffffffu, enc_ordered(lo));
     if (lane == 0) {
-      Top2 cur = sh.best[warp][r];
+      Top2 cur = sh.best[buf][warp][r];
       top2_offer(cur, m.s1, m.i1);
       top2_offer(cur, m.s2, m.i2);
-      sh.best[warp][r] = cur;
-      const uint32_t old = atomicMax(&sh.ctx[r].m_enc, enc);
-      if (enc > old) atomicMax(A.hints + sh.ctx[r].row, enc);
+      sh.best[buf][warp][r] = cur;
+      const uint32_t old = atomicMax(&sh.ctx[buf][r].m_enc, enc);
+      if (enc > old) atomicMax(A.hints + sh.ctx[buf][r].row, enc);
     }
   }
   __syncwarp();
@@ -187,8 +188,9 @@ gauss_sweep_kernel(const __grid_constant__ SweepArgs A, int n_ranges, int rows_p
   constexpr int kPlane = 128 * kGPad;
   const size_t quad_bytes = gauss_quad_bytes(n_streams);
   GaussQuad& sh = *reinterpret_cast<GaussQuad*>(gls_smem_raw + (size_t)quad * quad_bytes);
-  uint32_t (*const xw)[4][32] =
+  uint32_t (*const xw_all)[4][32] =  // [2 * kGRows * n_streams][4][32]: buffer p starts at p * kGRows * n_streams
       reinterpret_cast<uint32_t(*)[4][32]>(gls_smem_raw + (size_t)quad * quad_bytes + sizeof(GaussQuad));
+  const int xw_stride = kGRows * n_streams;
   uint32_t (*const labels)[4] =
       reinterpret_cast<uint32_t(*)[4]>(gls_smem_raw + (size_t)n_quads * quad_bytes);
   float* const us = reinterpret_cast<float*>(gls_smem_raw + (size_t)n_quads * quad_bytes + 128 * 4 * sizeof(uint32_t));
@@ -249,17 +251,16 @@ gauss_sweep_kernel(const __grid_constant__ SweepArgs A, int n_ranges, int rows_p
       }
     }
   };
-  auto commit = [&](int row0) {
+  auto commit = [&](int row0, int buf) {
     const int idx = tq;
     if (idx < kGRows * D) {
       const int r = idx / D, d = idx - r * D;
-      sh.mu[d][r] = pf_mu[0];
+      sh.mu[buf][d][r] = pf_mu[0];
     }
     if (tq < kGRows) {
       const int r = tq;
       const int row = row0 + r;
       GaussRowCtx cx;
-      cx.pad = 0;
       cx.row = row < row_hi ? row : -1;
       const int b = ENC ? row : row / K;
       const int k = ENC ? 0 : row - b * K;
@@ -269,13 +270,12 @@ gauss_sweep_kernel(const __grid_constant__ SweepArgs A, int n_ranges, int rows_p
       cx.seq = pf_seq;
       cx.msg = pf_msg;
       cx.m_enc = cx.row >= 0 ? pf_hint : 0u;
-      sh.ctx[r] = cx;
-#pragma unroll
-      for (int w2 = 0; w2 < kGWarps; ++w2) top2_init(sh.best[w2][r]);
+      cx.nms = scaled_offset(filter_offset(dec_ordered(cx.m_enc)) + 4.0f);
+      sh.ctx[buf][r] = cx;
     }
   };
   // coarse words of the block's stream-rows: warp w computes stream-rows sr = w, w + 4, ...
-  auto coarse_words = [&](int row0) {
+  auto coarse_words = [&](int row0, int buf) {
     for (int sr = warp; sr < kGRows * n_streams; sr += kGWarps) {
       const int r = sr / n_streams, ks = sr - r * n_streams;
       const int row = row0 + r;
@@ -286,10 +286,11 @@ gauss_sweep_kernel(const __grid_constant__ SweepArgs A, int n_ranges, int rows_p
       const uint32_t seq = A.seq_ids ? __ldg(A.seq_ids + b) : A.seq_base + (uint32_t)b;
       uint32_t cw[4];
       philox4x32<ROUNDS>(A.rk, A.rounds, ((uint32_t)tile << 5) | (uint32_t)lane, c1, A.pos_base, seq, cw);
-      xw[sr][0][lane] = cw[0];
-      xw[sr][1][lane] = cw[1];
-      xw[sr][2][lane] = cw[2];
-      xw[sr][3][lane] = cw[3];
+      uint32_t (*const xo)[32] = xw_all[buf * xw_stride + sr];
+      xo[0][lane] = cw[0];
+      xo[1][lane] = cw[1];
+      xo[2][lane] = cw[2];
+      xo[3][lane] = cw[3];
     }
   };
   // The blocks of rows are walked in a rotated order that differs from tile to tile: CTAs that run
@@ -301,10 +302,12 @@ gauss_sweep_kernel(const __grid_constant__ SweepArgs A, int n_ranges, int rows_p
   const int rot = (int)(((uint32_t)tile * 2654435761u >> 8) % (uint32_t)n_blocks);
   auto block_row = [&](int it) { return row_lo + ((it + rot) % n_blocks) * kGRows; };
   __syncthreads();  // the tile is in shared memory
+  // every row slot's running results start empty in both buffers
+  if (tq < 2 * kGWarps * kGRows) top2_init((&sh.best[0][0][0])[tq]);
   if (quad < n_blocks) {
     fetch(block_row(quad));
-    commit(block_row(quad));
-    coarse_words(block_row(quad));
+    commit(block_row(quad), 0);
+    coarse_words(block_row(quad), 0);
   }
   quad_sync();
 
@@ -315,8 +318,10 @@ gauss_sweep_kernel(const __grid_constant__ SweepArgs A, int n_ranges, int rows_p
   GaussEntry* const queue = sh.queue[warp];
   const bool group_in_range = cand0 + (long long)gl * 16 < N;
 
-  for (int it = quad; it < n_blocks; it += n_quads) {
+  int buf = 0;  // the buffer of the block being worked on
+  for (int it = quad; it < n_blocks; it += n_quads, buf ^= 1) {
     const int row0 = block_row(it);
+    uint32_t (*const xw)[4][32] = xw_all + buf * xw_stride;
     if (it + n_quads < n_blocks) fetch(block_row(it + n_quads));
     // ---- weights of the lane's 16 candidates for the block's four rows -----------------------
     unsigned long long acc[kGRows][8];
@@ -326,7 +331,7 @@ gauss_sweep_kernel(const __grid_constant__ SweepArgs A, int n_ranges, int rows_p
       for (int p = 0; p < 8; ++p) acc[r][p] = 0ull;
 #pragma unroll 2
     for (int d = 0; d < D; ++d) {
-      const float2 m2 = *reinterpret_cast<const float2*>(&sh.mu[d][0]);
+      const float2 m2 = *reinterpret_cast<const float2*>(&sh.mu[buf][d][0]);
       unsigned long long up[8];
 #pragma unroll
       for (int q = 0; q < 4; ++q) {
@@ -362,7 +367,7 @@ gauss_sweep_kernel(const __grid_constant__ SweepArgs A, int n_ranges, int rows_p
     }
 #pragma unroll
     for (int r = 0; r < kGRows; ++r) {
-      const GaussRowCtx cx = sh.ctx[r];
+      const GaussRowCtx cx = sh.ctx[buf][r];
       if (cx.row < 0) continue;  // uniform over the CTA
       float wgt[16];
       float amax = -CUDART_INF_F;
@@ -373,17 +378,6 @@ gauss_sweep_kernel(const __grid_constant__ SweepArgs A, int n_ranges, int rows_p
         wgt[2 * p] = pn[2 * p] - s0;
         wgt[2 * p + 1] = pn[2 * p + 1] - s1;
         amax = fmaxf(amax, fmaxf(wgt[2 * p], wgt[2 * p + 1]));
-      }
-      if (use_labels) {  // maximum over the candidates that carry the transmitted label
-        const uint32_t m4 = (uint32_t)cx.msg * 0x01010101u;
-        amax = -CUDART_INF_F;
-#pragma unroll
-        for (int q = 0; q < 4; ++q) {
-          const uint32_t eq = __vcmpeq4(lab[q], m4);  // 0xff per matching byte
-#pragma unroll
-          for (int t = 0; t < 4; ++t)
-            if (eq & (1u << (8 * t))) amax = fmaxf(amax, wgt[4 * q + t]);
-        }
       }
       if (ENC) {
         // the lane's share of sum_i exp(weight_i), relative to its own maximum; lanes are merged
@@ -402,16 +396,29 @@ gauss_sweep_kernel(const __grid_constant__ SweepArgs A, int n_ranges, int rows_p
 #pragma unroll
         for (int dd = 16; dd > 0; dd >>= 1) ls += __shfl_xor_sync(0xffffffffu, ls, dd);
         if (lane == 0) {
-          sh.lse_m[warp][r] = wm;
-          sh.lse_s[warp][r] = ls;
+          sh.lse_m[buf][warp][r] = wm;
+          sh.lse_s[buf][warp][r] = ls;
         }
       }
-      const float nm4 = filter_offset(dec_ordered(cx.m_enc)) + 4.0f;
-      const float nms = scaled_offset(nm4);
-      const float thr = exp2_upper_from_scaled(amax, kLog2e * (1.0f / 126.0f), nms);
+      const float thr = exp2_upper_from_scaled(amax, kLog2e * (1.0f / 126.0f), cx.nms);
       for (int ks = 0; ks < n_streams; ++ks) {
         const uint32_t w = xw[r * n_streams + ks][warp][lane];
-        const bool pass = group_in_range && coarse_lower(w) <= thr;
+        bool pass = group_in_range && coarse_lower(w) <= thr;
+        if (use_labels && pass) {
+          // second look, for the few groups that pass on all sixteen: the maximum over the
+          // candidates that carry the transmitted label (with L_max labels the best eligible
+          // score lies about ln L_max lower, and that many more groups pass the first test)
+          const uint32_t m4 = (uint32_t)cx.msg * 0x01010101u;
+          float emax = -CUDART_INF_F;
+#pragma unroll
+          for (int q = 0; q < 4; ++q) {
+            const uint32_t eq = __vcmpeq4(lab[q], m4);  // 0xff per matching byte
+#pragma unroll
+            for (int t = 0; t < 4; ++t)
+              if (eq & (1u << (8 * t))) emax = fmaxf(emax, wgt[4 * q + t]);
+          }
+          pass = coarse_lower(w) <= exp2_upper_from_scaled(emax, kLog2e * (1.0f / 126.0f), cx.nms);
+        }
         const unsigned bal = __ballot_sync(0xffffffffu, pass);
         if (bal != 0u) {
           if (pass) {
@@ -428,7 +435,7 @@ gauss_sweep_kernel(const __grid_constant__ SweepArgs A, int n_ranges, int rows_p
             __syncwarp();
             const int nb = min(qn, 32);
             qn -= nb;
-            gauss_flush<ROUNDS, ENC>(A, sh, qn, nb);
+            gauss_flush<ROUNDS, ENC>(A, sh, buf, qn, nb);
           }
         }
       }
@@ -437,30 +444,39 @@ gauss_sweep_kernel(const __grid_constant__ SweepArgs A, int n_ranges, int rows_p
       __syncwarp();
       const int nb = min(qn, 32);
       qn -= nb;
-      gauss_flush<ROUNDS, ENC>(A, sh, qn, nb);
+      gauss_flush<ROUNDS, ENC>(A, sh, buf, qn, nb);
     }
-    quad_sync();  // every warp's results for this block are in shared memory
-    // ---- warp r (< rows per block) merges row slot r and writes its partial result; then the
-    //      next block is set up
+    // ---- the next block is set up in the other buffer (its global values were fetched before
+    //      this block's arithmetic); one barrier per block
+    if (it + n_quads < n_blocks) {
+      commit(block_row(it + n_quads), buf ^ 1);
+      coarse_words(block_row(it + n_quads), buf ^ 1);
+    }
+    quad_sync();  // this block's results and the next block's set-up are in shared memory
+    // ---- warp r (< rows per block) merges row slot r of this block, writes its partial result and
+    //      empties the slot for the block after next, while the other warps go on: buffer `buf` is
+    //      written again only after the next barrier, which this warp reaches after the merge
     {
       const int r = warp;
       const int row = row0 + r;
-      if (r < kGRows && row < row_hi && lane == 0) {
-        Top2 m = sh.best[0][r];
+      if (r < kGRows && lane == 0) {
+        Top2 m = sh.best[buf][0][r];
         float lm = kGroupLseFloor, ls = 0.f;
 #pragma unroll
         for (int w2 = 1; w2 < kGWarps; ++w2) {
-          top2_offer(m, sh.best[w2][r].s1, sh.best[w2][r].i1);
-          top2_offer(m, sh.best[w2][r].s2, sh.best[w2][r].i2);
+          top2_offer(m, sh.best[buf][w2][r].s1, sh.best[buf][w2][r].i1);
+          top2_offer(m, sh.best[buf][w2][r].s2, sh.best[buf][w2][r].i2);
         }
+#pragma unroll
+        for (int w2 = 0; w2 < kGWarps; ++w2) top2_init(sh.best[buf][w2][r]);
         if (ENC) {
 #pragma unroll
-          for (int w2 = 0; w2 < kGWarps; ++w2) lm = fmaxf(lm, sh.lse_m[w2][r]);
+          for (int w2 = 0; w2 < kGWarps; ++w2) lm = fmaxf(lm, sh.lse_m[buf][w2][r]);
 #pragma unroll
           for (int w2 = 0; w2 < kGWarps; ++w2)
-            ls += sh.lse_s[w2][r] * ex2_approx((sh.lse_m[w2][r] - lm) * kLog2e);
+            ls += sh.lse_s[buf][w2][r] * ex2_approx((sh.lse_m[buf][w2][r] - lm) * kLog2e);
         }
-        if (m.i1 >= 0 || (ENC && ls > 0.f)) {
+        if (row < row_hi && (m.i1 >= 0 || (ENC && ls > 0.f))) {
           Partial pr;
           pr.s1 = m.s1; pr.i1 = m.i1; pr.s2 = m.s2; pr.i2 = m.i2;
           pr.lm = lm; pr.ls = ls; pr.pad0 = 0; pr.pad1 = 0;
@@ -469,12 +485,6 @@ gauss_sweep_kernel(const __grid_constant__ SweepArgs A, int n_ranges, int rows_p
         }
       }
     }
-    quad_sync();  // the merge has read the block's results
-    if (it + n_quads < n_blocks) {
-      commit(block_row(it + n_quads));
-      coarse_words(block_row(it + n_quads));
-    }
-    quad_sync();
   }
   asm volatile("griddepcontrol.launch_dependents;");
 }
