@@ -41,13 +41,15 @@ struct TopmWarpBuf {
 
 // Keeps the M largest of the n buffered entries (ties: first come, i.e. lowest index), in their
 // order of arrival; returns the new count and the code of the M-th largest.  Requires n > M.
-__device__ __noinline__ int topm_prune(TopmWarpBuf* wb, int n, int M, uint32_t* kth_out) {
+// last_pass: 0 for fp32 logits; 2 for bf16 logits, whose codes differ in their upper 16 bits only
+// (the lower 16 are all zero or all one with the sign), so two of the four radix passes suffice.
+__device__ __noinline__ unsigned long long topm_prune(TopmWarpBuf* wb, int n, int M, int last_pass) {
   const int lane = threadIdx.x & 31;
   const uint32_t lt = (1u << lane) - 1u;
   uint32_t prefix = 0u;
   int remaining = M;  // rank still to find among the entries that share `prefix`
 #pragma unroll 1
-  for (int pass = 3; pass >= 0; --pass) {
+  for (int pass = 3; pass >= last_pass; --pass) {
     for (int i = lane; i < 256; i += 32) wb->hist[i] = 0u;
     __syncwarp();
     const int shift = 8 * pass;
@@ -89,7 +91,8 @@ __device__ __noinline__ int topm_prune(TopmWarpBuf* wb, int n, int M, uint32_t* 
     prefix = (prefix << 8) | (uint32_t)bin;
     __syncwarp();
   }
-  const uint32_t kth = prefix;
+  // bf16: complete the code (its lower half repeats the inverted top bit)
+  const uint32_t kth = last_pass == 2 ? (prefix << 16) | ((prefix & 0x8000u) ? 0u : 0xffffu) : prefix;
   int out = 0, ties_seen = 0;
 #pragma unroll 1
   for (int base = 0; base < n; base += 32) {
@@ -111,19 +114,19 @@ __device__ __noinline__ int topm_prune(TopmWarpBuf* wb, int n, int M, uint32_t* 
     ties_seen += __popc(eqb);
     __syncwarp();
   }
-  *kth_out = kth;
-  return out;
+  return ((unsigned long long)kth << 32) | (unsigned)out;  // (code of the M-th largest, new count)
 }
 
 // Batched examination of queued groups: lane l < nb takes group queue[first + l], reads its 16
 // logits again (L2 hits) and appends the tokens above the current threshold to the token buffer,
 // in index order (the queue is in index order, lanes append in lane order).  Then the buffer is
 // pruned if it has grown past M + 64.  Returns the new count; *thr is raised by a prune.
+// Returns (threshold bits << 32) | new count; the threshold is raised by a prune.
 template <int DT>
-__device__ __noinline__ int topm_expand(TopmWarpBuf* wb, const int* queue, const char* rowp, int V,
-                                        int first, int nb, int n, int M, float* thr_io) {
+__device__ __noinline__ unsigned long long topm_expand(TopmWarpBuf* wb, const int* queue,
+                                                       const char* rowp, int V, int first, int nb,
+                                                       int n, int M, float thr) {
   const int lane = threadIdx.x & 31;
-  const float thr = *thr_io;
   float a[16];
   uint32_t m = 0u;
   int tok = 0;
@@ -156,11 +159,11 @@ __device__ __noinline__ int topm_expand(TopmWarpBuf* wb, const int* queue, const
   n += __shfl_sync(0xffffffffu, incl, 31);
   __syncwarp();
   if (n > M + 64) {
-    uint32_t kth;
-    n = topm_prune(wb, n, M, &kth);
-    *thr_io = dec_ordered(kth);
+    const unsigned long long r = topm_prune(wb, n, M, DT == kBF16 ? 2 : 0);
+    n = (int)(unsigned)r;
+    thr = dec_ordered((uint32_t)(r >> 32));
   }
-  return n;
+  return ((unsigned long long)__float_as_uint(thr) << 32) | (unsigned)n;
 }
 
 template <int DT>
@@ -227,15 +230,15 @@ topm_select_kernel(const TopmArgs T) {
       }
       if (qn == 0 && s >= n_steps) break;
       __syncwarp();
-      for (int first = 0; first < qn; first += 32)
-        n = topm_expand<DT>(wb, queue, rowp, T.V, first, min(32, qn - first), n, T.M, &thr);
+      for (int first = 0; first < qn; first += 32) {
+        const unsigned long long r = topm_expand<DT>(wb, queue, rowp, T.V, first, min(32, qn - first), n, T.M, thr);
+        n = (int)(unsigned)r;
+        thr = __uint_as_float((uint32_t)(r >> 32));
+      }
       qn = 0;
       if (s >= n_steps) break;
     }
-    if (n > T.M) {
-      uint32_t kth;
-      n = topm_prune(wb, n, T.M, &kth);
-    }
+    if (n > T.M) n = (int)(unsigned)topm_prune(wb, n, T.M, DT == kBF16 ? 2 : 0);
     __syncwarp();
     for (int i = lane; i < T.M; i += 32) {
       T.ids[row * T.M + i] = i < n ? wb->idx[i] : -1;
