@@ -127,6 +127,9 @@ typedef struct {
 #define GLS_COMBINE_ACTIVE 0u /* Algorithm 2 as printed: the min over k runs over the active set */
 #define GLS_COMBINE_ALL 1u    /* Appendix B, strong drafter invariance: min over all k           */
 #define GLS_NO_BONUS 2u       /* target rows cover positions 0..L-1 only; no bonus token         */
+/* How gls_target_sample_verify walks Algorithm 2 (same results either way; default: by size).  */
+#define GLS_VERIFY_ALL_ROWS 4u    /* race every target row, then run the loop on the row results  */
+#define GLS_VERIFY_ACTIVE_ROWS 8u /* position by position: only rows of active drafts are read    */
 
 /* Library version, major * 10000 + minor * 100 + patch. */
 int gls_version(void);
@@ -218,7 +221,8 @@ int gls_compress_gaussian(const float* candidates, const float* source, const fl
  * still belong to the caller.
  *
  * Limits and rules:
- *   - A problem whose scratch need, gls_workspace_bytes(B, K, J, V), exceeds
+ *   - A problem whose scratch need (that of gls_draft_sample: hints, partial results and row
+ *     results of the B * K * J rows; never more than gls_workspace_bytes(B, K, J, V)) exceeds
  *     GLS_STATIC_SCRATCH_BYTES is refused with GLS_ERR_STATIC_LIMIT and nothing is enqueued
  *     (gls_static_scratch_bytes() returns the limit at run time).
  *   - The first call on each device looks up the buffer's device address (one

@@ -12,6 +12,7 @@ _SRC_DIR = os.path.join(_HERE, "csrc")
 _LIB = os.path.join(_HERE, "libgls.so")
 
 COMBINE_ACTIVE, COMBINE_ALL, NO_BONUS = 0, 1, 2
+VERIFY_ALL_ROWS, VERIFY_ACTIVE_ROWS = 4, 8  # how the dense verify call walks Algorithm 2
 NOISE_SHARED_ACROSS_K = 1
 DEV_EMPTY_SUPPORT = 1
 F32, BF16 = 0, 1

@@ -42,6 +42,11 @@ static int num_sms() {
 }
 constexpr int kMinChunk = 2048;
 constexpr int kMaxChunk = 16384;
+// Target rows of a verify call, in bytes, from which Algorithm 2 is walked position by position
+#ifndef GLS_STEPWISE_MIN_BYTES
+#define GLS_STEPWISE_MIN_BYTES 256e6
+#endif
+constexpr int kMaxPhases = 4;  // phases of such a walk (two are used: position 0, the rest)
 
 struct Plan {
   int chunk, splits, parts;
@@ -155,6 +160,29 @@ static Plan make_plan_step(long long rows1, long long rows2, long long V, int dt
   return p;
 }
 
+// Position-by-position verification (noise_spec 4): partial-result slots for the finest slicing a
+// position can get, and after the hints and partials the state of the walk (active sets, row
+// lists and their lengths) in place of the per-row results.
+template <int SH>
+static Plan make_plan_stepwise_t(int B, int K, int J, long long V) {
+  Plan p = Plan();
+  p.rows = (long long)B * K * J;
+  p.chunk = 0;
+  p.splits = listed_max_splits((int)V, S4Cfg<SH>::kCtaTokens);
+  p.per_slice = S4Cfg<SH>::kWarps;
+  p.parts = p.splits * S4Cfg<SH>::kWarps;
+  plan_layout(p);
+  p.total = p.off_rows + align_up((size_t)B * sizeof(unsigned long long), 256) +
+            align_up((size_t)kMaxPhases * sizeof(int), 256) + align_up((size_t)J * B * K * sizeof(int), 256);
+  return p;
+}
+static Plan make_plan_stepwise(int B, int K, int J, long long V, int dtype, bool multi = false) {
+  const int sh = s4_shape(dtype, V, multi);
+  return sh == kS4ShapeBf16 ? make_plan_stepwise_t<kS4ShapeBf16>(B, K, J, V)
+         : sh == kS4ShapeF32Wide ? make_plan_stepwise_t<kS4ShapeF32Wide>(B, K, J, V)
+                                 : make_plan_stepwise_t<kS4ShapeF32Narrow>(B, K, J, V);
+}
+
 static Plan make_plan(long long rows, long long V, int spec, int dtype, bool multi = false) {
   return spec == 4 ? make_plan4(rows, V, dtype, multi) : make_plan1(rows, V);
 }
@@ -167,7 +195,8 @@ static Plan make_plan(long long rows, long long V, int spec, int dtype, bool mul
 // Warp-collective; the result is valid in lane 0.
 template <int DT, int SPEC, int ROUNDS>
 __device__ __forceinline__ RowResult finalize_row(const SweepArgs& A, int row, int with_lse,
-                                                  uint32_t* __restrict__ dev_status) {
+                                                  uint32_t* __restrict__ dev_status,
+                                                  int parts_in_use = 0) {
   const int lane = threadIdx.x & 31;
   constexpr int ES = DT == kBF16 ? 2 : 4;
   const RowLoc rl = locate_row<ES>(A, row);
@@ -175,7 +204,7 @@ __device__ __forceinline__ RowResult finalize_row(const SweepArgs& A, int row, i
   const float inv_t = rl.inv_t;
   const float c2 = inv_t * kLog2e;
 
-  const int used = rl.second ? A.parts2 : A.parts1;
+  const int used = parts_in_use > 0 ? parts_in_use : rl.second ? A.parts2 : A.parts1;
   const int n_parts = used > 0 ? used : A.parts;  // slots in use
   Top2 best;
   top2_init(best);
@@ -433,6 +462,146 @@ finalize_verify_kernel(const __grid_constant__ SweepArgs A, const VerifyArgs va)
   if (threadIdx.x < 32)
     verify_sequence_warp(srows, b, va.K, va.L, va.J, va.flags, va.multi_rows, dtok, va.out_tokens,
                          va.out_num, va.accept, va.out_scores, va.dev_status);
+}
+
+// ------------------------------------------------------------------------------------------
+// Algorithm 2 in phases.  Y_j needs the target rows of the drafts that are still active at
+// position j and nothing else, and nothing at all is needed past the stopping time, so the
+// verification can read far fewer rows than the call is given.  The positions are cut into
+// phases [j0, j1); a phase sweeps the rows (b, k, j) of its positions for the drafts k active
+// when it starts (sweep4_listed_kernel over a row list in device memory), then one kernel reduces
+// them, walks the phase's positions (emits Y_j, prunes the active set) and lists the rows of the
+// next phase.  The first phase is position 0 alone, where every draft is active; most drafts
+// are pruned there, so the second phase takes all remaining positions of the few survivors.
+// State in the workspace: the active set of every sequence, a row list and its length per phase.
+// ------------------------------------------------------------------------------------------
+struct PhasedState {
+  unsigned long long* active;  // [B]
+  int* counts;                 // [kMaxPhases]
+  int* lists;                  // phase p at lists + B * K * (its first position): row numbers
+};
+
+__global__ void phased_init_kernel(const VerifyArgs va, const PhasedState S, int first_end,
+                                   uint32_t* __restrict__ hints) {
+  const long long t = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  const long long BK = (long long)va.B * va.K;
+  // first phase: every draft is active at positions [0, first_end); Appendix B on a row per draft
+  // reads the row of the lowest active draft only, draft 0 at position 0
+  if (va.multi_rows) {
+    if (t < (long long)va.B * first_end) S.lists[t] = (int)((t / first_end) * va.K * va.J + t % first_end);
+  } else if (t < BK * first_end) {
+    S.lists[t] = (int)((t / first_end) * va.J + t % first_end);
+  }
+  if (t < va.B) {
+    S.active[t] = va.K >= 64 ? ~0ull : ((1ull << va.K) - 1ull);
+    va.out_num[t] = 0;
+  }
+  if (t < kMaxPhases) S.counts[t] = t == 0 ? (int)((va.multi_rows ? va.B : BK) * first_end) : 0;
+  if (t < BK * va.J) hints[t] = 0u;
+  if (t < (long long)va.B * va.J) {
+    va.out_tokens[t] = -1;
+    if (va.out_scores) va.out_scores[t] = 0.f;
+  }
+  if (t < BK * va.L) va.accept[t] = 0;
+}
+
+// Phase `phase` = positions [j0, j1) of every sequence that is still running; the next phase (if
+// any) is [j1, j2).  A CTA per sequence, a warp per listed row, then one warp walks the positions.
+template <int DT, int ROUNDS>
+__global__ void __launch_bounds__(kFusedVerifyMaxWarps * 32)
+phased_verify_kernel(const __grid_constant__ SweepArgs A, const VerifyArgs va, const PhasedState S,
+                     int phase, int j0, int j1, int j2, int cta_tokens, int sweep_grid,
+                     int warps_per_slice) {
+  RowResult* srows = reinterpret_cast<RowResult*>(gls_smem_raw);  // [K][j1 - j0]
+  const int b = blockIdx.x;
+  const int lane = threadIdx.x & 31;
+  unsigned long long active = S.active[b];  // written by the previous phase, complete by now
+  asm volatile("griddepcontrol.wait;" ::: "memory");  // the sweep before this launch is complete
+  if (active == 0ull) return;
+  const int K = va.K, L = va.L, J = va.J, W = j1 - j0;
+  const ListedSlicing sl = listed_slicing(S.counts[phase], A.V, cta_tokens, sweep_grid);
+  for (int r = threadIdx.x >> 5; r < K * W; r += (int)(blockDim.x >> 5)) {
+    const int k = r / W, j = j0 + r % W;
+    if (!((active >> k) & 1ull)) continue;
+    if (va.multi_rows && j0 == 0 && k != 0) continue;  // the first phase listed draft 0 only
+    const RowResult rr = finalize_row<DT, 4, ROUNDS>(A, (b * K + k) * J + j, 1, nullptr,
+                                                     sl.splits * warps_per_slice);
+    if (lane == 0) srows[r] = rr;
+  }
+  __syncthreads();
+  if (threadIdx.x >= 32) return;
+  int n_out = j0;
+  for (int j = j0; j < j1; ++j) {
+    // Y_j: the best of the active rows' winners after subtracting each row's log-sum-exp; ties:
+    // lowest token, then lowest k.  Appendix B on a row per draft: the row of the lowest active
+    // draft, which was raced under all K streams.
+    const int kref = va.multi_rows ? __ffsll((long long)active) - 1 : -1;
+    double bs = -CUDART_INF;
+    int bi = -1;
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+      const int k = lane + 32 * h;
+      if (k >= K || !((active >> k) & 1ull)) continue;
+      if (va.multi_rows && k != kref) continue;
+      const RowResult r = srows[k * W + (j - j0)];
+      if (r.idx < 0) continue;
+      const double sc = r.score - r.lse;
+      if (bi < 0 || sc > bs || (sc == bs && r.idx < bi)) {
+        bs = sc;
+        bi = r.idx;
+      }
+    }
+#pragma unroll
+    for (int d = 16; d > 0; d >>= 1) {
+      const double os = __shfl_xor_sync(0xffffffffu, bs, d);
+      const int oi = __shfl_xor_sync(0xffffffffu, bi, d);
+      if (oi >= 0 && (bi < 0 || os > bs || (os == bs && oi < bi))) {
+        bs = os;
+        bi = oi;
+      }
+    }
+    if (lane == 0) {
+      va.out_tokens[(long long)b * J + j] = bi;
+      if (va.out_scores) va.out_scores[(long long)b * J + j] = bi >= 0 ? (float)bs : CUDART_NAN_F;
+      if (bi < 0 && va.dev_status) atomicOr(va.dev_status, GLS_DEV_EMPTY_SUPPORT);
+    }
+    n_out = j + 1;
+    if (j == L) {  // bonus token
+      active = 0ull;
+      break;
+    }
+    unsigned long long next = 0ull;
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+      const int k = lane + 32 * h;
+      const bool ok = k < K && ((active >> k) & 1ull) && bi >= 0 &&
+                      va.draft_tokens[((long long)b * K + k) * L + j] == bi;
+      if (ok) va.accept[((long long)b * K + k) * L + j] = 1;
+      next |= (unsigned long long)__ballot_sync(0xffffffffu, ok) << (32 * h);
+    }
+    active = next;
+    if (active == 0ull) break;
+  }
+  if (n_out >= J) active = 0ull;
+  if (active != 0ull) {  // the survivors' rows at the positions of the next phase
+    const int W2 = j2 - j1;
+    int base = 0;
+    if (lane == 0) base = atomicAdd(&S.counts[phase + 1], __popcll(active) * W2);
+    base = __shfl_sync(0xffffffffu, base, 0);
+    int* list = S.lists + (long long)va.B * K * j1;
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+      const int k = lane + 32 * h;
+      if (k < K && ((active >> k) & 1ull)) {
+        const int rank = __popcll(active & ((1ull << k) - 1ull));
+        for (int jj = 0; jj < W2; ++jj) list[base + rank * W2 + jj] = (b * K + k) * J + j1 + jj;
+      }
+    }
+  }
+  if (lane == 0) {
+    S.active[b] = active;
+    if (active == 0ull) va.out_num[b] = n_out;
+  }
 }
 
 // The fused draft + verify call: a CTA per sequence finalises the sequence's K x L draft rows
@@ -826,6 +995,69 @@ static int run_rows(SweepArgs& A, int dtype, int spec, const Plan& P, void* work
   return err == cudaSuccess ? GLS_OK : GLS_ERR_CUDA;
 }
 
+// Algorithm 2 in phases: per phase a sweep over the listed rows and the kernel that walks the
+// phase's positions.
+template <int SH, int ROUNDS, bool MULTI>
+static int run_verify_stepwise_t(SweepArgs& A, const VerifyArgs& va, const Plan& P, void* workspace,
+                                 cudaStream_t st) {
+  constexpr int DT = S4Cfg<SH>::kDT;
+  char* ws = (char*)workspace;
+  A.chunk = 0;
+  A.splits = 0;
+  A.parts = P.parts;
+  A.rows = (int)P.rows;
+  A.hints = (uint32_t*)(ws + P.off_hints);
+  A.partials = (Partial*)(ws + P.off_partials);
+  PhasedState S;
+  size_t off = P.off_rows;
+  S.active = (unsigned long long*)(ws + off);
+  off += align_up((size_t)va.B * sizeof(unsigned long long), 256);
+  S.counts = (int*)(ws + off);
+  off += align_up((size_t)kMaxPhases * sizeof(int), 256);
+  S.lists = (int*)(ws + off);
+  const long long BK = (long long)va.B * va.K;
+  // phases: position 0, then everything else
+  int ends[kMaxPhases];
+  int n_phases = 0;
+  ends[n_phases++] = 1;
+  if (va.J > 1) ends[n_phases++] = va.J;
+  {
+    const long long n = BK * va.J;  // the largest index range the initialisation covers
+    phased_init_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(va, S, ends[0], A.hints);
+  }
+  const long long cap = (long long)num_sms() * S4Cfg<SH>::kCtasPerSM;
+  const int warps = kFusedVerifyMaxWarps;
+  int j0 = 0;
+  for (int p = 0; p < n_phases; ++p) {
+    const int j1 = ends[p], j2 = p + 1 < n_phases ? ends[p + 1] : j1;
+    const long long most = BK * (j1 - j0) * P.splits;  // items if every row of the phase is listed
+    const int grid = (int)(most < cap ? most : cap);
+    sweep4_listed_kernel<SH, ROUNDS, MULTI><<<grid, S4Cfg<SH>::kWarps * 32, sizeof(S4Shared<SH>), st>>>(
+        A, S.lists + BK * j0, S.counts + p);
+    const int nrows = va.K * (j1 - j0);
+    cudaLaunchAttribute attr;
+    cudaLaunchConfig_t cfg = dependent_launch(&attr, va.B, (nrows < warps ? nrows : warps) * 32,
+                                              (size_t)nrows * sizeof(RowResult), st);
+    if (cudaLaunchKernelEx(&cfg, phased_verify_kernel<DT, ROUNDS>, A, va, S, p, j0, j1, j2,
+                           (int)S4Cfg<SH>::kCtaTokens, grid, (int)S4Cfg<SH>::kWarps) != cudaSuccess)
+      return GLS_ERR_CUDA;
+    j0 = j1;
+  }
+  return cudaGetLastError() == cudaSuccess ? GLS_OK : GLS_ERR_CUDA;
+}
+static int run_verify_stepwise(SweepArgs& A, int dtype, const VerifyArgs& va, const Plan& P,
+                               void* workspace, cudaStream_t st) {
+  const int sh = s4_shape(dtype, A.V, va.multi_rows);
+  const bool r10 = A.rounds == 10;
+#define STEPWISE(SH, M) (r10 ? run_verify_stepwise_t<SH, 10, M>(A, va, P, workspace, st) \
+                             : run_verify_stepwise_t<SH, 0, M>(A, va, P, workspace, st))
+  if (va.multi_rows) return sh == kS4ShapeBf16 ? STEPWISE(kS4ShapeBf16, true) : STEPWISE(kS4ShapeF32Narrow, true);
+  if (sh == kS4ShapeBf16) return STEPWISE(kS4ShapeBf16, false);
+  if (sh == kS4ShapeF32Wide) return STEPWISE(kS4ShapeF32Wide, false);
+  return STEPWISE(kS4ShapeF32Narrow, false);
+#undef STEPWISE
+}
+
 static bool sizes_ok(int B, int K, int J, int64_t V) {
   if (B <= 0 || K <= 0 || K > GLS_MAX_K || J <= 0 || V <= 0) return false;
   if (V >= (1LL << 31) - 4 * kS4MaxCtaTokens) return false;
@@ -867,9 +1099,9 @@ const char* gls_status_string(int status) {
   }
 }
 
-size_t gls_workspace_bytes(int B, int K, int J, int64_t V) {
-  if (!sizes_ok(B, K, J, V)) return 0;
-  // the largest need over the noise layouts and element types (the call may use any of them)
+// scratch of a call that races every row it is given: the largest need over the noise layouts and
+// element types (the call may use any of them)
+static size_t all_rows_workspace(int B, int K, int J, int64_t V) {
   size_t need = make_plan1((long long)B * K * J, V).total;
   for (int dt = 0; dt < 2; ++dt) {
     const size_t d = make_plan4((long long)B * K * J, V, dt, false).total;
@@ -882,9 +1114,21 @@ size_t gls_workspace_bytes(int B, int K, int J, int64_t V) {
   return need;
 }
 
+size_t gls_workspace_bytes(int B, int K, int J, int64_t V) {
+  if (!sizes_ok(B, K, J, V)) return 0;
+  size_t need = all_rows_workspace(B, K, J, V);
+  for (int dt = 0; dt < 2; ++dt) {
+    for (int multi = 0; multi < 2; ++multi) {  // verification in phases
+      const size_t g = make_plan_stepwise(B, K, J, V, dt, multi != 0).total;
+      if (g > need) need = g;
+    }
+  }
+  return need;
+}
+
 size_t gls_draft_verify_workspace_bytes(int B, int K, int L, int J, int64_t V) {
   if (L < 1 || J < L || J > L + 1 || !sizes_ok(B, K, L + J, V)) return 0;
-  size_t need = 0;
+  size_t need = gls_workspace_bytes(B, K, J, V);  // large inputs: a draft call, then a verify call
   for (int dt = 0; dt < 2; ++dt) {
     const size_t t = make_plan_step((long long)B * K * L, (long long)B * K * J, V, dt).total;
     if (t > need) need = t;
@@ -927,7 +1171,9 @@ int gls_target_sample_verify(const gls_rows_t* target_logits, int B, int K, int 
                              uint32_t flags, int32_t* out_tokens, int32_t* out_num_tokens,
                              uint8_t* out_accept, float* out_scores, void* workspace,
                              size_t workspace_bytes, uint32_t* device_status, void* stream) {
-  if (flags & ~(GLS_COMBINE_ALL | GLS_NO_BONUS)) return GLS_ERR_INVALID_ARG;
+  if (flags & ~(GLS_COMBINE_ALL | GLS_NO_BONUS | GLS_VERIFY_ALL_ROWS | GLS_VERIFY_ACTIVE_ROWS))
+    return GLS_ERR_INVALID_ARG;
+  if ((flags & GLS_VERIFY_ALL_ROWS) && (flags & GLS_VERIFY_ACTIVE_ROWS)) return GLS_ERR_INVALID_ARG;
   const int J = L + ((flags & GLS_NO_BONUS) ? 0 : 1);
   if (!noise || !out_tokens || !out_num_tokens || L < 0 || !sizes_ok(B, K, J, V))
     return GLS_ERR_INVALID_ARG;
@@ -947,7 +1193,17 @@ int gls_target_sample_verify(const gls_rows_t* target_logits, int B, int K, int 
   // and the epilogue reads the row of the lowest active draft.
   const bool multi = (flags & GLS_COMBINE_ALL) && target_logits->stride_k != 0 && K > 1;
   if (multi && (spec != 4 || K > 8 || V >= (1LL << 28))) return GLS_ERR_UNSUPPORTED;
-  const Plan P = make_plan((long long)B * K * J, V, spec, target_logits->dtype, multi);
+  // Position by position (only the rows of active drafts are read) when the walk can prune
+  // anything and the rows are large enough for its J rounds of launches to pay.
+  const bool can_step = spec == 4 && (multi || !(flags & GLS_COMBINE_ALL)) && L >= 1 && J >= 2 &&
+                        (size_t)K * (J - 1) * sizeof(RowResult) <= kFusedVerifyMaxSmem;
+  if ((flags & GLS_VERIFY_ACTIVE_ROWS) && !can_step) return GLS_ERR_UNSUPPORTED;
+  const double bytes = (double)B * K * J * (double)V * (target_logits->dtype == GLS_BF16 ? 2.0 : 4.0);
+  const bool stepwise = can_step && ((flags & GLS_VERIFY_ACTIVE_ROWS) ||
+                                     (!(flags & GLS_VERIFY_ALL_ROWS) && bytes >= GLS_STEPWISE_MIN_BYTES));
+  flags &= ~(GLS_VERIFY_ALL_ROWS | GLS_VERIFY_ACTIVE_ROWS);
+  const Plan P = stepwise ? make_plan_stepwise(B, K, J, V, target_logits->dtype, multi)
+                          : make_plan((long long)B * K * J, V, spec, target_logits->dtype, multi);
   if (!workspace || workspace_bytes < P.total) return GLS_ERR_WORKSPACE;
   if (multi) A.multi_k = K;
   A.data = target_logits->data;
@@ -968,6 +1224,7 @@ int gls_target_sample_verify(const gls_rows_t* target_logits, int B, int K, int 
   va.accept = out_accept;
   va.out_scores = out_scores;
   va.dev_status = device_status;
+  if (stepwise) return run_verify_stepwise(A, target_logits->dtype, va, P, workspace, st);
   bool fused = false;
   rc = run_rows(A, target_logits->dtype, spec, P, workspace, true, nullptr, nullptr, nullptr, st,
                 &va, &fused);
@@ -1015,6 +1272,20 @@ int gls_draft_verify(const gls_rows_t* draft_logits, const gls_rows_t* target_lo
   if ((flags & GLS_COMBINE_ALL) && target_logits->stride_k != 0 && K > 1) return GLS_ERR_UNSUPPORTED;
   if (fused_verify_smem(K, L, J) > kFusedVerifyMaxSmem) return GLS_ERR_UNSUPPORTED;
   const long long rows_d = (long long)B * K * L, rows_t = (long long)B * K * J;
+  // Large target rows: the draft rows first, then Algorithm 2 in phases, which reads the target
+  // rows of active drafts only (the draft tokens it needs are this call's own output).
+  if (J >= 2 && !(flags & GLS_COMBINE_ALL) &&
+      (double)rows_t * (double)V * (target_logits->dtype == GLS_BF16 ? 2.0 : 4.0) >= GLS_STEPWISE_MIN_BYTES) {
+    if (!workspace || workspace_bytes < gls_draft_verify_workspace_bytes(B, K, L, J, V)) return GLS_ERR_WORKSPACE;
+    rc = gls_draft_sample(draft_logits, B, K, L, V, inv_temp_draft, inv_temp_per_draft_host, noise,
+                          out_draft_tokens, out_draft_scores, workspace, workspace_bytes, device_status,
+                          stream);
+    if (rc != GLS_OK) return rc;
+    return gls_target_sample_verify(target_logits, B, K, L, V, inv_temp_target, out_draft_tokens, noise,
+                                    flags | GLS_VERIFY_ACTIVE_ROWS, out_tokens, out_num_tokens,
+                                    out_accept, out_scores, workspace, workspace_bytes, device_status,
+                                    stream);
+  }
   const Plan P = make_plan_step(rows_d, rows_t, V, draft_logits->dtype);
   if (!workspace || workspace_bytes < P.total) return GLS_ERR_WORKSPACE;
   A.data = draft_logits->data;
@@ -1532,7 +1803,7 @@ int gls_draft_sample_static(const gls_rows_t* draft_logits, int B, int K, int J,
                             const gls_noise_t* noise, int32_t* out_tokens, float* out_scores,
                             uint32_t* device_status, void* stream) {
   if (!gls::sizes_ok(B, K, J, V)) return GLS_ERR_INVALID_ARG;
-  const size_t need = gls_workspace_bytes(B, K, J, V);
+  const size_t need = all_rows_workspace(B, K, J, V);  // what gls_draft_sample may use
   if (need == 0) return GLS_ERR_INVALID_ARG;
   if (need > (size_t)GLS_STATIC_SCRATCH_BYTES) return GLS_ERR_STATIC_LIMIT;
   void* scratch = nullptr;

@@ -235,9 +235,11 @@ __device__ __noinline__ void lse4_redo_careful(const char* rowp, int tok0, int n
 // ------------------------------------------------------------------------------------------
 // The kernel
 // ------------------------------------------------------------------------------------------
-// One work item: slice `split` of row `row`, swept by the calling CTA.
+// One work item: slice `split` of row `row`, swept by the calling CTA; rows are cut into `splits`
+// slices of `chunk` tokens.
 template <int SH, bool LSE, int ROUNDS, bool MULTI>
-__device__ __forceinline__ void s4_item(const SweepArgs& A, int row, int split, uint32_t tag) {
+__device__ __forceinline__ void s4_item(const SweepArgs& A, int row, int split, uint32_t tag,
+                                        const int chunk, const int splits) {
   constexpr int DT = S4Cfg<SH>::kDT;
   S4Shared<SH>& sh = s4_shared<SH>();
   const int lane = threadIdx.x & 31;
@@ -249,8 +251,8 @@ __device__ __forceinline__ void s4_item(const SweepArgs& A, int row, int split, 
   uint2* const queue = sh.queue[warp];
   volatile unsigned long long* const m_tag = &sh.m_tag;
   {
-    const int tok_begin = split * A.chunk;  // a multiple of 2048
-    const int tok_end = min(A.V, tok_begin + A.chunk);
+    const int tok_begin = split * chunk;  // a multiple of 2048
+    const int tok_end = min(A.V, tok_begin + chunk);
     uint32_t c1, pos, seq;
     const char* rowp;
     float c2;
@@ -288,7 +290,7 @@ __device__ __forceinline__ void s4_item(const SweepArgs& A, int row, int split, 
     const int tok0 = base_w + lane * 16;  // the lane's first group; its others follow at +512 tokens
 
     // bound published by earlier slices of the row (the hint words are cleared only when rows are cut)
-    uint32_t m_enc = A.splits > 1 ? __ldcg(A.hints + row) : 0u;
+    uint32_t m_enc = splits > 1 ? __ldcg(A.hints + row) : 0u;
     float lm = kGroupLseFloor;
     unsigned long long ls2 = 0ull;
     int qn = 0;
@@ -380,7 +382,7 @@ __device__ __forceinline__ void s4_item(const SweepArgs& A, int row, int split, 
       // the slices of a row trade their bounds through the row's hint word at batch time (not
       // after the item's last batch: nothing is left to filter, and the item publishes its bound
       // when it ends)
-      if (A.splits > 1 && !last) {
+      if (splits > 1 && !last) {
         uint32_t h = 0u;
         if (lane == 0) h = e > m_enc ? atomicMax(A.hints + row, e) : __ldcg(A.hints + row);
         e = max(e, __shfl_sync(0xffffffffu, h, 0));
@@ -493,7 +495,7 @@ __device__ __forceinline__ void s4_item(const SweepArgs& A, int row, int split, 
       pr.lm = lm; pr.ls = ls; pr.pad0 = 0; pr.pad1 = 0;
       if (GLS_IN_RANGE(split * kWarps + warp, 0, A.parts, 23u) && GLS_IN_RANGE(row, 0, A.rows, 24u))
         A.partials[(long long)row * A.parts + split * kWarps + warp] = pr;
-      if (A.splits > 1 && m_enc > 0u) atomicMax(A.hints + row, m_enc);
+      if (splits > 1 && m_enc > 0u) atomicMax(A.hints + row, m_enc);
     }
   }
 }
@@ -514,14 +516,64 @@ sweep4_kernel(const __grid_constant__ SweepArgs A) {
     const int row = A.row_begin + (int)(item - (long long)split * A.row_count);
     if constexpr (LSEMODE == 2) {
       if (row >= A.rows1)
-        s4_item<SH, true, ROUNDS, false>(A, row, split, tag);
+        s4_item<SH, true, ROUNDS, false>(A, row, split, tag, A.chunk, A.splits);
       else
-        s4_item<SH, false, ROUNDS, false>(A, row, split, tag);
+        s4_item<SH, false, ROUNDS, false>(A, row, split, tag, A.chunk, A.splits);
     } else {
-      s4_item<SH, LSEMODE == 1, ROUNDS, MULTI>(A, row, split, tag);
+      s4_item<SH, LSEMODE == 1, ROUNDS, MULTI>(A, row, split, tag, A.chunk, A.splits);
     }
   }
   // this block has no more work: a dependent launch (the reduction) may start to be scheduled
+  asm volatile("griddepcontrol.launch_dependents;");
+}
+
+// ------------------------------------------------------------------------------------------
+// Rows named by a list in device memory (the position-by-position verification of Algorithm 2:
+// the rows of a position are those of the drafts still active there, known only on the device).
+// The slicing follows from the number of listed rows: as many slices per row as let one round of
+// work items fill the launch, each at least four steps long.
+// ------------------------------------------------------------------------------------------
+struct ListedSlicing {
+  int chunk, splits;
+};
+__host__ __device__ __forceinline__ int listed_max_splits(int V, int cta_tokens) {
+  const int steps = (V + cta_tokens - 1) / cta_tokens;
+  return steps >= 8 ? steps / 4 : 1;
+}
+__host__ __device__ __forceinline__ ListedSlicing listed_slicing(int n_rows, int V, int cta_tokens,
+                                                                 int grid) {
+  const int steps = (V + cta_tokens - 1) / cta_tokens;
+  int want = n_rows > 0 ? grid / n_rows : 1;
+  const int cap = listed_max_splits(V, cta_tokens);
+  if (want > cap) want = cap;
+  if (want < 1) want = 1;
+  const int chunk_steps = (steps + want - 1) / want;
+  ListedSlicing r;
+  r.chunk = chunk_steps * cta_tokens;
+  r.splits = (steps + chunk_steps - 1) / chunk_steps;
+  return r;
+}
+
+// Races and log-sum-exp of the rows list[0 .. *count): the target side of one phase (MULTI: every
+// row under all of the call's noise streams at once, Appendix B).
+template <int SH, int ROUNDS, bool MULTI>
+__global__ void __launch_bounds__(S4Cfg<SH>::kWarps * 32, S4Cfg<SH>::kCtasPerSM)
+sweep4_listed_kernel(const __grid_constant__ SweepArgs A, const int* __restrict__ list,
+                     const int* __restrict__ count) {
+  S4Shared<SH>& sh = s4_shared<SH>();
+  if (threadIdx.x == 0) sh.m_tag = 0ull;
+  __syncthreads();
+  const int n = __ldcg(count);
+  const ListedSlicing sl = listed_slicing(n, A.V, S4Cfg<SH>::kCtaTokens, (int)gridDim.x);
+  const long long n_items = (long long)n * sl.splits;
+  uint32_t tag = 0u;
+  for (long long item = blockIdx.x; item < n_items; item += gridDim.x) {
+    ++tag;
+    const int split = (int)(item / n);
+    const int row = __ldcg(list + (int)(item - (long long)split * n));
+    if (GLS_IN_RANGE(row, 0, A.rows, 27u))
+      s4_item<SH, true, ROUNDS, MULTI>(A, row, split, tag, sl.chunk, sl.splits);
+  }
   asm volatile("griddepcontrol.launch_dependents;");
 }
 

@@ -403,7 +403,7 @@ def test_host_detectable_errors(gls):
     with pytest.raises(gls.GlsError):
         gls.draft_sample(x.cpu())
     with pytest.raises(gls.GlsError):
-        gls.target_sample_verify(x, tok, flags=8)
+        gls.target_sample_verify(x, tok, flags=16)
     with pytest.raises(gls.GlsError):
         gls.draft_sample(torch.zeros(1, 65, 1, 8, device="cuda"))
     # the context is still usable afterwards
@@ -445,3 +445,45 @@ def test_draft_verify_in_one_call(gls, oracle, dtype):
         gls.draft_verify(x, x[:, :, :2].repeat(1, 1, 2, 1)[:, :, :3], spec=1)
     with pytest.raises(gls.GlsError):  # both sets must have one element type
         gls.draft_verify(x, x[:, :, :2].repeat(1, 1, 2, 1)[:, :, :3].to(torch.bfloat16))
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+def test_verify_position_by_position(gls, oracle, dtype):
+    """Algorithm 2 walked position by position (only the rows of active drafts are read) against
+    the oracle and against the walk that races every row first: rows long enough to be cut into
+    several slices, one draft, no bonus row, a sequence count that is not a multiple of anything."""
+    for cfg, B, K, L, V in ((3, 9, 8, 5, 70001), (4, 7, 8, 8, 40000), (2, 16, 4, 4, 3000),
+                            (3, 5, 1, 3, 20000), (2, 3, 33, 2, 2500)):
+        w = synth.verify_workload(cfg, "cuda", B=B, K=K, L=L, V=V)
+        d, t = w.draft_logits.to(dtype), w.target_logits.to(dtype)
+        kw = dict(seed=w.noise_seed, inv_temp=w.inv_temp)
+        refd = oracle.draft_sample(synth.to_numpy_rows(d), **kw)
+        dtok = torch.from_numpy(refd["tokens"]).cuda()
+        for extra, tt in ((0, t), (gls.NO_BONUS, t[:, :, :L])):
+            ref = oracle.target_sample_verify(synth.to_numpy_rows(tt.contiguous()), dtok.cpu().numpy(),
+                                              flags=extra, **kw)
+            outs = {}
+            for how in (gls.VERIFY_ACTIVE_ROWS, gls.VERIFY_ALL_ROWS):
+                status = torch.zeros(1, dtype=torch.int32, device="cuda")
+                out = parity.to_np(gls.target_sample_verify(tt, dtok, flags=extra | how, status=status, **kw))
+                parity.check_verify(out, ref, "cfg%d flags %d" % (cfg, extra | how))
+                assert int(status.item()) == 0
+                outs[how] = out
+            a, e = outs[gls.VERIFY_ACTIVE_ROWS], outs[gls.VERIFY_ALL_ROWS]
+            same = (a["tokens"] == e["tokens"]).all(axis=1)
+            assert same.mean() > 0.9  # they may part only at a near-tie
+            assert (a["tau"][same] == e["tau"][same]).all()
+            assert (a["accept"][same] == e["accept"][same]).all()
+            if 1 < K <= 8:  # Appendix B on a row per draft: the row of the lowest active draft only
+                refb = oracle.target_sample_verify(synth.to_numpy_rows(tt.contiguous()), dtok.cpu().numpy(),
+                                                   flags=extra | gls.COMBINE_ALL, **kw)
+                for how in (gls.VERIFY_ACTIVE_ROWS, gls.VERIFY_ALL_ROWS):
+                    out = parity.to_np(gls.target_sample_verify(tt, dtok, flags=extra | gls.COMBINE_ALL | how, **kw))
+                    parity.check_verify(out, refb, "cfg%d Appendix B flags %d" % (cfg, extra | how))
+    # the walk in phases needs the default noise layout and rows that it can leave out
+    with pytest.raises(gls.GlsError):
+        gls.target_sample_verify(t[:, :1].expand_as(t), dtok, flags=gls.VERIFY_ACTIVE_ROWS | gls.COMBINE_ALL, **kw)
+    with pytest.raises(gls.GlsError):
+        gls.target_sample_verify(t, dtok, flags=gls.VERIFY_ACTIVE_ROWS, spec=1, **kw)
+    with pytest.raises(gls.GlsError):
+        gls.target_sample_verify(t, dtok, flags=gls.VERIFY_ACTIVE_ROWS | gls.VERIFY_ALL_ROWS, **kw)
