@@ -235,6 +235,23 @@ def _event_ms(fn, steps, flush=None, warmup=3):
     return statistics.mean(a.elapsed_time(b) for a, b in ev)
 
 
+def _verify_call_record(pkg, target_logits, L, out, ms, peak, flags=0, spec=4):
+    """Time, rows and bytes of one verify call whose results are in `out`.  Walked in phases the
+    call reads position 0 of every draft (under Appendix B on a row per draft: of draft 0) and the
+    remaining positions of the drafts that survive position 0; otherwise every row."""
+    B, K, J, V = target_logits.shape
+    es = target_logits.element_size()
+    walk = pkg.verify_walk(target_logits, L, flags, spec) if spec == 4 else 0
+    rows = B * K * J
+    if walk == 1:
+        survivors = int(out["accept"][:, :, 0].sum().item())
+        rows = (B if (flags & pkg.COMBINE_ALL) else B * K) + survivors * (J - 1)
+    r = _fracs(rows * V * es, ms, peak)
+    r.update(walk="phases" if walk == 1 else "every row", rows_read=rows, rows_given=B * K * J,
+             bytes_read=rows * V * es)
+    return r
+
+
 def _measure_verify(cfg_id, steps, peak, spec=4):
     """One verification workload: draft call, verify call, the fused call and (small inputs) a
     replayed CUDA graph, L2-cold; Appendix B's variant of the verify call."""
@@ -263,17 +280,27 @@ def _measure_verify(cfg_id, steps, peak, spec=4):
         pkg.draft_verify(w.draft_logits, w.target_logits, out_draft_tokens=buf.draft_tokens,
                          out_draft_scores=buf.draft_scores, out=buf.out, **kw)
 
+    def verify_every_row():
+        pkg.target_sample_verify(w.target_logits, buf.draft_tokens, out=buf.out,
+                                 flags=pkg.VERIFY_ALL_ROWS, **kw)
+
     def verify_all():
         pkg.target_sample_verify(w.target_logits, buf.draft_tokens, out=buf.out,
                                  flags=pkg.COMBINE_ALL, **kw)
 
     res = {"workload": WORKLOAD_DESC["cfg%d" % cfg_id],
            "l2": "flushed between calls" if small else "inputs larger than L2",
-           "draft_call": _fracs(db, _event_ms(draft, steps, flush), peak),
-           "verify_call": _fracs(tb, _event_ms(verify, steps, flush), peak),
-           "one_call": _fracs(db + tb, _event_ms(fused, steps, flush), peak)}
-    res["verified_positions_per_s"] = B * L / (res["one_call"]["ms"] * 1e-3)
-    res["verify_call_appendix_b"] = _fracs(tb, _event_ms(verify_all, max(3, steps // 4), flush), peak)
+           "draft_call": _fracs(db, _event_ms(draft, steps, flush), peak)}
+    v_ms = _event_ms(verify, steps, flush)
+    res["verify_call"] = _verify_call_record(pkg, w.target_logits, L, buf.out, v_ms, peak)
+    one_ms = _event_ms(fused, steps, flush)
+    res["one_call"] = _fracs(db + res["verify_call"]["bytes_read"], one_ms, peak)
+    res["verified_positions_per_s"] = B * L / (one_ms * 1e-3)
+    if res["verify_call"]["walk"] == "phases":
+        res["verify_call_every_row_raced"] = _fracs(tb, _event_ms(verify_every_row, steps, flush), peak)
+    ab_ms = _event_ms(verify_all, max(3, steps // 4), flush)
+    res["verify_call_appendix_b"] = _verify_call_record(pkg, w.target_logits, L, buf.out, ab_ms, peak,
+                                                        flags=pkg.COMBINE_ALL)
     if small:
         res["l2_warm"] = {"draft_call_ms": _event_ms(draft, steps), "verify_call_ms": _event_ms(verify, steps),
                           "one_call_ms": _event_ms(fused, steps)}
@@ -541,38 +568,54 @@ def run_ours(args):
         return
 
     peak, which = _peaks()
-    achieved = tbytes / (verify_ms * 1e-3) / 1e9
-    kname = {4: "sweep4_kernel", 3: "sweep3_kernel"}.get(args.spec, "sweep_kernel") + "<%s, lse>" % (
-        "bf16" if w.target_logits.dtype == torch.bfloat16 else "f32")
+    bf = w.target_logits.dtype == torch.bfloat16
+    vrec = None
     if args.topm:
-        kname = "topm_select_kernel<%s> + sparse_verify_kernel" % (
-            "bf16" if w.target_logits.dtype == torch.bfloat16 else "f32")
-    kdesc = (" (target side: selection of the top-M tokens of every row, then the race on the lists; "
-             "the event bracket is the whole call)") if args.topm else (
-        " (target side: the dominant kernel; the event bracket "
-        "is the whole call, which also runs finalize_verify_kernel, ~4 % of it, so the "
-        "kernel alone is slightly faster than reported)")
-    roofline = {"bound": "hbm", "kernel": kname + kdesc,
+        achieved, k_ms, k_bytes = tbytes / (verify_ms * 1e-3) / 1e9, verify_ms, tbytes
+        kname = "topm_select_kernel<%s> + sparse_verify_kernel (target side: selection of the top-M " \
+                "tokens of every row, then the race on the lists; the event bracket is the whole call)" % (
+                    "bf16" if bf else "f32")
+    else:
+        vrec = _verify_call_record(pkg, w.target_logits, L, buf.out, verify_ms, peak, spec=args.spec)
+        sweep = {4: "sweep4_kernel", 3: "sweep3_kernel"}.get(args.spec, "sweep_kernel")
+        if draft_ms >= verify_ms:
+            # the verify call reads few rows: the draft rows' sweep is the dominant kernel
+            achieved, k_ms, k_bytes = dbytes / (draft_ms * 1e-3) / 1e9, draft_ms, dbytes
+            kname = "%s<%s> (draft side: the dominant kernel; the event bracket is the whole draft call, " \
+                    "which also runs finalize_rows_kernel, ~3 %% of it)" % (sweep, "bf16" if bf else "f32")
+        else:
+            achieved, k_ms, k_bytes = vrec["gbs"], verify_ms, vrec["bytes_read"]
+            kname = "%s<%s, lse> (target side: the dominant kernel; the event bracket is the whole verify " \
+                    "call, reduction and Algorithm 2's loop included)" % (sweep, "bf16" if bf else "f32")
+    step_bytes = dbytes + (vrec["bytes_read"] if vrec else tbytes)
+    roofline = {"bound": "hbm", "kernel": kname,
                 "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                 "peak_source": "of " + which,
                 "frac_of_nominal_8TBs": achieved / 8000.0,
-                "traffic": (TRAFFIC_RATIO * tbytes) if (TRAFFIC_RATIO and args.spec == 4 and not args.topm) else None,
-                "algorithmic_bytes": tbytes, "ms": verify_ms,
-                "draft_side": {"achieved": dbytes / (draft_ms * 1e-3) / 1e9, "ms": draft_ms,
-                               "frac": dbytes / (draft_ms * 1e-3) / 1e9 / peak,
-                               "frac_of_nominal_8TBs": dbytes / (draft_ms * 1e-3) / 8e12},
-                "step": {"achieved": (dbytes + tbytes) / (ms_per_step * 1e-3) / 1e9,
-                         "frac_of_nominal_8TBs": (dbytes + tbytes) / (ms_per_step * 1e-3) / 8e12}}
+                "traffic": (TRAFFIC_RATIO * k_bytes) if (TRAFFIC_RATIO and args.spec == 4 and not args.topm) else None,
+                "algorithmic_bytes": k_bytes, "ms": k_ms,
+                "draft_call": _fracs(dbytes, draft_ms, peak),
+                "verify_call": vrec if vrec else _fracs(tbytes, verify_ms, peak),
+                "step": _fracs(step_bytes, ms_per_step, peak)}
     if rank == 0 and world == 1 and not args.topm and not args.no_extras:
-        # Appendix B's variant of the verify call (every target row raced under all K streams)
+        n_x = max(3, min(args.steps, 10))
+        if vrec["walk"] == "phases":
+            # the walk that races every target row first: what the call cost before Algorithm 2's
+            # active sets were used to leave rows unread
+            er_ms = _event_ms(lambda: pkg.target_sample_verify(
+                w.target_logits, buf.draft_tokens, out=buf.out, workspace=buf.workspace, status=buf.status,
+                flags=pkg.VERIFY_ALL_ROWS, **kw), n_x, flush)
+            roofline["verify_call_every_row_raced"] = _fracs(tbytes, er_ms, peak)
+        # Appendix B's variant of the verify call (rows raced under all K streams)
         ab_ms = _event_ms(lambda: pkg.target_sample_verify(
             w.target_logits, buf.draft_tokens, out=buf.out, workspace=buf.workspace, status=buf.status,
-            flags=pkg.COMBINE_ALL, **kw), max(3, min(args.steps, 10)), flush)
-        roofline["verify_call_appendix_b"] = _fracs(tbytes, ab_ms, peak)
+            flags=pkg.COMBINE_ALL, **kw), n_x, flush)
+        roofline["verify_call_appendix_b"] = _verify_call_record(pkg, w.target_logits, L, buf.out, ab_ms,
+                                                                 peak, flags=pkg.COMBINE_ALL, spec=args.spec)
     if sustained is not None:
-        sustained["verify_call"] = _fracs(tbytes, sustained["verify_call_ms"], peak)
+        sustained["verify_call"] = _fracs(vrec["bytes_read"], sustained["verify_call_ms"], peak)
         sustained["draft_call"] = _fracs(dbytes, sustained["draft_call_ms"], peak)
-        sustained["step"] = _fracs(dbytes + tbytes, sustained["ms_per_step"], peak)
+        sustained["step"] = _fracs(step_bytes, sustained["ms_per_step"], peak)
         roofline["sustained"] = sustained
     del w, buf
     torch.cuda.empty_cache()
@@ -610,9 +653,13 @@ def run_ours(args):
                        "l2_warm": l2_warm, "cuda_graph_replay": graphed,
                        "l2": "flushed between steps" if flush is not None
                        else "inputs (%.2f GB) larger than L2" % ((dbytes + tbytes) / 1e9),
+                       "bytes_given": dbytes + tbytes, "bytes_read": step_bytes,
                        "mean_tau": tau_mean, "other_workloads": others},
-            "hbm_gbs": (dbytes + tbytes) / (ms_per_step * 1e-3) / 1e9,
-            "clocks": clocks, "e2e": e2e, "gpu_launches": 4 * args.steps,
+            "hbm_gbs": step_bytes / (ms_per_step * 1e-3) / 1e9,
+            # draft call: sweep + reduction; verify call: sweep + reduction with Algorithm 2's
+            # loop, or in phases: initialisation + 2 x (sweep over the listed rows + walk)
+            "clocks": clocks, "e2e": e2e,
+            "gpu_launches": (4 if args.topm else 7 if vrec["walk"] == "phases" else 2 if args.fused else 4) * args.steps,
             "roofline": roofline, "cpu_baseline": cpu}
     print(json.dumps(line))
     if dist is not None:

@@ -273,6 +273,20 @@ int gls_target_sample_verify(const gls_rows_t* target_logits, int B, int K, int 
                              size_t workspace_bytes, uint32_t* device_status, void* stream);
 
 /*
+ * Which way gls_target_sample_verify would walk Algorithm 2 for these arguments (no counterpart
+ * in the paper; the results do not depend on it).  0: every target row is raced, then the loop
+ * runs on the row results.  1: in phases -- position 0 of every draft, then the remaining positions
+ * of the drafts still active -- so that a target row is read only while Algorithm 2 can still use
+ * it: B * K rows plus (J - 1) rows per draft that survives position 0, instead of B * K * J
+ * (under GLS_COMBINE_ALL on a row per draft: B rows plus (J - 1) per survivor).  Chosen by size
+ * unless `flags` carries GLS_VERIFY_ALL_ROWS or GLS_VERIFY_ACTIVE_ROWS; the walk in phases
+ * needs the default noise layout, L >= 1 and J >= 2, and under GLS_COMBINE_ALL a row per draft.
+ * row_per_draft: target rows' stride_k != 0.  Returns -1 for arguments the call would refuse.
+ */
+int gls_verify_walk(int dtype, int row_per_draft, int B, int K, int L, int64_t V, int noise_spec,
+                    uint32_t flags);
+
+/*
  * Draft phase and verification in one call -- Algorithm 2 from its draft loop to its end, for the
  * case where both sets of logits are resident (all L draft positions are known, e.g. a drafter
  * that is not autoregressive in the tokens sampled here, a replayed or re-scored step, or the
@@ -280,7 +294,9 @@ int gls_target_sample_verify(const gls_rows_t* target_logits, int B, int K, int 
  * gls_draft_sample(draft_logits, J = L) followed by gls_target_sample_verify(target_logits, the
  * tokens just drawn), bit for bit, but one sweep launch covers both sets of rows and one
  * reduction launch finalises the draft rows, the target rows and Algorithm 2's loop, which halves
- * the number of launches of a step (what bounds small batches).
+ * the number of launches of a step (what bounds small batches).  Inputs for which
+ * gls_verify_walk() answers 1 are large enough that launches do not matter: there the call runs
+ * the draft rows first and then Algorithm 2 in phases on the tokens just drawn.
  *
  *   draft_logits       [B,K,L,V] rows, temperature inv_temp_draft (or per draft, host array [K])
  *   target_logits      [B,K,J,V] rows, J = L + 1 (J = L with GLS_NO_BONUS), temperature

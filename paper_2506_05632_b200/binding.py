@@ -419,6 +419,21 @@ def target_sample_verify(logits, draft_tokens, inv_temp=1.0, flags=0, seed=0, se
     return out
 
 
+def verify_walk(target_logits, L, flags=0, spec=4):
+    """1 if target_sample_verify would walk Algorithm 2 in phases for these rows (reading the rows
+    of active drafts only), 0 if it would race every row first; GlsError for refused arguments."""
+    B, K, J, V = target_logits.shape
+    lib = load()
+    lib.gls_verify_walk.restype = C.c_int
+    lib.gls_verify_walk.argtypes = [C.c_int, C.c_int, C.c_int, C.c_int, C.c_int, C.c_int64, C.c_int,
+                                    C.c_uint32]
+    rc = int(lib.gls_verify_walk(BF16 if target_logits.dtype == torch.bfloat16 else F32,
+                                 int(target_logits.stride(1) != 0), B, K, int(L), V, int(spec), int(flags)))
+    if rc < 0:
+        raise GlsError("gls_verify_walk: arguments that the verify call refuses")
+    return rc
+
+
 def draft_verify_workspace_bytes(B, K, L, J, V):
     return int(load().gls_draft_verify_workspace_bytes(int(B), int(K), int(L), int(J), int(V)))
 

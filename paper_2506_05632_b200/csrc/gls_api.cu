@@ -42,9 +42,11 @@ static int num_sms() {
 }
 constexpr int kMinChunk = 2048;
 constexpr int kMaxChunk = 16384;
-// Target rows of a verify call, in bytes, from which Algorithm 2 is walked position by position
+// Target rows of a verify call, in bytes, from which Algorithm 2 is walked in phases (measured
+// break-even with the walk that races every row first: 200 MB; 100 MB for Appendix B on a row per
+// draft, whose rows cost K times the noise arithmetic)
 #ifndef GLS_STEPWISE_MIN_BYTES
-#define GLS_STEPWISE_MIN_BYTES 256e6
+#define GLS_STEPWISE_MIN_BYTES 192e6
 #endif
 constexpr int kMaxPhases = 4;  // phases of such a walk (two are used: position 0, the rest)
 
@@ -1058,6 +1060,23 @@ static int run_verify_stepwise(SweepArgs& A, int dtype, const VerifyArgs& va, co
 #undef STEPWISE
 }
 
+// How gls_target_sample_verify walks Algorithm 2: 0 = every row is raced, then the loop; 1 = in
+// phases (only the rows of active drafts are read): when the walk can prune anything and the rows
+// are large enough for its extra launches to pay; -1 = GLS_VERIFY_ACTIVE_ROWS asked for and
+// not possible.
+static int verify_walk(int dtype, bool row_per_draft, int B, int K, int L, int64_t V, int spec,
+                       uint32_t flags) {
+  const int J = L + ((flags & GLS_NO_BONUS) ? 0 : 1);
+  const bool multi = (flags & GLS_COMBINE_ALL) && row_per_draft && K > 1;
+  if (multi && (spec != 4 || K > 8 || V >= (1LL << 28))) return -1;  // the call refuses these
+  const bool can = spec == 4 && (multi || !(flags & GLS_COMBINE_ALL)) && L >= 1 && J >= 2 &&
+                   (size_t)K * (J - 1) * sizeof(RowResult) <= kFusedVerifyMaxSmem;
+  if (flags & GLS_VERIFY_ACTIVE_ROWS) return can ? 1 : -1;
+  if (!can || (flags & GLS_VERIFY_ALL_ROWS)) return 0;
+  const double bytes = (double)B * K * J * (double)V * (dtype == GLS_BF16 ? 2.0 : 4.0);
+  return bytes >= (multi ? 0.5 : 1.0) * GLS_STEPWISE_MIN_BYTES ? 1 : 0;
+}
+
 static bool sizes_ok(int B, int K, int J, int64_t V) {
   if (B <= 0 || K <= 0 || K > GLS_MAX_K || J <= 0 || V <= 0) return false;
   if (V >= (1LL << 31) - 4 * kS4MaxCtaTokens) return false;
@@ -1124,6 +1143,15 @@ size_t gls_workspace_bytes(int B, int K, int J, int64_t V) {
     }
   }
   return need;
+}
+
+int gls_verify_walk(int dtype, int row_per_draft, int B, int K, int L, int64_t V, int noise_spec,
+                    uint32_t flags) {
+  if (flags & ~(GLS_COMBINE_ALL | GLS_NO_BONUS | GLS_VERIFY_ALL_ROWS | GLS_VERIFY_ACTIVE_ROWS)) return -1;
+  if ((flags & GLS_VERIFY_ALL_ROWS) && (flags & GLS_VERIFY_ACTIVE_ROWS)) return -1;
+  const int J = L + ((flags & GLS_NO_BONUS) ? 0 : 1);
+  if (L < 0 || !sizes_ok(B, K, J, V) || (dtype != GLS_F32 && dtype != GLS_BF16)) return -1;
+  return verify_walk(dtype, row_per_draft != 0, B, K, L, V, noise_spec, flags);
 }
 
 size_t gls_draft_verify_workspace_bytes(int B, int K, int L, int J, int64_t V) {
@@ -1193,14 +1221,9 @@ int gls_target_sample_verify(const gls_rows_t* target_logits, int B, int K, int 
   // and the epilogue reads the row of the lowest active draft.
   const bool multi = (flags & GLS_COMBINE_ALL) && target_logits->stride_k != 0 && K > 1;
   if (multi && (spec != 4 || K > 8 || V >= (1LL << 28))) return GLS_ERR_UNSUPPORTED;
-  // Position by position (only the rows of active drafts are read) when the walk can prune
-  // anything and the rows are large enough for its J rounds of launches to pay.
-  const bool can_step = spec == 4 && (multi || !(flags & GLS_COMBINE_ALL)) && L >= 1 && J >= 2 &&
-                        (size_t)K * (J - 1) * sizeof(RowResult) <= kFusedVerifyMaxSmem;
-  if ((flags & GLS_VERIFY_ACTIVE_ROWS) && !can_step) return GLS_ERR_UNSUPPORTED;
-  const double bytes = (double)B * K * J * (double)V * (target_logits->dtype == GLS_BF16 ? 2.0 : 4.0);
-  const bool stepwise = can_step && ((flags & GLS_VERIFY_ACTIVE_ROWS) ||
-                                     (!(flags & GLS_VERIFY_ALL_ROWS) && bytes >= GLS_STEPWISE_MIN_BYTES));
+  const int walk = verify_walk(target_logits->dtype, target_logits->stride_k != 0, B, K, L, V, spec, flags);
+  if (walk < 0) return GLS_ERR_UNSUPPORTED;
+  const bool stepwise = walk == 1;
   flags &= ~(GLS_VERIFY_ALL_ROWS | GLS_VERIFY_ACTIVE_ROWS);
   const Plan P = stepwise ? make_plan_stepwise(B, K, J, V, target_logits->dtype, multi)
                           : make_plan((long long)B * K * J, V, spec, target_logits->dtype, multi);
@@ -1274,8 +1297,7 @@ int gls_draft_verify(const gls_rows_t* draft_logits, const gls_rows_t* target_lo
   const long long rows_d = (long long)B * K * L, rows_t = (long long)B * K * J;
   // Large target rows: the draft rows first, then Algorithm 2 in phases, which reads the target
   // rows of active drafts only (the draft tokens it needs are this call's own output).
-  if (J >= 2 && !(flags & GLS_COMBINE_ALL) &&
-      (double)rows_t * (double)V * (target_logits->dtype == GLS_BF16 ? 2.0 : 4.0) >= GLS_STEPWISE_MIN_BYTES) {
+  if (verify_walk(target_logits->dtype, target_logits->stride_k != 0, B, K, L, V, spec, flags) == 1) {
     if (!workspace || workspace_bytes < gls_draft_verify_workspace_bytes(B, K, L, J, V)) return GLS_ERR_WORKSPACE;
     rc = gls_draft_sample(draft_logits, B, K, L, V, inv_temp_draft, inv_temp_per_draft_host, noise,
                           out_draft_tokens, out_draft_scores, workspace, workspace_bytes, device_status,

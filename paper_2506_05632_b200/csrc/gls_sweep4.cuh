@@ -530,8 +530,8 @@ sweep4_kernel(const __grid_constant__ SweepArgs A) {
 // ------------------------------------------------------------------------------------------
 // Rows named by a list in device memory (the position-by-position verification of Algorithm 2:
 // the rows of a position are those of the drafts still active there, known only on the device).
-// The slicing follows from the number of listed rows: as many slices per row as let one round of
-// work items fill the launch, each at least four steps long.
+// The slicing follows from the number of listed rows, by the rule of the host-side plan; slices
+// are at least four steps long.
 // ------------------------------------------------------------------------------------------
 struct ListedSlicing {
   int chunk, splits;
@@ -543,10 +543,25 @@ __host__ __device__ __forceinline__ int listed_max_splits(int V, int cta_tokens)
 __host__ __device__ __forceinline__ ListedSlicing listed_slicing(int n_rows, int V, int cta_tokens,
                                                                  int grid) {
   const int steps = (V + cta_tokens - 1) / cta_tokens;
-  int want = n_rows > 0 ? grid / n_rows : 1;
   const int cap = listed_max_splits(V, cta_tokens);
-  if (want > cap) want = cap;
-  if (want < 1) want = 1;
+  // Few rows (less than half a launch): as many slices per row as keep the items within one
+  // round.  Otherwise the fewest slices for which the items fill the launch and the last round of
+  // items leaves at most 15 % of it idle (or every CTA gets a dozen items).
+  int want = cap;
+  if (2 * (long long)n_rows < grid) {
+    want = n_rows > 0 ? grid / n_rows : 1;
+    if (want > cap) want = cap;
+  } else {
+    for (int sp = 1; sp < cap; ++sp) {
+      const long long items = (long long)n_rows * sp;
+      if (items < grid) continue;
+      const long long rounds = (items + grid - 1) / grid;
+      if (items >= 12LL * grid || (rounds * grid - items) * 100 <= 15 * rounds * grid) {
+        want = sp;
+        break;
+      }
+    }
+  }
   const int chunk_steps = (steps + want - 1) / want;
   ListedSlicing r;
   r.chunk = chunk_steps * cta_tokens;

@@ -29,7 +29,7 @@ def _report(tally):
     print(line)
 
 
-def _verify_case(gls, oracle, cfg, chunk, **shape):
+def _verify_case(gls, oracle, cfg, chunk, walk=0, **shape):
     """Every sequence of the configuration: the GPU runs the full-size call, the oracle recomputes
     it from the same logits in chunks of `chunk` sequences (results are keyed by the absolute
     sequence id, so a chunk's oracle result does not depend on the rest of the batch)."""
@@ -37,7 +37,7 @@ def _verify_case(gls, oracle, cfg, chunk, **shape):
     B, K, L, V = w.shape
     kw = dict(seed=w.noise_seed, inv_temp=w.inv_temp)
     tok, sc = gls.draft_sample(w.draft_logits, **kw)
-    out = gls.target_sample_verify(w.target_logits, tok, **kw)
+    out = gls.target_sample_verify(w.target_logits, tok, flags=walk, **kw)
     torch.cuda.synchronize()
     o = parity.to_np(out)
     tok_h, sc_h = tok.cpu().numpy(), sc.cpu().numpy()
@@ -81,6 +81,12 @@ def test_config2_full(gls, oracle):
 def test_config3_full(gls, oracle):
     """B=64, K=8, L=5, V=128256, bf16, T=0.7: all 64 sequences (5632 rows)."""
     _verify_case(gls, oracle, 3, chunk=16)
+
+
+def test_config3_full_every_row_raced(gls, oracle):
+    """Configuration 3 again with the walk that races all 3072 target rows before Algorithm 2's
+    loop (the default at this size reads the rows of active drafts only)."""
+    _verify_case(gls, oracle, 3, chunk=16, walk=gls.VERIFY_ALL_ROWS)
 
 
 def test_config4_full(gls, oracle):
@@ -138,10 +144,12 @@ def test_autoregressive_draft_shape(gls, oracle):
     assert np.array_equal(tok.cpu().numpy()[idx], ref["tokens"])
 
 
-def test_config3_one_call_equals_two_calls(gls):
-    """gls_draft_verify at full size (one sweep launch per set of rows, each sliced for its own
-    row count, one reduction launch): bit-identical to the draft call followed by the verify call."""
-    w = synth.verify_workload(3, "cuda")
+@pytest.mark.parametrize("B", [64, 12])
+def test_config3_one_call_equals_two_calls(gls, B):
+    """gls_draft_verify on configuration 3: at full size (the draft rows, then Algorithm 2 in
+    phases) and at a fifth of it (one sweep launch per set of rows, each sliced for its own row
+    count, one reduction launch): bit-identical to the draft call followed by the verify call."""
+    w = synth.verify_workload(3, "cuda", B=B)
     kw = dict(seed=w.noise_seed, inv_temp=w.inv_temp)
     tok, sc = gls.draft_sample(w.draft_logits, **kw)
     out = gls.target_sample_verify(w.target_logits, tok, **kw)
