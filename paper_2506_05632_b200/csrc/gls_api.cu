@@ -485,6 +485,7 @@ struct PhasedState {
 
 __global__ void phased_init_kernel(const VerifyArgs va, const PhasedState S, int first_end,
                                    uint32_t* __restrict__ hints) {
+  asm volatile("griddepcontrol.launch_dependents;");  // the first sweep may be scheduled
   const long long t = (long long)blockIdx.x * blockDim.x + threadIdx.x;
   const long long BK = (long long)va.B * va.K;
   // first phase: every draft is active at positions [0, first_end); Appendix B on a row per draft
@@ -519,6 +520,7 @@ phased_verify_kernel(const __grid_constant__ SweepArgs A, const VerifyArgs va, c
   const int lane = threadIdx.x & 31;
   unsigned long long active = S.active[b];  // written by the previous phase, complete by now
   asm volatile("griddepcontrol.wait;" ::: "memory");  // the sweep before this launch is complete
+  asm volatile("griddepcontrol.launch_dependents;");  // the next phase's sweep may be scheduled
   if (active == 0ull) return;
   const int K = va.K, L = va.L, J = va.J, W = j1 - j0;
   const ListedSlicing sl = listed_slicing(S.counts[phase], A.V, cta_tokens, sweep_grid);
@@ -1034,8 +1036,16 @@ static int run_verify_stepwise_t(SweepArgs& A, const VerifyArgs& va, const Plan&
     const int j1 = ends[p], j2 = p + 1 < n_phases ? ends[p + 1] : j1;
     const long long most = BK * (j1 - j0) * P.splits;  // items if every row of the phase is listed
     const int grid = (int)(most < cap ? most : cap);
-    sweep4_listed_kernel<SH, ROUNDS, MULTI><<<grid, S4Cfg<SH>::kWarps * 32, sizeof(S4Shared<SH>), st>>>(
-        A, S.lists + BK * j0, S.counts + p);
+    {
+      // a programmatic dependent of the kernel before it (the initialisation or the previous
+      // phase's walk): it waits for that kernel before it reads the list
+      cudaLaunchAttribute sattr;
+      cudaLaunchConfig_t scfg = dependent_launch(&sattr, grid, S4Cfg<SH>::kWarps * 32, sizeof(S4Shared<SH>), st);
+      const int* list = S.lists + BK * j0;
+      const int* count = S.counts + p;
+      if (cudaLaunchKernelEx(&scfg, sweep4_listed_kernel<SH, ROUNDS, MULTI>, A, list, count) != cudaSuccess)
+        return GLS_ERR_CUDA;
+    }
     const int nrows = va.K * (j1 - j0);
     cudaLaunchAttribute attr;
     cudaLaunchConfig_t cfg = dependent_launch(&attr, va.B, (nrows < warps ? nrows : warps) * 32,

@@ -578,6 +578,8 @@ sweep4_listed_kernel(const __grid_constant__ SweepArgs A, const int* __restrict_
   S4Shared<SH>& sh = s4_shared<SH>();
   if (threadIdx.x == 0) sh.m_tag = 0ull;
   __syncthreads();
+  // the kernel that wrote the list (launched before this one) is complete
+  asm volatile("griddepcontrol.wait;" ::: "memory");
   const int n = __ldcg(count);
   const ListedSlicing sl = listed_slicing(n, A.V, S4Cfg<SH>::kCtaTokens, (int)gridDim.x);
   const long long n_items = (long long)n * sl.splits;
