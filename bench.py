@@ -427,6 +427,7 @@ def run_ours(args):
     small = dbytes + tbytes < 512e6  # fits the 126 MB L2 several times over? then flush
     flush = torch.zeros(64 << 20, dtype=torch.float32, device="cuda") if small else None
 
+    walk_flags = {"auto": 0, "all": pkg.VERIFY_ALL_ROWS, "phases": pkg.VERIFY_ACTIVE_ROWS}[args.walk]
     topm_ws = None
     if args.topm:
         # extra workload: every row truncated to its top-M logits in front of the races
@@ -455,7 +456,7 @@ def run_ours(args):
                          workspace=buf.workspace, status=buf.status, **kw)
         _mark(marks)
         pkg.target_sample_verify(w.target_logits, buf.draft_tokens, out=buf.out,
-                                 workspace=buf.workspace, status=buf.status, **kw)
+                                 workspace=buf.workspace, status=buf.status, flags=walk_flags, **kw)
         _mark(marks)
 
     for _ in range(max(args.warmup, 3)):
@@ -576,7 +577,8 @@ def run_ours(args):
                 "tokens of every row, then the race on the lists; the event bracket is the whole call)" % (
                     "bf16" if bf else "f32")
     else:
-        vrec = _verify_call_record(pkg, w.target_logits, L, buf.out, verify_ms, peak, spec=args.spec)
+        vrec = _verify_call_record(pkg, w.target_logits, L, buf.out, verify_ms, peak, flags=walk_flags,
+                                   spec=args.spec)
         sweep = {4: "sweep4_kernel", 3: "sweep3_kernel"}.get(args.spec, "sweep_kernel")
         if draft_ms >= verify_ms:
             # the verify call reads few rows: the draft rows' sweep is the dominant kernel
@@ -719,6 +721,9 @@ def main():
     ap.add_argument("--topm", type=int, default=0,
                     help="extra workload: truncate every row to its top-M logits first (Sec. 4.4)")
     ap.add_argument("--fused", action="store_true", help="one gls_draft_verify call per step")
+    ap.add_argument("--walk", choices=("auto", "all", "phases"), default="auto",
+                    help="how the verify call walks Algorithm 2: every target row raced first, in "
+                         "phases (only rows of active drafts are read), or the library's choice by size")
     ap.add_argument("--no-sustained", action="store_true", help="skip the two-second back-to-back loop")
     ap.add_argument("--no-extras", action="store_true", help="skip the other configurations")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg")
