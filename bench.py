@@ -561,6 +561,8 @@ def run_ours(args):
         assert torch.equal(res["tau"], buf.out["tau"].cpu())
         e2e = {"value": world * B * L / (e_ms * 1e-3), "unit": UNIT,
                "h2d_bytes_per_step": hs.h2d_bytes, "d2h_bytes_per_step": hs.d2h_bytes,
+               # only the rows Algorithm 2 reads are copied; the step is given this many bytes:
+               "host_bytes_given_per_step": hs.h2d_bytes_all,
                "ms_per_step": e_ms, "steps": n_e2e}
         del h_d, h_t, hs
     if rank != 0:

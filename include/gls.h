@@ -129,7 +129,15 @@ typedef struct {
 #define GLS_NO_BONUS 2u       /* target rows cover positions 0..L-1 only; no bonus token         */
 /* How gls_target_sample_verify walks Algorithm 2 (same results either way; default: by size).  */
 #define GLS_VERIFY_ALL_ROWS 4u    /* race every target row, then run the loop on the row results  */
-#define GLS_VERIFY_ACTIVE_ROWS 8u /* position by position: only rows of active drafts are read    */
+#define GLS_VERIFY_ACTIVE_ROWS 8u /* in phases: only rows of active drafts are read               */
+/* The walk in phases as two calls with the same arguments and the same, untouched workspace, for a
+ * caller that fetches target rows on demand (e.g. from host memory).  GLS_VERIFY_FIRST_PHASE reads
+ * the rows at position 0 only and writes out_tokens[:,0], out_accept[:,:,0] and out_num_tokens
+ * (the emitted count for sequences that stopped, 0 for those still running).  GLS_VERIFY_REST
+ * reads, of the other rows, exactly those (b, k, 1..J-1) with out_accept[b,k,0] == 1 and
+ * completes all outputs; rows it does not read need not hold valid data.                         */
+#define GLS_VERIFY_FIRST_PHASE 16u
+#define GLS_VERIFY_REST 32u
 
 /* Library version, major * 10000 + minor * 100 + patch. */
 int gls_version(void);

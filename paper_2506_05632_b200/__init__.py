@@ -11,7 +11,8 @@ kernels of csrc/.  There is no CPU fallback: if libgls.so cannot be loaded the c
     compress_gaussian(u, a, t, bins, ...)     the same from the source: Appendix C weights computed in the kernels
 """
 from .binding import (  # noqa: F401
-    COMBINE_ACTIVE, COMBINE_ALL, NO_BONUS, VERIFY_ALL_ROWS, VERIFY_ACTIVE_ROWS, NOISE_SHARED_ACROSS_K,
+    COMBINE_ACTIVE, COMBINE_ALL, NO_BONUS, VERIFY_ALL_ROWS, VERIFY_ACTIVE_ROWS, VERIFY_FIRST_PHASE,
+    VERIFY_REST, NOISE_SHARED_ACROSS_K,
     DEV_EMPTY_SUPPORT, GlsError,
     build, debug_bounds, compress_gaussian, compress_gaussian_workspace_bytes, compress_select, draft_sample, draft_sample_sparse, draft_sample_static,
     draft_sample_topm, draft_verify, draft_verify_workspace_bytes, lib_path, load,

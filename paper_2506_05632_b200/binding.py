@@ -13,6 +13,7 @@ _LIB = os.path.join(_HERE, "libgls.so")
 
 COMBINE_ACTIVE, COMBINE_ALL, NO_BONUS = 0, 1, 2
 VERIFY_ALL_ROWS, VERIFY_ACTIVE_ROWS = 4, 8  # how the dense verify call walks Algorithm 2
+VERIFY_FIRST_PHASE, VERIFY_REST = 16, 32   # the walk in phases as two calls (rows fetched on demand)
 NOISE_SHARED_ACROSS_K = 1
 DEV_EMPTY_SUPPORT = 1
 F32, BF16 = 0, 1

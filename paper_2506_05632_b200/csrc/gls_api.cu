@@ -1003,7 +1003,7 @@ static int run_rows(SweepArgs& A, int dtype, int spec, const Plan& P, void* work
 // phase's positions.
 template <int SH, int ROUNDS, bool MULTI>
 static int run_verify_stepwise_t(SweepArgs& A, const VerifyArgs& va, const Plan& P, void* workspace,
-                                 cudaStream_t st) {
+                                 cudaStream_t st, int part) {
   constexpr int DT = S4Cfg<SH>::kDT;
   char* ws = (char*)workspace;
   A.chunk = 0;
@@ -1025,14 +1025,17 @@ static int run_verify_stepwise_t(SweepArgs& A, const VerifyArgs& va, const Plan&
   int n_phases = 0;
   ends[n_phases++] = 1;
   if (va.J > 1) ends[n_phases++] = va.J;
-  {
+  // part 0: the whole walk; 1: the first phase only (the state stays in the workspace); 2: the
+  // phases after the first, from that state
+  const int p_begin = part == 2 ? 1 : 0, p_end = part == 1 ? 1 : n_phases;
+  if (p_begin == 0) {
     const long long n = BK * va.J;  // the largest index range the initialisation covers
     phased_init_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(va, S, ends[0], A.hints);
   }
   const long long cap = (long long)num_sms() * S4Cfg<SH>::kCtasPerSM;
   const int warps = kFusedVerifyMaxWarps;
-  int j0 = 0;
-  for (int p = 0; p < n_phases; ++p) {
+  int j0 = p_begin > 0 ? ends[p_begin - 1] : 0;
+  for (int p = p_begin; p < p_end; ++p) {
     const int j1 = ends[p], j2 = p + 1 < n_phases ? ends[p + 1] : j1;
     const long long most = BK * (j1 - j0) * P.splits;  // items if every row of the phase is listed
     const int grid = (int)(most < cap ? most : cap);
@@ -1058,16 +1061,25 @@ static int run_verify_stepwise_t(SweepArgs& A, const VerifyArgs& va, const Plan&
   return cudaGetLastError() == cudaSuccess ? GLS_OK : GLS_ERR_CUDA;
 }
 static int run_verify_stepwise(SweepArgs& A, int dtype, const VerifyArgs& va, const Plan& P,
-                               void* workspace, cudaStream_t st) {
+                               void* workspace, cudaStream_t st, int part) {
   const int sh = s4_shape(dtype, A.V, va.multi_rows);
   const bool r10 = A.rounds == 10;
-#define STEPWISE(SH, M) (r10 ? run_verify_stepwise_t<SH, 10, M>(A, va, P, workspace, st) \
-                             : run_verify_stepwise_t<SH, 0, M>(A, va, P, workspace, st))
+#define STEPWISE(SH, M) (r10 ? run_verify_stepwise_t<SH, 10, M>(A, va, P, workspace, st, part) \
+                             : run_verify_stepwise_t<SH, 0, M>(A, va, P, workspace, st, part))
   if (va.multi_rows) return sh == kS4ShapeBf16 ? STEPWISE(kS4ShapeBf16, true) : STEPWISE(kS4ShapeF32Narrow, true);
   if (sh == kS4ShapeBf16) return STEPWISE(kS4ShapeBf16, false);
   if (sh == kS4ShapeF32Wide) return STEPWISE(kS4ShapeF32Wide, false);
   return STEPWISE(kS4ShapeF32Narrow, false);
 #undef STEPWISE
+}
+
+constexpr uint32_t kWalkFlags =
+    GLS_VERIFY_ALL_ROWS | GLS_VERIFY_ACTIVE_ROWS | GLS_VERIFY_FIRST_PHASE | GLS_VERIFY_REST;
+// known bits only, and at most one request about the walk
+static bool verify_flags_ok(uint32_t flags) {
+  if (flags & ~(GLS_COMBINE_ALL | GLS_NO_BONUS | kWalkFlags)) return false;
+  const uint32_t w = flags & kWalkFlags;
+  return (w & (w - 1u)) == 0u;
 }
 
 // How gls_target_sample_verify walks Algorithm 2: 0 = every row is raced, then the loop; 1 = in
@@ -1081,7 +1093,7 @@ static int verify_walk(int dtype, bool row_per_draft, int B, int K, int L, int64
   if (multi && (spec != 4 || K > 8 || V >= (1LL << 28))) return -1;  // the call refuses these
   const bool can = spec == 4 && (multi || !(flags & GLS_COMBINE_ALL)) && L >= 1 && J >= 2 &&
                    (size_t)K * (J - 1) * sizeof(RowResult) <= kFusedVerifyMaxSmem;
-  if (flags & GLS_VERIFY_ACTIVE_ROWS) return can ? 1 : -1;
+  if (flags & (GLS_VERIFY_ACTIVE_ROWS | GLS_VERIFY_FIRST_PHASE | GLS_VERIFY_REST)) return can ? 1 : -1;
   if (!can || (flags & GLS_VERIFY_ALL_ROWS)) return 0;
   const double bytes = (double)B * K * J * (double)V * (dtype == GLS_BF16 ? 2.0 : 4.0);
   return bytes >= (multi ? 0.5 : 1.0) * GLS_STEPWISE_MIN_BYTES ? 1 : 0;
@@ -1157,8 +1169,7 @@ size_t gls_workspace_bytes(int B, int K, int J, int64_t V) {
 
 int gls_verify_walk(int dtype, int row_per_draft, int B, int K, int L, int64_t V, int noise_spec,
                     uint32_t flags) {
-  if (flags & ~(GLS_COMBINE_ALL | GLS_NO_BONUS | GLS_VERIFY_ALL_ROWS | GLS_VERIFY_ACTIVE_ROWS)) return -1;
-  if ((flags & GLS_VERIFY_ALL_ROWS) && (flags & GLS_VERIFY_ACTIVE_ROWS)) return -1;
+  if (!verify_flags_ok(flags)) return -1;
   const int J = L + ((flags & GLS_NO_BONUS) ? 0 : 1);
   if (L < 0 || !sizes_ok(B, K, J, V) || (dtype != GLS_F32 && dtype != GLS_BF16)) return -1;
   return verify_walk(dtype, row_per_draft != 0, B, K, L, V, noise_spec, flags);
@@ -1209,9 +1220,7 @@ int gls_target_sample_verify(const gls_rows_t* target_logits, int B, int K, int 
                              uint32_t flags, int32_t* out_tokens, int32_t* out_num_tokens,
                              uint8_t* out_accept, float* out_scores, void* workspace,
                              size_t workspace_bytes, uint32_t* device_status, void* stream) {
-  if (flags & ~(GLS_COMBINE_ALL | GLS_NO_BONUS | GLS_VERIFY_ALL_ROWS | GLS_VERIFY_ACTIVE_ROWS))
-    return GLS_ERR_INVALID_ARG;
-  if ((flags & GLS_VERIFY_ALL_ROWS) && (flags & GLS_VERIFY_ACTIVE_ROWS)) return GLS_ERR_INVALID_ARG;
+  if (!verify_flags_ok(flags)) return GLS_ERR_INVALID_ARG;
   const int J = L + ((flags & GLS_NO_BONUS) ? 0 : 1);
   if (!noise || !out_tokens || !out_num_tokens || L < 0 || !sizes_ok(B, K, J, V))
     return GLS_ERR_INVALID_ARG;
@@ -1234,7 +1243,8 @@ int gls_target_sample_verify(const gls_rows_t* target_logits, int B, int K, int 
   const int walk = verify_walk(target_logits->dtype, target_logits->stride_k != 0, B, K, L, V, spec, flags);
   if (walk < 0) return GLS_ERR_UNSUPPORTED;
   const bool stepwise = walk == 1;
-  flags &= ~(GLS_VERIFY_ALL_ROWS | GLS_VERIFY_ACTIVE_ROWS);
+  const int part = (flags & GLS_VERIFY_FIRST_PHASE) ? 1 : (flags & GLS_VERIFY_REST) ? 2 : 0;
+  flags &= ~kWalkFlags;
   const Plan P = stepwise ? make_plan_stepwise(B, K, J, V, target_logits->dtype, multi)
                           : make_plan((long long)B * K * J, V, spec, target_logits->dtype, multi);
   if (!workspace || workspace_bytes < P.total) return GLS_ERR_WORKSPACE;
@@ -1257,7 +1267,7 @@ int gls_target_sample_verify(const gls_rows_t* target_logits, int B, int K, int 
   va.accept = out_accept;
   va.out_scores = out_scores;
   va.dev_status = device_status;
-  if (stepwise) return run_verify_stepwise(A, target_logits->dtype, va, P, workspace, st);
+  if (stepwise) return run_verify_stepwise(A, target_logits->dtype, va, P, workspace, st, part);
   bool fused = false;
   rc = run_rows(A, target_logits->dtype, spec, P, workspace, true, nullptr, nullptr, nullptr, st,
                 &va, &fused);

@@ -81,53 +81,129 @@ class GraphedStep:
 
 
 class HostStepper:
-    """Hot path from HOST logits: chunked, double-buffered H2D copies overlapped with the sweeps."""
+    """Hot path from HOST logits, in chunks of sequences whose copies overlap the sweeps of other
+    chunks.  Only what Algorithm 2 reads crosses the host link: a chunk's draft rows and its
+    target rows at position 0 go first; the verify call's first phase then tells which drafts
+    survived position 0, and only their remaining target rows are copied before the rest of the
+    walk runs (`VERIFY_FIRST_PHASE` / `VERIFY_REST`).  The host waits once per chunk, for that
+    list of survivors, while the copies of the next chunk are already queued."""
+
+    STAGES = 3
 
     def __init__(self, B, K, L, V, dtype, chunk_seqs=16, device="cuda"):
         self.B, self.K, self.L, self.V = B, K, L, V
         self.chunk = min(chunk_seqs, B)
         self.copy_stream = torch.cuda.Stream(device=device)
-        self.stage = [dict(d=torch.empty((self.chunk, K, L, V), dtype=dtype, device=device),
-                           t=torch.empty((self.chunk, K, L + 1, V), dtype=dtype, device=device),
-                           ready=torch.cuda.Event(), free=torch.cuda.Event(),
-                           buf=StepBuffers(self.chunk, K, L, V, device))
-                      for _ in range(2)]
+        c = self.chunk
+        self.stage = [dict(d=torch.empty((c, K, L, V), dtype=dtype, device=device),
+                           t=torch.empty((c, K, L + 1, V), dtype=dtype, device=device),
+                           ready=torch.cuda.Event(), rest=torch.cuda.Event(),
+                           first=torch.cuda.Event(), free=torch.cuda.Event(),
+                           acc0=torch.empty((c, K), dtype=torch.uint8).pin_memory(),
+                           buf=StepBuffers(c, K, L, V, device))
+                      for _ in range(self.STAGES)]
         # a ragged last chunk has buffers of its own, allocated here and not inside step()
-        self.ragged = StepBuffers(B % self.chunk, K, L, V, device) if B % self.chunk else None
+        self.ragged = StepBuffers(B % c, K, L, V, device) if B % c else None
         self.h_tokens = torch.empty((B, L + 1), dtype=torch.int32).pin_memory()
         self.h_tau = torch.empty((B,), dtype=torch.int32).pin_memory()
         self.h_accept = torch.empty((B, K, L), dtype=torch.uint8).pin_memory()
-        elt = torch.empty(0, dtype=dtype).element_size()
-        self.h2d_bytes = B * K * (2 * L + 1) * V * elt
-        self.d2h_bytes = self.h_tokens.numel() * 4 + self.h_tau.numel() * 4 + self.h_accept.numel()
+        self.elt = torch.empty(0, dtype=dtype).element_size()
+        self.h2d_bytes_all = B * K * (2 * L + 1) * V * self.elt  # every row the step is given
+        self.h2d_bytes = self.h2d_bytes_all                       # what the last step() copied
+        self.d2h_bytes = (self.h_tokens.numel() * 4 + self.h_tau.numel() * 4 + self.h_accept.numel()
+                          + B * K)
+
+    def _chunks(self):
+        return [(b0, min(self.B, b0 + self.chunk)) for b0 in range(0, self.B, self.chunk)]
 
     def step(self, h_draft, h_target, inv_temp=1.0, seed=0, seq_base=0, spec=4, rounds=10):
         """h_draft [B,K,L,V], h_target [B,K,L+1,V]: pinned host tensors.  Returns host results."""
+        L, K = self.L, self.K
+        if L < 1 or spec != 4:
+            return self._step_all_rows(h_draft, h_target, inv_temp, seed, seq_base, spec, rounds)
         main = torch.cuda.current_stream()
-        n = 0
-        for b0 in range(0, self.B, self.chunk):
-            b1 = min(self.B, b0 + self.chunk)
-            s = self.stage[n & 1]
+        chunks = self._chunks()
+        copied = 0
+        row_bytes = self.V * self.elt
+
+        def views(n):
+            b0, b1 = chunks[n]
+            s = self.stage[n % self.STAGES]
+            nb = b1 - b0
+            bb = s["buf"] if nb == self.chunk else self.ragged
+            return b0, b1, nb, s, s["d"][:nb], s["t"][:nb], bb
+
+        def first_part(n):
+            """Copies of the chunk's draft rows and position-0 target rows; draft call; first phase."""
+            b0, b1, nb, s, d, t, bb = views(n)
+            with torch.cuda.stream(self.copy_stream):
+                if n >= self.STAGES:
+                    self.copy_stream.wait_event(s["free"])
+                d.copy_(h_draft[b0:b1], non_blocking=True)
+                for i in range(nb):
+                    for k in range(K):
+                        t[i, k, 0].copy_(h_target[b0 + i, k, 0], non_blocking=True)
+                s["ready"].record(self.copy_stream)
+            main.wait_event(s["ready"])
+            kw = dict(inv_temp=inv_temp, seed=seed, seq_base=seq_base + b0, spec=spec, rounds=rounds,
+                      workspace=bb.workspace, status=bb.status)
+            binding.draft_sample(d, out_tokens=bb.draft_tokens, out_scores=bb.draft_scores, **kw)
+            binding.target_sample_verify(t, bb.draft_tokens, out=bb.out,
+                                         flags=binding.VERIFY_FIRST_PHASE, **kw)
+            s["acc0"][:nb].copy_(bb.out["accept"][:, :, 0], non_blocking=True)
+            s["first"].record(main)
+            return nb * K * (L + 1) * row_bytes
+
+        def second_part(n):
+            """The survivors' remaining target rows, the rest of the walk, results to the host."""
+            b0, b1, nb, s, d, t, bb = views(n)
+            s["first"].synchronize()
+            alive = torch.nonzero(s["acc0"][:nb]).tolist()
+            with torch.cuda.stream(self.copy_stream):
+                for i, k in alive:
+                    t[i, k, 1:].copy_(h_target[b0 + i, k, 1:], non_blocking=True)
+                s["rest"].record(self.copy_stream)
+            main.wait_event(s["rest"])
+            kw = dict(inv_temp=inv_temp, seed=seed, seq_base=seq_base + b0, spec=spec, rounds=rounds,
+                      workspace=bb.workspace, status=bb.status)
+            out = binding.target_sample_verify(t, bb.draft_tokens, out=bb.out,
+                                               flags=binding.VERIFY_REST, **kw)
+            self.h_tokens[b0:b1].copy_(out["tokens"], non_blocking=True)
+            self.h_tau[b0:b1].copy_(out["tau"], non_blocking=True)
+            self.h_accept[b0:b1].copy_(out["accept"], non_blocking=True)
+            s["free"].record(main)
+            return len(alive) * L * row_bytes
+
+        # chunk n + 1's first part is queued before the host waits for chunk n's survivors
+        copied += first_part(0)
+        for n in range(len(chunks)):
+            if n + 1 < len(chunks):
+                copied += first_part(n + 1)
+            copied += second_part(n)
+        main.synchronize()
+        self.h2d_bytes = copied
+        return dict(tokens=self.h_tokens, tau=self.h_tau, accept=self.h_accept)
+
+    def _step_all_rows(self, h_draft, h_target, inv_temp, seed, seq_base, spec, rounds):
+        """Every row copied, one draft call and one verify call per chunk."""
+        main = torch.cuda.current_stream()
+        for n, (b0, b1) in enumerate(self._chunks()):
+            s = self.stage[n % self.STAGES]
             nb = b1 - b0
             with torch.cuda.stream(self.copy_stream):
-                if n >= 2:
+                if n >= self.STAGES:
                     self.copy_stream.wait_event(s["free"])
                 s["d"][:nb].copy_(h_draft[b0:b1], non_blocking=True)
                 s["t"][:nb].copy_(h_target[b0:b1], non_blocking=True)
                 s["ready"].record(self.copy_stream)
             main.wait_event(s["ready"])
-            buf = s["buf"]
-            if nb == self.chunk:
-                d, t, bb = s["d"], s["t"], buf
-            else:  # ragged last chunk
-                d, t = s["d"][:nb], s["t"][:nb]
-                bb = self.ragged
-            out = spec_step(d, t, bb, inv_temp=inv_temp, seed=seed, seq_base=seq_base + b0,
-                            spec=spec, rounds=rounds)
+            bb = s["buf"] if nb == self.chunk else self.ragged
+            out = spec_step(s["d"][:nb], s["t"][:nb], bb, inv_temp=inv_temp, seed=seed,
+                            seq_base=seq_base + b0, spec=spec, rounds=rounds)
             self.h_tokens[b0:b1].copy_(out["tokens"], non_blocking=True)
             self.h_tau[b0:b1].copy_(out["tau"], non_blocking=True)
             self.h_accept[b0:b1].copy_(out["accept"], non_blocking=True)
             s["free"].record(main)
-            n += 1
         main.synchronize()
+        self.h2d_bytes = self.h2d_bytes_all
         return dict(tokens=self.h_tokens, tau=self.h_tau, accept=self.h_accept)

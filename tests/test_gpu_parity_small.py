@@ -403,7 +403,7 @@ def test_host_detectable_errors(gls):
     with pytest.raises(gls.GlsError):
         gls.draft_sample(x.cpu())
     with pytest.raises(gls.GlsError):
-        gls.target_sample_verify(x, tok, flags=16)
+        gls.target_sample_verify(x, tok, flags=64)
     with pytest.raises(gls.GlsError):
         gls.draft_sample(torch.zeros(1, 65, 1, 8, device="cuda"))
     # the context is still usable afterwards
@@ -487,3 +487,38 @@ def test_verify_position_by_position(gls, oracle, dtype):
         gls.target_sample_verify(t, dtok, flags=gls.VERIFY_ACTIVE_ROWS, spec=1, **kw)
     with pytest.raises(gls.GlsError):
         gls.target_sample_verify(t, dtok, flags=gls.VERIFY_ACTIVE_ROWS | gls.VERIFY_ALL_ROWS, **kw)
+
+
+def test_walk_in_two_calls_and_from_host_buffers(gls):
+    """The walk in phases split into its two calls, with every target row that the second call
+    does not read overwritten by NaN in between, equals the one-call walk; and the step from
+    pinned host buffers, which copies only those rows, equals the step on device tensors."""
+    from paper_2506_05632_b200 import pipeline
+
+    w = synth.verify_workload(3, "cuda", B=11, K=8, L=5, V=30011)
+    B, K, L, V = w.shape
+    kw = dict(seed=w.noise_seed, inv_temp=w.inv_temp)
+    tok, _ = gls.draft_sample(w.draft_logits, **kw)
+    ref = gls.target_sample_verify(w.target_logits, tok, flags=gls.VERIFY_ACTIVE_ROWS, **kw)
+    ref = {k: v.clone() for k, v in ref.items()}
+    ws = torch.empty(gls.workspace_bytes(B, K, L + 1, V), dtype=torch.uint8, device="cuda")
+    t = w.target_logits.clone()
+    out = gls.target_sample_verify(t, tok, flags=gls.VERIFY_FIRST_PHASE, workspace=ws, **kw)
+    assert torch.equal(out["accept"][:, :, 0], ref["accept"][:, :, 0])
+    assert torch.equal(out["tokens"][:, 0], ref["tokens"][:, 0])
+    alive = out["accept"][:, :, 0].bool()
+    assert 0 < int(alive.sum()) < B * K
+    t[:, :, 1:][~alive] = float("nan")  # rows of pruned drafts: never read again
+    out = gls.target_sample_verify(t, tok, flags=gls.VERIFY_REST, workspace=ws, out=out, **kw)
+    for key in ("tokens", "tau", "accept"):
+        assert torch.equal(out[key], ref[key]), key
+    assert torch.equal(out["scores"].nan_to_num(7.0), ref["scores"].nan_to_num(7.0))
+    hs = pipeline.HostStepper(B, K, L, V, w.draft_logits.dtype, chunk_seqs=4)
+    h_d, h_t = w.draft_logits.cpu().pin_memory(), w.target_logits.cpu().pin_memory()
+    for _ in range(2):  # the second pass reuses the staging buffers
+        res = hs.step(h_d, h_t, **kw)
+        for key in ("tokens", "tau", "accept"):
+            assert torch.equal(res[key], ref[key].cpu()), key
+    assert hs.h2d_bytes == (B * K * (L + 1) + int(alive.sum()) * L) * V * 2 < hs.h2d_bytes_all
+    with pytest.raises(gls.GlsError):
+        gls.target_sample_verify(t, tok, flags=gls.VERIFY_FIRST_PHASE | gls.VERIFY_REST, **kw)
