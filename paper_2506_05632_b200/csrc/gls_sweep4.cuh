@@ -314,12 +314,23 @@ __device__ __forceinline__ void s4_item(const SweepArgs& A, int row, int split, 
       philox4x32<ROUNDS>(A.rk, A.rounds, s4_call_index(g0), c1s, pos, seq, cw);
     };
 
+    // shapes that keep the next step's loads in flight request the first step now, so that it
+    // arrives while the warm start computes (which then takes its data from the same registers)
+    constexpr bool PREFETCH = S4Cfg<SH>::kPrefetch && !MULTI;
+    G nxt[PREFETCH ? kS4LaneGroups : 1];
+    if (PREFETCH && n_steps > 0) load_step(nxt, 0);
+
     // ---- warm start: evaluate, per lane, the most promising group of the first step; skipped
     //      when an earlier slice of the row has already published a bound ---------------------
     if (n_steps > 0 && m_enc == 0u) {
       G g[kS4LaneGroups];
       uint32_t cw[4];
-      load_step(g, 0);
+      if constexpr (PREFETCH) {
+#pragma unroll
+        for (int j = 0; j < kS4LaneGroups; ++j) g[j] = nxt[j];
+      } else {
+        load_step(g, 0);
+      }
       coarse_step(cw, 0, c1);
       float bkey = -CUDART_INF_F;
       int bj = -1;
@@ -435,9 +446,6 @@ __device__ __forceinline__ void s4_item(const SweepArgs& A, int row, int split, 
       // ---- the sweep.  The inner loop runs until 32 groups are queued; the batched evaluation
       //      is called from the outer loop so that the inner loop carries no call.
       int s = 0;
-      constexpr bool PREFETCH = S4Cfg<SH>::kPrefetch;
-      G nxt[PREFETCH ? kS4LaneGroups : 1];
-      if (PREFETCH && n_steps > 0) load_step(nxt, 0);
       for (;;) {
 #pragma unroll 1
         for (; s < n_steps && qn < 32; ++s) {
