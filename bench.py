@@ -574,8 +574,10 @@ def run_ours(args):
     bf = w.target_logits.dtype == torch.bfloat16
     vrec = None
     if args.topm:
-        achieved, k_ms, k_bytes = tbytes / (verify_ms * 1e-3) / 1e9, verify_ms, tbytes
-        kname = "topm_select_kernel<%s> + sparse_verify_kernel (target side: selection of the top-M " \
+        # the verify call truncates (and so reads) only the rows its walk of Algorithm 2 needs
+        vrec = _verify_call_record(pkg, w.target_logits, L, buf.out, verify_ms, peak)
+        achieved, k_ms, k_bytes = dbytes / (draft_ms * 1e-3) / 1e9, draft_ms, dbytes
+        kname = "topm_select_kernel<%s> + sparse_draft_kernel (draft side: selection of the top-M " \
                 "tokens of every row, then the race on the lists; the event bracket is the whole call)" % (
                     "bf16" if bf else "f32")
     else:
@@ -663,7 +665,7 @@ def run_ours(args):
             # draft call: sweep + reduction; verify call: sweep + reduction with Algorithm 2's
             # loop, or in phases: initialisation + 2 x (sweep over the listed rows + walk)
             "clocks": clocks, "e2e": e2e,
-            "gpu_launches": (4 if args.topm else 7 if vrec["walk"] == "phases" else 2 if args.fused else 4) * args.steps,
+            "gpu_launches": (7 if vrec["walk"] == "phases" else 2 if args.fused and not args.topm else 4) * args.steps,
             "roofline": roofline, "cpu_baseline": cpu}
     print(json.dumps(line))
     if dist is not None:

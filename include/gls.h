@@ -369,7 +369,12 @@ int gls_target_sample_verify_sparse(const gls_sparse_rows_t* target_rows, int B,
  * 1 <= M <= 256.  `workspace` (device, gls_topm_workspace_bytes) receives the lists: int32 ids
  * [B,K,J,M] followed, 256-byte aligned, by fp32 logits [B,K,J,M], in index order, id -1 past the
  * kept count; the caller may read them after the call.  Errors as for the dense entry points;
- * K * (L + 1) must not exceed 1536 for the verify call.
+ * K * (L + 1) must not exceed 1536 for the verify call.  The verify call on a row per draft walks
+ * Algorithm 2 in phases when gls_verify_walk() says so for the dense rows (or `flags` carries
+ * GLS_VERIFY_ACTIVE_ROWS; GLS_VERIFY_ALL_ROWS forbids it): the selection, which is what the call
+ * costs, then runs only over the rows the walk reads -- position 0 of every draft, then the
+ * remaining positions of the drafts that survived it -- and the lists of the other rows are left
+ * unwritten.  After the lists the workspace holds the state of that walk.
  */
 size_t gls_topm_workspace_bytes(int B, int K, int J, int M);
 int gls_draft_sample_topm(const gls_rows_t* draft_logits, int B, int K, int J, int64_t V, int M,

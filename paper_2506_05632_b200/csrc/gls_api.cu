@@ -500,7 +500,7 @@ __global__ void phased_init_kernel(const VerifyArgs va, const PhasedState S, int
     va.out_num[t] = 0;
   }
   if (t < kMaxPhases) S.counts[t] = t == 0 ? (int)((va.multi_rows ? va.B : BK) * first_end) : 0;
-  if (t < BK * va.J) hints[t] = 0u;
+  if (hints != nullptr && t < BK * va.J) hints[t] = 0u;
   if (t < (long long)va.B * va.J) {
     va.out_tokens[t] = -1;
     if (va.out_scores) va.out_scores[t] = 0.f;
@@ -508,32 +508,13 @@ __global__ void phased_init_kernel(const VerifyArgs va, const PhasedState S, int
   if (t < BK * va.L) va.accept[t] = 0;
 }
 
-// Phase `phase` = positions [j0, j1) of every sequence that is still running; the next phase (if
-// any) is [j1, j2).  A CTA per sequence, a warp per listed row, then one warp walks the positions.
-template <int DT, int ROUNDS>
-__global__ void __launch_bounds__(kFusedVerifyMaxWarps * 32)
-phased_verify_kernel(const __grid_constant__ SweepArgs A, const VerifyArgs va, const PhasedState S,
-                     int phase, int j0, int j1, int j2, int cta_tokens, int sweep_grid,
-                     int warps_per_slice) {
-  RowResult* srows = reinterpret_cast<RowResult*>(gls_smem_raw);  // [K][j1 - j0]
-  const int b = blockIdx.x;
+// One warp walks positions [j0, j1) of sequence b on the row results srows[k * (j1 - j0) + j - j0]
+// (valid for the drafts in `active`): emits Y_j, prunes the active set, and either lists the
+// survivors' rows at the next phase's positions [j1, j2) or closes the sequence.
+__device__ void phased_walk(const RowResult* srows, unsigned long long active, const VerifyArgs& va,
+                            const PhasedState& S, int b, int phase, int j0, int j1, int j2) {
   const int lane = threadIdx.x & 31;
-  unsigned long long active = S.active[b];  // written by the previous phase, complete by now
-  asm volatile("griddepcontrol.wait;" ::: "memory");  // the sweep before this launch is complete
-  asm volatile("griddepcontrol.launch_dependents;");  // the next phase's sweep may be scheduled
-  if (active == 0ull) return;
   const int K = va.K, L = va.L, J = va.J, W = j1 - j0;
-  const ListedSlicing sl = listed_slicing(S.counts[phase], A.V, cta_tokens, sweep_grid);
-  for (int r = threadIdx.x >> 5; r < K * W; r += (int)(blockDim.x >> 5)) {
-    const int k = r / W, j = j0 + r % W;
-    if (!((active >> k) & 1ull)) continue;
-    if (va.multi_rows && j0 == 0 && k != 0) continue;  // the first phase listed draft 0 only
-    const RowResult rr = finalize_row<DT, 4, ROUNDS>(A, (b * K + k) * J + j, 1, nullptr,
-                                                     sl.splits * warps_per_slice);
-    if (lane == 0) srows[r] = rr;
-  }
-  __syncthreads();
-  if (threadIdx.x >= 32) return;
   int n_out = j0;
   for (int j = j0; j < j1; ++j) {
     // Y_j: the best of the active rows' winners after subtracting each row's log-sum-exp; ties:
@@ -606,6 +587,34 @@ phased_verify_kernel(const __grid_constant__ SweepArgs A, const VerifyArgs va, c
     S.active[b] = active;
     if (active == 0ull) va.out_num[b] = n_out;
   }
+}
+
+// Phase `phase` = positions [j0, j1) of every sequence that is still running; the next phase (if
+// any) is [j1, j2).  A CTA per sequence, a warp per listed row, then one warp walks the positions.
+template <int DT, int ROUNDS>
+__global__ void __launch_bounds__(kFusedVerifyMaxWarps * 32)
+phased_verify_kernel(const __grid_constant__ SweepArgs A, const VerifyArgs va, const PhasedState S,
+                     int phase, int j0, int j1, int j2, int cta_tokens, int sweep_grid,
+                     int warps_per_slice) {
+  RowResult* srows = reinterpret_cast<RowResult*>(gls_smem_raw);  // [K][j1 - j0]
+  const int b = blockIdx.x;
+  const int lane = threadIdx.x & 31;
+  unsigned long long active = S.active[b];  // written by the previous phase, complete by now
+  asm volatile("griddepcontrol.wait;" ::: "memory");  // the sweep before this launch is complete
+  asm volatile("griddepcontrol.launch_dependents;");  // the next phase's sweep may be scheduled
+  if (active == 0ull) return;
+  const int K = va.K, J = va.J, W = j1 - j0;
+  const ListedSlicing sl = listed_slicing(S.counts[phase], A.V, cta_tokens, sweep_grid);
+  for (int r = threadIdx.x >> 5; r < K * W; r += (int)(blockDim.x >> 5)) {
+    const int k = r / W, j = j0 + r % W;
+    if (!((active >> k) & 1ull)) continue;
+    if (va.multi_rows && j0 == 0 && k != 0) continue;  // the first phase listed draft 0 only
+    const RowResult rr = finalize_row<DT, 4, ROUNDS>(A, (b * K + k) * J + j, 1, nullptr,
+                                                     sl.splits * warps_per_slice);
+    if (lane == 0) srows[r] = rr;
+  }
+  __syncthreads();
+  if (threadIdx.x < 32) phased_walk(srows, active, va, S, b, phase, j0, j1, j2);
 }
 
 // The fused draft + verify call: a CTA per sequence finalises the sequence's K x L draft rows
@@ -796,6 +805,28 @@ sparse_verify_kernel(const __grid_constant__ SweepArgs A, const SparseArgs S, co
   if (threadIdx.x < 32)
     verify_sequence_warp(srows, b, va.K, va.L, va.J, va.flags, va.multi_rows, dtok, va.out_tokens,
                          va.out_num, va.accept, va.out_scores, va.dev_status);
+}
+
+// Algorithm 2 in phases on sparse rows (the lists of a phase were selected just before): as
+// phased_verify_kernel, with the row results computed from the lists.
+template <int SPEC, int ROUNDS>
+__global__ void __launch_bounds__(kFusedVerifyMaxWarps * 32)
+sparse_phased_kernel(const __grid_constant__ SweepArgs A, const SparseArgs Sp, const VerifyArgs va,
+                     const PhasedState S, int phase, int j0, int j1, int j2) {
+  RowResult* srows = reinterpret_cast<RowResult*>(gls_smem_raw);  // [K][j1 - j0]
+  const int b = blockIdx.x;
+  const unsigned long long active = S.active[b];
+  if (active == 0ull) return;
+  const int K = va.K, J = va.J, W = j1 - j0;
+  for (int r = threadIdx.x >> 5; r < K * W; r += (int)(blockDim.x >> 5)) {
+    const int k = r / W, j = j0 + r % W;
+    if (!((active >> k) & 1ull)) continue;
+    if (va.multi_rows && j0 == 0 && k != 0) continue;  // the first phase listed draft 0 only
+    const RowResult rr = sparse_row<SPEC, ROUNDS>(A, Sp, (b * K + k) * J + j, nullptr);
+    if ((threadIdx.x & 31) == 0) srows[r] = rr;
+  }
+  __syncthreads();
+  if (threadIdx.x < 32) phased_walk(srows, active, va, S, b, phase, j0, j1, j2);
 }
 
 // ------------------------------------------------------------------------------------------
@@ -1757,16 +1788,23 @@ size_t gls_static_scratch_bytes(void) { return (size_t)GLS_STATIC_SCRATCH_BYTES;
 // ------------------------------------------------------------------------------------------
 size_t gls_topm_workspace_bytes(int B, int K, int J, int M) {
   if (B <= 0 || K <= 0 || J <= 0 || M <= 0 || M > gls::kTopmMaxM) return 0;
+  // the lists, then the state of a verification in phases (active sets, row lists, their lengths)
   return gls::align_up((size_t)B * K * J * M * sizeof(int32_t), 256) +
-         gls::align_up((size_t)B * K * J * M * sizeof(float), 256);
+         gls::align_up((size_t)B * K * J * M * sizeof(float), 256) +
+         gls::align_up((size_t)B * sizeof(unsigned long long), 256) +
+         gls::align_up((size_t)gls::kMaxPhases * sizeof(int), 256) +
+         gls::align_up((size_t)B * K * J * sizeof(int), 256);
 }
 
 }  // extern "C"
 
 namespace gls {
 // selects into the workspace and describes the result as sparse rows
+// list / count: NULL, or the rows to select (device memory), at most max_listed of them
 static int topm_select(const gls_rows_t* rows, int B, int K, int J, int64_t V, int M, void* workspace,
-                       size_t workspace_bytes, cudaStream_t st, gls_sparse_rows_t* out) {
+                       size_t workspace_bytes, cudaStream_t st, gls_sparse_rows_t* out,
+                       const int* list = nullptr, const int* count = nullptr,
+                       long long max_listed = 0) {
   if (M <= 0 || M > kTopmMaxM || !sizes_ok(B, K, J, V)) return GLS_ERR_INVALID_ARG;
   const int rc = check_rows(rows);
   if (rc != GLS_OK) return rc;
@@ -1784,7 +1822,9 @@ static int topm_select(const gls_rows_t* rows, int B, int K, int J, int64_t V, i
   T.rows = (long long)B * K * J;
   T.ids = (int32_t*)workspace;
   T.logits = (float*)((char*)workspace + align_up((size_t)T.rows * M * sizeof(int32_t), 256));
-  const long long want = (T.rows + kTopmWarps - 1) / kTopmWarps;
+  T.list = list;
+  T.count = count;
+  const long long want = ((list ? max_listed : T.rows) + kTopmWarps - 1) / kTopmWarps;
   const long long cap = (long long)num_sms() * kTopmCtasPerSM;
   const int grid = (int)(want < cap ? want : cap);
   if (rows->dtype == GLS_BF16)
@@ -1799,6 +1839,76 @@ static int topm_select(const gls_rows_t* rows, int B, int K, int J, int64_t V, i
   out->stride_j = M;
   out->M = M;
   return GLS_OK;
+}
+
+// The top-M verify call in phases: select + race position 0 of every draft, walk it, then select
+// + race the remaining positions of the surviving drafts and finish the walk.
+static int topm_verify_phased(const gls_rows_t* rows, int B, int K, int L, int J, int64_t V, int M,
+                              float inv_temp, const int32_t* draft_tokens, const gls_noise_t* noise,
+                              uint32_t flags, int32_t* out_tokens, int32_t* out_num_tokens,
+                              uint8_t* out_accept, float* out_scores, void* workspace,
+                              size_t workspace_bytes, uint32_t* device_status, cudaStream_t st) {
+  if (!out_tokens || !out_num_tokens || !draft_tokens || !out_accept) return GLS_ERR_INVALID_ARG;
+  if (!finite_pos(inv_temp)) return GLS_ERR_INVALID_ARG;
+  if (M <= 0 || M > kTopmMaxM) return GLS_ERR_INVALID_ARG;
+  if (!workspace || workspace_bytes < gls_topm_workspace_bytes(B, K, J, M)) return GLS_ERR_WORKSPACE;
+  const bool multi = (flags & GLS_COMBINE_ALL) && K > 1;
+  SweepArgs A;
+  std::memset(&A, 0, sizeof(A));
+  for (int k = 0; k < K; ++k) A.inv_t[k] = inv_temp;
+  int spec;
+  int rc = fill_noise(A, noise, 0u, &spec);
+  if (rc != GLS_OK) return rc;
+  A.K = K;
+  A.J = J;
+  if (multi) A.multi_k = K;
+  VerifyArgs va;
+  va.B = B; va.K = K; va.L = L; va.J = J;
+  va.flags = flags & (GLS_COMBINE_ALL | GLS_NO_BONUS);
+  va.multi_rows = multi;
+  va.draft_tokens = draft_tokens;
+  va.out_tokens = out_tokens;
+  va.out_num = out_num_tokens;
+  va.accept = out_accept;
+  va.out_scores = out_scores;
+  va.dev_status = device_status;
+  const long long BK = (long long)B * K;
+  char* ws = (char*)workspace;
+  size_t off = align_up((size_t)BK * J * M * sizeof(int32_t), 256) + align_up((size_t)BK * J * M * sizeof(float), 256);
+  PhasedState S;
+  S.active = (unsigned long long*)(ws + off);
+  off += align_up((size_t)B * sizeof(unsigned long long), 256);
+  S.counts = (int*)(ws + off);
+  off += align_up((size_t)kMaxPhases * sizeof(int), 256);
+  S.lists = (int*)(ws + off);
+  const int ends[2] = {1, J};
+  phased_init_kernel<<<(unsigned)((BK * J + 255) / 256), 256, 0, st>>>(va, S, ends[0], nullptr);
+  int j0 = 0;
+  for (int p = 0; p < 2; ++p) {
+    const int j1 = ends[p], j2 = p == 0 ? ends[1] : j1;
+    gls_sparse_rows_t sp;
+    rc = topm_select(rows, B, K, J, V, M, workspace, workspace_bytes, st, &sp, S.lists + BK * j0,
+                     S.counts + p, BK * (j1 - j0));
+    if (rc != GLS_OK) return rc;
+    SparseArgs Sp;
+    Sp.ids = sp.token_ids;
+    Sp.logits = sp.logits;
+    Sp.sb = sp.stride_b;
+    Sp.sk = sp.stride_k;
+    Sp.sj = sp.stride_j;
+    Sp.M = sp.M;
+    const int nrows = K * (j1 - j0);
+    const int warps = nrows < kFusedVerifyMaxWarps ? nrows : kFusedVerifyMaxWarps;
+    const size_t smem = (size_t)nrows * sizeof(RowResult);
+    const bool r10 = A.rounds == 10;
+#define SPARSE_PHASED(SPEC, R) \
+  sparse_phased_kernel<SPEC, R><<<B, warps * 32, smem, st>>>(A, Sp, va, S, p, j0, j1, j2)
+    if (spec == 1) { if (r10) SPARSE_PHASED(1, 10); else SPARSE_PHASED(1, 0); }
+    else { if (r10) SPARSE_PHASED(4, 10); else SPARSE_PHASED(4, 0); }
+#undef SPARSE_PHASED
+    j0 = j1;
+  }
+  return cudaGetLastError() == cudaSuccess ? GLS_OK : GLS_ERR_CUDA;
 }
 }  // namespace gls
 
@@ -1824,13 +1934,27 @@ int gls_target_sample_verify_topm(const gls_rows_t* target_logits, int B, int K,
                                   int32_t* out_num_tokens, uint8_t* out_accept, float* out_scores,
                                   void* workspace, size_t workspace_bytes, uint32_t* device_status,
                                   void* stream) {
-  if (flags & ~(GLS_COMBINE_ALL | GLS_NO_BONUS)) return GLS_ERR_INVALID_ARG;
+  if (!gls::verify_flags_ok(flags) || (flags & (GLS_VERIFY_FIRST_PHASE | GLS_VERIFY_REST)))
+    return GLS_ERR_INVALID_ARG;
+  const uint32_t walk_flags = flags & (GLS_VERIFY_ALL_ROWS | GLS_VERIFY_ACTIVE_ROWS);
+  flags &= ~walk_flags;
   const int J = L + ((flags & GLS_NO_BONUS) ? 0 : 1);
   if (!noise || !out_tokens || !out_num_tokens || L < 0) return GLS_ERR_INVALID_ARG;
   if ((long long)K * J > 1536) return GLS_ERR_UNSUPPORTED;
   gls_sparse_rows_t sp;
   // rows shared by all drafts (stride_k == 0) are truncated once and stay shared
   const int ksel = (target_logits && target_logits->stride_k == 0) ? 1 : K;
+  // Large inputs with a row per draft: Algorithm 2 in phases, so that only the rows it reads are
+  // truncated (the selection is what the call costs).  Same rule as the dense verify call.
+  int walk = 0;
+  if (target_logits && noise && ksel == K && gls::sizes_ok(B, K, J, V) &&
+      (target_logits->dtype == GLS_F32 || target_logits->dtype == GLS_BF16))
+    walk = gls::verify_walk(target_logits->dtype, true, B, K, L, V, 4, flags | walk_flags);
+  if ((walk_flags & GLS_VERIFY_ACTIVE_ROWS) && walk != 1) return GLS_ERR_UNSUPPORTED;
+  if (walk == 1)
+    return gls::topm_verify_phased(target_logits, B, K, L, J, V, M, inv_temp, draft_tokens, noise, flags,
+                                   out_tokens, out_num_tokens, out_accept, out_scores, workspace,
+                                   workspace_bytes, device_status, (cudaStream_t)stream);
   const int rc = gls::topm_select(target_logits, B, ksel, J, V, M, workspace, workspace_bytes,
                                   (cudaStream_t)stream, &sp);
   if (rc != GLS_OK) return rc;
@@ -1839,6 +1963,7 @@ int gls_target_sample_verify_topm(const gls_rows_t* target_logits, int B, int K,
                                          out_tokens, out_num_tokens, out_accept, out_scores,
                                          device_status, stream);
 }
+
 
 int gls_draft_sample_static(const gls_rows_t* draft_logits, int B, int K, int J, int64_t V,
                             float inv_temp, const float* inv_temp_per_draft_host,

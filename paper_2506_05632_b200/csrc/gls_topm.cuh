@@ -31,6 +31,10 @@ struct TopmArgs {
   long long rows;
   int32_t* ids;           // [rows][M]
   float* logits;          // [rows][M]
+  // NULL, or the rows to truncate: row numbers (b * K + k) * J + j in device memory and their
+  // count (the verification in phases truncates only the rows it will read)
+  const int* list;
+  const int* count;
 };
 
 struct TopmWarpBuf {
@@ -179,8 +183,11 @@ topm_select_kernel(const TopmArgs T) {
   TopmWarpBuf* const wb = &bufs[warp];
   int* const queue = queues[warp];
 
-  for (long long row = (long long)blockIdx.x * kTopmWarps + warp; row < T.rows;
-       row += (long long)gridDim.x * kTopmWarps) {
+  const long long n_rows = T.list != nullptr ? (long long)__ldcg(T.count) : T.rows;
+  for (long long it = (long long)blockIdx.x * kTopmWarps + warp; it < n_rows;
+       it += (long long)gridDim.x * kTopmWarps) {
+    const long long row = T.list != nullptr ? (long long)__ldcg(T.list + it) : it;
+    if (!GLS_IN_RANGE(row, 0, T.rows, 42u)) continue;
     const int j = (int)(row % T.J);
     const long long bk = row / T.J;
     const int k = (int)(bk % T.K);

@@ -106,3 +106,35 @@ def test_topm_argument_errors(gls):
             gls.draft_sample_topm(x, M)
     with pytest.raises(gls.GlsError):
         gls.draft_sample_topm(x, 10, workspace=torch.empty(16, dtype=torch.uint8, device="cuda"))
+
+
+@pytest.mark.parametrize("spec", [1, 4])
+def test_topm_verify_in_phases(gls, oracle, spec):
+    """The top-M verify call walked in phases (only the rows Algorithm 2 reads are truncated)
+    against the oracle on masked rows and against the walk that truncates every row; also
+    Appendix B on a row per draft and a call without the bonus row."""
+    B, K, L, V, M = 9, 8, 4, 30011, 50
+    w = synth.verify_workload(3, "cuda", B=B, K=K, L=L, V=V)
+    kw = dict(seed=w.noise_seed, inv_temp=w.inv_temp, spec=spec)
+    dmask, _ = _masked(w.draft_logits, M)
+    dtok, _, _ = gls.draft_sample_topm(w.draft_logits, M, **kw)
+    refd = oracle.draft_sample(dmask, **kw)
+    assert np.array_equal(dtok.cpu().numpy(), refd["tokens"])
+    for extra, t in ((0, w.target_logits), (gls.NO_BONUS, w.target_logits[:, :, :L]),
+                     (gls.COMBINE_ALL, w.target_logits)):
+        tmask, _ = _masked(t.contiguous(), M)
+        refv = oracle.target_sample_verify(tmask, refd["tokens"], flags=extra, **kw)
+        outs = []
+        for how in (gls.VERIFY_ACTIVE_ROWS, gls.VERIFY_ALL_ROWS):
+            out = parity.to_np(gls.target_sample_verify_topm(t, dtok, M, flags=extra | how, **kw))
+            parity.check_verify(out, refv, "top-M flags %d" % (extra | how))
+            outs.append(out)
+        for key in ("tokens", "tau", "accept"):  # fp64 races on the same lists: identical
+            assert np.array_equal(outs[0][key], outs[1][key]), key
+        if extra == 0:
+            assert (refv["tau"] > 1).any() and (refv["tau"] < L + 1).any()
+    with pytest.raises(gls.GlsError):  # rows shared by the drafts leave nothing to skip
+        gls.target_sample_verify_topm(w.target_logits[:, :1].expand(B, K, L + 1, V), dtok, M,
+                                      flags=gls.VERIFY_ACTIVE_ROWS, **kw)
+    with pytest.raises(gls.GlsError):
+        gls.target_sample_verify_topm(w.target_logits, dtok, M, flags=gls.VERIFY_REST, **kw)
