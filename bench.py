@@ -441,7 +441,7 @@ def run_ours(args):
             dtok = pkg.draft_sample_topm(w.draft_logits, args.topm, workspace=topm_ws,
                                          status=buf.status, **kw)[0]
             _mark(marks)
-            buf.out = pkg.target_sample_verify_topm(w.target_logits, dtok, args.topm,
+            buf.out = pkg.target_sample_verify_topm(w.target_logits, dtok, args.topm, flags=walk_flags,
                                                     workspace=topm_ws, status=buf.status, **kw)
             _mark(marks)
             return
@@ -575,7 +575,7 @@ def run_ours(args):
     vrec = None
     if args.topm:
         # the verify call truncates (and so reads) only the rows its walk of Algorithm 2 needs
-        vrec = _verify_call_record(pkg, w.target_logits, L, buf.out, verify_ms, peak)
+        vrec = _verify_call_record(pkg, w.target_logits, L, buf.out, verify_ms, peak, flags=walk_flags)
         achieved, k_ms, k_bytes = dbytes / (draft_ms * 1e-3) / 1e9, draft_ms, dbytes
         kname = "topm_select_kernel<%s> + sparse_draft_kernel (draft side: selection of the top-M " \
                 "tokens of every row, then the race on the lists; the event bracket is the whole call)" % (
