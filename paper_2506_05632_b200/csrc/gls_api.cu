@@ -905,6 +905,15 @@ static cudaError_t launch_finalize_t(const SweepArgs& A, int rows, bool lse, Row
 }
 
 // sweep + split reduction of one batch of rows
+// The launch size for n_items work items dealt round-robin to at most `cap` resident CTAs: the
+// smallest grid that needs no more rounds than `cap` would, so that every CTA gets the same
+// number of items (to within one) and no last round runs on a fraction of the machine.
+static int even_grid(long long n_items, long long cap) {
+  if (n_items <= cap) return (int)(n_items > 0 ? n_items : 1);
+  const long long rounds = (n_items + cap - 1) / cap;
+  return (int)((n_items + rounds - 1) / rounds);
+}
+
 template <int DT, int SPEC, int ROUNDS>
 static cudaError_t launch_fused_verify_t(const SweepArgs& A, const VerifyArgs& va, cudaStream_t st) {
   const size_t smem = fused_verify_smem(va.K, va.L, va.J);
@@ -967,7 +976,7 @@ static int run_rows(SweepArgs& A, int dtype, int spec, const Plan& P, void* work
 #define SWEEP4(SH, R)                                                                       \
   do {                                                                                      \
     const long long cap = (long long)num_sms() * S4Cfg<SH>::kCtasPerSM;                       \
-    const int grid = (int)(P.n_items < cap ? P.n_items : cap);                              \
+    const int grid = even_grid(P.n_items, cap);                                             \
     const size_t smem = sizeof(S4Shared<SH>);                                               \
     if (A.multi_k > 0)                                                                      \
       sweep4_kernel<SH, 1, R, true><<<grid, S4Cfg<SH>::kWarps * 32, smem, st>>>(A);         \
@@ -984,8 +993,8 @@ static int run_rows(SweepArgs& A, int dtype, int spec, const Plan& P, void* work
       A2.chunk = P.chunk2;                                                                  \
       A2.splits = P.splits2;                                                                \
       A2.n_items = (long long)A2.row_count * P.splits2;                                     \
-      const int g1 = (int)(A1.n_items < cap ? A1.n_items : cap);                            \
-      const int g2 = (int)(A2.n_items < cap ? A2.n_items : cap);                            \
+      const int g1 = even_grid(A1.n_items, cap);                                            \
+      const int g2 = even_grid(A2.n_items, cap);                                            \
       sweep4_kernel<SH, 0, R><<<g1, S4Cfg<SH>::kWarps * 32, smem, st>>>(A1);                \
       sweep4_kernel<SH, 1, R><<<g2, S4Cfg<SH>::kWarps * 32, smem, st>>>(A2);                \
     }                                                                                       \
