@@ -382,6 +382,31 @@ def test_step_replayed_as_cuda_graph_matches_eager(gls):
     assert (out["tau"] == L + 1).all()  # identical rows on both sides accept every position
 
 
+def test_walk_in_phases_replayed_as_cuda_graph(gls):
+    """The verify call in phases (a chain of programmatic dependent launches whose sizes are read
+    on the device) can be captured and replayed, also after the inputs changed in place."""
+    B, K, L, V = 6, 4, 3, 20000
+    w = synth.verify_workload(3, "cuda", B=B, K=K, L=L, V=V)
+    t = w.target_logits.clone()
+    kw = dict(seed=w.noise_seed, inv_temp=w.inv_temp)
+    tok, _ = gls.draft_sample(w.draft_logits, **kw)
+    ws = torch.empty(gls.workspace_bytes(B, K, L + 1, V), dtype=torch.uint8, device="cuda")
+    out = gls.target_sample_verify(t, tok, flags=gls.VERIFY_ACTIVE_ROWS, workspace=ws, **kw)
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        gls.target_sample_verify(t, tok, flags=gls.VERIFY_ACTIVE_ROWS, workspace=ws, out=out, **kw)
+    for refill in (False, True):
+        if refill:  # other rows, other survivors
+            t.copy_(torch.roll(w.target_logits, 1, dims=0))
+        graph.replay()
+        got = {k: v.clone() for k, v in out.items()}
+        ref = gls.target_sample_verify(t, tok, flags=gls.VERIFY_ALL_ROWS, **kw)
+        torch.cuda.synchronize()
+        for key in ("tokens", "tau", "accept"):
+            assert torch.equal(got[key], ref[key]), key
+
+
 def test_host_detectable_errors(gls):
     x = torch.zeros(2, 2, 2, 64, device="cuda")
     tok = torch.zeros(2, 2, 1, dtype=torch.int32, device="cuda")
