@@ -295,6 +295,18 @@ int gls_verify_walk(int dtype, int row_per_draft, int B, int K, int L, int64_t V
                     uint32_t flags);
 
 /*
+ * Plumbing for callers whose logits live in (pinned) host memory and who fetch only the rows a
+ * call will read (no counterpart in the paper): n_rows rows of row_bytes bytes each, the rows
+ * src_pitch bytes apart on the host and dst_pitch bytes apart on the device, copied host to
+ * device on `stream` as one strided copy -- e.g. the position-0 rows of a [B,K,J,V] tensor
+ * (pitch J * V * element size) ahead of GLS_VERIFY_FIRST_PHASE.  Asynchronous for pinned host
+ * memory.  Returns GLS_OK, GLS_ERR_INVALID_ARG (null pointer, a pitch below row_bytes) or
+ * GLS_ERR_CUDA.
+ */
+int gls_copy_rows_to_device(void* dst_device, size_t dst_pitch, const void* src_host, size_t src_pitch,
+                            size_t row_bytes, size_t n_rows, void* stream);
+
+/*
  * Draft phase and verification in one call -- Algorithm 2 from its draft loop to its end, for the
  * case where both sets of logits are resident (all L draft positions are known, e.g. a drafter
  * that is not autoregressive in the tokens sampled here, a replayed or re-scored step, or the

@@ -420,6 +420,25 @@ def target_sample_verify(logits, draft_tokens, inv_temp=1.0, flags=0, seed=0, se
     return out
 
 
+def copy_rows_to_device(dst, src, stream=None):
+    """dst (device) and src (pinned host): tensors of the same shape [n, row] and dtype whose rows
+    are contiguous and a constant stride apart (e.g. t[:, :, 0].flatten(0, 1) of a [B,K,J,V]
+    tensor): one strided host-to-device copy on `stream` (default: the current stream)."""
+    assert dst.dim() == 2 and dst.shape == src.shape and dst.dtype == src.dtype
+    assert dst.is_cuda and not src.is_cuda
+    if dst.shape[1] > 1 and (dst.stride(1) != 1 or src.stride(1) != 1):
+        raise GlsError("rows must be contiguous")
+    es = dst.element_size()
+    lib = load()
+    lib.gls_copy_rows_to_device.restype = C.c_int
+    lib.gls_copy_rows_to_device.argtypes = [C.c_void_p, C.c_size_t, C.c_void_p, C.c_size_t, C.c_size_t,
+                                            C.c_size_t, C.c_void_p]
+    n, row = dst.shape
+    st = stream.cuda_stream if stream is not None else _stream()
+    _check(lib.gls_copy_rows_to_device(dst.data_ptr(), max(dst.stride(0), row) * es, src.data_ptr(),
+                                       max(src.stride(0), row) * es, row * es, n, st))
+
+
 def verify_walk(target_logits, L, flags=0, spec=4):
     """1 if target_sample_verify would walk Algorithm 2 in phases for these rows (reading the rows
     of active drafts only), 0 if it would race every row first; GlsError for refused arguments."""

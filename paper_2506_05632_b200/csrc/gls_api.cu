@@ -1207,6 +1207,17 @@ size_t gls_workspace_bytes(int B, int K, int J, int64_t V) {
   return need;
 }
 
+int gls_copy_rows_to_device(void* dst_device, size_t dst_pitch, const void* src_host, size_t src_pitch,
+                            size_t row_bytes, size_t n_rows, void* stream) {
+  if (!dst_device || !src_host || row_bytes == 0 || dst_pitch < row_bytes || src_pitch < row_bytes)
+    return GLS_ERR_INVALID_ARG;
+  if (n_rows == 0) return GLS_OK;
+  return cudaMemcpy2DAsync(dst_device, dst_pitch, src_host, src_pitch, row_bytes, n_rows,
+                           cudaMemcpyHostToDevice, (cudaStream_t)stream) == cudaSuccess
+             ? GLS_OK
+             : GLS_ERR_CUDA;
+}
+
 int gls_verify_walk(int dtype, int row_per_draft, int B, int K, int L, int64_t V, int noise_spec,
                     uint32_t flags) {
   if (!verify_flags_ok(flags)) return -1;

@@ -140,9 +140,10 @@ class HostStepper:
                 if n >= self.STAGES:
                     self.copy_stream.wait_event(s["free"])
                 d.copy_(h_draft[b0:b1], non_blocking=True)
-                for i in range(nb):
-                    for k in range(K):
-                        t[i, k, 0].copy_(h_target[b0 + i, k, 0], non_blocking=True)
+                # the chunk's nb * K rows at position 0, (L + 1) * V elements apart: one strided copy
+                rows0 = (nb * K, self.V), ((L + 1) * self.V, 1)
+                binding.copy_rows_to_device(t.as_strided(*rows0), h_target[b0:b1].as_strided(*rows0),
+                                            stream=self.copy_stream)
                 s["ready"].record(self.copy_stream)
             main.wait_event(s["ready"])
             kw = dict(inv_temp=inv_temp, seed=seed, seq_base=seq_base + b0, spec=spec, rounds=rounds,
