@@ -324,8 +324,9 @@ int gls_copy_rows_to_device(void* dst_device, size_t dst_pitch, const void* src_
  *   out_draft_tokens   [B,K,L] int32, out_draft_scores NULL or [B,K,L] fp32 (as gls_draft_sample)
  *   out_tokens, out_num_tokens, out_accept, out_scores: as gls_target_sample_verify
  *   workspace          at least gls_draft_verify_workspace_bytes(B, K, L, J, V) bytes
- * L >= 1.  Default noise layout only; GLS_COMBINE_ALL only with target rows shared by all k; K, L
- * such that K * (32 J + 4 L) bytes fit in 48 KB (GLS_ERR_UNSUPPORTED otherwise: use the two calls).
+ * L >= 1.  Default noise layout only; K, L such that K * (32 J + 4 L) bytes fit in 48 KB
+ * (GLS_ERR_UNSUPPORTED otherwise: use the two calls).  GLS_COMBINE_ALL with a target row per draft
+ * runs as the two calls internally (and has their limits: K <= 8).
  */
 size_t gls_draft_verify_workspace_bytes(int B, int K, int L, int J, int64_t V);
 int gls_draft_verify(const gls_rows_t* draft_logits, const gls_rows_t* target_logits, int B, int K,

@@ -1363,21 +1363,23 @@ int gls_draft_verify(const gls_rows_t* draft_logits, const gls_rows_t* target_lo
   // row per draft and sequences whose row results exceed the epilogue's shared memory take the
   // two separate calls
   if (spec != 4) return GLS_ERR_UNSUPPORTED;
-  if ((flags & GLS_COMBINE_ALL) && target_logits->stride_k != 0 && K > 1) return GLS_ERR_UNSUPPORTED;
   if (fused_verify_smem(K, L, J) > kFusedVerifyMaxSmem) return GLS_ERR_UNSUPPORTED;
   const long long rows_d = (long long)B * K * L, rows_t = (long long)B * K * J;
   // Large target rows: the draft rows first, then Algorithm 2 in phases, which reads the target
-  // rows of active drafts only (the draft tokens it needs are this call's own output).
-  if (verify_walk(target_logits->dtype, target_logits->stride_k != 0, B, K, L, V, spec, flags) == 1) {
+  // rows of active drafts only (the draft tokens it needs are this call's own output).  Appendix
+  // B on a row per draft (every row under all K streams) takes the two calls at any size.
+  const bool multi = (flags & GLS_COMBINE_ALL) && target_logits->stride_k != 0 && K > 1;
+  const int walk = verify_walk(target_logits->dtype, target_logits->stride_k != 0, B, K, L, V, spec, flags);
+  if (walk < 0) return GLS_ERR_UNSUPPORTED;
+  if (walk == 1 || multi) {
     if (!workspace || workspace_bytes < gls_draft_verify_workspace_bytes(B, K, L, J, V)) return GLS_ERR_WORKSPACE;
     rc = gls_draft_sample(draft_logits, B, K, L, V, inv_temp_draft, inv_temp_per_draft_host, noise,
                           out_draft_tokens, out_draft_scores, workspace, workspace_bytes, device_status,
                           stream);
     if (rc != GLS_OK) return rc;
     return gls_target_sample_verify(target_logits, B, K, L, V, inv_temp_target, out_draft_tokens, noise,
-                                    flags | GLS_VERIFY_ACTIVE_ROWS, out_tokens, out_num_tokens,
-                                    out_accept, out_scores, workspace, workspace_bytes, device_status,
-                                    stream);
+                                    flags, out_tokens, out_num_tokens, out_accept, out_scores,
+                                    workspace, workspace_bytes, device_status, stream);
   }
   const Plan P = make_plan_step(rows_d, rows_t, V, draft_logits->dtype);
   if (!workspace || workspace_bytes < P.total) return GLS_ERR_WORKSPACE;

@@ -450,7 +450,8 @@ def test_draft_verify_in_one_call(gls, oracle, dtype):
         for flags, tt, kw in (
                 (0, t, dict(seed=SEED + 21, inv_temp=0.9, seq_base=3, pos_base=1)),
                 (gls.NO_BONUS, t[:, :, :L], dict(seed=SEED + 22, inv_temp_per_draft=its, inv_temp=1.3)),
-                (gls.COMBINE_ALL, t[:, :1].expand(B, K, L + 1, V), dict(seed=SEED + 23, inv_temp=1.0))):
+                (gls.COMBINE_ALL, t[:, :1].expand(B, K, L + 1, V), dict(seed=SEED + 23, inv_temp=1.0)),
+                (gls.COMBINE_ALL, t, dict(seed=SEED + 24, inv_temp=1.1))):  # Appendix B, a row per draft
             dtok, dsc, out = gls.draft_verify(d, tt, flags=flags, **kw)
             tok2, sc2 = gls.draft_sample(d, **kw)
             vkw = {k: v for k, v in kw.items() if k != "inv_temp_per_draft"}
