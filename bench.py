@@ -241,14 +241,17 @@ def _verify_call_record(pkg, target_logits, L, out, ms, peak, flags=0, spec=4):
     remaining positions of the drafts that survive position 0; otherwise every row."""
     B, K, J, V = target_logits.shape
     es = target_logits.element_size()
-    walk = pkg.verify_walk(target_logits, L, flags, spec) if spec == 4 else 0
+    ends = pkg.verify_phases(target_logits, L, flags, spec) if spec == 4 else []
     rows = B * K * J
-    if walk == 1:
-        survivors = int(out["accept"][:, :, 0].sum().item())
-        rows = (B if (flags & pkg.COMBINE_ALL) else B * K) + survivors * (J - 1)
+    if ends:
+        # phase p reads its positions' rows of the drafts active when it starts
+        rows, j0 = (B if (flags & pkg.COMBINE_ALL) else B * K) * ends[0], ends[0]
+        for e in ends[1:]:
+            rows += int(out["accept"][:, :, j0 - 1].sum().item()) * (e - j0)
+            j0 = e
     r = _fracs(rows * V * es, ms, peak)
-    r.update(walk="phases" if walk == 1 else "every row", rows_read=rows, rows_given=B * K * J,
-             bytes_read=rows * V * es)
+    r.update(walk="phases" if ends else "every row", phase_ends=ends or None, rows_read=rows,
+             rows_given=B * K * J, bytes_read=rows * V * es)
     return r
 
 
@@ -665,7 +668,8 @@ def run_ours(args):
             # draft call: sweep + reduction; verify call: sweep + reduction with Algorithm 2's
             # loop, or in phases: initialisation + 2 x (sweep over the listed rows + walk)
             "clocks": clocks, "e2e": e2e,
-            "gpu_launches": (7 if vrec["walk"] == "phases" else 2 if args.fused and not args.topm else 4) * args.steps,
+            "gpu_launches": (3 + 2 * len(vrec["phase_ends"]) if vrec["walk"] == "phases"
+                             else 2 if args.fused and not args.topm else 4) * args.steps,
             "roofline": roofline, "cpu_baseline": cpu}
     print(json.dumps(line))
     if dist is not None:

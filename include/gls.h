@@ -134,10 +134,14 @@ typedef struct {
  * caller that fetches target rows on demand (e.g. from host memory).  GLS_VERIFY_FIRST_PHASE reads
  * the rows at position 0 only and writes out_tokens[:,0], out_accept[:,:,0] and out_num_tokens
  * (the emitted count for sequences that stopped, 0 for those still running).  GLS_VERIFY_REST
- * reads, of the other rows, exactly those (b, k, 1..J-1) with out_accept[b,k,0] == 1 and
- * completes all outputs; rows it does not read need not hold valid data.                         */
+ * reads, of the other rows, only rows (b, k, 1..J-1) with out_accept[b,k,0] == 1 (all of them,
+ * or fewer where a further phase can leave some out) and completes all outputs; rows of drafts
+ * that did not survive position 0 need not hold valid data.                                      */
 #define GLS_VERIFY_FIRST_PHASE 16u
 #define GLS_VERIFY_REST 32u
+/* The walk in phases with positions 1 and 2 as a phase of their own whatever the size (by default
+ * only very large inputs take it: see gls_verify_phases).                                        */
+#define GLS_VERIFY_THREE_PHASES 64u
 
 /* Library version, major * 10000 + minor * 100 + patch. */
 int gls_version(void);
@@ -293,6 +297,15 @@ int gls_target_sample_verify(const gls_rows_t* target_logits, int B, int K, int 
  */
 int gls_verify_walk(int dtype, int row_per_draft, int B, int K, int L, int64_t V, int noise_spec,
                     uint32_t flags);
+/*
+ * The phases of that walk: returns their number (0 when every row is raced, -1 for refused
+ * arguments) and writes to the HOST array ends[p] = one past the last position of phase p.  Phase
+ * p reads the rows (b, k, j), j in [ends[p-1], ends[p]), of the drafts k still active when it
+ * starts (phase 0: every draft, position 0).  Two phases normally; very large inputs take
+ * positions 1 and 2 as a phase of their own before the rest.
+ */
+int gls_verify_phases(int dtype, int row_per_draft, int B, int K, int L, int64_t V, int noise_spec,
+                      uint32_t flags, int ends_host[4]);
 
 /*
  * Plumbing for callers whose logits live in (pinned) host memory and who fetch only the rows a

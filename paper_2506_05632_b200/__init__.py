@@ -12,9 +12,9 @@ kernels of csrc/.  There is no CPU fallback: if libgls.so cannot be loaded the c
 """
 from .binding import (  # noqa: F401
     COMBINE_ACTIVE, COMBINE_ALL, NO_BONUS, VERIFY_ALL_ROWS, VERIFY_ACTIVE_ROWS, VERIFY_FIRST_PHASE,
-    VERIFY_REST, NOISE_SHARED_ACROSS_K,
+    VERIFY_REST, VERIFY_THREE_PHASES, NOISE_SHARED_ACROSS_K,
     DEV_EMPTY_SUPPORT, GlsError,
     build, copy_rows_to_device, debug_bounds, compress_gaussian, compress_gaussian_workspace_bytes, compress_select, draft_sample, draft_sample_sparse, draft_sample_static,
     draft_sample_topm, draft_verify, draft_verify_workspace_bytes, lib_path, load,
     static_scratch_bytes, status_string, target_sample_verify, target_sample_verify_sparse,
-    target_sample_verify_topm, topm_workspace_bytes, verify_walk, version, workspace_bytes)
+    target_sample_verify_topm, topm_workspace_bytes, verify_phases, verify_walk, version, workspace_bytes)

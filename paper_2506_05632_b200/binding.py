@@ -14,6 +14,7 @@ _LIB = os.path.join(_HERE, "libgls.so")
 COMBINE_ACTIVE, COMBINE_ALL, NO_BONUS = 0, 1, 2
 VERIFY_ALL_ROWS, VERIFY_ACTIVE_ROWS = 4, 8  # how the dense verify call walks Algorithm 2
 VERIFY_FIRST_PHASE, VERIFY_REST = 16, 32   # the walk in phases as two calls (rows fetched on demand)
+VERIFY_THREE_PHASES = 64                   # positions 1 and 2 as a phase of their own
 NOISE_SHARED_ACROSS_K = 1
 DEV_EMPTY_SUPPORT = 1
 F32, BF16 = 0, 1
@@ -452,6 +453,23 @@ def verify_walk(target_logits, L, flags=0, spec=4):
     if rc < 0:
         raise GlsError("gls_verify_walk: arguments that the verify call refuses")
     return rc
+
+
+def verify_phases(target_logits, L, flags=0, spec=4):
+    """Phase boundaries of target_sample_verify's walk for these rows: [] if every row is raced,
+    else [e0, e1, ...] with phase p covering positions [e(p-1), ep)."""
+    B, K, J, V = target_logits.shape
+    lib = load()
+    ends = (C.c_int * 4)()
+    lib.gls_verify_phases.restype = C.c_int
+    lib.gls_verify_phases.argtypes = [C.c_int, C.c_int, C.c_int, C.c_int, C.c_int, C.c_int64, C.c_int,
+                                      C.c_uint32, C.c_void_p]
+    n = int(lib.gls_verify_phases(BF16 if target_logits.dtype == torch.bfloat16 else F32,
+                                  int(target_logits.stride(1) != 0), B, K, int(L), V, int(spec),
+                                  int(flags), ends))
+    if n < 0:
+        raise GlsError("gls_verify_phases: arguments that the verify call refuses")
+    return [int(ends[i]) for i in range(n)]
 
 
 def draft_verify_workspace_bytes(B, K, L, J, V):

@@ -48,6 +48,9 @@ constexpr int kMaxChunk = 16384;
 #ifndef GLS_STEPWISE_MIN_BYTES
 #define GLS_STEPWISE_MIN_BYTES 192e6
 #endif
+#ifndef GLS_THIRD_PHASE_MIN_BYTES
+#define GLS_THIRD_PHASE_MIN_BYTES 256e6
+#endif
 constexpr int kMaxPhases = 4;  // phases of such a walk (two are used: position 0, the rest)
 
 struct Plan {
@@ -431,6 +434,7 @@ struct VerifyArgs {
   int B, K, L, J;
   uint32_t flags;
   bool multi_rows;  // every row result is the best over all K noise streams (Appendix B)
+  bool three_phases;  // the walk in phases: positions 1 and 2 as a phase of their own (forced)
   const int32_t* draft_tokens;
   int32_t* out_tokens;
   int32_t* out_num;
@@ -477,6 +481,16 @@ finalize_verify_kernel(const __grid_constant__ SweepArgs A, const VerifyArgs va)
 // are pruned there, so the second phase takes all remaining positions of the few survivors.
 // State in the workspace: the active set of every sequence, a row list and its length per phase.
 // ------------------------------------------------------------------------------------------
+// The phases of such a walk over J positions: ends[p] = one past the last position of phase p.
+static int phase_ends(int B, int J, long long V, int elt_bytes, int ends[kMaxPhases], bool three = false) {
+  int n = 0;
+  ends[n++] = 1;
+  if (J > 3 && (three || (double)B * (J - 3) * (double)V * elt_bytes >= GLS_THIRD_PHASE_MIN_BYTES))
+    ends[n++] = 3;
+  if (J > 1) ends[n++] = J;
+  return n;
+}
+
 struct PhasedState {
   unsigned long long* active;  // [B]
   int* counts;                 // [kMaxPhases]
@@ -1060,11 +1074,11 @@ static int run_verify_stepwise_t(SweepArgs& A, const VerifyArgs& va, const Plan&
   off += align_up((size_t)kMaxPhases * sizeof(int), 256);
   S.lists = (int*)(ws + off);
   const long long BK = (long long)va.B * va.K;
-  // phases: position 0, then everything else
+  // phases: position 0, then everything else; very large inputs take positions 1 and 2 before
+  // the rest (most survivors of position 0 are pruned there, and a phase's fixed cost is small
+  // against the rows that a sequence of B survivors would read at the remaining positions)
   int ends[kMaxPhases];
-  int n_phases = 0;
-  ends[n_phases++] = 1;
-  if (va.J > 1) ends[n_phases++] = va.J;
+  const int n_phases = phase_ends(va.B, va.J, A.V, DT == kBF16 ? 2 : 4, ends, va.three_phases);
   // part 0: the whole walk; 1: the first phase only (the state stays in the workspace); 2: the
   // phases after the first, from that state
   const int p_begin = part == 2 ? 1 : 0, p_end = part == 1 ? 1 : n_phases;
@@ -1113,8 +1127,8 @@ static int run_verify_stepwise(SweepArgs& A, int dtype, const VerifyArgs& va, co
 #undef STEPWISE
 }
 
-constexpr uint32_t kWalkFlags =
-    GLS_VERIFY_ALL_ROWS | GLS_VERIFY_ACTIVE_ROWS | GLS_VERIFY_FIRST_PHASE | GLS_VERIFY_REST;
+constexpr uint32_t kWalkFlags = GLS_VERIFY_ALL_ROWS | GLS_VERIFY_ACTIVE_ROWS | GLS_VERIFY_FIRST_PHASE |
+                                GLS_VERIFY_REST | GLS_VERIFY_THREE_PHASES;
 // known bits only, and at most one request about the walk
 static bool verify_flags_ok(uint32_t flags) {
   if (flags & ~(GLS_COMBINE_ALL | GLS_NO_BONUS | kWalkFlags)) return false;
@@ -1133,7 +1147,8 @@ static int verify_walk(int dtype, bool row_per_draft, int B, int K, int L, int64
   if (multi && (spec != 4 || K > 8 || V >= (1LL << 28))) return -1;  // the call refuses these
   const bool can = spec == 4 && (multi || !(flags & GLS_COMBINE_ALL)) && L >= 1 && J >= 2 &&
                    (size_t)K * (J - 1) * sizeof(RowResult) <= kFusedVerifyMaxSmem;
-  if (flags & (GLS_VERIFY_ACTIVE_ROWS | GLS_VERIFY_FIRST_PHASE | GLS_VERIFY_REST)) return can ? 1 : -1;
+  if (flags & (GLS_VERIFY_ACTIVE_ROWS | GLS_VERIFY_FIRST_PHASE | GLS_VERIFY_REST | GLS_VERIFY_THREE_PHASES))
+    return can ? 1 : -1;
   if (!can || (flags & GLS_VERIFY_ALL_ROWS)) return 0;
   const double bytes = (double)B * K * J * (double)V * (dtype == GLS_BF16 ? 2.0 : 4.0);
   return bytes >= (multi ? 0.5 : 1.0) * GLS_STEPWISE_MIN_BYTES ? 1 : 0;
@@ -1226,6 +1241,14 @@ int gls_verify_walk(int dtype, int row_per_draft, int B, int K, int L, int64_t V
   return verify_walk(dtype, row_per_draft != 0, B, K, L, V, noise_spec, flags);
 }
 
+int gls_verify_phases(int dtype, int row_per_draft, int B, int K, int L, int64_t V, int noise_spec,
+                      uint32_t flags, int ends_host[4]) {
+  const int walk = gls_verify_walk(dtype, row_per_draft, B, K, L, V, noise_spec, flags);
+  if (walk <= 0 || !ends_host) return walk < 0 ? -1 : 0;
+  const int J = L + ((flags & GLS_NO_BONUS) ? 0 : 1);
+  return phase_ends(B, J, V, dtype == GLS_BF16 ? 2 : 4, ends_host, (flags & GLS_VERIFY_THREE_PHASES) != 0);
+}
+
 size_t gls_draft_verify_workspace_bytes(int B, int K, int L, int J, int64_t V) {
   if (L < 1 || J < L || J > L + 1 || !sizes_ok(B, K, L + J, V)) return 0;
   size_t need = gls_workspace_bytes(B, K, J, V);  // large inputs: a draft call, then a verify call
@@ -1295,6 +1318,7 @@ int gls_target_sample_verify(const gls_rows_t* target_logits, int B, int K, int 
   if (walk < 0) return GLS_ERR_UNSUPPORTED;
   const bool stepwise = walk == 1;
   const int part = (flags & GLS_VERIFY_FIRST_PHASE) ? 1 : (flags & GLS_VERIFY_REST) ? 2 : 0;
+  const bool three = (flags & GLS_VERIFY_THREE_PHASES) != 0;
   flags &= ~kWalkFlags;
   const Plan P = stepwise ? make_plan_stepwise(B, K, J, V, target_logits->dtype, multi)
                           : make_plan((long long)B * K * J, V, spec, target_logits->dtype, multi);
@@ -1312,6 +1336,7 @@ int gls_target_sample_verify(const gls_rows_t* target_logits, int B, int K, int 
   va.B = B; va.K = K; va.L = L; va.J = J;
   va.flags = flags;
   va.multi_rows = multi;
+  va.three_phases = three;
   va.draft_tokens = draft_tokens;
   va.out_tokens = out_tokens;
   va.out_num = out_num_tokens;
@@ -1401,6 +1426,7 @@ int gls_draft_verify(const gls_rows_t* draft_logits, const gls_rows_t* target_lo
   va.B = B; va.K = K; va.L = L; va.J = J;
   va.flags = flags;
   va.multi_rows = false;
+  va.three_phases = false;
   va.draft_tokens = nullptr;  // taken from the draft rows of this very call
   va.out_tokens = out_tokens;
   va.out_num = out_num_tokens;
@@ -1496,6 +1522,7 @@ int gls_target_sample_verify_sparse(const gls_sparse_rows_t* target_rows, int B,
   va.B = B; va.K = K; va.L = L; va.J = J;
   va.flags = flags;
   va.multi_rows = multi;
+  va.three_phases = false;
   va.draft_tokens = draft_tokens;
   va.out_tokens = out_tokens;
   va.out_num = out_num_tokens;
@@ -1888,6 +1915,7 @@ static int topm_verify_phased(const gls_rows_t* rows, int B, int K, int L, int J
   va.B = B; va.K = K; va.L = L; va.J = J;
   va.flags = flags & (GLS_COMBINE_ALL | GLS_NO_BONUS);
   va.multi_rows = multi;
+  va.three_phases = (flags & GLS_VERIFY_THREE_PHASES) != 0;
   va.draft_tokens = draft_tokens;
   va.out_tokens = out_tokens;
   va.out_num = out_num_tokens;
@@ -1903,11 +1931,12 @@ static int topm_verify_phased(const gls_rows_t* rows, int B, int K, int L, int J
   S.counts = (int*)(ws + off);
   off += align_up((size_t)kMaxPhases * sizeof(int), 256);
   S.lists = (int*)(ws + off);
-  const int ends[2] = {1, J};
+  int ends[kMaxPhases];
+  const int n_phases = phase_ends(B, J, V, rows->dtype == GLS_BF16 ? 2 : 4, ends, va.three_phases);
   phased_init_kernel<<<(unsigned)((BK * J + 255) / 256), 256, 0, st>>>(va, S, ends[0], nullptr);
   int j0 = 0;
-  for (int p = 0; p < 2; ++p) {
-    const int j1 = ends[p], j2 = p == 0 ? ends[1] : j1;
+  for (int p = 0; p < n_phases; ++p) {
+    const int j1 = ends[p], j2 = p + 1 < n_phases ? ends[p + 1] : j1;
     gls_sparse_rows_t sp;
     rc = topm_select(rows, B, K, J, V, M, workspace, workspace_bytes, st, &sp, S.lists + BK * j0,
                      S.counts + p, BK * (j1 - j0));
@@ -1958,7 +1987,7 @@ int gls_target_sample_verify_topm(const gls_rows_t* target_logits, int B, int K,
                                   void* stream) {
   if (!gls::verify_flags_ok(flags) || (flags & (GLS_VERIFY_FIRST_PHASE | GLS_VERIFY_REST)))
     return GLS_ERR_INVALID_ARG;
-  const uint32_t walk_flags = flags & (GLS_VERIFY_ALL_ROWS | GLS_VERIFY_ACTIVE_ROWS);
+  const uint32_t walk_flags = flags & (GLS_VERIFY_ALL_ROWS | GLS_VERIFY_ACTIVE_ROWS | GLS_VERIFY_THREE_PHASES);
   flags &= ~walk_flags;
   const int J = L + ((flags & GLS_NO_BONUS) ? 0 : 1);
   if (!noise || !out_tokens || !out_num_tokens || L < 0) return GLS_ERR_INVALID_ARG;
@@ -1972,9 +2001,10 @@ int gls_target_sample_verify_topm(const gls_rows_t* target_logits, int B, int K,
   if (target_logits && noise && ksel == K && gls::sizes_ok(B, K, J, V) &&
       (target_logits->dtype == GLS_F32 || target_logits->dtype == GLS_BF16))
     walk = gls::verify_walk(target_logits->dtype, true, B, K, L, V, 4, flags | walk_flags);
-  if ((walk_flags & GLS_VERIFY_ACTIVE_ROWS) && walk != 1) return GLS_ERR_UNSUPPORTED;
+  if ((walk_flags & (GLS_VERIFY_ACTIVE_ROWS | GLS_VERIFY_THREE_PHASES)) && walk != 1) return GLS_ERR_UNSUPPORTED;
   if (walk == 1)
-    return gls::topm_verify_phased(target_logits, B, K, L, J, V, M, inv_temp, draft_tokens, noise, flags,
+    return gls::topm_verify_phased(target_logits, B, K, L, J, V, M, inv_temp, draft_tokens, noise,
+                                   flags | (walk_flags & GLS_VERIFY_THREE_PHASES),
                                    out_tokens, out_num_tokens, out_accept, out_scores, workspace,
                                    workspace_bytes, device_status, (cudaStream_t)stream);
   const int rc = gls::topm_select(target_logits, B, ksel, J, V, M, workspace, workspace_bytes,

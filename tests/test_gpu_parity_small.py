@@ -428,7 +428,7 @@ def test_host_detectable_errors(gls):
     with pytest.raises(gls.GlsError):
         gls.draft_sample(x.cpu())
     with pytest.raises(gls.GlsError):
-        gls.target_sample_verify(x, tok, flags=64)
+        gls.target_sample_verify(x, tok, flags=128)
     with pytest.raises(gls.GlsError):
         gls.draft_sample(torch.zeros(1, 65, 1, 8, device="cuda"))
     # the context is still usable afterwards
@@ -489,7 +489,7 @@ def test_verify_position_by_position(gls, oracle, dtype):
             ref = oracle.target_sample_verify(synth.to_numpy_rows(tt.contiguous()), dtok.cpu().numpy(),
                                               flags=extra, **kw)
             outs = {}
-            for how in (gls.VERIFY_ACTIVE_ROWS, gls.VERIFY_ALL_ROWS):
+            for how in (gls.VERIFY_ACTIVE_ROWS, gls.VERIFY_ALL_ROWS, gls.VERIFY_THREE_PHASES):
                 status = torch.zeros(1, dtype=torch.int32, device="cuda")
                 out = parity.to_np(gls.target_sample_verify(tt, dtok, flags=extra | how, status=status, **kw))
                 parity.check_verify(out, ref, "cfg%d flags %d" % (cfg, extra | how))
@@ -503,7 +503,7 @@ def test_verify_position_by_position(gls, oracle, dtype):
             if 1 < K <= 8:  # Appendix B on a row per draft: the row of the lowest active draft only
                 refb = oracle.target_sample_verify(synth.to_numpy_rows(tt.contiguous()), dtok.cpu().numpy(),
                                                    flags=extra | gls.COMBINE_ALL, **kw)
-                for how in (gls.VERIFY_ACTIVE_ROWS, gls.VERIFY_ALL_ROWS):
+                for how in (gls.VERIFY_ACTIVE_ROWS, gls.VERIFY_ALL_ROWS, gls.VERIFY_THREE_PHASES):
                     out = parity.to_np(gls.target_sample_verify(tt, dtok, flags=extra | gls.COMBINE_ALL | how, **kw))
                     parity.check_verify(out, refb, "cfg%d Appendix B flags %d" % (cfg, extra | how))
     # the walk in phases needs the default noise layout and rows that it can leave out

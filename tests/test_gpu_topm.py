@@ -125,12 +125,12 @@ def test_topm_verify_in_phases(gls, oracle, spec):
         tmask, _ = _masked(t.contiguous(), M)
         refv = oracle.target_sample_verify(tmask, refd["tokens"], flags=extra, **kw)
         outs = []
-        for how in (gls.VERIFY_ACTIVE_ROWS, gls.VERIFY_ALL_ROWS):
+        for how in (gls.VERIFY_ACTIVE_ROWS, gls.VERIFY_ALL_ROWS, gls.VERIFY_THREE_PHASES):
             out = parity.to_np(gls.target_sample_verify_topm(t, dtok, M, flags=extra | how, **kw))
             parity.check_verify(out, refv, "top-M flags %d" % (extra | how))
             outs.append(out)
         for key in ("tokens", "tau", "accept"):  # fp64 races on the same lists: identical
-            assert np.array_equal(outs[0][key], outs[1][key]), key
+            assert np.array_equal(outs[0][key], outs[1][key]) and np.array_equal(outs[0][key], outs[2][key]), key
         if extra == 0:
             assert (refv["tau"] > 1).any() and (refv["tau"] < L + 1).any()
     with pytest.raises(gls.GlsError):  # rows shared by the drafts leave nothing to skip
