@@ -45,8 +45,8 @@ constexpr int kMaxChunk = 16384;
 // Target rows of a verify call, in bytes, from which Algorithm 2 is walked in phases (measured
 // break-even with the walk that races every row first: 200 MB; 100 MB for Appendix B on a row per
 // draft, whose rows cost K times the noise arithmetic)
-#ifndef GLS_STEPWISE_MIN_BYTES
-#define GLS_STEPWISE_MIN_BYTES 192e6
+#ifndef GLS_PHASED_MIN_BYTES
+#define GLS_PHASED_MIN_BYTES 192e6
 #endif
 #ifndef GLS_THIRD_PHASE_MIN_BYTES
 #define GLS_THIRD_PHASE_MIN_BYTES 256e6
@@ -169,7 +169,7 @@ static Plan make_plan_step(long long rows1, long long rows2, long long V, int dt
 // position can get, and after the hints and partials the state of the walk (active sets, row
 // lists and their lengths) in place of the per-row results.
 template <int SH>
-static Plan make_plan_stepwise_t(int B, int K, int J, long long V) {
+static Plan make_plan_phased_t(int B, int K, int J, long long V) {
   Plan p = Plan();
   p.rows = (long long)B * K * J;
   p.chunk = 0;
@@ -181,11 +181,11 @@ static Plan make_plan_stepwise_t(int B, int K, int J, long long V) {
             align_up((size_t)kMaxPhases * sizeof(int), 256) + align_up((size_t)J * B * K * sizeof(int), 256);
   return p;
 }
-static Plan make_plan_stepwise(int B, int K, int J, long long V, int dtype, bool multi = false) {
+static Plan make_plan_phased(int B, int K, int J, long long V, int dtype, bool multi = false) {
   const int sh = s4_shape(dtype, V, multi);
-  return sh == kS4ShapeBf16 ? make_plan_stepwise_t<kS4ShapeBf16>(B, K, J, V)
-         : sh == kS4ShapeF32Wide ? make_plan_stepwise_t<kS4ShapeF32Wide>(B, K, J, V)
-                                 : make_plan_stepwise_t<kS4ShapeF32Narrow>(B, K, J, V);
+  return sh == kS4ShapeBf16 ? make_plan_phased_t<kS4ShapeBf16>(B, K, J, V)
+         : sh == kS4ShapeF32Wide ? make_plan_phased_t<kS4ShapeF32Wide>(B, K, J, V)
+                                 : make_plan_phased_t<kS4ShapeF32Narrow>(B, K, J, V);
 }
 
 static Plan make_plan(long long rows, long long V, int spec, int dtype, bool multi = false) {
@@ -1064,7 +1064,7 @@ static int run_rows(SweepArgs& A, int dtype, int spec, const Plan& P, void* work
 // Algorithm 2 in phases: per phase a sweep over the listed rows and the kernel that walks the
 // phase's positions.
 template <int SH, int ROUNDS, bool MULTI>
-static int run_verify_stepwise_t(SweepArgs& A, const VerifyArgs& va, const Plan& P, void* workspace,
+static int run_verify_phased_t(SweepArgs& A, const VerifyArgs& va, const Plan& P, void* workspace,
                                  cudaStream_t st, int part) {
   constexpr int DT = S4Cfg<SH>::kDT;
   char* ws = (char*)workspace;
@@ -1122,17 +1122,17 @@ static int run_verify_stepwise_t(SweepArgs& A, const VerifyArgs& va, const Plan&
   }
   return cudaGetLastError() == cudaSuccess ? GLS_OK : GLS_ERR_CUDA;
 }
-static int run_verify_stepwise(SweepArgs& A, int dtype, const VerifyArgs& va, const Plan& P,
+static int run_verify_phased(SweepArgs& A, int dtype, const VerifyArgs& va, const Plan& P,
                                void* workspace, cudaStream_t st, int part) {
   const int sh = s4_shape(dtype, A.V, va.multi_rows);
   const bool r10 = A.rounds == 10;
-#define STEPWISE(SH, M) (r10 ? run_verify_stepwise_t<SH, 10, M>(A, va, P, workspace, st, part) \
-                             : run_verify_stepwise_t<SH, 0, M>(A, va, P, workspace, st, part))
-  if (va.multi_rows) return sh == kS4ShapeBf16 ? STEPWISE(kS4ShapeBf16, true) : STEPWISE(kS4ShapeF32Narrow, true);
-  if (sh == kS4ShapeBf16) return STEPWISE(kS4ShapeBf16, false);
-  if (sh == kS4ShapeF32Wide) return STEPWISE(kS4ShapeF32Wide, false);
-  return STEPWISE(kS4ShapeF32Narrow, false);
-#undef STEPWISE
+#define PHASED(SH, M) (r10 ? run_verify_phased_t<SH, 10, M>(A, va, P, workspace, st, part) \
+                             : run_verify_phased_t<SH, 0, M>(A, va, P, workspace, st, part))
+  if (va.multi_rows) return sh == kS4ShapeBf16 ? PHASED(kS4ShapeBf16, true) : PHASED(kS4ShapeF32Narrow, true);
+  if (sh == kS4ShapeBf16) return PHASED(kS4ShapeBf16, false);
+  if (sh == kS4ShapeF32Wide) return PHASED(kS4ShapeF32Wide, false);
+  return PHASED(kS4ShapeF32Narrow, false);
+#undef PHASED
 }
 
 constexpr uint32_t kWalkFlags = GLS_VERIFY_ALL_ROWS | GLS_VERIFY_ACTIVE_ROWS | GLS_VERIFY_FIRST_PHASE |
@@ -1159,7 +1159,7 @@ static int verify_walk(int dtype, bool row_per_draft, int B, int K, int L, int64
     return can ? 1 : -1;
   if (!can || (flags & GLS_VERIFY_ALL_ROWS)) return 0;
   const double bytes = (double)B * K * J * (double)V * (dtype == GLS_BF16 ? 2.0 : 4.0);
-  return bytes >= (multi ? 0.5 : 1.0) * GLS_STEPWISE_MIN_BYTES ? 1 : 0;
+  return bytes >= (multi ? 0.5 : 1.0) * GLS_PHASED_MIN_BYTES ? 1 : 0;
 }
 
 static bool sizes_ok(int B, int K, int J, int64_t V) {
@@ -1223,7 +1223,7 @@ size_t gls_workspace_bytes(int B, int K, int J, int64_t V) {
   size_t need = all_rows_workspace(B, K, J, V);
   for (int dt = 0; dt < 2; ++dt) {
     for (int multi = 0; multi < 2; ++multi) {  // verification in phases
-      const size_t g = make_plan_stepwise(B, K, J, V, dt, multi != 0).total;
+      const size_t g = make_plan_phased(B, K, J, V, dt, multi != 0).total;
       if (g > need) need = g;
     }
   }
@@ -1324,11 +1324,11 @@ int gls_target_sample_verify(const gls_rows_t* target_logits, int B, int K, int 
   if (multi && (spec != 4 || K > 8 || V >= (1LL << 28))) return GLS_ERR_UNSUPPORTED;
   const int walk = verify_walk(target_logits->dtype, target_logits->stride_k != 0, B, K, L, V, spec, flags);
   if (walk < 0) return GLS_ERR_UNSUPPORTED;
-  const bool stepwise = walk == 1;
+  const bool in_phases = walk == 1;
   const int part = (flags & GLS_VERIFY_FIRST_PHASE) ? 1 : (flags & GLS_VERIFY_REST) ? 2 : 0;
   const bool three = (flags & GLS_VERIFY_THREE_PHASES) != 0;
   flags &= ~kWalkFlags;
-  const Plan P = stepwise ? make_plan_stepwise(B, K, J, V, target_logits->dtype, multi)
+  const Plan P = in_phases ? make_plan_phased(B, K, J, V, target_logits->dtype, multi)
                           : make_plan((long long)B * K * J, V, spec, target_logits->dtype, multi);
   if (!workspace || workspace_bytes < P.total) return GLS_ERR_WORKSPACE;
   if (multi) A.multi_k = K;
@@ -1351,7 +1351,7 @@ int gls_target_sample_verify(const gls_rows_t* target_logits, int B, int K, int 
   va.accept = out_accept;
   va.out_scores = out_scores;
   va.dev_status = device_status;
-  if (stepwise) return run_verify_stepwise(A, target_logits->dtype, va, P, workspace, st, part);
+  if (in_phases) return run_verify_phased(A, target_logits->dtype, va, P, workspace, st, part);
   bool fused = false;
   rc = run_rows(A, target_logits->dtype, spec, P, workspace, true, nullptr, nullptr, nullptr, st,
                 &va, &fused);
