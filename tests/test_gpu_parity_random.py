@@ -47,7 +47,15 @@ def test_random_shapes(gls, oracle, seed):
             dtok = torch.zeros(B, K, 0, dtype=torch.int32, device="cuda")
         # Appendix B: on shared rows under either layout; on a row per draft under the default one
         flags = gls.COMBINE_ALL if ((shared or spec == 4) and rng.random() < 0.4) else 0
-        out = gls.target_sample_verify(t, dtok, flags=flags, **kw)
+        # how Algorithm 2 is walked: the library's choice (every row raced at these sizes) or,
+        # where it can be, in two or three phases
+        walk = int(rng.choice([0, gls.VERIFY_ACTIVE_ROWS, gls.VERIFY_THREE_PHASES]))
+        try:
+            gls.verify_walk(t, L, flags | walk, spec)
+        except gls.GlsError:  # nothing to leave out (e.g. Appendix B on one draft or shared rows)
+            walk = 0
+        what += " walk %d" % walk
+        out = gls.target_sample_verify(t, dtok, flags=flags | walk, **kw)
         refv = oracle.target_sample_verify(synth.to_numpy_rows(t.contiguous()), dtok.cpu().numpy(),
                                            flags=flags, **kw)
         mismatches += parity.check_verify(parity.to_np(out), refv, what)
