@@ -252,6 +252,9 @@ def _verify_call_record(pkg, target_logits, L, out, ms, peak, flags=0, spec=4):
     r = _fracs(rows * V * es, ms, peak)
     r.update(walk="phases" if ends else "every row", phase_ends=ends or None, rows_read=rows,
              rows_given=B * K * J, bytes_read=rows * V * es)
+    # for comparison with a call that reads all it is given: the rows GIVEN per second, as bytes
+    # (not a bandwidth: the walk in phases leaves most of them unread)
+    r["rows_given_gbs"] = B * K * J * V * es / (ms * 1e-3) / 1e9
     return r
 
 
