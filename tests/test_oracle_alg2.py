@@ -216,3 +216,39 @@ def test_appendix_b_acceptance_with_j_of_k_active(oracle):
     # fewer active drafts of the same K: the strongly invariant variant accepts less often than
     # the printed algorithm would with those J drafts alone
     assert theory.exact_acceptance_active(p, q, K, 1) < theory.exact_acceptance(p, q, 1)
+
+
+def test_only_the_rows_of_active_drafts_matter(oracle):
+    """Algorithm 2's Y_j is a minimum over the drafts still active at position j, and the loop ends
+    when none is left: replacing every target row q^(j,k) of a draft that was pruned before
+    position j (and every row past the stopping time) by an unrelated distribution changes no
+    emitted token, no accept flag and no stopping time.  Appendix B's variant reads, per position,
+    the row of the lowest active draft under all K streams: the same replacement, sparing that row
+    only, changes nothing either.  (This is what lets an implementation leave those rows unread.)"""
+    rng = np.random.default_rng(29)
+    Ms, Mb = _tables(rng, 0.8), _tables(rng, 0.8)
+    K, L, n = 4, 4, 4000
+    lMs, lMb = np.log(Ms).astype(np.float32), np.log(Mb).astype(np.float32)
+    X, o = _run(oracle, Ms, Mb, K, L, n)
+    ctx = np.concatenate([np.full((n, K, 1), START, dtype=np.int64), X.astype(np.int64)], axis=2)
+    tl = np.ascontiguousarray(lMb[ctx])  # [n,K,L+1,V], as _run built it
+    acc = o["accept"].astype(bool)
+    # active[b,k,j]: draft k takes part in Y_j
+    active = np.ones((n, K, L + 1), dtype=bool)
+    active[:, :, 1:] = acc
+    assert 0.2 < active.mean() < 0.9  # the case prunes a good share of the rows
+    junk = np.log(rng.dirichlet(np.ones(V), size=(n, K, L + 1))).astype(np.float32)
+    o2 = oracle.target_sample_verify(np.where(active[..., None], tl, junk), X, seed=SEED)
+    for key in ("tokens", "tau", "accept"):
+        assert np.array_equal(o2[key], o[key]), key
+    emitted = np.arange(L + 1)[None, :] < o["tau"][:, None]
+    assert np.allclose(o2["scores"][emitted], o["scores"][emitted], rtol=0, atol=0)
+    # Appendix B on a row per draft: only the lowest active draft's row is read
+    ob = oracle.target_sample_verify(tl, X, flags=COMBINE_ALL, seed=SEED)
+    actb = np.ones((n, K, L + 1), dtype=bool)
+    actb[:, :, 1:] = ob["accept"].astype(bool)
+    lowest = actb & (np.cumsum(actb, axis=1) == 1)
+    ob2 = oracle.target_sample_verify(np.where(lowest[..., None], tl, junk), X, flags=COMBINE_ALL,
+                                      seed=SEED)
+    for key in ("tokens", "tau", "accept"):
+        assert np.array_equal(ob2[key], ob[key]), key
