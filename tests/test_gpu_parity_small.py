@@ -479,7 +479,8 @@ def test_verify_position_by_position(gls, oracle, dtype):
     the oracle and against the walk that races every row first: rows long enough to be cut into
     several slices, one draft, no bonus row, a sequence count that is not a multiple of anything."""
     for cfg, B, K, L, V in ((3, 9, 8, 5, 70001), (4, 7, 8, 8, 40000), (2, 16, 4, 4, 3000),
-                            (3, 5, 1, 3, 20000), (2, 3, 33, 2, 2500)):
+                            (3, 5, 1, 3, 20000), (2, 3, 33, 2, 2500),
+                            (2, 2, 3, 2, (1 << 19) + 777)):  # fp32: the eight-warp launch shape
         w = synth.verify_workload(cfg, "cuda", B=B, K=K, L=L, V=V)
         d, t = w.draft_logits.to(dtype), w.target_logits.to(dtype)
         kw = dict(seed=w.noise_seed, inv_temp=w.inv_temp)
