@@ -366,10 +366,11 @@ def _measure_compress(steps, peak, B=None):
                        max(3, steps // 5))
     eb, db = w.enc_logw.numel() * 4, w.dec_logw.numel() * 4
     agree = float((out["enc_index"] == gout["enc_index"]).float().mean().item())
-    # from the source the path is bound by fp32 arithmetic: (1 + K) rows per sample, N candidates,
-    # D coordinates, one two-wide add and one two-wide multiply-add per coordinate and PAIR of
-    # candidates; peak = SMs x 4 schedulers x 32 lanes x clock, one instruction per lane and clock
-    lane_instr = B * (1 + K) * N * D * 2 / 2
+    # from the source the path is bound by fp32 arithmetic: per sample one encoder row (per
+    # coordinate and PAIR of candidates one two-wide difference and one two-wide multiply-add) and K
+    # decoder rows (one two-wide multiply-add: the dot-product form), N candidates, D coordinates;
+    # peak = SMs x 4 schedulers x 32 lanes x clock, one instruction per lane and clock
+    lane_instr = B * (2 + K) * N * D / 2
     alu_peak = 148 * 4 * 32 * 1.965e9
     assert int(status.item()) == 0
     return {"workload": WORKLOAD_DESC["cfg5"],

@@ -47,14 +47,15 @@ struct __align__(16) GaussEntry {  // a queued group: coarse word, group | strea
 // [stream-row][word][lane] follow it, then the next quad's block.
 struct __align__(16) GaussQuad {
   // [2]: the block being worked on and the next one, which is set up meanwhile
-  float mu[2][kGMaxD][kGRows];                    // scaled means of the block's rows
+  float mu[2][kGMaxD][kGRows];                    // twice the scaled means of the block's rows
   GaussRowCtx ctx[2][kGRows];
   Top2 best[2][kGWarps][kGRows];                  // per warp and row slot
   float lse_m[2][kGWarps][kGRows], lse_s[2][kGWarps][kGRows];
   GaussEntry queue[kGWarps][kGQueue];
 };
 // Layout: quads x (GaussQuad, coarse words [2][kGRows * streams][4][32]), labels [128][4], then the
-// tile [(D + 1)][128 * kGPad] floats, plane D holding |u|^2 / (2 s2_prior).
+// tile [(D + 1)][128 * kGPad] floats, plane D holding the part of a weight that depends on the
+// candidate alone.
 __host__ __device__ inline size_t gauss_quad_bytes(int streams) {
   return sizeof(GaussQuad) + (size_t)2 * kGRows * streams * 4 * 32 * sizeof(uint32_t);
 }
@@ -196,21 +197,26 @@ gauss_sweep_kernel(const __grid_constant__ SweepArgs A, int n_ranges, int rows_p
   float* const us = reinterpret_cast<float*>(gls_smem_raw + (size_t)n_quads * quad_bytes + 128 * 4 * sizeof(uint32_t));
   auto quad_sync = [&]() { asm volatile("bar.sync %0, %1;" ::"r"(quad + 1), "r"(kGWarps * 32) : "memory"); };
 
-  // ---- the tile's coordinates, scaled, to shared memory; plane D holds |u|^2 / (2 s2_prior),
-  //      -inf for candidates past the end (their weights become -inf)
+  // ---- the tile's coordinates, scaled, to shared memory; plane D holds the candidate's own part
+  //      of the weight, -inf for candidates past the end (their weights become -inf)
   {
     const float half_inv_prior = (float)(0.5 / A.g_s2_prior);
     for (int c = threadIdx.x; c < kGTile; c += (int)blockDim.x) {
       const long long i = cand0 + c;
       const int grp = c >> 4, t = c & 15;
       const int at = grp * kGPad + 4 * ((t >> 2) ^ ((grp >> 1) & 3)) + (t & 3);
-      float nrm = 0.f;
+      float nrm = 0.f, nrm_s = 0.f;
       for (int d = 0; d < D; ++d) {
         const float x = i < N ? __ldg(A.gu + i * D + d) : 0.f;
+        const float xs = x * scale;
         nrm = fmaf(x, x, nrm);
-        us[d * kPlane + at] = x * scale;
+        nrm_s = fmaf(xs, xs, nrm_s);
+        us[d * kPlane + at] = xs;
       }
-      us[D * kPlane + at] = i < N ? nrm * half_inv_prior : -CUDART_INF_F;
+      // the part of the weight that does not depend on the row: |u|^2 / (2 s2_prior), in the
+      // decoder pass (dot-product form, below) less |u s|^2
+      us[D * kPlane + at] = i < N ? (ENC ? nrm * half_inv_prior : fmaf(nrm, half_inv_prior, -nrm_s))
+                                  : -CUDART_INF_F;
     }
   }
   // decoder pass with one label array for all samples: the tile's labels, so that the group test
@@ -255,7 +261,7 @@ gauss_sweep_kernel(const __grid_constant__ SweepArgs A, int n_ranges, int rows_p
     const int idx = tq;
     if (idx < kGRows * D) {
       const int r = idx / D, d = idx - r * D;
-      sh.mu[buf][d][r] = pf_mu[0];
+      sh.mu[buf][d][r] = ENC ? pf_mu[0] : 2.0f * pf_mu[0];  // decoder pass: doubled, the cross term's factor
     }
     if (tq < kGRows) {
       const int r = tq;
@@ -324,11 +330,23 @@ gauss_sweep_kernel(const __grid_constant__ SweepArgs A, int n_ranges, int rows_p
     uint32_t (*const xw)[4][32] = xw_all + buf * xw_stride;
     if (it + n_quads < n_blocks) fetch(block_row(it + n_quads));
     // ---- weights of the lane's 16 candidates for the block's four rows -----------------------
+    // With us = u s and ms = m s (s = 1 / sqrt(2 v)) the weight is
+    //   |u|^2 / (2 s2_prior) - |us - ms|^2 = (|u|^2 / (2 s2_prior) - |us|^2) + us . (2 ms) - |ms|^2.
+    // Decoder pass: the first term sits in plane D of the tile, the last is one number per row, and
+    // the middle one is a dot product, one two-wide multiply-add per coordinate and pair of
+    // candidates instead of a difference and a multiply-add.  The cancellation costs eps times the
+    // size of the terms (a few 1e-6 for the decoders' wide conditionals), inside the margin of the
+    // group test and the window in which the reduction re-scores the leaders in fp64.  The encoder
+    // pass keeps the differences: its weights also feed the log-sum-exp that normalises the
+    // encoder's score, and a narrow encoder target (large s) would cost it its 1e-5.
     unsigned long long acc[kGRows][8];
+    float m2acc[kGRows];
 #pragma unroll
-    for (int r = 0; r < kGRows; ++r)
+    for (int r = 0; r < kGRows; ++r) {
+      m2acc[r] = 0.f;
 #pragma unroll
       for (int p = 0; p < 8; ++p) acc[r][p] = 0ull;
+    }
 #pragma unroll 2
     for (int d = 0; d < D; ++d) {
       const float2 m2 = *reinterpret_cast<const float2*>(&sh.mu[buf][d][0]);
@@ -342,14 +360,21 @@ gauss_sweep_kernel(const __grid_constant__ SweepArgs A, int n_ranges, int rows_p
       const float mr[kGRows] = {m2.x, m2.y};
 #pragma unroll
       for (int r = 0; r < kGRows; ++r) {
-        // all differences first, then all multiply-adds: with one warp per scheduler a dependent
-        // pair issued back to back would stall on its own latency
-        const unsigned long long nm2 = pack_f32x2(-mr[r], -mr[r]);
-        unsigned long long diff[8];
+        if constexpr (ENC) {
+          // all differences first, then all multiply-adds: a dependent pair issued back to back
+          // would stall on its own latency
+          const unsigned long long nm2 = pack_f32x2(-mr[r], -mr[r]);
+          unsigned long long diff[8];
 #pragma unroll
-        for (int p = 0; p < 8; ++p) diff[p] = add_f32x2(up[p], nm2);
+          for (int p = 0; p < 8; ++p) diff[p] = add_f32x2(up[p], nm2);
 #pragma unroll
-        for (int p = 0; p < 8; ++p) acc[r][p] = fma_f32x2(diff[p], diff[p], acc[r][p]);
+          for (int p = 0; p < 8; ++p) acc[r][p] = fma_f32x2(diff[p], diff[p], acc[r][p]);
+        } else {
+          const unsigned long long tm2 = pack_f32x2(mr[r], mr[r]);
+          m2acc[r] = fmaf(mr[r], mr[r], m2acc[r]);
+#pragma unroll
+          for (int p = 0; p < 8; ++p) acc[r][p] = fma_f32x2(up[p], tm2, acc[r][p]);
+        }
       }
     }
     float pn[16];
@@ -371,12 +396,13 @@ gauss_sweep_kernel(const __grid_constant__ SweepArgs A, int n_ranges, int rows_p
       if (cx.row < 0) continue;  // uniform over the CTA
       float wgt[16];
       float amax = -CUDART_INF_F;
+      const float nm2 = -0.25f * m2acc[r];  // decoder pass: -|ms|^2 (the means are stored doubled)
 #pragma unroll
       for (int p = 0; p < 8; ++p) {
         float s0, s1;
         unpack_f32x2(acc[r][p], s0, s1);
-        wgt[2 * p] = pn[2 * p] - s0;
-        wgt[2 * p + 1] = pn[2 * p + 1] - s1;
+        wgt[2 * p] = ENC ? pn[2 * p] - s0 : (pn[2 * p] + nm2) + s0;
+        wgt[2 * p + 1] = ENC ? pn[2 * p + 1] - s1 : (pn[2 * p + 1] + nm2) + s1;
         amax = fmaxf(amax, fmaxf(wgt[2 * p], wgt[2 * p + 1]));
       }
       if (ENC) {
