@@ -17,6 +17,7 @@
 #include "gls_sweep4.cuh"
 #include "gls_topm.cuh"
 #include "gls_gauss.cuh"
+#include "gls_gauss_mma.cuh"
 
 namespace gls {
 
@@ -50,6 +51,9 @@ constexpr int kMaxChunk = 16384;
 #endif
 #ifndef GLS_THIRD_PHASE_MIN_BYTES
 #define GLS_THIRD_PHASE_MIN_BYTES 256e6
+#endif
+#ifndef GLS_GAUSS_MMA
+#define GLS_GAUSS_MMA 1
 #endif
 constexpr int kMaxPhases = 4;  // phases of such a walk (two are used: position 0, the rest)
 
@@ -1784,7 +1788,33 @@ int gls_compress_gaussian(const float* candidates, const float* source, const fl
   A.bins = bins;
   A.bins_sb = bins_stride_b;
   A.msg = out_message;
-  GAUSS_SWEEP(false, B * K, P.rows_per_range_dec, 1.0 / std::sqrt(2.0 * var_dec));
+  if (D == kMD && GLS_GAUSS_MMA) {
+    // sixteen coordinates: the rows' dot products with the candidates on the tensor cores
+    const int rows = B * K;
+    long long want = (4LL * num_sms() + P.tiles - 1) / P.tiles;  // CTAs for several waves
+    const long long blocks = (rows + kMRows - 1) / kMRows;
+    if (want > blocks) want = blocks;
+    if (want < 1) want = 1;
+    const int per_range = (int)(((blocks + want - 1) / want) * kMRows);
+    const int n_ranges = (rows + per_range - 1) / per_range;
+    const size_t smem = gauss_mma_smem_bytes();
+    if (cudaMemsetAsync(A.hints, 0, (size_t)rows * sizeof(uint32_t), st) != cudaSuccess ||
+        cudaMemsetAsync(A.partials, 0xff, (size_t)rows * P.tiles * sizeof(Partial), st) != cudaSuccess)
+      return GLS_ERR_CUDA;
+    const float scale_dec = (float)(1.0 / std::sqrt(2.0 * var_dec));
+    if (r10) {
+      cudaFuncSetAttribute(gauss_dec_mma_kernel<10>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+      gauss_dec_mma_kernel<10><<<P.tiles * n_ranges, kMWarps * 32, smem, st>>>(A, n_ranges, per_range,
+                                                                                (long long)N, scale_dec);
+    } else {
+      cudaFuncSetAttribute(gauss_dec_mma_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+      gauss_dec_mma_kernel<0><<<P.tiles * n_ranges, kMWarps * 32, smem, st>>>(A, n_ranges, per_range,
+                                                                               (long long)N, scale_dec);
+    }
+    if (cudaGetLastError() != cudaSuccess) return GLS_ERR_CUDA;
+  } else {
+    GAUSS_SWEEP(false, B * K, P.rows_per_range_dec, 1.0 / std::sqrt(2.0 * var_dec));
+  }
 #undef GAUSS_SWEEP
   err = r10 ? launch_finalize_t<kF32, 4, 10>(A, B * K, false, rowres, nullptr, nullptr, device_status, st)
             : launch_finalize_t<kF32, 4, 0>(A, B * K, false, rowres, nullptr, nullptr, device_status, st);

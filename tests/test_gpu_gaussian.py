@@ -37,11 +37,11 @@ def _compare(gls, oracle, u, a, t, bins, what, **kw):
 
 @pytest.mark.parametrize("shape", [
     (5, 1, 100, 1, 1), (7, 2, 2048, 3, 4), (9, 4, 2049, 16, 16), (6, 3, 5000, 5, 2),
-    (13, 8, 40001, 16, 8), (3, 4, 2048 * 7 + 15, 8, 1),
+    (13, 8, 40001, 16, 8), (3, 4, 2048 * 7 + 15, 8, 1), (4, 3, 3000, 16, 1), (21, 5, 9000, 16, 64),
 ])
 def test_small_shapes(gls, oracle, shape):
-    """Tiles with ragged ends, row counts that are not multiples of four, every D up to 16, with
-    and without labels."""
+    """Tiles with ragged ends, row counts that are not multiples of four or sixteen, every D up to
+    16 (sixteen coordinates: the decoder rows go through the tensor cores), with and without labels."""
     B, K, N, D, l_max = shape
     u, a, t, bins = _case(B, K, N, D, l_max, 11 + N % 13)
     _compare(gls, oracle, u, a, t, bins, "gauss %s" % (shape,), seed=SEED, seq_base=4)
