@@ -1802,15 +1802,16 @@ int gls_compress_gaussian(const float* candidates, const float* source, const fl
         cudaMemsetAsync(A.partials, 0xff, (size_t)rows * P.tiles * sizeof(Partial), st) != cudaSuccess)
       return GLS_ERR_CUDA;
     const float scale_dec = (float)(1.0 / std::sqrt(2.0 * var_dec));
-    if (r10) {
-      cudaFuncSetAttribute(gauss_dec_mma_kernel<10>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-      gauss_dec_mma_kernel<10><<<P.tiles * n_ranges, kMWarps * 32, smem, st>>>(A, n_ranges, per_range,
-                                                                                (long long)N, scale_dec);
-    } else {
-      cudaFuncSetAttribute(gauss_dec_mma_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-      gauss_dec_mma_kernel<0><<<P.tiles * n_ranges, kMWarps * 32, smem, st>>>(A, n_ranges, per_range,
-                                                                               (long long)N, scale_dec);
-    }
+    const bool lab = bins != nullptr && bins_stride_b == 0;
+#define GAUSS_MMA(R, LAB)                                                                                  \
+  do {                                                                                                     \
+    cudaFuncSetAttribute(gauss_dec_mma_kernel<R, LAB>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem); \
+    gauss_dec_mma_kernel<R, LAB><<<P.tiles * n_ranges, kMWarps * 32, smem, st>>>(A, n_ranges, per_range,     \
+                                                                                (long long)N, scale_dec);  \
+  } while (0)
+    if (r10) { if (lab) GAUSS_MMA(10, true); else GAUSS_MMA(10, false); }
+    else { if (lab) GAUSS_MMA(0, true); else GAUSS_MMA(0, false); }
+#undef GAUSS_MMA
     if (cudaGetLastError() != cudaSuccess) return GLS_ERR_CUDA;
   } else {
     GAUSS_SWEEP(false, B * K, P.rows_per_range_dec, 1.0 / std::sqrt(2.0 * var_dec));

@@ -197,7 +197,7 @@ __device__ __noinline__ void gauss_mma_flush(const SweepArgs& A, GaussMmaWarp& w
 // The kernel.  Grid: tiles x row ranges (as gauss_sweep_kernel); rows are decoder rows (b, k)
 // under stream k, restricted to the candidates labelled A.msg[b].  D = 16.
 // ------------------------------------------------------------------------------------------
-template <int ROUNDS>
+template <int ROUNDS, bool LABELS /* one label array for all samples: test eligible candidates only */>
 __global__ void __launch_bounds__(kMWarps * 32, 1)
 gauss_dec_mma_kernel(const __grid_constant__ SweepArgs A, int n_ranges, int rows_per_range, long long N,
                      float scale /* 1 / sqrt(2 v) of the decoders' conditional */) {
@@ -215,7 +215,7 @@ gauss_dec_mma_kernel(const __grid_constant__ SweepArgs A, int n_ranges, int rows
   GaussMmaWarp& wp = reinterpret_cast<GaussMmaWarp*>(labels + kGTile)[warp];
   __shared__ uint32_t umax_bits;  // largest |u s| of the tile (as ordered bits of a non-negative float)
   const float half_inv_prior = (float)(0.5 / A.g_s2_prior);
-  const bool use_labels = A.bins != nullptr && A.bins_sb == 0;
+  constexpr bool use_labels = LABELS;
   if (threadIdx.x == 0) umax_bits = 0u;
   __syncthreads();
   // ---- the tile: scaled coordinates rounded to tf32, P(u), labels
@@ -312,7 +312,8 @@ gauss_dec_mma_kernel(const __grid_constant__ SweepArgs A, int n_ranges, int rows
     }
     // per-row constants of the lane's two rows (accumulator rows g and g + 8)
     const float nm2_lo = -wp.ctx[g].m2, nm2_hi = -wp.ctx[g + 8].m2;
-    const int msg_lo = wp.ctx[g].msg, msg_hi = wp.ctx[g + 8].msg;
+    // the rows' labels, replicated over the bytes of a word for a four-way compare
+    const uint32_t msg_lo = (uint32_t)wp.ctx[g].msg * 0x01010101u, msg_hi = (uint32_t)wp.ctx[g + 8].msg * 0x01010101u;
     // ... and of the row this lane tests
     const bool tester = q < 2 && wp.ctx[my_row].row >= 0;
     const float margin = wp.ctx[my_row].margin;
@@ -335,6 +336,7 @@ gauss_dec_mma_kernel(const __grid_constant__ SweepArgs A, int n_ranges, int rows
           const uint32_t w = __shfl_sync(0xffffffffu, cw[j], my_row + 16 * h);
           // approximate weights of the group's 16 candidates for the lane's two rows
           float mlo = -CUDART_INF_F, mhi = -CUDART_INF_F;
+          float wl[4], wh[4];  // the lane's four candidates of the group, lower and upper row
 #pragma unroll
           for (int nt = 0; nt < 2; ++nt) {
             const int cbase = grp * 16 + nt * 8;
@@ -343,18 +345,22 @@ gauss_dec_mma_kernel(const __grid_constant__ SweepArgs A, int n_ranges, int rows
             mma_tf32_16x8x8(c, af[0], __float_as_uint(bv.x), __float_as_uint(bv.y));
             mma_tf32_16x8x8(c, af[1], __float_as_uint(bv.z), __float_as_uint(bv.w));
             const float2 pv = *reinterpret_cast<const float2*>(pc + cbase + 2 * q);
-            float w0 = c[0] + pv.x, w1 = c[1] + pv.y, w2 = c[2] + pv.x, w3 = c[3] + pv.y;
-            if (use_labels) {
-              const uint32_t lb = *reinterpret_cast<const unsigned short*>(labels + cbase + 2 * q);
-              const int l0 = (int)(lb & 0xffu), l1 = (int)(lb >> 8);
-              if (l0 != msg_lo) w0 = -CUDART_INF_F;
-              if (l1 != msg_lo) w1 = -CUDART_INF_F;
-              if (l0 != msg_hi) w2 = -CUDART_INF_F;
-              if (l1 != msg_hi) w3 = -CUDART_INF_F;
-            }
-            mlo = fmaxf(mlo, fmaxf(w0, w1));
-            mhi = fmaxf(mhi, fmaxf(w2, w3));
+            wl[2 * nt] = c[0] + pv.x; wl[2 * nt + 1] = c[1] + pv.y;
+            wh[2 * nt] = c[2] + pv.x; wh[2 * nt + 1] = c[3] + pv.y;
           }
+          if (use_labels) {
+            // labels of the lane's candidates (2 q, 2 q + 1 of each half of the group) in one word
+            const uint32_t lb = (uint32_t)*reinterpret_cast<const unsigned short*>(labels + grp * 16 + 2 * q) |
+                                ((uint32_t)*reinterpret_cast<const unsigned short*>(labels + grp * 16 + 8 + 2 * q) << 16);
+            const uint32_t el = __vcmpeq4(lb, msg_lo), eh = __vcmpeq4(lb, msg_hi);  // 0xff per match
+#pragma unroll
+            for (int t = 0; t < 4; ++t) {
+              if (!(el & (1u << (8 * t)))) wl[t] = -CUDART_INF_F;
+              if (!(eh & (1u << (8 * t)))) wh[t] = -CUDART_INF_F;
+            }
+          }
+          mlo = fmaxf(fmaxf(wl[0], wl[1]), fmaxf(wl[2], wl[3]));
+          mhi = fmaxf(fmaxf(wh[0], wh[1]), fmaxf(wh[2], wh[3]));
           mlo += nm2_lo;
           mhi += nm2_hi;
           // maxima over the quad's four column pairs: odd q keeps the upper row, even q the lower
